@@ -1,0 +1,187 @@
+"""CPU oracle for the RAPID verify step -- TEST INFRASTRUCTURE ONLY.
+
+A ctypes wrapper over ``rapid_oracle.c`` (plain fp64 C written from the paper:
+Algorithm 1, Eq. (new_target), Eq. (delta), the tail rule of Section 2.4).
+It shares nothing with the CUDA library and must not be imported by the
+product package; only tests, the smoke check and the benchmark's CPU-baseline
+leg may use it.
+
+Arrays are numpy; bf16 tensors are passed as their raw bits (uint16).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rapid_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+RESIDUAL_PAPER = 0  # norm(max(p - phat, p - q, 0)): Algorithm 1, residual step
+RESIDUAL_PHAT = 1   # norm(max(phat - q, 0)): Section 2.1's residual with phat as the target
+FLAG_RESIDUAL_FALLBACK = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP) if the shared object is missing or stale.
+
+    ``RAPID_ORACLE_LIB`` may name another build of the same source; the tests
+    use it to show that planted mistakes are caught by the pins.
+    """
+    override = os.environ.get("RAPID_ORACLE_LIB")
+    if override:
+        return override
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        subprocess.run(
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"],
+            check=True,
+        )
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        c_i64 = ctypes.c_int64
+        c_dbl = ctypes.c_double
+        vp = ctypes.c_void_p
+        lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_verify_attention.restype = ctypes.c_int
+        lib.oracle_verify_attention.argtypes = [
+            vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, c_i64,
+            ctypes.c_int, c_i64, c_i64, c_i64, c_dbl, vp, c_i64, vp, vp,
+        ]
+        lib.oracle_rapid_distributions.restype = None
+        lib.oracle_rapid_distributions.argtypes = [vp, vp, c_i64, c_dbl, c_dbl, c_dbl, vp, vp, vp, vp]
+        lib.oracle_residual_weights.restype = None
+        lib.oracle_residual_weights.argtypes = [vp, vp, vp, c_i64, ctypes.c_int, vp]
+        lib.oracle_inverse_cdf.restype = c_i64
+        lib.oracle_inverse_cdf.argtypes = [vp, c_i64, c_dbl]
+        lib.oracle_accept.restype = ctypes.c_int
+        lib.oracle_accept.argtypes = [
+            vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, c_i64, c_dbl, c_dbl, c_dbl, ctypes.c_int,
+            vp, vp, vp, vp,
+        ]
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def verify_attention(q_bits, k_bits, v_bits, ctx_lens, gamma, scale=0.0, units=None,
+                     kv_strides=None):
+    """Definition of verify attention.
+
+    q_bits [B,R,Hq,D] uint16 (bf16 bits); k_bits, v_bits [B,Hkv,Lmax,D] uint16
+    (or flat arrays when ``kv_strides=(stride_b, stride_h, stride_l, Lmax, Hkv)``
+    in elements is given); ctx_lens [B] int32.  Returns (out [B,R,Hq,D]
+    float64, lse [B,R,Hq] float64).  ``units`` optionally lists the
+    (b*Hq+h)*R+i units to compute; other rows are NaN.
+    """
+    lib = _load()
+    q_bits = _c(q_bits, np.uint16)
+    B, R, Hq, D = q_bits.shape
+    assert R == gamma + 1
+    if kv_strides is None:
+        k_bits = _c(k_bits, np.uint16)
+        v_bits = _c(v_bits, np.uint16)
+        _, Hkv, Lmax, Dk = k_bits.shape
+        assert Dk == D and v_bits.shape == k_bits.shape and k_bits.shape[0] == B
+        sb, sh, sl = Hkv * Lmax * D, Lmax * D, D
+    else:
+        sb, sh, sl, Lmax, Hkv = kv_strides
+        assert k_bits.dtype == np.uint16 and v_bits.dtype == np.uint16
+        assert k_bits.flags.c_contiguous and v_bits.flags.c_contiguous
+    ctx_lens = _c(ctx_lens, np.int32)
+    out = np.full((B, R, Hq, D), np.nan, dtype=np.float64)
+    lse = np.full((B, R, Hq), np.nan, dtype=np.float64)
+    if units is not None:
+        units = _c(units, np.int64)
+        n_units = units.size
+    else:
+        n_units = 0
+    rc = lib.oracle_verify_attention(
+        _ptr(q_bits), _ptr(k_bits), _ptr(v_bits), _ptr(ctx_lens), B, Hq, Hkv, D, Lmax, gamma,
+        sb, sh, sl, float(scale), _ptr(units), n_units, _ptr(out), _ptr(lse))
+    if rc != 0:
+        raise ValueError(f"oracle_verify_attention failed with {rc}")
+    return out, lse
+
+
+def rapid_distributions(z, d, T=1.0, eta=0.0, tail_alpha=0.1):
+    """(p, q, phat_patched, phat_raw) for one draft position, all float64 [V]."""
+    lib = _load()
+    z = _c(z, np.float32)
+    d = _c(d, np.float32)
+    V = z.size
+    assert d.size == V
+    p = np.empty(V)
+    q = np.empty(V)
+    phat = np.empty(V)
+    raw = np.empty(V)
+    lib.oracle_rapid_distributions(_ptr(z), _ptr(d), V, float(T), float(eta), float(tail_alpha),
+                                   _ptr(p), _ptr(q), _ptr(phat), _ptr(raw))
+    return p, q, phat, raw
+
+
+def residual_weights(p, q, phat, mode=RESIDUAL_PAPER):
+    lib = _load()
+    p = _c(p, np.float64)
+    q = _c(q, np.float64)
+    phat = _c(phat, np.float64)
+    w = np.empty(p.size)
+    lib.oracle_residual_weights(_ptr(p), _ptr(q), _ptr(phat), p.size, int(mode), _ptr(w))
+    return w
+
+
+def inverse_cdf(w, u) -> int:
+    lib = _load()
+    w = _c(w, np.float64)
+    return int(lib.oracle_inverse_cdf(_ptr(w), w.size, float(u)))
+
+
+def accept(target_logits, draft_logits, draft_tokens, uniforms, eta, T=1.0, tail_alpha=0.1,
+           residual_mode=RESIDUAL_PAPER, want_ratios=True):
+    """Algorithm 1's validation loop + residual draw.
+
+    target_logits [B,gamma+1,V] f32, draft_logits [B,gamma,V] f32,
+    draft_tokens [B,gamma] i32, uniforms [B,gamma+1] f32.
+    Returns dict(accept_len [B] i32, next_token [B] i32, flags [B] i32,
+    ratios [B,gamma] f64 or None).
+    """
+    lib = _load()
+    z = _c(target_logits, np.float32)
+    B, R, V = z.shape
+    gamma = R - 1
+    d = _c(draft_logits, np.float32).reshape(B, gamma, V)
+    tok = _c(draft_tokens, np.int32).reshape(B, gamma)
+    u = _c(uniforms, np.float32).reshape(B, R)
+    accept_len = np.empty(B, dtype=np.int32)
+    next_token = np.empty(B, dtype=np.int32)
+    flags = np.empty(B, dtype=np.int32)
+    ratios = np.full((B, gamma), np.nan) if want_ratios else None
+    rc = lib.oracle_accept(_ptr(z), _ptr(d), _ptr(tok), _ptr(u), B, gamma, V, float(eta), float(T),
+                           float(tail_alpha), int(residual_mode), _ptr(accept_len),
+                           _ptr(next_token), _ptr(flags), _ptr(ratios))
+    if rc != 0:
+        raise ValueError(f"oracle_accept failed with {rc}")
+    return dict(accept_len=accept_len, next_token=next_token, flags=flags, ratios=ratios)
