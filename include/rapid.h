@@ -1,0 +1,246 @@
+/*
+ * rapid.h -- C ABI of the RAPID verify-step library (NVIDIA B200, sm_100a).
+ *
+ * The library computes the target model's verification step of
+ * retrieval-augmented speculative decoding (Algorithm 1 of the RAPID paper):
+ *
+ *   1. verify attention: the gamma+1 newest query rows of every sequence attend
+ *      over that sequence's whole bf16 KV cache in one pass (Algorithm 1, the
+ *      LogitsOf step; Section 2.1 "validated by the target model in a single
+ *      forward pass"), causally masked among themselves;
+ *   2. accept / residual: the validation loop of Algorithm 1 with the
+ *      retrieval-augmented target distribution of Eq. (new_target), the tail
+ *      rule of Section 2.4 and the residual draw of Algorithm 1's last step.
+ *
+ * Conventions shared by every entry point
+ *   - Pointers are DEVICE pointers owned by the caller unless a parameter is
+ *     documented as host memory.  Structs are read on the host during the call.
+ *   - Nothing is allocated and nothing is freed.  Scratch lives in a caller
+ *     workspace whose size the *_workspace_bytes() functions give.  A workspace
+ *     must be prepared once with rapid_workspace_init() before its first use
+ *     and must not be shared by calls that can overlap on the GPU.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL is the default stream).  There is no host synchronisation
+ *     unless an entry point says so.
+ *   - Return value: RAPID_OK or one of the RAPID_ERR_* codes.  No exception
+ *     crosses the boundary.  rapid_last_error() describes the last failure on
+ *     the calling thread.
+ *   - Problems only the device can see (a context length outside
+ *     [gamma+1, Lmax], a draft token outside [0, V), an empty residual) set a
+ *     bit of the sticky status word stored in the first 4 bytes of the
+ *     workspace; the kernels never trap and always write defined outputs.
+ */
+#ifndef RAPID_H
+#define RAPID_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RAPID_VERSION 100
+
+/* return codes */
+#define RAPID_OK 0
+#define RAPID_ERR_INVALID_ARG 1 /* NULL pointer, non-positive size, T <= 0, ...              */
+#define RAPID_ERR_UNSUPPORTED 2 /* head_dim not 64/128, too many grouped rows, misalignment   */
+#define RAPID_ERR_WORKSPACE 3   /* workspace missing or smaller than *_workspace_bytes()      */
+#define RAPID_ERR_CUDA 4        /* a CUDA runtime / driver call failed (see rapid_last_error) */
+
+/* bits of the device status word (first int32 of a workspace; sticky) */
+#define RAPID_STATUS_BAD_CTX_LEN 1        /* ctx_lens[b] outside [gamma+1, Lmax]: clamped into range  */
+#define RAPID_STATUS_BAD_DRAFT_TOKEN 2    /* draft token outside [0, V): clamped into range           */
+#define RAPID_STATUS_RESIDUAL_FALLBACK 4  /* residual mass was 0 / not finite: token drawn from p    */
+#define RAPID_STATUS_PIPELINE_TIMEOUT 8   /* an on-chip wait hit its time limit: outputs invalid      */
+
+/* residual_mode */
+#define RAPID_RESIDUAL_PAPER 0 /* norm(max(p - phat, p - q, 0)): Algorithm 1, residual step               */
+#define RAPID_RESIDUAL_PHAT 1  /* norm(max(phat - q, 0)): the residual of Section 2.1 with phat as target */
+
+/*
+ * Geometry of one attention call.
+ *   q, out : [B, R, Hq, D] bf16, dense, R = gamma + 1.  Row i of sequence b is
+ *            the query at absolute position ctx_lens[b] - R + i.
+ *   k, v   : [B, Hkv, Lmax, D] bf16 with D contiguous; element strides between
+ *            sequences / KV heads / tokens as given (0 = dense).  Strides must be
+ *            multiples of 8 elements and the base pointers 16-byte aligned.
+ *            Entries at token positions >= ctx_lens[b] are never used, whatever
+ *            their bits.
+ *   ctx_lens[b] counts the R newest tokens too (their K/V were appended by the
+ *            caller) and must lie in [R, Lmax].
+ *   Hq must be a multiple of Hkv; (Hq/Hkv) * R grouped rows per KV head may
+ *   not exceed 128; D is 64 or 128.
+ */
+typedef struct rapid_attn_shape {
+    int32_t B;
+    int32_t Hq;
+    int32_t Hkv;
+    int32_t D;
+    int64_t Lmax;
+    int64_t kv_stride_b;
+    int64_t kv_stride_h;
+    int64_t kv_stride_l;
+} rapid_attn_shape;
+
+/* Optional knobs and extra outputs of the attention call (NULL = defaults). */
+typedef struct rapid_attn_params {
+    float scale;      /* softmax scale; 0 = 1/sqrt(D)                                             */
+    int32_t num_ctas; /* CTAs the KV length is split over; 0 = one per SM; at most 512            */
+    float* lse_out;   /* device [B, R, Hq] fp32 natural-log sum-exp of the scaled scores, or NULL */
+    float* out_f32;   /* device [B, R, Hq, D] fp32 output before bf16 rounding, or NULL           */
+} rapid_attn_params;
+
+/*
+ * Geometry of one accept call.
+ *   target_logits : [B, gamma+1, V] fp32, row stride target_row_stride elements (0 = V)
+ *   draft_logits  : [B, gamma,   V] fp32, row stride draft_row_stride elements (0 = V)
+ *   V and both row strides are multiples of 4 and the bases 16-byte aligned.
+ */
+typedef struct rapid_accept_shape {
+    int32_t B;
+    int32_t gamma;
+    int64_t V;
+    int64_t target_row_stride;
+    int64_t draft_row_stride;
+} rapid_accept_shape;
+
+/* Parameters of the accept rule (NULL = T 1, tail_alpha 0.1, RAPID_RESIDUAL_PAPER, no extras). */
+typedef struct rapid_accept_params {
+    float temperature;     /* T > 0 of Algorithm 1; the same T scales target and draft logits   */
+    float tail_alpha;      /* Section 2.4: entries of phat below tail_alpha * max(phat) keep p;
+                              0 disables the rule                                              */
+    int32_t residual_mode; /* RAPID_RESIDUAL_*                                                  */
+    int32_t reserved;
+    float* ratio_out;      /* device [B, gamma] fp32: phat(x')/q(x') of every position, or NULL */
+} rapid_accept_params;
+
+/* ---- workspaces ---------------------------------------------------------------------------- */
+
+/* Bytes of scratch rapid_verify_attention() needs for this geometry (0 on invalid arguments). */
+size_t rapid_attention_workspace_bytes(const rapid_attn_shape* shape, int gamma);
+
+/* Bytes of scratch rapid_accept() needs (0 on invalid arguments). */
+size_t rapid_accept_workspace_bytes(const rapid_accept_shape* shape);
+
+/*
+ * Prepares a workspace (device memory, 256-byte aligned): clears the status
+ * word and the small bookkeeping header.  Asynchronous on the stream.  Call
+ * once after allocating, and again whenever the status word should be cleared.
+ */
+int rapid_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Copies the status word to *host_status.  Synchronises the stream. */
+int rapid_workspace_status(const void* workspace, void* cuda_stream, int32_t* host_status);
+
+/* ---- the verify step ------------------------------------------------------------------------- */
+
+/*
+ * Verify attention (Algorithm 1, the target's LogitsOf pass; Section 2.1).
+ *
+ * For every sequence b, query head h (KV head h / (Hq/Hkv)) and row i:
+ *   out[b,i,h,:] = sum_j softmax_j(scale * q[b,i,h,:] . k[b,kvh,j,:]) * v[b,kvh,j,:]
+ * over the keys 0 <= j <= ctx_lens[b] - R + i.  fp32 accumulation, bf16
+ * probabilities in the second product, bf16 output.
+ *
+ * The KV length is split over the CTAs of one launch (each K/V tile is read
+ * from HBM once per KV head, shared by all grouped rows) and the partial
+ * results are merged by their log-sum-exp in a second launch.
+ *
+ *   q, k_cache, v_cache, out : device, see rapid_attn_shape
+ *   ctx_lens : device int32 [B]
+ *   gamma    : number of draft tokens (>= 0); gamma = 0 is a plain one-row decode
+ *   params   : host, may be NULL
+ *   workspace: device, >= rapid_attention_workspace_bytes(), initialised
+ */
+int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cache,
+                           const int32_t* ctx_lens, int gamma, void* out,
+                           const rapid_attn_shape* shape, const rapid_attn_params* params,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Accept / residual (Algorithm 1, validation loop and residual step;
+ * Eq. (new_target); Section 2.4).
+ *
+ * For each sequence b and position k = 0..gamma-1 with z = target_logits[b,k],
+ * d = draft_logits[b,k], x' = draft_tokens[b,k]:
+ *   p = softmax(z/T), q = softmax(d/T), phat = softmax(z/T + eta*(q - p)),
+ *   phat_v := p_v wherever phat_v < tail_alpha * max(phat)   (not renormalised),
+ *   position k is accepted iff uniforms[b,k] <= min(1, phat(x')/q(x')).
+ * out_accept_len[b] = number of leading accepted positions n.
+ * out_next_token[b] = inverse-CDF draw with uniforms[b,gamma] from
+ *   norm(max(p - phat, p - q, 0)) of position n   if n < gamma  (or the
+ *   RAPID_RESIDUAL_PHAT variant), else from softmax(target_logits[b,gamma]/T).
+ * The draw returns the smallest token whose running sum of weights exceeds
+ * uniforms[b,gamma] * total.
+ *
+ *   draft_tokens : device int32 [B, gamma];  uniforms : device fp32 [B, gamma+1] in [0,1)
+ *   eta          : transfer strength of Eq. (new_target); 0 gives standard speculative sampling
+ *   out_accept_len, out_next_token : device int32 [B]
+ *   params : host, may be NULL;  workspace: device, >= rapid_accept_workspace_bytes(), initialised
+ */
+int rapid_accept(const float* target_logits, const float* draft_logits,
+                 const int32_t* draft_tokens, const float* uniforms, float eta,
+                 int32_t* out_accept_len, int32_t* out_next_token,
+                 const rapid_accept_shape* shape, const rapid_accept_params* params,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * One verify step: rapid_verify_attention followed by rapid_accept on the same
+ * stream, with no host synchronisation in between (Algorithm 1, one iteration
+ * of the outer loop after drafting).  The projections and the LM head that turn
+ * attention outputs into logits belong to the caller's model, so the logits are
+ * inputs here.  Arguments are those of the two calls.
+ */
+int rapid_verify_step(const void* q, const void* k_cache, const void* v_cache,
+                      const int32_t* ctx_lens, int gamma, void* out,
+                      const rapid_attn_shape* attn_shape, const rapid_attn_params* attn_params,
+                      void* attn_workspace, size_t attn_workspace_bytes,
+                      const float* target_logits, const float* draft_logits,
+                      const int32_t* draft_tokens, const float* uniforms, float eta,
+                      int32_t* out_accept_len, int32_t* out_next_token,
+                      const rapid_accept_shape* accept_shape,
+                      const rapid_accept_params* accept_params, void* accept_workspace,
+                      size_t accept_workspace_bytes, void* cuda_stream);
+
+/*
+ * The same step (Algorithm 1, one verification) for callers whose tensors live
+ * in HOST memory (pinned memory makes the copies asynchronous).  Every h_*
+ * pointer is host memory; K/V must be dense.  Inputs are copied into
+ * `device_arena` (device memory, at least rapid_verify_step_host_arena_bytes(),
+ * 256-byte aligned; it also holds both workspaces and is initialised by the
+ * call), the step runs, and out / accept_len / next_token are copied back.
+ * The call returns after the stream has been synchronised, so the host outputs
+ * are valid on return.  *h_status (may be NULL) receives the OR of both status
+ * words.
+ */
+int rapid_verify_step_host(const void* h_q, const void* h_k_cache, const void* h_v_cache,
+                           const int32_t* h_ctx_lens, int gamma, void* h_out,
+                           const rapid_attn_shape* attn_shape, const rapid_attn_params* attn_params,
+                           const float* h_target_logits, const float* h_draft_logits,
+                           const int32_t* h_draft_tokens, const float* h_uniforms, float eta,
+                           int32_t* h_accept_len, int32_t* h_next_token,
+                           const rapid_accept_shape* accept_shape,
+                           const rapid_accept_params* accept_params, void* device_arena,
+                           size_t device_arena_bytes, int32_t* h_status, void* cuda_stream);
+
+size_t rapid_verify_step_host_arena_bytes(const rapid_attn_shape* attn_shape, int gamma,
+                                          const rapid_accept_shape* accept_shape);
+
+/* ---- misc ------------------------------------------------------------------------------------ */
+
+/* Description of the last error on this thread ("" if none).  Never NULL. */
+const char* rapid_last_error(void);
+
+/* RAPID_VERSION of the built library. */
+int rapid_version(void);
+
+/* Kernels launched by this library on the calling thread since the last reset (for accounting). */
+int64_t rapid_kernel_launch_count(void);
+void rapid_kernel_launch_count_reset(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAPID_H */
