@@ -1,0 +1,288 @@
+"""ctypes binding of include/rapid.h -- argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "librapid.so")
+
+STATUS_BAD_CTX_LEN = 1
+STATUS_BAD_DRAFT_TOKEN = 2
+STATUS_RESIDUAL_FALLBACK = 4
+STATUS_PIPELINE_TIMEOUT = 8
+RESIDUAL_PAPER = 0
+RESIDUAL_PHAT = 1
+
+EXPORTS = [
+    "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_accept", "rapid_verify_step",
+    "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_last_error",
+    "rapid_version", "rapid_kernel_launch_count", "rapid_kernel_launch_count_reset",
+]
+
+
+class RapidError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"rapid error {code}: {message}")
+        self.code = code
+
+
+class _AttnShape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32),
+                ("D", ctypes.c_int32), ("Lmax", ctypes.c_int64), ("kv_stride_b", ctypes.c_int64),
+                ("kv_stride_h", ctypes.c_int64), ("kv_stride_l", ctypes.c_int64)]
+
+
+class _AttnParams(ctypes.Structure):
+    _fields_ = [("scale", ctypes.c_float), ("num_ctas", ctypes.c_int32),
+                ("lse_out", ctypes.c_void_p), ("out_f32", ctypes.c_void_p)]
+
+
+class _AcceptShape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("gamma", ctypes.c_int32), ("V", ctypes.c_int64),
+                ("target_row_stride", ctypes.c_int64), ("draft_row_stride", ctypes.c_int64)]
+
+
+class _AcceptParams(ctypes.Structure):
+    _fields_ = [("temperature", ctypes.c_float), ("tail_alpha", ctypes.c_float),
+                ("residual_mode", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("ratio_out", ctypes.c_void_p)]
+
+
+@dataclass
+class AttnParams:
+    scale: float = 0.0
+    num_ctas: int = 0
+    lse_out: Optional[torch.Tensor] = None   # [B,R,Hq] float32
+    out_f32: Optional[torch.Tensor] = None   # [B,R,Hq,D] float32
+
+
+@dataclass
+class AcceptParams:
+    temperature: float = 1.0
+    tail_alpha: float = 0.1
+    residual_mode: int = RESIDUAL_PAPER
+    ratio_out: Optional[torch.Tensor] = None  # [B,gamma] float32
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Loads librapid.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2502_20330_b200.build` "
+                "(this package has no CPU or PyTorch fallback)")
+        lib = ctypes.CDLL(_LIB_PATH)
+        vp, i32, i64, sz, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t, ctypes.c_float
+        lib.rapid_attention_workspace_bytes.restype = sz
+        lib.rapid_attention_workspace_bytes.argtypes = [ctypes.POINTER(_AttnShape), i32]
+        lib.rapid_accept_workspace_bytes.restype = sz
+        lib.rapid_accept_workspace_bytes.argtypes = [ctypes.POINTER(_AcceptShape)]
+        lib.rapid_workspace_init.restype = i32
+        lib.rapid_workspace_init.argtypes = [vp, sz, vp]
+        lib.rapid_workspace_status.restype = i32
+        lib.rapid_workspace_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+        attn_args = [vp, vp, vp, vp, i32, vp, ctypes.POINTER(_AttnShape), ctypes.POINTER(_AttnParams)]
+        acc_args = [vp, vp, vp, vp, f32, vp, vp, ctypes.POINTER(_AcceptShape), ctypes.POINTER(_AcceptParams)]
+        lib.rapid_verify_attention.restype = i32
+        lib.rapid_verify_attention.argtypes = attn_args + [vp, sz, vp]
+        lib.rapid_accept.restype = i32
+        lib.rapid_accept.argtypes = acc_args + [vp, sz, vp]
+        lib.rapid_verify_step.restype = i32
+        lib.rapid_verify_step.argtypes = attn_args + [vp, sz] + acc_args + [vp, sz, vp]
+        lib.rapid_verify_step_host.restype = i32
+        lib.rapid_verify_step_host.argtypes = attn_args + acc_args + [vp, sz, ctypes.POINTER(ctypes.c_int32), vp]
+        lib.rapid_verify_step_host_arena_bytes.restype = sz
+        lib.rapid_verify_step_host_arena_bytes.argtypes = [ctypes.POINTER(_AttnShape), i32, ctypes.POINTER(_AcceptShape)]
+        lib.rapid_last_error.restype = ctypes.c_char_p
+        lib.rapid_version.restype = i32
+        lib.rapid_kernel_launch_count.restype = i64
+        lib.rapid_kernel_launch_count_reset.restype = None
+        _lib = lib
+    return _lib
+
+
+def last_error() -> str:
+    return load_library().rapid_last_error().decode()
+
+
+def version() -> int:
+    return int(load_library().rapid_version())
+
+
+def kernel_launch_count() -> int:
+    return int(load_library().rapid_kernel_launch_count())
+
+
+def kernel_launch_count_reset() -> None:
+    load_library().rapid_kernel_launch_count_reset()
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise RapidError(rc, last_error())
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _attn_shape(q: torch.Tensor, k: torch.Tensor) -> _AttnShape:
+    B, R, Hq, D = q.shape
+    Bk, Hkv, Lmax, Dk = k.shape
+    if Bk != B or Dk != D:
+        raise ValueError("q and k_cache disagree on batch or head_dim")
+    if k.stride(3) != 1:
+        raise ValueError("k_cache / v_cache must have a contiguous head_dim")
+    return _AttnShape(B, Hq, Hkv, D, Lmax, k.stride(0), k.stride(1), k.stride(2))
+
+
+def _attn_params(p: Optional[AttnParams]):
+    if p is None:
+        return None
+    return ctypes.byref(_AttnParams(p.scale, p.num_ctas, p.lse_out.data_ptr() if p.lse_out is not None else None,
+                                    p.out_f32.data_ptr() if p.out_f32 is not None else None))
+
+
+def _accept_shape(target_logits: torch.Tensor, draft_logits: torch.Tensor) -> _AcceptShape:
+    B, R, V = target_logits.shape
+    if target_logits.stride(2) != 1 or (draft_logits.numel() and draft_logits.stride(-1) != 1):
+        raise ValueError("logits must be contiguous along the vocabulary")
+    zs = target_logits.stride(1)
+    ds = draft_logits.stride(1) if R > 1 else V
+    if R > 1 and (target_logits.stride(0) != R * zs or draft_logits.stride(0) != (R - 1) * ds):
+        raise ValueError("logit rows must be equally spaced")
+    return _AcceptShape(B, R - 1, V, zs, ds)
+
+
+def _accept_params(p: Optional[AcceptParams]):
+    if p is None:
+        return None
+    return ctypes.byref(_AcceptParams(p.temperature, p.tail_alpha, p.residual_mode, 0,
+                                      p.ratio_out.data_ptr() if p.ratio_out is not None else None))
+
+
+def attention_workspace_bytes(B, Hq, Hkv, D, Lmax, gamma) -> int:
+    s = _AttnShape(B, Hq, Hkv, D, Lmax, 0, 0, 0)
+    return int(load_library().rapid_attention_workspace_bytes(ctypes.byref(s), gamma))
+
+
+def accept_workspace_bytes(B, gamma, V) -> int:
+    s = _AcceptShape(B, gamma, V, 0, 0)
+    return int(load_library().rapid_accept_workspace_bytes(ctypes.byref(s)))
+
+
+def verify_step_host_arena_bytes(B, Hq, Hkv, D, Lmax, gamma, V) -> int:
+    a = _AttnShape(B, Hq, Hkv, D, Lmax, 0, 0, 0)
+    c = _AcceptShape(B, gamma, V, 0, 0)
+    return int(load_library().rapid_verify_step_host_arena_bytes(ctypes.byref(a), gamma, ctypes.byref(c)))
+
+
+def workspace_init(workspace: torch.Tensor, stream=None) -> None:
+    _check(load_library().rapid_workspace_init(_p(workspace), workspace.numel() * workspace.element_size(),
+                                               _stream_ptr(stream)))
+
+
+def new_workspace(nbytes: int, device="cuda", stream=None) -> torch.Tensor:
+    """Allocates (with torch) and initialises a workspace of at least nbytes."""
+    if nbytes <= 0:
+        raise ValueError("workspace size query failed (invalid shape?)")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    workspace_init(ws, stream)
+    return ws
+
+
+def workspace_status(workspace: torch.Tensor, stream=None) -> int:
+    out = ctypes.c_int32(0)
+    _check(load_library().rapid_workspace_status(_p(workspace), _stream_ptr(stream), ctypes.byref(out)))
+    return int(out.value)
+
+
+def _nbytes(t: torch.Tensor) -> int:
+    return t.numel() * t.element_size()
+
+
+def rapid_verify_attention(q, k_cache, v_cache, ctx_lens, gamma, out, workspace, params: Optional[AttnParams] = None,
+                           stream=None) -> None:
+    """out[B,R,Hq,D] <- verify attention of q[B,R,Hq,D] over k_cache/v_cache[B,Hkv,Lmax,D] (bf16, CUDA)."""
+    if q.dtype != torch.bfloat16 or k_cache.dtype != torch.bfloat16 or v_cache.dtype != torch.bfloat16 \
+            or out.dtype != torch.bfloat16 or ctx_lens.dtype != torch.int32:
+        raise TypeError("q/k/v/out must be bfloat16 and ctx_lens int32")
+    if not (q.is_contiguous() and out.is_contiguous()) or q.shape[1] != gamma + 1 or out.shape != q.shape:
+        raise ValueError("q and out must be dense [B, gamma+1, Hq, D]")
+    if k_cache.stride() != v_cache.stride() or k_cache.shape != v_cache.shape:
+        raise ValueError("k_cache and v_cache must share shape and strides")
+    shape = _attn_shape(q, k_cache)
+    _check(load_library().rapid_verify_attention(_p(q), _p(k_cache), _p(v_cache), _p(ctx_lens), gamma, _p(out),
+                                                 ctypes.byref(shape), _attn_params(params), _p(workspace),
+                                                 _nbytes(workspace), _stream_ptr(stream)))
+
+
+def rapid_accept(target_logits, draft_logits, draft_tokens, uniforms, eta, out_accept_len, out_next_token,
+                 workspace, params: Optional[AcceptParams] = None, stream=None) -> None:
+    """Algorithm 1's validation loop + residual draw on device tensors (see include/rapid.h)."""
+    if target_logits.dtype != torch.float32 or draft_logits.dtype != torch.float32 or uniforms.dtype != torch.float32:
+        raise TypeError("logits and uniforms must be float32")
+    if draft_tokens.dtype != torch.int32 or out_accept_len.dtype != torch.int32 or out_next_token.dtype != torch.int32:
+        raise TypeError("tokens and outputs must be int32")
+    shape = _accept_shape(target_logits, draft_logits)
+    _check(load_library().rapid_accept(_p(target_logits), _p(draft_logits), _p(draft_tokens), _p(uniforms),
+                                       float(eta), _p(out_accept_len), _p(out_next_token), ctypes.byref(shape),
+                                       _accept_params(params), _p(workspace), _nbytes(workspace),
+                                       _stream_ptr(stream)))
+
+
+def rapid_verify_step(q, k_cache, v_cache, ctx_lens, gamma, out, attn_workspace, target_logits, draft_logits,
+                      draft_tokens, uniforms, eta, out_accept_len, out_next_token, accept_workspace,
+                      attn_params: Optional[AttnParams] = None, accept_params: Optional[AcceptParams] = None,
+                      stream=None) -> None:
+    """Attention then accept on one stream, no host synchronisation."""
+    ashape = _attn_shape(q, k_cache)
+    cshape = _accept_shape(target_logits, draft_logits)
+    _check(load_library().rapid_verify_step(
+        _p(q), _p(k_cache), _p(v_cache), _p(ctx_lens), gamma, _p(out), ctypes.byref(ashape), _attn_params(attn_params),
+        _p(attn_workspace), _nbytes(attn_workspace),
+        _p(target_logits), _p(draft_logits), _p(draft_tokens), _p(uniforms), float(eta), _p(out_accept_len),
+        _p(out_next_token), ctypes.byref(cshape), _accept_params(accept_params), _p(accept_workspace),
+        _nbytes(accept_workspace), _stream_ptr(stream)))
+
+
+def rapid_verify_step_host(q, k_cache, v_cache, ctx_lens, gamma, out, target_logits, draft_logits, draft_tokens,
+                           uniforms, eta, out_accept_len, out_next_token, device_arena,
+                           attn_params: Optional[AttnParams] = None, accept_params: Optional[AcceptParams] = None,
+                           stream=None) -> int:
+    """The step on HOST tensors (ideally pinned): copies in, runs, copies back, synchronises. Returns the status word."""
+    for t in (q, k_cache, v_cache, ctx_lens, out, target_logits, draft_logits, draft_tokens, uniforms,
+              out_accept_len, out_next_token):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("rapid_verify_step_host takes dense host tensors")
+    B, R, Hq, D = q.shape
+    _, Hkv, Lmax, _ = k_cache.shape
+    ashape = _AttnShape(B, Hq, Hkv, D, Lmax, 0, 0, 0)
+    cshape = _AcceptShape(B, gamma, target_logits.shape[2], 0, 0)
+    status = ctypes.c_int32(0)
+    _check(load_library().rapid_verify_step_host(
+        _p(q), _p(k_cache), _p(v_cache), _p(ctx_lens), gamma, _p(out), ctypes.byref(ashape), _attn_params(attn_params),
+        _p(target_logits), _p(draft_logits), _p(draft_tokens), _p(uniforms), float(eta), _p(out_accept_len),
+        _p(out_next_token), ctypes.byref(cshape), _accept_params(accept_params), _p(device_arena),
+        _nbytes(device_arena), ctypes.byref(status), _stream_ptr(stream)))
+    return int(status.value)

@@ -1,0 +1,492 @@
+// Accept / residual step (Algorithm 1, validation loop and residual draw; Eq. (new_target);
+// tail rule of Section 2.4), vocabulary-parallel.
+//
+// Every logit row is cut into NCH chunks; a grid of (chunk, row) CTAs makes four short passes
+// over rows that stay resident in L2 after the first one:
+//   1. stats    : per-chunk (max, sum exp) of z/T and d/T                      -> p, q
+//   2. shift    : per-chunk (max, sum exp) of y = z/T + eta (q - p)            -> phat
+//   3. residual : per-chunk sums of w = max(p - phat', p - q, 0) (phat' = phat with the tail
+//                 rule applied) and the ratio phat'(x')/q(x') at the draft token
+//   4. select   : per sequence, the number of leading accepted drafts n, then an inverse-CDF
+//                 search: chunk sums first, then a block scan inside the one chunk that holds
+//                 the target mass
+// Every position is processed speculatively (also those after the first rejection); pass 4
+// picks the row that Algorithm 1 would have reached.  All reductions run in a fixed order, so
+// results are bit-identical from run to run.  exp is evaluated in base 2: x2 = x * log2(e)/T.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace rapid {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kMaxChunks = 64;
+
+struct AcceptArgs {
+    const float* z;  // target logits [B, R, V]
+    const float* d;  // draft logits  [B, gamma, V]
+    const int32_t* tokens;
+    const float* uniforms;
+    int32_t* accept_len;
+    int32_t* next_token;
+    float* ratio_out;  // optional [B, gamma]
+    int32_t* status;
+    float4* stats;    // [B*R][NCH]  (max z2, sum z, max d2, sum d)
+    float2* ystats;   // [B*gamma][NCH] (max y2, sum)
+    float2* wsums;    // [B*R][NCH] (sum w, sum p)
+    float* ratio;     // [B*gamma]
+    int B, gamma, R, V, NCH, chunk;  // chunk = elements per chunk (multiple of 4)
+    long long zs, ds;                // row strides
+    float inv_T_log2;                // log2(e) / T
+    float eta_log2;                  // eta * log2(e)
+    float log2_alpha;                // log2(tail_alpha), -inf disables the tail rule
+    int mode;
+};
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Block-wide (max, rescaled sum) reduction of per-thread online-softmax states; fixed order.
+__device__ __forceinline__ void block_reduce_ms(float& m, float& s, float* sh_m, float* sh_s) {
+    const float wm = warp_max(m);
+    s = (m == -INFINITY) ? 0.f : s * exp2f(m - wm);
+    s = warp_sum(s);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) {
+        sh_m[warp] = wm;
+        sh_s[warp] = s;
+    }
+    __syncthreads();
+    float M = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < kThreads / 32; ++i) M = fmaxf(M, sh_m[i]);
+    float S = 0.f;
+#pragma unroll
+    for (int i = 0; i < kThreads / 32; ++i)
+        S += (sh_m[i] == -INFINITY) ? 0.f : sh_s[i] * exp2f(sh_m[i] - M);
+    m = M;
+    s = S;
+}
+
+__device__ __forceinline__ float block_reduce_sum(float v, float* sh) {
+    v = warp_sum(v);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) sh[warp] = v;
+    __syncthreads();
+    float S = 0.f;
+#pragma unroll
+    for (int i = 0; i < kThreads / 32; ++i) S += sh[i];
+    return S;
+}
+
+// Combine the per-chunk (max, sum) partials of a row, in chunk order (every thread does it).
+__device__ __forceinline__ void combine_ms(const float* m, const float* s, int n, int stride,
+                                           float& M, float& S) {
+    M = -INFINITY;
+    for (int c = 0; c < n; ++c) M = fmaxf(M, m[c * stride]);
+    S = 0.f;
+    for (int c = 0; c < n; ++c) {
+        const float mc = m[c * stride];
+        S += (mc == -INFINITY) ? 0.f : s[c * stride] * exp2f(mc - M);
+    }
+}
+
+__device__ __forceinline__ void online_add(float& m, float& s, float x) {
+    if (x > m) {
+        s = s * exp2f(m - x) + 1.f;  // exp2f(-inf) = 0 covers the first element
+        m = x;
+    } else if (x != -INFINITY) {  // a logit of -inf carries no mass (and -inf - -inf is NaN)
+        s += exp2f(x - m);
+    }
+}
+
+// ---- pass 1 ----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) accept_stats_kernel(const AcceptArgs a) {
+    __shared__ float sh_m[kThreads / 32], sh_s[kThreads / 32];
+    const int c = blockIdx.x, row = blockIdx.y;
+    const int b = row / a.R, k = row % a.R;
+    const int v0 = c * a.chunk, v1 = min(v0 + a.chunk, a.V);
+    const float* z = a.z + (size_t)row * a.zs;
+    float mz = -INFINITY, sz = 0.f, md = -INFINITY, sd = 0.f;
+    for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
+        const float4 x = *reinterpret_cast<const float4*>(z + v);
+        online_add(mz, sz, x.x * a.inv_T_log2);
+        online_add(mz, sz, x.y * a.inv_T_log2);
+        online_add(mz, sz, x.z * a.inv_T_log2);
+        online_add(mz, sz, x.w * a.inv_T_log2);
+    }
+    if (k < a.gamma) {
+        const float* d = a.d + (size_t)(b * a.gamma + k) * a.ds;
+        for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
+            const float4 x = *reinterpret_cast<const float4*>(d + v);
+            online_add(md, sd, x.x * a.inv_T_log2);
+            online_add(md, sd, x.y * a.inv_T_log2);
+            online_add(md, sd, x.z * a.inv_T_log2);
+            online_add(md, sd, x.w * a.inv_T_log2);
+        }
+    }
+    block_reduce_ms(mz, sz, sh_m, sh_s);
+    block_reduce_ms(md, sd, sh_m, sh_s);
+    if (threadIdx.x == 0) a.stats[(size_t)row * a.NCH + c] = make_float4(mz, sz, md, sd);
+}
+
+struct RowStats {
+    float Mz, inv_Sz, Md, inv_Sd;
+};
+
+__device__ __forceinline__ RowStats load_row_stats(const AcceptArgs& a, int row, bool has_draft) {
+    const float* st = reinterpret_cast<const float*>(a.stats + (size_t)row * a.NCH);
+    RowStats r;
+    float S;
+    combine_ms(st + 0, st + 1, a.NCH, 4, r.Mz, S);
+    r.inv_Sz = 1.f / S;
+    r.Md = 0.f;
+    r.inv_Sd = 0.f;
+    if (has_draft) {
+        combine_ms(st + 2, st + 3, a.NCH, 4, r.Md, S);
+        r.inv_Sd = 1.f / S;
+    }
+    return r;
+}
+
+// y in base-2 units: (z/T + eta (q - p)) * log2(e)
+__device__ __forceinline__ float shifted_logit2(const AcceptArgs& a, const RowStats& r, float z,
+                                                float d, float& p, float& q) {
+    const float z2 = z * a.inv_T_log2;
+    p = exp2f(z2 - r.Mz) * r.inv_Sz;
+    q = exp2f(d * a.inv_T_log2 - r.Md) * r.inv_Sd;
+    return fmaf(a.eta_log2, q - p, z2);
+}
+
+// ---- pass 2 ----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) accept_shift_stats_kernel(const AcceptArgs a) {
+    __shared__ float sh_m[kThreads / 32], sh_s[kThreads / 32];
+    const int c = blockIdx.x, drow = blockIdx.y;  // drow over B*gamma
+    const int b = drow / a.gamma, k = drow % a.gamma;
+    const int row = b * a.R + k;
+    const RowStats r = load_row_stats(a, row, true);
+    const int v0 = c * a.chunk, v1 = min(v0 + a.chunk, a.V);
+    const float* z = a.z + (size_t)row * a.zs;
+    const float* d = a.d + (size_t)drow * a.ds;
+    float my = -INFINITY, sy = 0.f;
+    for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
+        const float4 x = *reinterpret_cast<const float4*>(z + v);
+        const float4 y = *reinterpret_cast<const float4*>(d + v);
+        float p, q;
+        online_add(my, sy, shifted_logit2(a, r, x.x, y.x, p, q));
+        online_add(my, sy, shifted_logit2(a, r, x.y, y.y, p, q));
+        online_add(my, sy, shifted_logit2(a, r, x.z, y.z, p, q));
+        online_add(my, sy, shifted_logit2(a, r, x.w, y.w, p, q));
+    }
+    block_reduce_ms(my, sy, sh_m, sh_s);
+    if (threadIdx.x == 0) a.ystats[(size_t)drow * a.NCH + c] = make_float2(my, sy);
+}
+
+// Residual weight of one vocabulary entry of a draft row; also returns phat' (tail rule applied).
+__device__ __forceinline__ float residual_weight(const AcceptArgs& a, const RowStats& r, float My,
+                                                 float inv_Sy, float z, float d, float& p,
+                                                 float& q, float& ph) {
+    const float y2 = shifted_logit2(a, r, z, d, p, q);
+    const float rel = y2 - My;
+    ph = (rel < a.log2_alpha) ? p : exp2f(rel) * inv_Sy;
+    float w;
+    if (a.mode == RAPID_RESIDUAL_PHAT)
+        w = ph - q;
+    else
+        w = fmaxf(p - ph, p - q);
+    return fmaxf(w, 0.f);
+}
+
+// ---- pass 3 ----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) accept_residual_kernel(const AcceptArgs a) {
+    __shared__ float sh[kThreads / 32];
+    const int c = blockIdx.x, row = blockIdx.y;
+    const int b = row / a.R, k = row % a.R;
+    const bool draft = k < a.gamma;
+    const RowStats r = load_row_stats(a, row, draft);
+    const int v0 = c * a.chunk, v1 = min(v0 + a.chunk, a.V);
+    const float* z = a.z + (size_t)row * a.zs;
+    float sw = 0.f, sp = 0.f;
+    if (draft) {
+        const int drow = b * a.gamma + k;
+        const float* d = a.d + (size_t)drow * a.ds;
+        const float* ys = reinterpret_cast<const float*>(a.ystats + (size_t)drow * a.NCH);
+        float My, Sy;
+        combine_ms(ys, ys + 1, a.NCH, 2, My, Sy);
+        const float inv_Sy = 1.f / Sy;
+        int tok = a.tokens[drow];
+        if (tok < 0 || tok >= a.V) {
+            if (c == 0 && threadIdx.x == 0) atomicOr(a.status, RAPID_STATUS_BAD_DRAFT_TOKEN);
+            tok = tok < 0 ? 0 : a.V - 1;
+        }
+        for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
+            const float4 x = *reinterpret_cast<const float4*>(z + v);
+            const float4 y = *reinterpret_cast<const float4*>(d + v);
+            const float xs[4] = {x.x, x.y, x.z, x.w};
+            const float ys4[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float p, q, ph;
+                sw += residual_weight(a, r, My, inv_Sy, xs[e], ys4[e], p, q, ph);
+                sp += p;
+                if (v + e == tok) {
+                    const float ratio = q > 0.f ? ph / q : INFINITY;
+                    a.ratio[drow] = ratio;
+                    if (a.ratio_out) a.ratio_out[drow] = ratio;
+                }
+            }
+        }
+    } else {
+        for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
+            const float4 x = *reinterpret_cast<const float4*>(z + v);
+            sp += exp2f(x.x * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+            sp += exp2f(x.y * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+            sp += exp2f(x.z * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+            sp += exp2f(x.w * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+        }
+        sw = sp;
+    }
+    sw = block_reduce_sum(sw, sh);
+    sp = block_reduce_sum(sp, sh);
+    if (threadIdx.x == 0) a.wsums[(size_t)row * a.NCH + c] = make_float2(sw, sp);
+}
+
+// ---- pass 4 ----------------------------------------------------------------------------------
+// One CTA per sequence.  Thread t owns a run of consecutive entries of the chosen chunk so that
+// the prefix order inside the chunk is the vocabulary order.
+__global__ void __launch_bounds__(kThreads) accept_select_kernel(const AcceptArgs a) {
+    __shared__ float sh_scan[kThreads];
+    __shared__ int sh_tok;
+    __shared__ int sh_last;
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x;
+
+    // number of leading accepted drafts
+    int n = 0;
+    for (; n < a.gamma; ++n) {
+        const float ratio = a.ratio[b * a.gamma + n];
+        const float u = a.uniforms[b * a.R + n];
+        if (!(u <= fminf(1.f, ratio))) break;
+    }
+    const int row = b * a.R + n;
+    const bool draft = n < a.gamma;
+    const float u = a.uniforms[b * a.R + a.gamma];
+    const float2* ws = a.wsums + (size_t)row * a.NCH;
+
+    float W = 0.f;
+    for (int c = 0; c < a.NCH; ++c) W += ws[c].x;
+    bool use_p = !draft;
+    if (!(W > 0.f) || !isfinite(W)) {  // empty residual: defined fallback, draw from p
+        use_p = true;
+        W = 0.f;
+        for (int c = 0; c < a.NCH; ++c) W += ws[c].y;
+        if (tid == 0) atomicOr(a.status, RAPID_STATUS_RESIDUAL_FALLBACK);
+    }
+    const float target = u * W;
+
+    // chunk that holds the target mass; if rounding leaves none, the last chunk with mass
+    int chunk = -1, last_pos = -1;
+    float before = 0.f, run = 0.f, before_last = 0.f;
+    for (int c = 0; c < a.NCH; ++c) {
+        const float wc = use_p ? ws[c].y : ws[c].x;
+        if (wc > 0.f) {
+            if (chunk < 0 && run + wc > target) {
+                chunk = c;
+                before = run;
+            }
+            last_pos = c;
+            before_last = run;
+            run += wc;
+        }
+    }
+    bool want_last = false;
+    if (chunk < 0) {
+        chunk = last_pos;
+        before = before_last;
+        want_last = true;
+    }
+    if (chunk < 0) {  // nothing has mass at all (non-finite logits): defined output
+        if (tid == 0) {
+            a.accept_len[b] = n;
+            a.next_token[b] = 0;
+        }
+        return;
+    }
+
+    const RowStats r = load_row_stats(a, row, draft);
+    float My = 0.f, inv_Sy = 0.f;
+    const float* z = a.z + (size_t)row * a.zs;
+    const float* d = nullptr;
+    if (draft) {
+        const int drow = b * a.gamma + n;
+        d = a.d + (size_t)drow * a.ds;
+        const float* ys = reinterpret_cast<const float*>(a.ystats + (size_t)drow * a.NCH);
+        float Sy;
+        combine_ms(ys, ys + 1, a.NCH, 2, My, Sy);
+        inv_Sy = 1.f / Sy;
+    }
+    const int v0 = chunk * a.chunk, v1 = min(v0 + a.chunk, a.V);
+    const int per = (((v1 - v0) + kThreads - 1) / kThreads + 3) & ~3;  // multiple of 4
+    const int t0 = v0 + tid * per, t1 = min(t0 + per, v1);
+
+    auto weight = [&](int v) -> float {
+        float p, q, ph;
+        if (draft) {
+            const float w = residual_weight(a, r, My, inv_Sy, z[v], d[v], p, q, ph);
+            return use_p ? p : w;
+        }
+        return exp2f(z[v] * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+    };
+
+    float mine = 0.f;
+    for (int v = t0; v < t1; ++v) mine += weight(v);
+    sh_scan[tid] = mine;
+    if (tid == 0) {
+        sh_tok = 0x7fffffff;
+        sh_last = -1;
+    }
+    __syncthreads();
+    float prefix = before;  // mass before this thread's run, summed in thread order
+    for (int t = 0; t < tid; ++t) prefix += sh_scan[t];
+    int found = 0x7fffffff, last = -1;
+    float cum = prefix;
+    for (int v = t0; v < t1; ++v) {
+        const float w = weight(v);
+        if (w > 0.f) {
+            cum += w;
+            last = v;
+            if (!want_last && cum > target && found == 0x7fffffff) found = v;
+        }
+    }
+    if (found != 0x7fffffff) atomicMin(&sh_tok, found);
+    if (last >= 0) atomicMax(&sh_last, last);
+    __syncthreads();
+    if (tid == 0) {
+        a.accept_len[b] = n;
+        const int tok = sh_tok != 0x7fffffff ? sh_tok : (sh_last >= 0 ? sh_last : v0);
+        a.next_token[b] = tok;
+    }
+}
+
+bool accept_shape_ok(const rapid_accept_shape* s) {
+    return s && s->B > 0 && s->gamma >= 0 && s->V > 0 && s->V <= 0x7ffffff0LL &&
+           (int64_t)s->B * (s->gamma + 1) <= 65535;
+}
+
+int pick_chunks(int64_t V) {
+    // about 8K entries per chunk keeps every CTA at a few iterations of 256 x float4
+    int n = (int)((V + 8191) / 8192);
+    return n < 1 ? 1 : (n > kMaxChunks ? kMaxChunks : n);
+}
+
+}  // namespace
+
+size_t accept_workspace_bytes(const rapid_accept_shape* s) {
+    if (!accept_shape_ok(s)) return 0;
+    const size_t rows = (size_t)s->B * (s->gamma + 1);
+    const size_t drows = (size_t)s->B * s->gamma;
+    size_t bytes = kWorkspaceHeaderBytes;
+    bytes += align_up(rows * kMaxChunks * sizeof(float4), 256);
+    bytes += align_up(drows * kMaxChunks * sizeof(float2), 256);
+    bytes += align_up(rows * kMaxChunks * sizeof(float2), 256);
+    bytes += align_up(drows * sizeof(float) + 4, 256);
+    return bytes;
+}
+
+int launch_accept(const float* target_logits, const float* draft_logits,
+                  const int32_t* draft_tokens, const float* uniforms, float eta,
+                  int32_t* out_accept_len, int32_t* out_next_token,
+                  const rapid_accept_shape* shape, const rapid_accept_params* params,
+                  void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (!accept_shape_ok(shape)) {
+        set_error("rapid_accept: invalid shape");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const rapid_accept_shape& s = *shape;
+    if (!target_logits || !uniforms || !out_accept_len || !out_next_token ||
+        (s.gamma > 0 && (!draft_logits || !draft_tokens))) {
+        set_error("rapid_accept: NULL argument");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const float T = params ? params->temperature : 1.0f;
+    const float alpha = params ? params->tail_alpha : 0.1f;
+    const int mode = params ? params->residual_mode : RAPID_RESIDUAL_PAPER;
+    if (!(T > 0.f) || !isfinite(T) || !(alpha >= 0.f) || !(alpha <= 1.f) || !isfinite(eta) ||
+        (mode != RAPID_RESIDUAL_PAPER && mode != RAPID_RESIDUAL_PHAT)) {
+        set_error("rapid_accept: need T > 0, 0 <= tail_alpha <= 1, finite eta, a known residual_mode");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const int64_t zs = s.target_row_stride ? s.target_row_stride : s.V;
+    const int64_t ds = s.draft_row_stride ? s.draft_row_stride : s.V;
+    if (s.V % 4 || zs % 4 || ds % 4 || zs < s.V || ds < s.V ||
+        ((uintptr_t)target_logits & 15) || ((uintptr_t)draft_logits & 15)) {
+        set_error("rapid_accept: V and row strides must be multiples of 4, logits 16-byte aligned");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const size_t need = accept_workspace_bytes(shape);
+    if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) {
+        set_error("rapid_accept: workspace of %zu bytes needed (256-byte aligned), got %zu", need,
+                  workspace_bytes);
+        return RAPID_ERR_WORKSPACE;
+    }
+    const int R = s.gamma + 1;
+    const size_t rows = (size_t)s.B * R, drows = (size_t)s.B * s.gamma;
+    uint8_t* p = static_cast<uint8_t*>(workspace);
+    AcceptArgs a;
+    a.status = reinterpret_cast<int32_t*>(p);
+    p += kWorkspaceHeaderBytes;
+    a.stats = reinterpret_cast<float4*>(p);
+    p += align_up(rows * kMaxChunks * sizeof(float4), 256);
+    a.ystats = reinterpret_cast<float2*>(p);
+    p += align_up(drows * kMaxChunks * sizeof(float2), 256);
+    a.wsums = reinterpret_cast<float2*>(p);
+    p += align_up(rows * kMaxChunks * sizeof(float2), 256);
+    a.ratio = reinterpret_cast<float*>(p);
+    a.z = target_logits;
+    a.d = draft_logits;
+    a.tokens = draft_tokens;
+    a.uniforms = uniforms;
+    a.accept_len = out_accept_len;
+    a.next_token = out_next_token;
+    a.ratio_out = params ? params->ratio_out : nullptr;
+    a.B = s.B;
+    a.gamma = s.gamma;
+    a.R = R;
+    a.V = (int)s.V;
+    a.NCH = pick_chunks(s.V);
+    a.chunk = (int)(((s.V / 4 + a.NCH - 1) / a.NCH) * 4);
+    a.zs = zs;
+    a.ds = ds;
+    a.inv_T_log2 = 1.4426950408889634f / T;
+    a.eta_log2 = eta * 1.4426950408889634f;
+    a.log2_alpha = alpha > 0.f ? log2f(alpha) : -INFINITY;
+    a.mode = mode;
+
+    int launches = 0;
+    accept_stats_kernel<<<dim3(a.NCH, (unsigned)rows), kThreads, 0, stream>>>(a);
+    ++launches;
+    if (s.gamma > 0) {
+        accept_shift_stats_kernel<<<dim3(a.NCH, (unsigned)drows), kThreads, 0, stream>>>(a);
+        ++launches;
+    }
+    accept_residual_kernel<<<dim3(a.NCH, (unsigned)rows), kThreads, 0, stream>>>(a);
+    accept_select_kernel<<<s.B, kThreads, 0, stream>>>(a);
+    launches += 2;
+    RAPID_CUDA_CHECK(cudaGetLastError());
+    count_launch(launches);
+    return RAPID_OK;
+}
+
+}  // namespace rapid

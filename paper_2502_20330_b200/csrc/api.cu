@@ -1,0 +1,244 @@
+// C ABI of the RAPID verify-step library: argument plumbing around the launchers.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace rapid {
+
+namespace {
+thread_local char g_error[512] = "";
+thread_local int64_t g_launches = 0;
+}  // namespace
+
+void set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof g_error, fmt, ap);
+    va_end(ap);
+}
+void clear_error() { g_error[0] = 0; }
+void count_launch(int n) { g_launches += n; }
+
+size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma);
+size_t accept_workspace_bytes(const rapid_accept_shape* s);
+
+}  // namespace rapid
+
+using namespace rapid;
+
+extern "C" {
+
+size_t rapid_attention_workspace_bytes(const rapid_attn_shape* shape, int gamma) {
+    return attention_workspace_bytes(shape, gamma);
+}
+
+size_t rapid_accept_workspace_bytes(const rapid_accept_shape* shape) {
+    return accept_workspace_bytes(shape);
+}
+
+int rapid_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    clear_error();
+    if (!workspace || workspace_bytes < kWorkspaceHeaderBytes || ((uintptr_t)workspace & 255)) {
+        set_error("rapid_workspace_init: need a 256-byte aligned workspace of at least %zu bytes",
+                  kWorkspaceHeaderBytes);
+        return RAPID_ERR_WORKSPACE;
+    }
+    RAPID_CUDA_CHECK(cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes,
+                                     static_cast<cudaStream_t>(cuda_stream)));
+    return RAPID_OK;
+}
+
+int rapid_workspace_status(const void* workspace, void* cuda_stream, int32_t* host_status) {
+    clear_error();
+    if (!workspace || !host_status) {
+        set_error("rapid_workspace_status: NULL argument");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(host_status, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    RAPID_CUDA_CHECK(cudaStreamSynchronize(st));
+    return RAPID_OK;
+}
+
+int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cache,
+                           const int32_t* ctx_lens, int gamma, void* out,
+                           const rapid_attn_shape* shape, const rapid_attn_params* params,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    clear_error();
+    return launch_verify_attention(q, k_cache, v_cache, ctx_lens, gamma, out, shape, params,
+                                   workspace, workspace_bytes,
+                                   static_cast<cudaStream_t>(cuda_stream));
+}
+
+int rapid_accept(const float* target_logits, const float* draft_logits,
+                 const int32_t* draft_tokens, const float* uniforms, float eta,
+                 int32_t* out_accept_len, int32_t* out_next_token,
+                 const rapid_accept_shape* shape, const rapid_accept_params* params,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    clear_error();
+    return launch_accept(target_logits, draft_logits, draft_tokens, uniforms, eta, out_accept_len,
+                         out_next_token, shape, params, workspace, workspace_bytes,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+int rapid_verify_step(const void* q, const void* k_cache, const void* v_cache,
+                      const int32_t* ctx_lens, int gamma, void* out,
+                      const rapid_attn_shape* attn_shape, const rapid_attn_params* attn_params,
+                      void* attn_workspace, size_t attn_workspace_bytes,
+                      const float* target_logits, const float* draft_logits,
+                      const int32_t* draft_tokens, const float* uniforms, float eta,
+                      int32_t* out_accept_len, int32_t* out_next_token,
+                      const rapid_accept_shape* accept_shape,
+                      const rapid_accept_params* accept_params, void* accept_workspace,
+                      size_t accept_workspace_bytes, void* cuda_stream) {
+    clear_error();
+    if (accept_shape && attn_shape &&
+        (accept_shape->gamma != gamma || accept_shape->B != attn_shape->B)) {
+        set_error("rapid_verify_step: attention and accept shapes disagree on B or gamma");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int rc = launch_verify_attention(q, k_cache, v_cache, ctx_lens, gamma, out, attn_shape,
+                                     attn_params, attn_workspace, attn_workspace_bytes, st);
+    if (rc != RAPID_OK) return rc;
+    return launch_accept(target_logits, draft_logits, draft_tokens, uniforms, eta, out_accept_len,
+                         out_next_token, accept_shape, accept_params, accept_workspace,
+                         accept_workspace_bytes, st);
+}
+
+namespace {
+struct HostArena {
+    size_t q, k, v, ctx, out, z, d, tok, u, alen, ntok, attn_ws, acc_ws, total;
+    size_t q_bytes, kv_bytes, ctx_bytes, z_bytes, d_bytes, tok_bytes, u_bytes, b_bytes;
+    size_t attn_ws_bytes, acc_ws_bytes;
+};
+
+bool plan_host_arena(const rapid_attn_shape* as, int gamma, const rapid_accept_shape* cs,
+                     HostArena& h) {
+    if (!as || !cs || gamma < 0) return false;
+    h.attn_ws_bytes = attention_workspace_bytes(as, gamma);
+    h.acc_ws_bytes = accept_workspace_bytes(cs);
+    if (!h.attn_ws_bytes || !h.acc_ws_bytes) return false;
+    const size_t R = gamma + 1;
+    h.q_bytes = (size_t)as->B * R * as->Hq * as->D * 2;
+    h.kv_bytes = (size_t)as->B * as->Hkv * as->Lmax * as->D * 2;
+    h.ctx_bytes = (size_t)as->B * 4;
+    h.z_bytes = (size_t)cs->B * R * cs->V * 4;
+    h.d_bytes = (size_t)cs->B * gamma * cs->V * 4;
+    h.tok_bytes = (size_t)cs->B * gamma * 4;
+    h.u_bytes = (size_t)cs->B * R * 4;
+    h.b_bytes = (size_t)cs->B * 4;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = off;
+        off += align_up(bytes ? bytes : 1, 256);
+        return at;
+    };
+    h.q = take(h.q_bytes);
+    h.k = take(h.kv_bytes);
+    h.v = take(h.kv_bytes);
+    h.ctx = take(h.ctx_bytes);
+    h.out = take(h.q_bytes);
+    h.z = take(h.z_bytes);
+    h.d = take(h.d_bytes);
+    h.tok = take(h.tok_bytes);
+    h.u = take(h.u_bytes);
+    h.alen = take(h.b_bytes);
+    h.ntok = take(h.b_bytes);
+    h.attn_ws = take(h.attn_ws_bytes);
+    h.acc_ws = take(h.acc_ws_bytes);
+    h.total = off;
+    return true;
+}
+}  // namespace
+
+size_t rapid_verify_step_host_arena_bytes(const rapid_attn_shape* attn_shape, int gamma,
+                                          const rapid_accept_shape* accept_shape) {
+    HostArena h;
+    return plan_host_arena(attn_shape, gamma, accept_shape, h) ? h.total : 0;
+}
+
+int rapid_verify_step_host(const void* h_q, const void* h_k_cache, const void* h_v_cache,
+                           const int32_t* h_ctx_lens, int gamma, void* h_out,
+                           const rapid_attn_shape* attn_shape, const rapid_attn_params* attn_params,
+                           const float* h_target_logits, const float* h_draft_logits,
+                           const int32_t* h_draft_tokens, const float* h_uniforms, float eta,
+                           int32_t* h_accept_len, int32_t* h_next_token,
+                           const rapid_accept_shape* accept_shape,
+                           const rapid_accept_params* accept_params, void* device_arena,
+                           size_t device_arena_bytes, int32_t* h_status, void* cuda_stream) {
+    clear_error();
+    HostArena h;
+    if (!plan_host_arena(attn_shape, gamma, accept_shape, h)) {
+        set_error("rapid_verify_step_host: invalid shapes");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (!h_q || !h_k_cache || !h_v_cache || !h_ctx_lens || !h_out || !h_target_logits ||
+        !h_uniforms || !h_accept_len || !h_next_token ||
+        (gamma > 0 && (!h_draft_logits || !h_draft_tokens))) {
+        set_error("rapid_verify_step_host: NULL argument");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (attn_shape->kv_stride_b || attn_shape->kv_stride_h || attn_shape->kv_stride_l ||
+        accept_shape->target_row_stride || accept_shape->draft_row_stride) {
+        set_error("rapid_verify_step_host: host tensors must be dense (all strides 0)");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    if (accept_shape->gamma != gamma || accept_shape->B != attn_shape->B) {
+        set_error("rapid_verify_step_host: attention and accept shapes disagree on B or gamma");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (!device_arena || device_arena_bytes < h.total || ((uintptr_t)device_arena & 255)) {
+        set_error("rapid_verify_step_host: device arena of %zu bytes needed (256-byte aligned), got %zu",
+                  h.total, device_arena_bytes);
+        return RAPID_ERR_WORKSPACE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* base = static_cast<uint8_t*>(device_arena);
+    const cudaMemcpyKind H2D = cudaMemcpyHostToDevice, D2H = cudaMemcpyDeviceToHost;
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(base + h.q, h_q, h.q_bytes, H2D, st));
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(base + h.k, h_k_cache, h.kv_bytes, H2D, st));
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(base + h.v, h_v_cache, h.kv_bytes, H2D, st));
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(base + h.ctx, h_ctx_lens, h.ctx_bytes, H2D, st));
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(base + h.z, h_target_logits, h.z_bytes, H2D, st));
+    if (gamma > 0) {
+        RAPID_CUDA_CHECK(cudaMemcpyAsync(base + h.d, h_draft_logits, h.d_bytes, H2D, st));
+        RAPID_CUDA_CHECK(cudaMemcpyAsync(base + h.tok, h_draft_tokens, h.tok_bytes, H2D, st));
+    }
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(base + h.u, h_uniforms, h.u_bytes, H2D, st));
+    RAPID_CUDA_CHECK(cudaMemsetAsync(base + h.attn_ws, 0, kWorkspaceHeaderBytes, st));
+    RAPID_CUDA_CHECK(cudaMemsetAsync(base + h.acc_ws, 0, kWorkspaceHeaderBytes, st));
+    int rc = launch_verify_attention(base + h.q, base + h.k, base + h.v,
+                                     reinterpret_cast<const int32_t*>(base + h.ctx), gamma,
+                                     base + h.out, attn_shape, attn_params, base + h.attn_ws,
+                                     h.attn_ws_bytes, st);
+    if (rc != RAPID_OK) return rc;
+    rc = launch_accept(reinterpret_cast<const float*>(base + h.z),
+                       reinterpret_cast<const float*>(base + h.d),
+                       reinterpret_cast<const int32_t*>(base + h.tok),
+                       reinterpret_cast<const float*>(base + h.u), eta,
+                       reinterpret_cast<int32_t*>(base + h.alen),
+                       reinterpret_cast<int32_t*>(base + h.ntok), accept_shape, accept_params,
+                       base + h.acc_ws, h.acc_ws_bytes, st);
+    if (rc != RAPID_OK) return rc;
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(h_out, base + h.out, h.q_bytes, D2H, st));
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(h_accept_len, base + h.alen, h.b_bytes, D2H, st));
+    RAPID_CUDA_CHECK(cudaMemcpyAsync(h_next_token, base + h.ntok, h.b_bytes, D2H, st));
+    int32_t st_words[2] = {0, 0};
+    if (h_status) {
+        RAPID_CUDA_CHECK(cudaMemcpyAsync(&st_words[0], base + h.attn_ws, 4, D2H, st));
+        RAPID_CUDA_CHECK(cudaMemcpyAsync(&st_words[1], base + h.acc_ws, 4, D2H, st));
+    }
+    RAPID_CUDA_CHECK(cudaStreamSynchronize(st));
+    if (h_status) *h_status = st_words[0] | st_words[1];
+    return RAPID_OK;
+}
+
+const char* rapid_last_error(void) { return g_error; }
+int rapid_version(void) { return RAPID_VERSION; }
+int64_t rapid_kernel_launch_count(void) { return g_launches; }
+void rapid_kernel_launch_count_reset(void) { g_launches = 0; }
+
+}  // extern "C"

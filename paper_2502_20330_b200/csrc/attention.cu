@@ -1,0 +1,625 @@
+// Verify attention (Algorithm 1, the target's single validation pass over the full context):
+// split-KV kernel + log-sum-exp merge.
+//
+// Work decomposition.  A "unit" is one (sequence, KV head) pair; its K/V cache is cut into
+// tiles of kTile keys.  All units' tiles form one flat list, cut into equal contiguous ranges,
+// one per CTA, so every CTA streams the same number of bytes whatever the context lengths are.
+// A CTA whose range crosses a unit boundary emits one partial result per unit it touches.
+// The G*R grouped query rows of a KV head (G = Hq/Hkv heads times R = gamma+1 draft rows) ride
+// together, so each K/V tile leaves HBM once.
+//
+// Inside a CTA one producer warp issues TMA tile loads (128-byte swizzle) into a ring of
+// shared-memory stages guarded by full/empty mbarriers; consumer warps are arranged as
+// MT row blocks (16 grouped rows each) x KS tile lanes: lane ks takes every KS-th tile, runs
+// QK^T and PV on the tensor cores with an fp32 online softmax, and keeps its own running
+// (max, sum, O).  Partials go to the workspace; the merge kernel combines them in a fixed
+// order, so results are bit-identical from run to run.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace rapid {
+
+namespace {
+
+constexpr int kTile = 64;  // keys per pipeline stage
+
+__host__ __device__ constexpr int tile_lanes(int MT) {
+    return MT == 1 ? 8 : MT == 2 ? 4 : MT == 3 ? 3 : MT <= 5 ? 2 : 1;
+}
+__host__ __device__ constexpr int num_stages(int D) { return D == 128 ? 6 : 8; }
+__host__ __device__ constexpr int stage_bytes(int D) { return 2 * kTile * D * 2; }
+
+struct AttnArgs {
+    const __nv_bfloat16* q;
+    const int32_t* ctx_lens;
+    float* partial;   // [slots][GR*(D+2)] fp32
+    int32_t* status;  // workspace status word
+    int B, Hq, Hkv, G, R, GR;
+    int Lmax;
+    int num_ctas;
+    float scale_log2;  // softmax scale * log2(e)
+};
+
+struct Walk {
+    int b, kvh, tile, ntiles, L;
+    long long remaining;
+    long long total;
+};
+
+__device__ __forceinline__ int clamp_len(int L, int R, int Lmax) {
+    return L < R ? R : (L > Lmax ? Lmax : L);
+}
+__device__ __forceinline__ int tiles_of(int L) { return (L + kTile - 1) / kTile; }
+
+// Flat tile range of CTA c of n: [c*T/n, (c+1)*T/n).
+__device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
+    long long T = 0;
+    for (int b = 0; b < a.B; ++b)
+        T += (long long)a.Hkv * tiles_of(clamp_len(a.ctx_lens[b], a.R, a.Lmax));
+    long long t0 = (long long)cta * T / a.num_ctas;
+    long long t1 = (long long)(cta + 1) * T / a.num_ctas;
+    w.total = T;
+    w.remaining = t1 - t0;
+    w.b = 0;
+    w.kvh = 0;
+    w.tile = 0;
+    w.L = 0;
+    w.ntiles = 0;
+    if (w.remaining <= 0) return;
+    long long t = t0;
+    for (int b = 0; b < a.B; ++b) {
+        const int L = clamp_len(a.ctx_lens[b], a.R, a.Lmax);
+        const int nt = tiles_of(L);
+        const long long span = (long long)a.Hkv * nt;
+        if (t < span) {
+            w.b = b;
+            w.kvh = (int)(t / nt);
+            w.tile = (int)(t % nt);
+            w.L = L;
+            w.ntiles = nt;
+            return;
+        }
+        t -= span;
+    }
+}
+
+__device__ __forceinline__ void walk_advance(const AttnArgs& a, Walk& w, int seg) {
+    w.remaining -= seg;
+    w.tile += seg;
+    if (w.tile >= w.ntiles) {
+        w.tile = 0;
+        if (++w.kvh == a.Hkv) {
+            w.kvh = 0;
+            ++w.b;
+            if (w.b < a.B) {
+                w.L = clamp_len(a.ctx_lens[w.b], a.R, a.Lmax);
+                w.ntiles = tiles_of(w.L);
+            }
+        }
+    }
+}
+
+template <int D, int MT>
+__global__ void __launch_bounds__((MT * tile_lanes(MT) + 1) * 32, 1)
+verify_attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmK,
+                           const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
+    constexpr int KS = tile_lanes(MT);
+    constexpr int NSTAGE = num_stages(D);
+    constexpr int STAGE = stage_bytes(D);
+    constexpr int HALF = kTile * 128;  // bytes of one 64-column box
+    constexpr int NHALF = D / 64;
+    constexpr int KSTEPS = D / 16;
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[NSTAGE];
+    __shared__ uint64_t empty_bar[NSTAGE];
+    __shared__ Walk s_walk;
+    __shared__ int s_abort;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int cta = blockIdx.x;
+
+    if (tid == 0) {
+        for (int s = 0; s < NSTAGE; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], MT);
+        }
+        fence_mbar_init();
+        s_abort = 0;
+        Walk w;
+        plan_cta(a, cta, w);
+        s_walk = w;
+        if (cta == 0) {
+            bool bad = false;
+            for (int b = 0; b < a.B; ++b) {
+                const int L = a.ctx_lens[b];
+                bad |= (L < a.R) || (L > a.Lmax);
+            }
+            if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
+        }
+    }
+    __syncthreads();
+    Walk w = s_walk;
+    volatile int* abort_flag = &s_abort;
+
+    if (warp == MT * KS) {
+        // ---------------- producer warp: one lane issues the TMA loads ----------------
+        if (lane == 0) {
+            prefetch_tensormap(&tmK);
+            prefetch_tensormap(&tmV);
+            int n = 0;
+            bool ok = true;
+            while (w.remaining > 0 && ok) {
+                const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+                for (int t = 0; t < seg && ok; ++t, ++n) {
+                    const int s = n % NSTAGE;
+                    if (n >= NSTAGE)
+                        ok = mbar_wait_bounded(&empty_bar[s], ((n / NSTAGE) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    uint8_t* dst = smem_gen + (size_t)s * STAGE;
+                    const int key0 = (w.tile + t) * kTile;
+                    mbar_arrive_expect_tx(&full_bar[s], STAGE);
+#pragma unroll
+                    for (int h = 0; h < NHALF; ++h) {
+                        tma_load_4d(dst + h * HALF, &tmK, &full_bar[s], h * 64, key0, w.kvh, w.b);
+                        tma_load_4d(dst + STAGE / 2 + h * HALF, &tmV, &full_bar[s], h * 64, key0,
+                                    w.kvh, w.b);
+                    }
+                }
+                walk_advance(a, w, seg);
+            }
+        }
+    } else {
+        // ---------------- consumer warps ----------------
+        const int mt = warp % MT;
+        const int ks = warp / MT;
+        const int gid = lane >> 2;
+        const int tig = lane & 3;
+        const int row0 = mt * 16 + gid;  // grouped rows of this thread: row0 and row0 + 8
+        const int slot_stride = a.GR * (D + 2);
+
+        int n = 0;
+        bool ok = true;
+        while (w.remaining > 0) {
+            const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+            const int L = w.L;
+
+            // A fragments of Q for this row block: grouped row m = i*G + g (i draft row, g head)
+            uint32_t qf[KSTEPS][4];
+            int lim[2];
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int m = row0 + 8 * r;
+                const bool valid = m < a.GR;
+                const int i = valid ? m / a.G : 0;
+                const int g = valid ? m % a.G : 0;
+                lim[r] = L - a.R + i;
+                const __nv_bfloat16* qrow =
+                    a.q + (((size_t)w.b * a.R + i) * a.Hq + (size_t)w.kvh * a.G + g) * D;
+#pragma unroll
+                for (int kk = 0; kk < KSTEPS; ++kk) {
+                    uint32_t lo = 0, hi = 0;
+                    if (valid) {
+                        lo = *reinterpret_cast<const uint32_t*>(qrow + kk * 16 + 2 * tig);
+                        hi = *reinterpret_cast<const uint32_t*>(qrow + kk * 16 + 8 + 2 * tig);
+                    }
+                    qf[kk][r] = lo;
+                    qf[kk][2 + r] = hi;
+                }
+            }
+
+            float o[D / 8][4];
+#pragma unroll
+            for (int j = 0; j < D / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+            float mrow[2] = {-INFINITY, -INFINITY};
+            float lrow[2] = {0.f, 0.f};
+
+            for (int t = 0; t < seg; ++t, ++n) {
+                if (n % KS != ks) continue;
+                const int s = n % NSTAGE;
+                if (ok) ok = mbar_wait_bounded(&full_bar[s], (n / NSTAGE) & 1, abort_flag);
+                if (!ok) continue;
+                const uint32_t kbase = smem_base + s * STAGE;
+                const uint32_t vbase = kbase + STAGE / 2;
+                const int key0 = (w.tile + t) * kTile;
+
+                // rows of V beyond the context may hold any bits (NaN included): zero them so
+                // that a zero probability times that row is exactly zero
+                if (key0 + kTile > L) {
+                    const int first_bad = L - key0;
+                    uint8_t* vgen = smem_gen + (size_t)s * STAGE + STAGE / 2;
+                    const int chunks = (kTile - first_bad) * 8;  // 16-byte chunks per half
+                    for (int h = 0; h < NHALF; ++h)
+                        for (int c = lane; c < chunks; c += 32)
+                            *reinterpret_cast<uint4*>(vgen + h * HALF + first_bad * 128 + c * 16) =
+                                make_uint4(0, 0, 0, 0);
+                    __syncwarp();
+                }
+
+                // ---- S = Q K^T ----
+                float sc[kTile / 8][4];
+#pragma unroll
+                for (int j = 0; j < kTile / 8; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
+#pragma unroll
+                for (int kk = 0; kk < KSTEPS; kk += 2) {
+                    const int chunk = 2 * kk + (lane >> 3);  // 16-byte chunk along D
+                    const int half = chunk >> 3;
+                    const int cc = chunk & 7;
+#pragma unroll
+                    for (int j = 0; j < kTile / 8; ++j) {
+                        const int key = 8 * j + (lane & 7);
+                        const uint32_t addr =
+                            kbase + half * HALF + key * 128 + ((cc ^ (key & 7)) << 4);
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4(b0, b1, b2, b3, addr);
+                        mma_bf16_16816(sc[j], qf[kk], b0, b1);
+                        mma_bf16_16816(sc[j], qf[kk + 1], b2, b3);
+                    }
+                }
+
+                // ---- causal mask among the draft rows and the ragged end of the context ----
+                if (key0 + kTile - 1 > L - a.R) {
+#pragma unroll
+                    for (int j = 0; j < kTile / 8; ++j)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int key = key0 + 8 * j + 2 * tig + (e & 1);
+                            if (key > lim[e >> 1]) sc[j][e] = -INFINITY;
+                        }
+                }
+
+                // ---- online softmax (base 2) ----
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    float mx = -INFINITY;
+#pragma unroll
+                    for (int j = 0; j < kTile / 8; ++j)
+                        mx = fmaxf(mx, fmaxf(sc[j][2 * r], sc[j][2 * r + 1]));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                    const float m_new = fmaxf(mrow[r], mx * a.scale_log2);
+                    const float m_safe = m_new == -INFINITY ? 0.f : m_new;
+                    const float corr = fast_exp2(mrow[r] - m_safe);
+                    mrow[r] = m_new;
+                    float sum = 0.f;
+#pragma unroll
+                    for (int j = 0; j < kTile / 8; ++j) {
+                        const float p0 = fast_exp2(fmaf(sc[j][2 * r], a.scale_log2, -m_safe));
+                        const float p1 = fast_exp2(fmaf(sc[j][2 * r + 1], a.scale_log2, -m_safe));
+                        sc[j][2 * r] = p0;
+                        sc[j][2 * r + 1] = p1;
+                        sum += p0 + p1;
+                    }
+                    lrow[r] = lrow[r] * corr + sum;
+#pragma unroll
+                    for (int j = 0; j < D / 8; ++j) {
+                        o[j][2 * r] *= corr;
+                        o[j][2 * r + 1] *= corr;
+                    }
+                }
+
+                // ---- O += P V ----
+#pragma unroll
+                for (int kk = 0; kk < kTile / 16; ++kk) {
+                    uint32_t pa[4];
+                    pa[0] = pack_bf16x2(sc[2 * kk][0], sc[2 * kk][1]);
+                    pa[1] = pack_bf16x2(sc[2 * kk][2], sc[2 * kk][3]);
+                    pa[2] = pack_bf16x2(sc[2 * kk + 1][0], sc[2 * kk + 1][1]);
+                    pa[3] = pack_bf16x2(sc[2 * kk + 1][2], sc[2 * kk + 1][3]);
+                    const int key = 16 * kk + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+                    for (int jn = 0; jn < D / 8; jn += 2) {
+                        const int chunk = jn + (lane >> 4);
+                        const int half = chunk >> 3;
+                        const int cc = chunk & 7;
+                        const uint32_t addr =
+                            vbase + half * HALF + key * 128 + ((cc ^ (key & 7)) << 4);
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4_trans(b0, b1, b2, b3, addr);
+                        mma_bf16_16816(o[jn], pa, b0, b1);
+                        mma_bf16_16816(o[jn + 1], pa, b2, b3);
+                    }
+                }
+
+                // hand the stage back to the producer
+                if (key0 + kTile > L) fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[s]);
+            }
+
+            // ---- write this warp's partial (unnormalised O, running max, running sum) ----
+            const int unit = w.b * a.Hkv + w.kvh;
+            float* slot = a.partial + ((size_t)(cta + unit) * KS + ks) * slot_stride;
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                float l = lrow[r];
+                l += __shfl_xor_sync(0xffffffffu, l, 1);
+                l += __shfl_xor_sync(0xffffffffu, l, 2);
+                const int m = row0 + 8 * r;
+                if (m < a.GR) {
+                    if (tig == 0) {
+                        slot[a.GR * D + m] = mrow[r];
+                        slot[a.GR * D + a.GR + m] = l;
+                    }
+                    if (mrow[r] != -INFINITY) {
+#pragma unroll
+                        for (int j = 0; j < D / 8; ++j)
+                            *reinterpret_cast<float2*>(slot + (size_t)m * D + 8 * j + 2 * tig) =
+                                make_float2(o[j][2 * r], o[j][2 * r + 1]);
+                    }
+                }
+            }
+            walk_advance(a, w, seg);
+        }
+    }
+
+    __syncthreads();
+    if (tid == 0 && s_abort) atomicOr(a.status, RAPID_STATUS_PIPELINE_TIMEOUT);
+}
+
+// Merge: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the partials of a unit, in slot
+// order.  grid (GR, units), block D threads.
+template <int D>
+__global__ void __launch_bounds__(D)
+verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* lse_out,
+                         float* out_f32) {
+    const int m = blockIdx.x;
+    const int unit = blockIdx.y;
+    const int b = unit / a.Hkv;
+    const int kvh = unit % a.Hkv;
+    const int d = threadIdx.x;
+
+    long long T = 0, t0 = 0;
+    int nt_b = 0;
+    for (int bb = 0; bb < a.B; ++bb) {
+        const int nt = tiles_of(clamp_len(a.ctx_lens[bb], a.R, a.Lmax));
+        if (bb < b) t0 += (long long)a.Hkv * nt;
+        if (bb == b) nt_b = nt;
+        T += (long long)a.Hkv * nt;
+    }
+    t0 += (long long)kvh * nt_b;
+    const long long t1 = t0 + nt_b;
+    const int c_first = (int)(((t0 + 1) * a.num_ctas - 1) / T);
+    const int c_last = (int)((t1 * a.num_ctas - 1) / T);
+    const int slot_stride = a.GR * (D + 2);
+
+    float M = -INFINITY;
+    for (int c = c_first; c <= c_last; ++c)
+        for (int ks = 0; ks < KS; ++ks) {
+            const float* slot = a.partial + ((size_t)(c + unit) * KS + ks) * slot_stride;
+            M = fmaxf(M, slot[a.GR * D + m]);
+        }
+    float acc = 0.f, lsum = 0.f;
+    for (int c = c_first; c <= c_last; ++c)
+        for (int ks = 0; ks < KS; ++ks) {
+            const float* slot = a.partial + ((size_t)(c + unit) * KS + ks) * slot_stride;
+            const float ms = slot[a.GR * D + m];
+            if (ms == -INFINITY) continue;
+            const float wgt = exp2f(ms - M);
+            lsum += wgt * slot[a.GR * D + a.GR + m];
+            acc += wgt * slot[(size_t)m * D + d];
+        }
+    const float val = acc / lsum;
+    const int i = m / a.G;
+    const int g = m % a.G;
+    const size_t row = ((size_t)b * a.R + i) * a.Hq + (size_t)kvh * a.G + g;
+    out[row * D + d] = __float2bfloat16_rn(val);
+    if (out_f32) out_f32[row * D + d] = val;
+    if (lse_out && d == 0) lse_out[row] = (M + log2f(lsum)) * 0.69314718055994530942f;
+}
+
+// ---- host side ----------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) !=
+                cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+int make_kv_map(CUtensorMap* map, const void* base, const rapid_attn_shape& s, int64_t sb,
+                int64_t sh, int64_t sl) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) {
+        set_error("cuTensorMapEncodeTiled is not available from the CUDA driver");
+        return RAPID_ERR_CUDA;
+    }
+    cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.Lmax, (cuuint64_t)s.Hkv, (cuuint64_t)s.B};
+    cuuint64_t strides[3] = {(cuuint64_t)sl * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)kTile, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return RAPID_ERR_CUDA;
+    }
+    return RAPID_OK;
+}
+
+template <int D, int MT>
+int launch_split(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
+                 cudaStream_t stream) {
+    constexpr int KS = tile_lanes(MT);
+    constexpr int threads = (MT * KS + 1) * 32;
+    constexpr int smem = num_stages(D) * stage_bytes(D) + 1024;
+    static bool configured[64] = {};
+    int dev = 0;
+    RAPID_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev >= 64 || !configured[dev]) {
+        RAPID_CUDA_CHECK(cudaFuncSetAttribute(verify_attn_splitkv_kernel<D, MT>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        if (dev < 64) configured[dev] = true;
+    }
+    verify_attn_splitkv_kernel<D, MT><<<a.num_ctas, threads, smem, stream>>>(tmK, tmV, a);
+    RAPID_CUDA_CHECK(cudaGetLastError());
+    return RAPID_OK;
+}
+
+template <int D>
+int dispatch_split(int MT, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
+                   cudaStream_t stream) {
+    switch (MT) {
+        case 1: return launch_split<D, 1>(tmK, tmV, a, stream);
+        case 2: return launch_split<D, 2>(tmK, tmV, a, stream);
+        case 3: return launch_split<D, 3>(tmK, tmV, a, stream);
+        case 4: return launch_split<D, 4>(tmK, tmV, a, stream);
+        case 5: return launch_split<D, 5>(tmK, tmV, a, stream);
+        case 6: return launch_split<D, 6>(tmK, tmV, a, stream);
+        case 7: return launch_split<D, 7>(tmK, tmV, a, stream);
+        case 8: return launch_split<D, 8>(tmK, tmV, a, stream);
+    }
+    set_error("unsupported number of grouped rows");
+    return RAPID_ERR_UNSUPPORTED;
+}
+
+int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+    }
+    return n;
+}
+
+bool attn_shape_ok(const rapid_attn_shape* s, int gamma) {
+    if (!s) return false;
+    if (s->B <= 0 || s->Hq <= 0 || s->Hkv <= 0 || s->Lmax <= 0 || gamma < 0) return false;
+    if (s->Hq % s->Hkv != 0) return false;
+    return true;
+}
+
+}  // namespace
+
+size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma) {
+    if (!attn_shape_ok(s, gamma)) return 0;
+    if (s->D != 64 && s->D != 128) return 0;
+    const int64_t GR = (int64_t)(s->Hq / s->Hkv) * (gamma + 1);
+    if (GR > 128) return 0;
+    const int MT = (int)((GR + 15) / 16);
+    const int64_t slots = ((int64_t)kMaxCtas + (int64_t)s->B * s->Hkv) * tile_lanes(MT);
+    return kWorkspaceHeaderBytes + (size_t)slots * GR * (s->D + 2) * sizeof(float);
+}
+
+int launch_verify_attention(const void* q, const void* k_cache, const void* v_cache,
+                            const int32_t* ctx_lens, int gamma, void* out,
+                            const rapid_attn_shape* shape, const rapid_attn_params* params,
+                            void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (!q || !k_cache || !v_cache || !ctx_lens || !out || !shape) {
+        set_error("rapid_verify_attention: NULL argument");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (!attn_shape_ok(shape, gamma)) {
+        set_error("rapid_verify_attention: invalid shape (B=%d Hq=%d Hkv=%d Lmax=%lld gamma=%d)",
+                  shape->B, shape->Hq, shape->Hkv, (long long)shape->Lmax, gamma);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const rapid_attn_shape& s = *shape;
+    const int R = gamma + 1;
+    const int G = s.Hq / s.Hkv;
+    const int GR = G * R;
+    if (s.D != 64 && s.D != 128) {
+        set_error("rapid_verify_attention: head_dim %d is not supported (64 or 128)", s.D);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    if (GR > 128) {
+        set_error("rapid_verify_attention: %d grouped rows per KV head exceed 128", GR);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    if (s.Lmax < R || s.Lmax > 0x7fffffffLL - kTile) {
+        set_error("rapid_verify_attention: Lmax %lld out of range", (long long)s.Lmax);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const int64_t sl = s.kv_stride_l ? s.kv_stride_l : s.D;
+    const int64_t sh = s.kv_stride_h ? s.kv_stride_h : s.Lmax * sl;
+    const int64_t sb = s.kv_stride_b ? s.kv_stride_b : s.Hkv * sh;
+    if (sl < s.D || sl % 8 || sh % 8 || sb % 8 || sh <= 0 || sb <= 0) {
+        set_error("rapid_verify_attention: K/V strides must be positive multiples of 8 elements");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q | (uintptr_t)out) & 15) {
+        set_error("rapid_verify_attention: q, k_cache, v_cache and out must be 16-byte aligned");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const size_t need = attention_workspace_bytes(shape, gamma);
+    if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) {
+        set_error("rapid_verify_attention: workspace of %zu bytes needed (256-byte aligned), got %zu",
+                  need, workspace_bytes);
+        return RAPID_ERR_WORKSPACE;
+    }
+    int num_ctas = params && params->num_ctas ? params->num_ctas : sm_count();
+    if (num_ctas <= 0 || num_ctas > kMaxCtas) {
+        set_error("rapid_verify_attention: num_ctas %d outside [1, %d]", num_ctas, kMaxCtas);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const float scale = params && params->scale != 0.f ? params->scale : 1.0f / sqrtf((float)s.D);
+    if (!(scale > 0.f) || !isfinite(scale)) {
+        set_error("rapid_verify_attention: scale must be positive and finite");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if ((int64_t)s.B * s.Hkv > 65535) {
+        set_error("rapid_verify_attention: B*Hkv above 65535 is not supported");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+
+    CUtensorMap tmK, tmV;
+    int rc = make_kv_map(&tmK, k_cache, s, sb, sh, sl);
+    if (rc != RAPID_OK) return rc;
+    rc = make_kv_map(&tmV, v_cache, s, sb, sh, sl);
+    if (rc != RAPID_OK) return rc;
+
+    AttnArgs a;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.ctx_lens = ctx_lens;
+    a.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kWorkspaceHeaderBytes);
+    a.status = static_cast<int32_t*>(workspace);
+    a.B = s.B;
+    a.Hq = s.Hq;
+    a.Hkv = s.Hkv;
+    a.G = G;
+    a.R = R;
+    a.GR = GR;
+    a.Lmax = (int)s.Lmax;
+    a.num_ctas = num_ctas;
+    a.scale_log2 = scale * 1.4426950408889634f;
+
+    const int MT = (GR + 15) / 16;
+    rc = s.D == 128 ? dispatch_split<128>(MT, tmK, tmV, a, stream)
+                    : dispatch_split<64>(MT, tmK, tmV, a, stream);
+    if (rc != RAPID_OK) return rc;
+
+    dim3 grid(GR, s.B * s.Hkv);
+    float* lse = params ? params->lse_out : nullptr;
+    float* o32 = params ? params->out_f32 : nullptr;
+    if (s.D == 128)
+        verify_attn_merge_kernel<128><<<grid, 128, 0, stream>>>(
+            a, tile_lanes(MT), static_cast<__nv_bfloat16*>(out), lse, o32);
+    else
+        verify_attn_merge_kernel<64><<<grid, 64, 0, stream>>>(
+            a, tile_lanes(MT), static_cast<__nv_bfloat16*>(out), lse, o32);
+    RAPID_CUDA_CHECK(cudaGetLastError());
+    count_launch(2);
+    return RAPID_OK;
+}
+
+}  // namespace rapid

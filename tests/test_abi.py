@@ -1,0 +1,61 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2502_20330_b200 import build
+    return ctypes.CDLL(build.build())
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "rapid.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rapid_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared()
+    assert "rapid_verify_attention" in names and "rapid_accept" in names and "rapid_verify_step" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in rapid.h but not exported"
+
+
+def test_binding_covers_the_header():
+    from paper_2502_20330_b200 import binding
+    assert sorted(binding.EXPORTS) == _declared()
+
+
+def test_host_only_calls(lib):
+    import paper_2502_20330_b200 as R
+    assert R.version() == 100
+    assert R.last_error() == ""
+    assert R.attention_workspace_bytes(1, 32, 8, 128, 131072, 8) > 0
+    assert R.attention_workspace_bytes(1, 32, 7, 128, 131072, 8) == 0     # Hq not a multiple of Hkv
+    assert R.accept_workspace_bytes(8, 4, 152064) > 0
+    assert R.accept_workspace_bytes(0, 4, 152064) == 0
+    a = R.verify_step_host_arena_bytes(1, 8, 2, 64, 4096, 4, 4096)
+    assert a > 2 * 2 * 4096 * 64 * 2
+
+
+def test_struct_layouts_match_the_header():
+    from paper_2502_20330_b200 import binding
+    assert ctypes.sizeof(binding._AttnShape) == 48
+    assert ctypes.sizeof(binding._AttnParams) == 24
+    assert ctypes.sizeof(binding._AcceptShape) == 32
+    assert ctypes.sizeof(binding._AcceptParams) == 24
+
+
+def test_product_does_not_touch_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2502_20330_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in src, f"{f} mentions the oracle"

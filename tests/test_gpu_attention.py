@@ -1,0 +1,162 @@
+"""Parity of the CUDA verify attention with the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import oracle
+from oracle import parity
+import workloads as wl
+from workloads import bf16_bits
+
+
+def _run(q, k, v, ctx, gamma, num_ctas=0, scale=0.0):
+    import paper_2502_20330_b200 as R
+    B, Rr, Hq, D = q.shape
+    Hkv, Lmax = k.shape[1], k.shape[2]
+    ws = R.new_workspace(R.attention_workspace_bytes(B, Hq, Hkv, D, Lmax, gamma))
+    out = torch.empty_like(q)
+    lse = torch.empty(B, Rr, Hq, dtype=torch.float32, device=q.device)
+    o32 = torch.empty(B, Rr, Hq, D, dtype=torch.float32, device=q.device)
+    R.rapid_verify_attention(q, k, v, ctx, gamma, out, ws,
+                             R.AttnParams(scale=scale, num_ctas=num_ctas, lse_out=lse, out_f32=o32))
+    torch.cuda.synchronize()
+    return out, lse, o32, R.workspace_status(ws)
+
+
+def _oracle(q, k, v, ctx, gamma, scale=0.0, units=None):
+    return oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx.cpu().numpy(), gamma,
+                                   scale=scale, units=units)
+
+
+def _compare(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, units=None):
+    out, lse, o32, status = _run(q, k, v, ctx, gamma, num_ctas, scale)
+    assert status == 0
+    ref, ref_lse = _oracle(q, k, v, ctx, gamma, scale, units)
+    rows = ~np.isnan(ref_lse)
+    rep = parity.check_attention(out.float().cpu().numpy(), ref, rows)
+    parity.check_attention(o32.cpu().numpy(), ref, rows)
+    assert np.abs(lse.cpu().numpy()[rows] - ref_lse[rows]).max() < 1e-3
+    return rep, out, o32
+
+
+def test_tiny_config():
+    cfg = wl.CONFIGS["tiny"]
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=1, device="cuda")
+    rep, _, _ = _compare(q, k, v, ctx, cfg.gamma)
+    assert rep["rows"] == cfg.B * cfg.R * cfg.Hq
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,gamma,L", [
+    (32, 8, 128, 8, 2048 + 37),     # 36 grouped rows, ragged tail
+    (64, 8, 128, 8, 1500),          # 72 grouped rows (five row blocks)
+    (28, 4, 128, 4, 3000),          # 35 grouped rows, G = 7
+    (32, 8, 128, 0, 777),           # one-row decode (drafter-side call)
+    (8, 2, 64, 4, 1000),            # head_dim 64
+    (16, 1, 64, 7, 513),            # 128 grouped rows: the maximum
+    (4, 4, 128, 2, 70),             # G = 1
+])
+def test_shapes_against_oracle(Hq, Hkv, D, gamma, L):
+    cfg = wl.VerifyConfig("t", B=2, Hq=Hq, Hkv=Hkv, D=D, gamma=gamma, V=4096, ctx_lens=(L, max(gamma + 1, L // 3)))
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=2, device="cuda", poison_padding=True)
+    _compare(q, k, v, ctx, gamma)
+
+
+@pytest.mark.parametrize("num_ctas", [1, 2, 7, 148, 509])
+def test_split_invariance(num_ctas):
+    """Any split of the KV length gives the oracle's answer, and fp32 results agree across splits."""
+    cfg = wl.VerifyConfig("t", B=3, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(4100, 9, 1111), Lmax=4200)
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=3, device="cuda", poison_padding=True)
+    _, _, o32 = _compare(q, k, v, ctx, cfg.gamma, num_ctas=num_ctas)
+    _, _, base, _ = _run(q, k, v, ctx, cfg.gamma, num_ctas=1)
+    rel = (o32 - base).norm(dim=-1) / base.norm(dim=-1)
+    assert rel.max().item() < 1e-4
+
+
+def test_minimum_context_equals_rows():
+    """L_b = R: row i sees exactly i+1 keys; row 0 returns the first value row."""
+    cfg = wl.VerifyConfig("t", B=2, Hq=8, Hkv=2, D=128, gamma=5, V=4096, ctx_lens=(6, 6), Lmax=64)
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=4, device="cuda", poison_padding=True)
+    _, out, o32 = _compare(q, k, v, ctx, cfg.gamma)
+    for h in range(8):
+        assert torch.equal(out[:, 0, h], v[:, h // 4, 0])
+
+
+def test_peaked_scores_and_planted_key():
+    cfg = wl.VerifyConfig("t", B=1, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(5000,), q_scale=4.0)
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=5, device="cuda")
+    k[0, :, 1234] = (q[0, 0, ::4] * 0.5)           # a key aligned with row 0 of each group's first head
+    _compare(q, k, v, ctx, cfg.gamma)
+
+
+def test_explicit_scale_and_strided_cache():
+    cfg = wl.VerifyConfig("t", B=2, Hq=8, Hkv=2, D=128, gamma=3, V=4096, ctx_lens=(900, 640), Lmax=1024)
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=6, device="cuda")
+    # token-major storage [B, L, Hkv, D] viewed as [B, Hkv, L, D]: non-dense strides
+    ks = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    vs = v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert not ks.is_contiguous()
+    out, lse, o32, status = _run(q, ks, vs, ctx, cfg.gamma, scale=0.05)
+    ref, _ = _oracle(q, k, v, ctx, cfg.gamma, scale=0.05)
+    parity.check_attention(o32.cpu().numpy(), ref)
+
+
+def test_run_to_run_bit_identity():
+    cfg = wl.VerifyConfig("t", B=2, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(6000, 3000))
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=7, device="cuda")
+    a = _run(q, k, v, ctx, cfg.gamma)
+    b = _run(q, k, v, ctx, cfg.gamma)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[2], b[2]) and torch.equal(a[1], b[1])
+
+
+def test_bad_context_length_sets_status_and_stays_defined():
+    cfg = wl.VerifyConfig("t", B=2, Hq=8, Hkv=2, D=64, gamma=2, V=4096, ctx_lens=(200, 100), Lmax=256)
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=8, device="cuda")
+    bad = ctx.clone(); bad[1] = 100000
+    out, _, _, status = _run(q, k, v, bad, cfg.gamma)
+    assert status & 1
+    assert torch.isfinite(out.float()).all()
+
+
+def test_argument_errors():
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("t", B=1, Hq=8, Hkv=2, D=64, gamma=2, V=4096, ctx_lens=(128,))
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=9, device="cuda")
+    out = torch.empty_like(q)
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(R.RapidError) as e:
+        R.rapid_verify_attention(q, k, v, ctx, 2, out, small)
+    assert e.value.code == 3
+    ws = R.new_workspace(R.attention_workspace_bytes(1, 8, 2, 64, 128, 2))
+    with pytest.raises(R.RapidError) as e:
+        R.rapid_verify_attention(q, k, v, ctx, 2, out, ws, R.AttnParams(num_ctas=100000))
+    assert e.value.code == 1
+    assert R.attention_workspace_bytes(1, 8, 2, 96, 128, 2) == 0          # unsupported head_dim
+    assert R.attention_workspace_bytes(1, 64, 1, 128, 128, 8) == 0        # 576 grouped rows
+
+
+def test_llama8b_32k_sampled_rows():
+    """The 32K workload in the bench's launch configuration; the oracle checks a sample of rows."""
+    cfg = wl.CONFIGS["llama8b_32k"]
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=10, device="cuda")
+    units = np.array([0, 8, 37, 100, 143, 200, 287], dtype=np.int64)
+    _compare(q, k, v, ctx, cfg.gamma, units=units)
+
+
+def test_llama8b_128k_and_70b_sampled_rows():
+    for name in ("llama8b_128k", "llama70b_128k"):
+        cfg = wl.CONFIGS[name]
+        q, k, v, ctx = wl.attention_inputs(cfg, seed=11, device="cuda")
+        n_units = cfg.B * cfg.Hq * cfg.R
+        units = np.array([0, 8, n_units // 2 + 3, n_units - 1], dtype=np.int64)
+        _compare(q, k, v, ctx, cfg.gamma, units=units)
+        del q, k, v
+
+
+def test_ragged_qwen_batch_sampled_rows():
+    cfg = wl.CONFIGS["qwen7b_ragged"]
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=12, device="cuda", poison_padding=True)
+    n_units = cfg.B * cfg.Hq * cfg.R
+    units = np.arange(3, n_units, n_units // 9, dtype=np.int64)
+    _compare(q, k, v, ctx, cfg.gamma, units=units)

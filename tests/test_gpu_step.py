@@ -1,0 +1,52 @@
+"""The chained verify step and its host-buffer form, against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import oracle
+from oracle import parity
+import workloads as wl
+from workloads import bf16_bits
+
+
+def _inputs(cfg, seed, device):
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=seed, device=device)
+    z, d, tok, u = wl.accept_inputs(cfg, seed=seed, device=device)
+    return q, k, v, ctx, z, d, tok, u
+
+
+def test_verify_step_chains_both_calls():
+    import paper_2502_20330_b200 as R
+    cfg = wl.CONFIGS["tiny"]
+    q, k, v, ctx, z, d, tok, u = _inputs(cfg, 21, "cuda")
+    aws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, k.shape[2], cfg.gamma))
+    cws = R.new_workspace(R.accept_workspace_bytes(cfg.B, cfg.gamma, cfg.V))
+    out = torch.empty_like(q)
+    alen = torch.zeros(cfg.B, dtype=torch.int32, device="cuda"); ntok = torch.zeros_like(alen)
+    R.kernel_launch_count_reset()
+    R.rapid_verify_step(q, k, v, ctx, cfg.gamma, out, aws, z, d, tok, u, cfg.eta, alen, ntok, cws)
+    torch.cuda.synchronize()
+    assert R.kernel_launch_count() == 6
+    ref, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx.cpu().numpy(), cfg.gamma)
+    parity.check_attention(out.float().cpu().numpy(), ref)
+    parity.check_accept(z.cpu().numpy(), d.cpu().numpy(), tok.cpu().numpy(), u.cpu().numpy(), cfg.eta, 1.0, 0.1, 0,
+                        alen.cpu().numpy(), ntok.cpu().numpy())
+    assert R.workspace_status(aws) == 0 and R.workspace_status(cws) == 0
+
+
+def test_verify_step_host_buffers():
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("t", B=2, Hq=8, Hkv=2, D=128, gamma=3, V=4096, ctx_lens=(700, 300), Lmax=768)
+    q, k, v, ctx, z, d, tok, u = [t.pin_memory() for t in _inputs(cfg, 22, "cpu")]
+    arena = torch.empty(R.verify_step_host_arena_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, 768, cfg.gamma, cfg.V),
+                        dtype=torch.uint8, device="cuda")
+    out = torch.empty_like(q).pin_memory()
+    alen = torch.zeros(cfg.B, dtype=torch.int32).pin_memory(); ntok = torch.zeros(cfg.B, dtype=torch.int32).pin_memory()
+    for _ in range(2):
+        status = R.rapid_verify_step_host(q, k, v, ctx, cfg.gamma, out, z, d, tok, u, 5.0, alen, ntok, arena)
+        assert status == 0
+        ref, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx.numpy(), cfg.gamma)
+        parity.check_attention(out.float().numpy(), ref)
+        parity.check_accept(z.numpy(), d.numpy(), tok.numpy(), u.numpy(), 5.0, 1.0, 0.1, 0, alen.numpy(), ntok.numpy())
