@@ -242,7 +242,14 @@ __global__ void __launch_bounds__(kThreads) accept_residual_kernel(const AcceptA
                 sw += residual_weight(a, r, My, inv_Sy, xs[e], ys4[e], p, q, ph);
                 sp += p;
                 if (v + e == tok) {
-                    const float ratio = q > 0.f ? ph / q : INFINITY;
+                    // the ratio is formed from log-probabilities: a draft token deep in the tail
+                    // has p, phat and q far below the fp32 normal range while their ratio is O(1)
+                    const float z2 = xs[e] * a.inv_T_log2;
+                    const float lq = (ys4[e] * a.inv_T_log2 - r.Md) + log2f(r.inv_Sd);
+                    const float y2 = fmaf(a.eta_log2, q - p, z2);
+                    const float lph = (y2 - My < a.log2_alpha) ? (z2 - r.Mz) + log2f(r.inv_Sz)
+                                                               : (y2 - My) + log2f(inv_Sy);
+                    const float ratio = (lq == -INFINITY) ? INFINITY : exp2f(lph - lq);
                     a.ratio[drow] = ratio;
                     if (a.ratio_out) a.ratio_out[drow] = ratio;
                 }

