@@ -90,6 +90,8 @@ typedef struct rapid_attn_params {
     int32_t num_ctas; /* CTAs the KV length is split over; 0 = one per SM; at most 512            */
     float* lse_out;   /* device [B, R, Hq] fp32 natural-log sum-exp of the scaled scores, or NULL */
     float* out_f32;   /* device [B, R, Hq, D] fp32 output before bf16 rounding, or NULL           */
+    void* split_done_event; /* a cudaEvent_t recorded on the stream between the split and the merge
+                               kernel (lets a caller time the two separately), or NULL          */
 } rapid_attn_params;
 
 /*

@@ -40,7 +40,8 @@ class _AttnShape(ctypes.Structure):
 
 class _AttnParams(ctypes.Structure):
     _fields_ = [("scale", ctypes.c_float), ("num_ctas", ctypes.c_int32),
-                ("lse_out", ctypes.c_void_p), ("out_f32", ctypes.c_void_p)]
+                ("lse_out", ctypes.c_void_p), ("out_f32", ctypes.c_void_p),
+                ("split_done_event", ctypes.c_void_p)]
 
 
 class _AcceptShape(ctypes.Structure):
@@ -60,6 +61,7 @@ class AttnParams:
     num_ctas: int = 0
     lse_out: Optional[torch.Tensor] = None   # [B,R,Hq] float32
     out_f32: Optional[torch.Tensor] = None   # [B,R,Hq,D] float32
+    split_done_event: Optional[int] = None   # cudaEvent_t handle recorded between split and merge
 
 
 @dataclass
@@ -160,7 +162,8 @@ def _attn_params(p: Optional[AttnParams]):
     if p is None:
         return None
     return ctypes.byref(_AttnParams(p.scale, p.num_ctas, p.lse_out.data_ptr() if p.lse_out is not None else None,
-                                    p.out_f32.data_ptr() if p.out_f32 is not None else None))
+                                    p.out_f32.data_ptr() if p.out_f32 is not None else None,
+                                    p.split_done_event))
 
 
 def _accept_shape(target_logits: torch.Tensor, draft_logits: torch.Tensor) -> _AcceptShape:

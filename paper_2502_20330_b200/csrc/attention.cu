@@ -618,6 +618,9 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
                     : dispatch_split<64>(MT, tmK, tmV, a, stream);
     if (rc != RAPID_OK) return rc;
 
+    if (params && params->split_done_event)
+        RAPID_CUDA_CHECK(cudaEventRecord(static_cast<cudaEvent_t>(params->split_done_event), stream));
+
     dim3 grid(GR, s.B * s.Hkv);
     float* lse = params ? params->lse_out : nullptr;
     float* o32 = params ? params->out_f32 : nullptr;

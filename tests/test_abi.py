@@ -47,7 +47,7 @@ def test_host_only_calls(lib):
 def test_struct_layouts_match_the_header():
     from paper_2502_20330_b200 import binding
     assert ctypes.sizeof(binding._AttnShape) == 48
-    assert ctypes.sizeof(binding._AttnParams) == 24
+    assert ctypes.sizeof(binding._AttnParams) == 32
     assert ctypes.sizeof(binding._AcceptShape) == 32
     assert ctypes.sizeof(binding._AcceptParams) == 24
 
