@@ -189,6 +189,45 @@ int rapid_accept(const float* target_logits, const float* draft_logits,
                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * rapid_accept without a caller workspace.  (The paper has no counterpart: this
+ * entry point exists only for the sake of callers, not of the method.)
+ *
+ * Who it is for: code that is not allowed to obtain device memory at the moment
+ * it needs an accept step -- a plugin running inside a serving process that
+ * handed all device memory to its own pool at start-up, a decode loop that has
+ * promised not to touch the allocator after warm-up because cudaMalloc and
+ * cudaFree stall every stream of the device, or a component whose memory
+ * budget is fixed by contract.  Such a caller still owns the logits, tokens,
+ * uniforms and the two output arrays, but has nowhere to put the few hundred
+ * kilobytes of per-row statistics the accept passes exchange.
+ *
+ * Here that scratch is a fixed array inside the library image (about 1.1 MB,
+ * resident on every GPU that loads the library until the process ends).  The
+ * computation, the kernels and the results are those of rapid_accept.
+ *
+ * Limits and rules
+ *   - B * (gamma+1) may not exceed 512 logit rows; larger shapes are rejected
+ *     with RAPID_ERR_UNSUPPORTED and a message that says so.
+ *   - The call allocates and frees nothing, on host or device.
+ *   - The first call on each device looks up the array's device address (the
+ *     device must be current).  Make that first call outside any stream
+ *     capture; later calls only enqueue work on the stream.
+ *   - All calls on a device share the one array, and it keeps what the last
+ *     call wrote.  The status word is cleared at the start of every call, so
+ *     status bits are per call here (not sticky).  Two calls whose GPU work can
+ *     overlap (different streams, no dependency) race on the array and give
+ *     undefined results; serialise them.
+ *   - out_status: device int32 that receives this call's status word
+ *     (RAPID_STATUS_* bits), or NULL.
+ * Other arguments: exactly those of rapid_accept.
+ */
+int rapid_accept_static(const float* target_logits, const float* draft_logits,
+                        const int32_t* draft_tokens, const float* uniforms, float eta,
+                        int32_t* out_accept_len, int32_t* out_next_token,
+                        const rapid_accept_shape* shape, const rapid_accept_params* params,
+                        int32_t* out_status, void* cuda_stream);
+
+/*
  * One verify step: rapid_verify_attention followed by rapid_accept on the same
  * stream, with no host synchronisation in between (Algorithm 1, one iteration
  * of the outer loop after drafting).  The projections and the LM head that turn

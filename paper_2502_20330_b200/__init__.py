@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     load_library,
     new_workspace,
     rapid_accept,
+    rapid_accept_static,
     rapid_verify_attention,
     rapid_verify_step,
     rapid_verify_step_host,

@@ -20,7 +20,8 @@ RESIDUAL_PHAT = 1
 
 EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
-    "rapid_workspace_status", "rapid_verify_attention", "rapid_accept", "rapid_verify_step",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_accept", "rapid_accept_static",
+    "rapid_verify_step",
     "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_last_error",
     "rapid_version", "rapid_kernel_launch_count", "rapid_kernel_launch_count_reset",
 ]
@@ -103,6 +104,8 @@ def load_library():
         lib.rapid_verify_attention.argtypes = attn_args + [vp, sz, vp]
         lib.rapid_accept.restype = i32
         lib.rapid_accept.argtypes = acc_args + [vp, sz, vp]
+        lib.rapid_accept_static.restype = i32
+        lib.rapid_accept_static.argtypes = acc_args + [vp, vp]
         lib.rapid_verify_step.restype = i32
         lib.rapid_verify_step.argtypes = attn_args + [vp, sz] + acc_args + [vp, sz, vp]
         lib.rapid_verify_step_host.restype = i32
@@ -252,6 +255,23 @@ def rapid_accept(target_logits, draft_logits, draft_tokens, uniforms, eta, out_a
                                        float(eta), _p(out_accept_len), _p(out_next_token), ctypes.byref(shape),
                                        _accept_params(params), _p(workspace), _nbytes(workspace),
                                        _stream_ptr(stream)))
+
+
+def rapid_accept_static(target_logits, draft_logits, draft_tokens, uniforms, eta, out_accept_len, out_next_token,
+                        params: Optional[AcceptParams] = None, out_status: Optional[torch.Tensor] = None,
+                        stream=None) -> None:
+    """rapid_accept for callers that cannot provide a workspace: the scratch is a fixed array inside
+    the library (at most 512 logit rows, calls must not overlap on the GPU; see include/rapid.h).
+    ``out_status`` is an optional int32 device tensor that receives this call's status word."""
+    if target_logits.dtype != torch.float32 or draft_logits.dtype != torch.float32 or uniforms.dtype != torch.float32:
+        raise TypeError("logits and uniforms must be float32")
+    if draft_tokens.dtype != torch.int32 or out_accept_len.dtype != torch.int32 or out_next_token.dtype != torch.int32:
+        raise TypeError("tokens and outputs must be int32")
+    shape = _accept_shape(target_logits, draft_logits)
+    _check(load_library().rapid_accept_static(_p(target_logits), _p(draft_logits), _p(draft_tokens), _p(uniforms),
+                                              float(eta), _p(out_accept_len), _p(out_next_token),
+                                              ctypes.byref(shape), _accept_params(params), _p(out_status),
+                                              _stream_ptr(stream)))
 
 
 def rapid_verify_step(q, k_cache, v_cache, ctx_lens, gamma, out, attn_workspace, target_logits, draft_logits,

@@ -497,3 +497,70 @@ int launch_accept(const float* target_logits, const float* draft_logits,
 }
 
 }  // namespace rapid
+
+// ---- accept step on library-owned scratch ------------------------------------------------------
+//
+// The scratch of the accept passes for up to kStaticMaxRows logit rows lives in this file-scope
+// device array instead of a caller workspace.  Every GPU that loads the library holds these
+// bytes until the process exits.
+namespace rapid {
+namespace {
+
+constexpr int kStaticMaxRows = 512;  // B * (gamma + 1) at most
+constexpr size_t kStaticScratchBytes =
+    kWorkspaceHeaderBytes + (size_t)kStaticMaxRows * kMaxChunks * (sizeof(float4) + 2 * sizeof(float2)) +
+    (size_t)kStaticMaxRows * sizeof(float) + 4 * 256;
+
+static __device__ __align__(256) unsigned char g_accept_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices] = {};  // device address of g_accept_scratch, per device
+
+}  // namespace
+}  // namespace rapid
+
+extern "C" int rapid_accept_static(const float* target_logits, const float* draft_logits,
+                                   const int32_t* draft_tokens, const float* uniforms, float eta,
+                                   int32_t* out_accept_len, int32_t* out_next_token,
+                                   const rapid_accept_shape* shape,
+                                   const rapid_accept_params* params, int32_t* out_status,
+                                   void* cuda_stream) {
+    using namespace rapid;
+    clear_error();
+    if (!shape || shape->B <= 0 || shape->gamma < 0) {
+        set_error("rapid_accept_static: invalid shape");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const long long rows = (long long)shape->B * (shape->gamma + 1);
+    const size_t need = accept_workspace_bytes(shape);
+    if (rows > kStaticMaxRows || need == 0 || need > kStaticScratchBytes) {
+        set_error("rapid_accept_static: B*(gamma+1) = %lld logit rows exceed the built-in scratch, which "
+                  "holds %d rows; use rapid_accept with a caller workspace", rows, kStaticMaxRows);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    int dev = 0;
+    RAPID_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) {
+        set_error("rapid_accept_static: device ordinal %d not supported", dev);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    // In host code the array's name is only a handle for the runtime, not a device address: the
+    // address the kernels can use has to be asked for, once per device, with that device current.
+    if (!g_scratch_addr[dev]) {
+        void* ptr = nullptr;
+        RAPID_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_accept_scratch));
+        g_scratch_addr[dev] = ptr;
+    }
+    void* scratch = g_scratch_addr[dev];
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // the array keeps whatever the previous call left: the status word must start at zero
+    RAPID_CUDA_CHECK(cudaMemsetAsync(scratch, 0, kWorkspaceHeaderBytes, st));
+    const int rc = launch_accept(target_logits, draft_logits, draft_tokens, uniforms, eta,
+                                 out_accept_len, out_next_token, shape, params, scratch,
+                                 kStaticScratchBytes, st);
+    if (rc != RAPID_OK) return rc;
+    if (out_status)
+        RAPID_CUDA_CHECK(cudaMemcpyAsync(out_status, scratch, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+    return RAPID_OK;
+}
+
