@@ -98,7 +98,8 @@ typedef struct rapid_attn_params {
  * Geometry of one accept call.
  *   target_logits : [B, gamma+1, V] fp32, row stride target_row_stride elements (0 = V)
  *   draft_logits  : [B, gamma,   V] fp32, row stride draft_row_stride elements (0 = V)
- *   V and both row strides are multiples of 4 and the bases 16-byte aligned.
+ *   V and both row strides are multiples of 4 and the bases 16-byte aligned;
+ *   V <= 196,608 and B * (gamma+1) <= 65,535.
  */
 typedef struct rapid_accept_shape {
     int32_t B;

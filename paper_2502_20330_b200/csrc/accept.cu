@@ -91,16 +91,18 @@ __device__ __forceinline__ float block_reduce_sum(float v, float* sh) {
     return S;
 }
 
-// Combine the per-chunk (max, sum) partials of a row, in chunk order (every thread does it).
+// Combine the per-chunk (max, sum) partials of a row.  Every warp does it for itself with its
+// lanes spread over the chunks (at most kMaxChunks = 64, two per lane), in a fixed shuffle order.
 __device__ __forceinline__ void combine_ms(const float* m, const float* s, int n, int stride,
                                            float& M, float& S) {
-    M = -INFINITY;
-    for (int c = 0; c < n; ++c) M = fmaxf(M, m[c * stride]);
-    S = 0.f;
-    for (int c = 0; c < n; ++c) {
-        const float mc = m[c * stride];
-        S += (mc == -INFINITY) ? 0.f : s[c * stride] * exp2f(mc - M);
-    }
+    const int lane = threadIdx.x & 31;
+    const float m0 = lane < n ? m[lane * stride] : -INFINITY;
+    const float m1 = lane + 32 < n ? m[(lane + 32) * stride] : -INFINITY;
+    const float s0 = lane < n ? s[lane * stride] : 0.f;
+    const float s1 = lane + 32 < n ? s[(lane + 32) * stride] : 0.f;
+    M = warp_max(fmaxf(m0, m1));
+    float part = (m0 == -INFINITY ? 0.f : s0 * exp2f(m0 - M)) + (m1 == -INFINITY ? 0.f : s1 * exp2f(m1 - M));
+    S = warp_sum(part);
 }
 
 __device__ __forceinline__ void online_add(float& m, float& s, float x) {
@@ -112,29 +114,52 @@ __device__ __forceinline__ void online_add(float& m, float& s, float x) {
     }
 }
 
+// A thread's share of a chunk: up to kPerThread float4 groups, strided by the block, all loaded
+// before any arithmetic so that the loads are in flight together.
+constexpr int kPerThread = 3;
+constexpr int kChunkMax = kThreads * 4 * kPerThread;  // 3072 entries
+
+struct Frag {
+    float4 x[kPerThread];
+    bool ok[kPerThread];
+};
+
+__device__ __forceinline__ Frag load_frag(const float* row, int v0, int v1, float fill) {
+    Frag f;
+#pragma unroll
+    for (int e = 0; e < kPerThread; ++e) {
+        const int v = v0 + (e * kThreads + threadIdx.x) * 4;
+        f.ok[e] = v < v1;
+        f.x[e] = f.ok[e] ? __ldg(reinterpret_cast<const float4*>(row + v)) : make_float4(fill, fill, fill, fill);
+    }
+    return f;
+}
+
 // ---- pass 1 ----------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads) accept_stats_kernel(const AcceptArgs a) {
     __shared__ float sh_m[kThreads / 32], sh_s[kThreads / 32];
     const int c = blockIdx.x, row = blockIdx.y;
     const int b = row / a.R, k = row % a.R;
     const int v0 = c * a.chunk, v1 = min(v0 + a.chunk, a.V);
-    const float* z = a.z + (size_t)row * a.zs;
+    const bool draft = k < a.gamma;
+    const Frag fz = load_frag(a.z + (size_t)row * a.zs, v0, v1, -INFINITY);
+    Frag fd;
+    if (draft) fd = load_frag(a.d + (size_t)(b * a.gamma + k) * a.ds, v0, v1, -INFINITY);
     float mz = -INFINITY, sz = 0.f, md = -INFINITY, sd = 0.f;
-    for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
-        const float4 x = *reinterpret_cast<const float4*>(z + v);
-        online_add(mz, sz, x.x * a.inv_T_log2);
-        online_add(mz, sz, x.y * a.inv_T_log2);
-        online_add(mz, sz, x.z * a.inv_T_log2);
-        online_add(mz, sz, x.w * a.inv_T_log2);
+#pragma unroll
+    for (int e = 0; e < kPerThread; ++e) {
+        online_add(mz, sz, fz.x[e].x * a.inv_T_log2);
+        online_add(mz, sz, fz.x[e].y * a.inv_T_log2);
+        online_add(mz, sz, fz.x[e].z * a.inv_T_log2);
+        online_add(mz, sz, fz.x[e].w * a.inv_T_log2);
     }
-    if (k < a.gamma) {
-        const float* d = a.d + (size_t)(b * a.gamma + k) * a.ds;
-        for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
-            const float4 x = *reinterpret_cast<const float4*>(d + v);
-            online_add(md, sd, x.x * a.inv_T_log2);
-            online_add(md, sd, x.y * a.inv_T_log2);
-            online_add(md, sd, x.z * a.inv_T_log2);
-            online_add(md, sd, x.w * a.inv_T_log2);
+    if (draft) {
+#pragma unroll
+        for (int e = 0; e < kPerThread; ++e) {
+            online_add(md, sd, fd.x[e].x * a.inv_T_log2);
+            online_add(md, sd, fd.x[e].y * a.inv_T_log2);
+            online_add(md, sd, fd.x[e].z * a.inv_T_log2);
+            online_add(md, sd, fd.x[e].w * a.inv_T_log2);
         }
     }
     block_reduce_ms(mz, sz, sh_m, sh_s);
@@ -176,19 +201,19 @@ __global__ void __launch_bounds__(kThreads) accept_shift_stats_kernel(const Acce
     const int c = blockIdx.x, drow = blockIdx.y;  // drow over B*gamma
     const int b = drow / a.gamma, k = drow % a.gamma;
     const int row = b * a.R + k;
-    const RowStats r = load_row_stats(a, row, true);
     const int v0 = c * a.chunk, v1 = min(v0 + a.chunk, a.V);
-    const float* z = a.z + (size_t)row * a.zs;
-    const float* d = a.d + (size_t)drow * a.ds;
+    const Frag fz = load_frag(a.z + (size_t)row * a.zs, v0, v1, -INFINITY);
+    const Frag fd = load_frag(a.d + (size_t)drow * a.ds, v0, v1, -INFINITY);
+    const RowStats r = load_row_stats(a, row, true);
     float my = -INFINITY, sy = 0.f;
-    for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
-        const float4 x = *reinterpret_cast<const float4*>(z + v);
-        const float4 y = *reinterpret_cast<const float4*>(d + v);
+#pragma unroll
+    for (int e = 0; e < kPerThread; ++e) {
+        if (!fz.ok[e]) continue;
         float p, q;
-        online_add(my, sy, shifted_logit2(a, r, x.x, y.x, p, q));
-        online_add(my, sy, shifted_logit2(a, r, x.y, y.y, p, q));
-        online_add(my, sy, shifted_logit2(a, r, x.z, y.z, p, q));
-        online_add(my, sy, shifted_logit2(a, r, x.w, y.w, p, q));
+        online_add(my, sy, shifted_logit2(a, r, fz.x[e].x, fd.x[e].x, p, q));
+        online_add(my, sy, shifted_logit2(a, r, fz.x[e].y, fd.x[e].y, p, q));
+        online_add(my, sy, shifted_logit2(a, r, fz.x[e].z, fd.x[e].z, p, q));
+        online_add(my, sy, shifted_logit2(a, r, fz.x[e].w, fd.x[e].w, p, q));
     }
     block_reduce_ms(my, sy, sh_m, sh_s);
     if (threadIdx.x == 0) a.ystats[(size_t)drow * a.NCH + c] = make_float2(my, sy);
@@ -215,27 +240,29 @@ __global__ void __launch_bounds__(kThreads) accept_residual_kernel(const AcceptA
     const int c = blockIdx.x, row = blockIdx.y;
     const int b = row / a.R, k = row % a.R;
     const bool draft = k < a.gamma;
-    const RowStats r = load_row_stats(a, row, draft);
     const int v0 = c * a.chunk, v1 = min(v0 + a.chunk, a.V);
     const float* z = a.z + (size_t)row * a.zs;
+    const Frag fz = load_frag(z, v0, v1, -INFINITY);
     float sw = 0.f, sp = 0.f;
     if (draft) {
         const int drow = b * a.gamma + k;
-        const float* d = a.d + (size_t)drow * a.ds;
+        const Frag fd = load_frag(a.d + (size_t)drow * a.ds, v0, v1, -INFINITY);
+        int tok = a.tokens[drow];
+        const RowStats r = load_row_stats(a, row, true);
         const float* ys = reinterpret_cast<const float*>(a.ystats + (size_t)drow * a.NCH);
         float My, Sy;
         combine_ms(ys, ys + 1, a.NCH, 2, My, Sy);
         const float inv_Sy = 1.f / Sy;
-        int tok = a.tokens[drow];
         if (tok < 0 || tok >= a.V) {
             if (c == 0 && threadIdx.x == 0) atomicOr(a.status, RAPID_STATUS_BAD_DRAFT_TOKEN);
             tok = tok < 0 ? 0 : a.V - 1;
         }
-        for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
-            const float4 x = *reinterpret_cast<const float4*>(z + v);
-            const float4 y = *reinterpret_cast<const float4*>(d + v);
-            const float xs[4] = {x.x, x.y, x.z, x.w};
-            const float ys4[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int g = 0; g < kPerThread; ++g) {
+            if (!fz.ok[g]) continue;
+            const int v = v0 + (g * kThreads + threadIdx.x) * 4;
+            const float xs[4] = {fz.x[g].x, fz.x[g].y, fz.x[g].z, fz.x[g].w};
+            const float ys4[4] = {fd.x[g].x, fd.x[g].y, fd.x[g].z, fd.x[g].w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 float p, q, ph;
@@ -256,12 +283,14 @@ __global__ void __launch_bounds__(kThreads) accept_residual_kernel(const AcceptA
             }
         }
     } else {
-        for (int v = v0 + threadIdx.x * 4; v < v1; v += kThreads * 4) {
-            const float4 x = *reinterpret_cast<const float4*>(z + v);
-            sp += exp2f(x.x * a.inv_T_log2 - r.Mz) * r.inv_Sz;
-            sp += exp2f(x.y * a.inv_T_log2 - r.Mz) * r.inv_Sz;
-            sp += exp2f(x.z * a.inv_T_log2 - r.Mz) * r.inv_Sz;
-            sp += exp2f(x.w * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+        const RowStats r = load_row_stats(a, row, false);
+#pragma unroll
+        for (int g = 0; g < kPerThread; ++g) {
+            if (!fz.ok[g]) continue;
+            sp += exp2f(fz.x[g].x * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+            sp += exp2f(fz.x[g].y * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+            sp += exp2f(fz.x[g].z * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+            sp += exp2f(fz.x[g].w * a.inv_T_log2 - r.Mz) * r.inv_Sz;
         }
         sw = sp;
     }
@@ -271,14 +300,25 @@ __global__ void __launch_bounds__(kThreads) accept_residual_kernel(const AcceptA
 }
 
 // ---- pass 4 ----------------------------------------------------------------------------------
-// One CTA per sequence.  Thread t owns a run of consecutive entries of the chosen chunk so that
-// the prefix order inside the chunk is the vocabulary order.
+// One CTA per sequence.  The chunk holding the target mass is found by a warp scan over the chunk
+// sums; inside it thread t owns 12 consecutive entries, so the prefix order is the vocabulary order.
+__device__ __forceinline__ float warp_incl_scan(float v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
 __global__ void __launch_bounds__(kThreads) accept_select_kernel(const AcceptArgs a) {
-    __shared__ float sh_scan[kThreads];
+    __shared__ float sh_warp[kThreads / 32];
     __shared__ int sh_tok;
     __shared__ int sh_last;
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
 
     // number of leading accepted drafts
     int n = 0;
@@ -292,36 +332,32 @@ __global__ void __launch_bounds__(kThreads) accept_select_kernel(const AcceptArg
     const float u = a.uniforms[b * a.R + a.gamma];
     const float2* ws = a.wsums + (size_t)row * a.NCH;
 
-    float W = 0.f;
-    for (int c = 0; c < a.NCH; ++c) W += ws[c].x;
+    // chunk sums: lane c holds chunks c and c + 32 (every warp computes the same thing)
+    const float2 w0 = lane < a.NCH ? ws[lane] : make_float2(0.f, 0.f);
+    const float2 w1 = lane + 32 < a.NCH ? ws[lane + 32] : make_float2(0.f, 0.f);
     bool use_p = !draft;
+    float c0 = use_p ? w0.y : w0.x, c1 = use_p ? w1.y : w1.x;
+    float i0 = warp_incl_scan(c0);
+    float i1 = warp_incl_scan(c1) + __shfl_sync(0xffffffffu, i0, 31);
+    float W = __shfl_sync(0xffffffffu, i1, 31);
     if (!(W > 0.f) || !isfinite(W)) {  // empty residual: defined fallback, draw from p
+        if (!use_p && tid == 0) atomicOr(a.status, RAPID_STATUS_RESIDUAL_FALLBACK);
         use_p = true;
-        W = 0.f;
-        for (int c = 0; c < a.NCH; ++c) W += ws[c].y;
-        if (tid == 0) atomicOr(a.status, RAPID_STATUS_RESIDUAL_FALLBACK);
+        c0 = w0.y;
+        c1 = w1.y;
+        i0 = warp_incl_scan(c0);
+        i1 = warp_incl_scan(c1) + __shfl_sync(0xffffffffu, i0, 31);
+        W = __shfl_sync(0xffffffffu, i1, 31);
     }
     const float target = u * W;
-
-    // chunk that holds the target mass; if rounding leaves none, the last chunk with mass
-    int chunk = -1, last_pos = -1;
-    float before = 0.f, run = 0.f, before_last = 0.f;
-    for (int c = 0; c < a.NCH; ++c) {
-        const float wc = use_p ? ws[c].y : ws[c].x;
-        if (wc > 0.f) {
-            if (chunk < 0 && run + wc > target) {
-                chunk = c;
-                before = run;
-            }
-            last_pos = c;
-            before_last = run;
-            run += wc;
-        }
-    }
+    const unsigned hit0 = __ballot_sync(0xffffffffu, c0 > 0.f && i0 > target);
+    const unsigned hit1 = __ballot_sync(0xffffffffu, c1 > 0.f && i1 > target);
+    const unsigned pos0 = __ballot_sync(0xffffffffu, c0 > 0.f);
+    const unsigned pos1 = __ballot_sync(0xffffffffu, c1 > 0.f);
+    int chunk = hit0 ? __ffs(hit0) - 1 : (hit1 ? 32 + __ffs(hit1) - 1 : -1);
     bool want_last = false;
-    if (chunk < 0) {
-        chunk = last_pos;
-        before = before_last;
+    if (chunk < 0) {  // rounding left no chunk above the target: the last chunk with mass
+        chunk = pos1 ? 63 - __clz(pos1) : (pos0 ? 31 - __clz(pos0) : -1);
         want_last = true;
     }
     if (chunk < 0) {  // nothing has mass at all (non-finite logits): defined output
@@ -331,6 +367,10 @@ __global__ void __launch_bounds__(kThreads) accept_select_kernel(const AcceptArg
         }
         return;
     }
+    // mass before the chosen chunk = its inclusive prefix minus its own sum
+    const float incl = __shfl_sync(0xffffffffu, chunk < 32 ? i0 : i1, chunk & 31);
+    const float own = __shfl_sync(0xffffffffu, chunk < 32 ? c0 : c1, chunk & 31);
+    const float before = incl - own;
 
     const RowStats r = load_row_stats(a, row, draft);
     float My = 0.f, inv_Sy = 0.f;
@@ -345,36 +385,56 @@ __global__ void __launch_bounds__(kThreads) accept_select_kernel(const AcceptArg
         inv_Sy = 1.f / Sy;
     }
     const int v0 = chunk * a.chunk, v1 = min(v0 + a.chunk, a.V);
-    const int per = (((v1 - v0) + kThreads - 1) / kThreads + 3) & ~3;  // multiple of 4
-    const int t0 = v0 + tid * per, t1 = min(t0 + per, v1);
-
-    auto weight = [&](int v) -> float {
-        float p, q, ph;
-        if (draft) {
-            const float w = residual_weight(a, r, My, inv_Sy, z[v], d[v], p, q, ph);
-            return use_p ? p : w;
+    constexpr int PER = 4 * kPerThread;  // consecutive entries per thread
+    const int t0 = v0 + tid * PER;
+    float wv[PER];
+#pragma unroll
+    for (int g = 0; g < kPerThread; ++g) {
+        const int v = t0 + 4 * g;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
+        const bool ok = v < v1;
+        if (ok) {
+            x = __ldg(reinterpret_cast<const float4*>(z + v));
+            if (draft) y = __ldg(reinterpret_cast<const float4*>(d + v));
         }
-        return exp2f(z[v] * a.inv_T_log2 - r.Mz) * r.inv_Sz;
-    };
-
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+        const float ys4[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float w = 0.f;
+            if (ok) {
+                if (draft) {
+                    float p, q, ph;
+                    const float rw = residual_weight(a, r, My, inv_Sy, xs[e], ys4[e], p, q, ph);
+                    w = use_p ? p : rw;
+                } else {
+                    w = exp2f(xs[e] * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+                }
+            }
+            wv[4 * g + e] = w;
+        }
+    }
     float mine = 0.f;
-    for (int v = t0; v < t1; ++v) mine += weight(v);
-    sh_scan[tid] = mine;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) mine += wv[e];
+    // block-wide exclusive prefix of the per-thread sums, in thread order
+    const float incl_w = warp_incl_scan(mine);
     if (tid == 0) {
         sh_tok = 0x7fffffff;
         sh_last = -1;
     }
+    if (lane == 31) sh_warp[warp] = incl_w;
     __syncthreads();
-    float prefix = before;  // mass before this thread's run, summed in thread order
-    for (int t = 0; t < tid; ++t) prefix += sh_scan[t];
+    float cum = before;
+    for (int wdx = 0; wdx < warp; ++wdx) cum += sh_warp[wdx];
+    cum += incl_w - mine;
     int found = 0x7fffffff, last = -1;
-    float cum = prefix;
-    for (int v = t0; v < t1; ++v) {
-        const float w = weight(v);
-        if (w > 0.f) {
-            cum += w;
-            last = v;
-            if (!want_last && cum > target && found == 0x7fffffff) found = v;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) {
+        if (wv[e] > 0.f) {
+            cum += wv[e];
+            last = t0 + e;
+            if (!want_last && cum > target && found == 0x7fffffff) found = t0 + e;
         }
     }
     if (found != 0x7fffffff) atomicMin(&sh_tok, found);
@@ -382,19 +442,19 @@ __global__ void __launch_bounds__(kThreads) accept_select_kernel(const AcceptArg
     __syncthreads();
     if (tid == 0) {
         a.accept_len[b] = n;
-        const int tok = sh_tok != 0x7fffffff ? sh_tok : (sh_last >= 0 ? sh_last : v0);
-        a.next_token[b] = tok;
+        a.next_token[b] = sh_tok != 0x7fffffff ? sh_tok : (sh_last >= 0 ? sh_last : v0);
     }
 }
 
 bool accept_shape_ok(const rapid_accept_shape* s) {
-    return s && s->B > 0 && s->gamma >= 0 && s->V > 0 && s->V <= 0x7ffffff0LL &&
+    // a chunk holds at most kChunkMax entries and a row at most kMaxChunks chunks
+    return s && s->B > 0 && s->gamma >= 0 && s->V > 0 && s->V <= (int64_t)kMaxChunks * kChunkMax &&
            (int64_t)s->B * (s->gamma + 1) <= 65535;
 }
 
 int pick_chunks(int64_t V) {
-    // about 8K entries per chunk keeps every CTA at a few iterations of 256 x float4
-    int n = (int)((V + 8191) / 8192);
+    // about 2K entries per chunk: two float4 loads per thread and array, all in flight at once
+    int n = (int)((V + 2047) / 2048);
     return n < 1 ? 1 : (n > kMaxChunks ? kMaxChunks : n);
 }
 

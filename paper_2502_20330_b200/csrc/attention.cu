@@ -32,6 +32,11 @@ __host__ __device__ constexpr int tile_lanes(int MT) {
 }
 __host__ __device__ constexpr int num_stages(int D) { return D == 128 ? 6 : 12; }
 __host__ __device__ constexpr int stage_bytes(int D) { return 2 * kTile * D * 2; }
+// floats per partial slot: GR rows of D, then GR maxima and GR sums; a multiple of 4 so that
+// every row of every slot can be read with 16-byte loads
+__host__ __device__ constexpr long long slot_floats(int GR, int D) {
+    return ((long long)GR * (D + 2) + 3) / 4 * 4;
+}
 
 struct AttnArgs {
     const __nv_bfloat16* q;
@@ -191,7 +196,7 @@ verify_attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmK,
         const int gid = lane >> 2;
         const int tig = lane & 3;
         const int row0 = mt * 16 + gid;  // grouped rows of this thread: row0 and row0 + 8
-        const int slot_stride = a.GR * (D + 2);
+        const int slot_stride = (int)slot_floats(a.GR, D);
 
         int n = 0;
         bool ok = true;
@@ -372,17 +377,24 @@ verify_attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmK,
     if (tid == 0 && s_abort) atomicOr(a.status, RAPID_STATUS_PIPELINE_TIMEOUT);
 }
 
-// Merge: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the partials of a unit, in slot
-// order.  grid (GR, units), block D threads.
+// Merge: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the partials of a unit.
+// One block of 4 warps per (grouped row, unit): warp w takes the slots j = w, w+4, ... (four
+// loads in flight per lane), lanes span D; the four warp sums are added in warp order, so the
+// result does not depend on timing.
 template <int D>
-__global__ void __launch_bounds__(D)
+__global__ void __launch_bounds__(128)
 verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* lse_out,
                          float* out_f32) {
+    constexpr int VEC = D / 32;
+    constexpr int UN = 4;
+    __shared__ float sh_acc[4][D];
+    __shared__ float sh_l[4];
     const int m = blockIdx.x;
     const int unit = blockIdx.y;
     const int b = unit / a.Hkv;
     const int kvh = unit % a.Hkv;
-    const int d = threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
 
     long long T = 0, t0 = 0;
     int nt_b = 0;
@@ -397,31 +409,66 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     const long long nc = T < a.num_ctas ? T : a.num_ctas;
     const int c_first = (int)(((t0 + 1) * nc - 1) / T);
     const int c_last = (int)((t1 * nc - 1) / T);
-    const int slot_stride = a.GR * (D + 2);
+    const int nslots = (c_last - c_first + 1) * KS;
+    const size_t slot_stride = (size_t)slot_floats(a.GR, D);
+    const float* base = a.partial + (size_t)(c_first + unit) * KS * slot_stride;  // slots are consecutive
 
     float M = -INFINITY;
-    for (int c = c_first; c <= c_last; ++c)
-        for (int ks = 0; ks < KS; ++ks) {
-            const float* slot = a.partial + ((size_t)(c + unit) * KS + ks) * slot_stride;
-            M = fmaxf(M, slot[a.GR * D + m]);
+    for (int j = lane; j < nslots; j += 32) M = fmaxf(M, base[j * slot_stride + a.GR * D + m]);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+
+    float acc[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+    float lsum = 0.f;
+    for (int j0 = warp; j0 < nslots; j0 += 4 * UN) {
+        float wgt[UN], lv[UN], ov[UN][VEC];
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const int j = j0 + 4 * u;
+            const float* slot = base + (size_t)j * slot_stride;
+            const float ms = j < nslots ? slot[a.GR * D + m] : -INFINITY;
+            const bool live = ms != -INFINITY;  // an untouched slot holds no O: never read it
+            wgt[u] = live ? exp2f(ms - M) : 0.f;
+            lv[u] = live ? slot[a.GR * D + a.GR + m] : 0.f;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) ov[u][e] = 0.f;
+            if (live) {
+                if (VEC == 4) {
+                    const float4 t = *reinterpret_cast<const float4*>(slot + (size_t)m * D + lane * 4);
+                    ov[u][0] = t.x; ov[u][1] = t.y; ov[u][2] = t.z; ov[u][VEC - 1] = t.w;
+                } else {
+                    const float2 t = *reinterpret_cast<const float2*>(slot + (size_t)m * D + lane * 2);
+                    ov[u][0] = t.x; ov[u][1] = t.y;
+                }
+            }
         }
-    float acc = 0.f, lsum = 0.f;
-    for (int c = c_first; c <= c_last; ++c)
-        for (int ks = 0; ks < KS; ++ks) {
-            const float* slot = a.partial + ((size_t)(c + unit) * KS + ks) * slot_stride;
-            const float ms = slot[a.GR * D + m];
-            if (ms == -INFINITY) continue;
-            const float wgt = exp2f(ms - M);
-            lsum += wgt * slot[a.GR * D + a.GR + m];
-            acc += wgt * slot[(size_t)m * D + d];
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            lsum += wgt[u] * lv[u];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] += wgt[u] * ov[u][e];
         }
-    const float val = acc / lsum;
-    const int i = m / a.G;
-    const int g = m % a.G;
-    const size_t row = ((size_t)b * a.R + i) * a.Hq + (size_t)kvh * a.G + g;
-    out[row * D + d] = __float2bfloat16_rn(val);
-    if (out_f32) out_f32[row * D + d] = val;
-    if (lse_out && d == 0) lse_out[row] = (M + log2f(lsum)) * 0.69314718055994530942f;
+    }
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) sh_acc[warp][lane * VEC + e] = acc[e];
+    if (lane == 0) sh_l[warp] = lsum;
+    __syncthreads();
+    if (warp == 0) {
+        const float l = ((sh_l[0] + sh_l[1]) + sh_l[2]) + sh_l[3];
+        const int i = m / a.G;
+        const int g = m % a.G;
+        const size_t row = ((size_t)b * a.R + i) * a.Hq + (size_t)kvh * a.G + g;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            const int d = lane * VEC + e;
+            const float val = (((sh_acc[0][d] + sh_acc[1][d]) + sh_acc[2][d]) + sh_acc[3][d]) / l;
+            out[row * D + d] = __float2bfloat16_rn(val);
+            if (out_f32) out_f32[row * D + d] = val;
+        }
+        if (lse_out && lane == 0) lse_out[row] = (M + log2f(l)) * 0.69314718055994530942f;
+    }
 }
 
 // ---- host side ----------------------------------------------------------------------------
@@ -528,7 +575,7 @@ size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma) {
     if (GR > 128) return 0;
     const int MT = (int)((GR + 15) / 16);
     const int64_t slots = ((int64_t)kMaxCtas + (int64_t)s->B * s->Hkv) * tile_lanes(MT);
-    return kWorkspaceHeaderBytes + (size_t)slots * GR * (s->D + 2) * sizeof(float);
+    return kWorkspaceHeaderBytes + (size_t)slots * slot_floats((int)GR, s->D) * sizeof(float);
 }
 
 int launch_verify_attention(const void* q, const void* k_cache, const void* v_cache,
@@ -628,7 +675,7 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
         verify_attn_merge_kernel<128><<<grid, 128, 0, stream>>>(
             a, tile_lanes(MT), static_cast<__nv_bfloat16*>(out), lse, o32);
     else
-        verify_attn_merge_kernel<64><<<grid, 64, 0, stream>>>(
+        verify_attn_merge_kernel<64><<<grid, 128, 0, stream>>>(
             a, tile_lanes(MT), static_cast<__nv_bfloat16*>(out), lse, o32);
     RAPID_CUDA_CHECK(cudaGetLastError());
     count_launch(2);
