@@ -15,8 +15,10 @@
 // (max, sum, O).  Partials go to the workspace; the merge kernel combines them in a fixed
 // order, so results are bit-identical from run to run.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
+#include "tcgen05.cuh"
 
 namespace rapid {
 
@@ -377,6 +379,345 @@ verify_attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmK,
     if (tid == 0 && s_abort) atomicOr(a.status, RAPID_STATUS_PIPELINE_TIMEOUT);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Split-KV kernel on the 5th-generation tensor cores.
+//
+// Same work decomposition, TMA ring and partial format as above (one partial per CTA and unit),
+// but the two products run as tcgen05.mma with accumulators in tensor memory:
+//   S[128 x 64]  = Q[128 x D] K_tile^T      (A = Q, B = K tile, both K-major, 128-byte swizzle)
+//   O[128 x D]  += P[128 x 64] V_tile       (A = P from shared memory, B = V tile, MN-major)
+// The grouped rows sit on the M axis (rows >= GR hold whatever shared memory holds; MMA rows
+// are independent, so they only produce rows nobody reads).  Warp roles:
+//   warps 0-3  softmax: thread t owns TMEM lane t = grouped row t: reads its S row, keeps the
+//              running max / sum, writes bf16 P into shared memory, rescales its O row only when
+//              the max has grown by more than 2^8 (so P stays within bf16 range), and writes the
+//              partial at the end of a unit;
+//   warp 4     TMA producer for K/V tiles;
+//   warp 5     allocates tensor memory, loads Q by TMA, issues every MMA and commits them to the
+//              mbarriers that hand S, P, O and the K/V stages between the roles.
+// S and P are double-buffered, so the QK^T product of tile n+1 runs under the softmax of tile n.
+// A wait whose outcome is the same for every lane of the warp (needed because the warp goes on
+// to warp-collective TMEM instructions).
+__device__ __forceinline__ bool warp_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait_bounded(bar, parity, abort_flag));
+}
+
+constexpr int kTcThreads = 192;
+constexpr int kTcMaxStages = 8;
+constexpr float kRescaleSlack = 8.f;  // log2 units
+
+struct TcLayout {
+    int rows_pad;   // GR rounded up to 8
+    int nstage;     // K/V stages in the ring
+    int n_active;   // softmax warps that own at least one grouped row
+    uint32_t off_q, off_p0, off_p1, off_stage;  // bytes from the 1024-aligned base
+};
+
+template <int D>
+__global__ void __launch_bounds__(kTcThreads, 1)
+verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+                              const __grid_constant__ CUtensorMap tmV,
+                              const __grid_constant__ CUtensorMap tmQ, const AttnArgs a,
+                              const TcLayout lay) {
+    constexpr int STAGE = stage_bytes(D);
+    constexpr int HALF = kTile * 128;
+    constexpr int NHALF = D / 64;
+    constexpr uint32_t TMEM_COLS = 256;
+    constexpr uint32_t COL_S0 = 0, COL_S1 = 64, COL_O = 128;
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[kTcMaxStages];
+    __shared__ uint64_t empty_bar[kTcMaxStages];
+    __shared__ uint64_t s_full[2], p_full[2], pv_done[2];
+    __shared__ uint64_t q_full, o_free;
+    __shared__ uint32_t tmem_slot;
+    __shared__ Walk s_walk;
+    __shared__ int s_abort;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int cta = blockIdx.x;
+    const int nstage = lay.nstage;
+
+    if (tid == 0) {
+        for (int s = 0; s < nstage; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s_full[i], 1);
+            mbar_init(&p_full[i], lay.n_active);
+            mbar_init(&pv_done[i], 1);
+        }
+        mbar_init(&q_full, 1);
+        mbar_init(&o_free, lay.n_active);
+        fence_mbar_init();
+        s_abort = 0;
+        Walk w;
+        plan_cta(a, cta, w);
+        s_walk = w;
+        if (cta == 0) {
+            bool bad = false;
+            for (int b = 0; b < a.B; ++b) {
+                const int L = a.ctx_lens[b];
+                bad |= (L < a.R) || (L > a.Lmax);
+            }
+            if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
+        }
+    }
+    if (warp == 5) tmem_alloc(&tmem_slot, TMEM_COLS);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+    Walk w = s_walk;
+    volatile int* abort_flag = &s_abort;
+
+    if (warp == 4) {
+        // ---------------- TMA producer for K/V tiles ----------------
+        if (lane == 0) {
+            prefetch_tensormap(&tmK);
+            prefetch_tensormap(&tmV);
+            int n = 0;
+            bool ok = true;
+            while (w.remaining > 0 && ok) {
+                const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+                for (int t = 0; t < seg && ok; ++t, ++n) {
+                    const int s = n % nstage;
+                    if (n >= nstage)
+                        ok = mbar_wait_bounded(&empty_bar[s], ((n / nstage) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    uint8_t* dst = smem_gen + lay.off_stage + (size_t)s * STAGE;
+                    const int key0 = (w.tile + t) * kTile;
+                    mbar_arrive_expect_tx(&full_bar[s], STAGE);
+#pragma unroll
+                    for (int h = 0; h < NHALF; ++h) {
+                        tma_load_4d(dst + h * HALF, &tmK, &full_bar[s], h * 64, key0, w.kvh, w.b);
+                        tma_load_4d(dst + STAGE / 2 + h * HALF, &tmV, &full_bar[s], h * 64, key0,
+                                    w.kvh, w.b);
+                    }
+                }
+                walk_advance(a, w, seg);
+            }
+        }
+    } else if (warp == 5) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            prefetch_tensormap(&tmQ);
+            const uint32_t idesc_qk = umma_idesc_bf16(128, kTile, 0, 0);
+            const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
+            const uint32_t q_base = smem_base + lay.off_q;
+            const uint32_t qhalf = (uint32_t)lay.rows_pad * 128u;
+            const uint32_t p_base[2] = {smem_base + lay.off_p0, smem_base + lay.off_p1};
+            const uint32_t st_base = smem_base + lay.off_stage;
+            const uint32_t tS[2] = {tmem_base + COL_S0, tmem_base + COL_S1};
+            const uint32_t tO = tmem_base + COL_O;
+            bool ok = true;
+
+            auto issue_qk = [&](int n_) {
+                const uint32_t kb = st_base + (uint32_t)(n_ % nstage) * STAGE;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t half = kk >> 2, ko = (kk & 3) * 32;
+                    umma_bf16_ss(tS[n_ & 1], umma_smem_desc(q_base + half * qhalf + ko, 16, 1024),
+                                 umma_smem_desc(kb + half * HALF + ko, 16, 1024), idesc_qk, kk > 0);
+                }
+                umma_commit(&s_full[n_ & 1]);
+            };
+
+            int n = 0, seg_idx = 0;
+            while (w.remaining > 0 && ok) {
+                const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+                // the previous unit's O row has been read out and its MMAs have all completed
+                if (seg_idx > 0) ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, abort_flag);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&q_full, (uint32_t)a.GR * D * 2);
+#pragma unroll
+                for (int h = 0; h < NHALF; ++h)
+                    tma_load_4d(smem_gen + lay.off_q + h * qhalf, &tmQ, &q_full, h * 64, w.kvh * a.G,
+                                0, w.b);
+                ok = mbar_wait_bounded(&q_full, seg_idx & 1, abort_flag);
+                if (ok) ok = mbar_wait_bounded(&full_bar[n % nstage], (n / nstage) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                issue_qk(n);
+                for (int t = 0; t < seg && ok; ++t, ++n) {
+                    if (t + 1 < seg) {
+                        ok = mbar_wait_bounded(&full_bar[(n + 1) % nstage], ((n + 1) / nstage) & 1,
+                                               abort_flag);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_qk(n + 1);
+                    }
+                    ok = mbar_wait_bounded(&p_full[n & 1], (n >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t vb = st_base + (uint32_t)(n % nstage) * STAGE + STAGE / 2;
+#pragma unroll
+                    for (int kk = 0; kk < kTile / 16; ++kk)
+                        umma_bf16_ss(tO, umma_smem_desc(p_base[n & 1] + kk * 32, 16, 1024),
+                                     umma_smem_desc(vb + kk * 2048, HALF, 1024), idesc_pv,
+                                     (t > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(&empty_bar[n % nstage]);
+                    umma_commit(&pv_done[n & 1]);
+                }
+                walk_advance(a, w, seg);
+                ++seg_idx;
+            }
+        }
+    } else if (warp < lay.n_active) {
+        // ---------------- softmax warps: thread t owns grouped row t ----------------
+        const int row = tid;
+        const bool row_valid = row < a.GR;
+        const int i_row = row_valid ? row / a.G : 0;
+        const int g_row = row_valid ? row % a.G : 0;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const uint32_t tS[2] = {tmem_base + lane_base + COL_S0, tmem_base + lane_base + COL_S1};
+        const uint32_t tO = tmem_base + lane_base + COL_O;
+        uint8_t* p_gen[2] = {smem_gen + lay.off_p0, smem_gen + lay.off_p1};
+        const float c = a.scale_log2;
+        const int slot_stride = (int)slot_floats(a.GR, D);
+        (void)g_row;
+
+        int n = 0, seg_idx = 0;
+        bool ok = true;
+        while (w.remaining > 0 && ok) {
+            const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+            const int L = w.L;
+            const int lim = L - a.R + i_row;
+            float m_ref = -INFINITY, l_run = 0.f;
+
+            for (int t = 0; t < seg && ok; ++t, ++n) {
+                const int sb = n & 1;
+                const int key0 = (w.tile + t) * kTile;
+                ok = warp_wait_bounded(&s_full[sb], (n >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                uint32_t sr[2][32];
+                tmem_ld_x32(tS[sb], sr[0]);
+                tmem_ld_x32(tS[sb] + 32, sr[1]);
+                tmem_wait_ld();
+
+                if (key0 + kTile - 1 > L - a.R) {  // causal rows and the ragged end of the context
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int k = 0; k < 32; ++k)
+                            if (key0 + h * 32 + k > lim) sr[h][k] = __float_as_uint(-INFINITY);
+                }
+                float mx = -INFINITY;
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(sr[h][k]));
+                const float m_new = row_valid ? fmaxf(m_ref, mx * c) : m_ref;
+                const bool grow = row_valid && (m_new > m_ref + kRescaleSlack);
+                float factor = 1.f;
+                if (grow) {
+                    factor = fast_exp2(m_ref - m_new);
+                    l_run *= factor;
+                    m_ref = m_new;
+                }
+                // the P buffer of tile n-2 must have been consumed
+                if (n >= 2) ok = warp_wait_bounded(&pv_done[sb], ((n - 2) >> 1) & 1, abort_flag);
+                if (!ok) break;
+                if (t > 0 && __any_sync(0xffffffffu, grow)) {
+                    // O must be at rest (PV of tile n-1 complete) while its rows are rescaled
+                    ok = warp_wait_bounded(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int c4 = 0; c4 < D / 32; ++c4) {
+                        uint32_t orow[32];
+                        tmem_ld_x32(tO + 32 * c4, orow);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k = 0; k < 32; ++k)
+                            orow[k] = __float_as_uint(__uint_as_float(orow[k]) * factor);
+                        tmem_st_x32(tO + 32 * c4, orow);
+                    }
+                    tmem_wait_st();
+                }
+                const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
+                float sum = 0.f;
+                uint32_t pk[32];
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int k = 0; k < 32; k += 2) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[h][k]), c, -m_use));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[h][k + 1]), c, -m_use));
+                        sum += p0 + p1;
+                        pk[h * 16 + (k >> 1)] = pack_bf16x2(p0, p1);
+                    }
+                l_run += sum;
+                if (row < lay.rows_pad) {
+                    uint8_t* prow = p_gen[sb] + row * 128;
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch)
+                        *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) =
+                            make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+                }
+                if (key0 + kTile > L) {
+                    // V rows beyond the context may hold any bits: zero them so that 0 * row = 0
+                    const int first_bad = L - key0;
+                    uint8_t* vgen = smem_gen + lay.off_stage + (size_t)(n % nstage) * STAGE + STAGE / 2;
+                    const int chunks = (kTile - first_bad) * 8;
+                    for (int h = 0; h < NHALF; ++h)
+                        for (int ch = tid; ch < chunks; ch += lay.n_active * 32)
+                            *reinterpret_cast<uint4*>(vgen + h * HALF + first_bad * 128 + ch * 16) =
+                                make_uint4(0, 0, 0, 0);
+                }
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_full[sb]);
+            }
+            if (!ok) break;
+
+            // ---- end of the unit: read the O row out of tensor memory and emit the partial ----
+            ok = warp_wait_bounded(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int unit = w.b * a.Hkv + w.kvh;
+            float* slot = a.partial + (size_t)(cta + unit) * slot_stride;
+#pragma unroll
+            for (int c4 = 0; c4 < D / 32; ++c4) {
+                uint32_t orow[32];
+                tmem_ld_x32(tO + 32 * c4, orow);
+                tmem_wait_ld();
+                if (row_valid && m_ref != -INFINITY) {
+#pragma unroll
+                    for (int k = 0; k < 32; k += 4)
+                        *reinterpret_cast<uint4*>(slot + (size_t)row * D + 32 * c4 + k) =
+                            make_uint4(orow[k], orow[k + 1], orow[k + 2], orow[k + 3]);
+                }
+            }
+            if (row_valid) {
+                slot[a.GR * D + row] = m_ref;
+                slot[a.GR * D + a.GR + row] = l_run;
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&o_free);
+            walk_advance(a, w, seg);
+            ++seg_idx;
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+    if (tid == 0 && s_abort) atomicOr(a.status, RAPID_STATUS_PIPELINE_TIMEOUT);
+}
+
 // Merge: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the partials of a unit.
 // One block of 4 warps per (grouped row, unit): warp w takes the slots j = w, w+4, ... (four
 // loads in flight per lane), lanes span D; the four warp sums are added in warp order, so the
@@ -532,6 +873,66 @@ int launch_split(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs&
     return RAPID_OK;
 }
 
+int make_q_map(CUtensorMap* map, const void* q, const rapid_attn_shape& s, int G, int R) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) {
+        set_error("cuTensorMapEncodeTiled is not available from the CUDA driver");
+        return RAPID_ERR_CUDA;
+    }
+    // q [B, R, Hq, D]: a box of (64 columns, G heads, R rows) lands as G*R rows of 128 bytes,
+    // row index i*G + g: the grouped-row order the kernels use
+    cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.Hq, (cuuint64_t)R, (cuuint64_t)s.B};
+    cuuint64_t strides[3] = {(cuuint64_t)s.D * 2, (cuuint64_t)s.Hq * s.D * 2,
+                             (cuuint64_t)R * s.Hq * s.D * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)G, (cuuint32_t)R, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled (q) failed with CUresult %d", (int)r);
+        return RAPID_ERR_CUDA;
+    }
+    return RAPID_OK;
+}
+
+constexpr int kMaxSmemOptin = 232448 - 1024;  // 227 KB per CTA on sm_100, less the static barriers
+
+template <int D>
+int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
+                    const AttnArgs& a, cudaStream_t stream) {
+    TcLayout lay;
+    lay.rows_pad = (a.GR + 7) / 8 * 8;
+    lay.n_active = (a.GR + 31) / 32;
+    const uint32_t qbytes = (uint32_t)(D / 64) * lay.rows_pad * 128;
+    const uint32_t pbytes = (uint32_t)lay.rows_pad * 128;
+    lay.off_q = 0;
+    lay.off_p0 = qbytes;
+    lay.off_p1 = qbytes + pbytes;
+    lay.off_stage = qbytes + 2 * pbytes;
+    int nstage = (kMaxSmemOptin - 1024 - (int)lay.off_stage) / stage_bytes(D);
+    if (nstage > kTcMaxStages) nstage = kTcMaxStages;
+    lay.nstage = nstage;
+    // the MMAs read 128 rows of Q and P whatever GR is: those reads must stay inside the allocation
+    const int smem = (int)lay.off_stage + nstage * stage_bytes(D) + 1024;
+    if (nstage < 2 || (int)lay.off_p1 + 128 * 128 > smem - 1024) {
+        set_error("shared-memory layout does not fit");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    static bool configured[64] = {};
+    int dev = 0;
+    RAPID_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev >= 64 || !configured[dev]) {
+        RAPID_CUDA_CHECK(cudaFuncSetAttribute(verify_attn_splitkv_tc_kernel<D>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              kMaxSmemOptin));
+        if (dev < 64) configured[dev] = true;
+    }
+    verify_attn_splitkv_tc_kernel<D><<<a.num_ctas, kTcThreads, smem, stream>>>(tmK, tmV, tmQ, a, lay);
+    RAPID_CUDA_CHECK(cudaGetLastError());
+    return RAPID_OK;
+}
+
 template <int D>
 int dispatch_split(int MT, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
                    cudaStream_t stream) {
@@ -661,8 +1062,19 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     a.scale_log2 = scale * 1.4426950408889634f;
 
     const int MT = (GR + 15) / 16;
-    rc = s.D == 128 ? dispatch_split<128>(MT, tmK, tmV, a, stream)
-                    : dispatch_split<64>(MT, tmK, tmV, a, stream);
+    static const bool legacy = getenv("RAPID_ATTN_LEGACY") != nullptr;
+    int KS = 1;
+    if (legacy) {
+        KS = tile_lanes(MT);
+        rc = s.D == 128 ? dispatch_split<128>(MT, tmK, tmV, a, stream)
+                        : dispatch_split<64>(MT, tmK, tmV, a, stream);
+    } else {
+        CUtensorMap tmQ;
+        rc = make_q_map(&tmQ, q, s, G, R);
+        if (rc != RAPID_OK) return rc;
+        rc = s.D == 128 ? launch_split_tc<128>(tmK, tmV, tmQ, a, stream)
+                        : launch_split_tc<64>(tmK, tmV, tmQ, a, stream);
+    }
     if (rc != RAPID_OK) return rc;
 
     if (params && params->split_done_event)
@@ -673,10 +1085,10 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     float* o32 = params ? params->out_f32 : nullptr;
     if (s.D == 128)
         verify_attn_merge_kernel<128><<<grid, 128, 0, stream>>>(
-            a, tile_lanes(MT), static_cast<__nv_bfloat16*>(out), lse, o32);
+            a, KS, static_cast<__nv_bfloat16*>(out), lse, o32);
     else
         verify_attn_merge_kernel<64><<<grid, 128, 0, stream>>>(
-            a, tile_lanes(MT), static_cast<__nv_bfloat16*>(out), lse, o32);
+            a, KS, static_cast<__nv_bfloat16*>(out), lse, o32);
     RAPID_CUDA_CHECK(cudaGetLastError());
     count_launch(2);
     return RAPID_OK;
