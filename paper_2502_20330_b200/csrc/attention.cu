@@ -382,54 +382,70 @@ verify_attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmK,
 // ---------------------------------------------------------------------------------------------
 // Split-KV kernel on the 5th-generation tensor cores.
 //
-// Same work decomposition, TMA ring and partial format as above (one partial per CTA and unit),
-// but the two products run as tcgen05.mma with accumulators in tensor memory:
-//   S[128 x 64]  = Q[128 x D] K_tile^T      (A = Q, B = K tile, both K-major, 128-byte swizzle)
-//   O[128 x D]  += P[128 x 64] V_tile       (A = P from shared memory, B = V tile, MN-major)
-// The grouped rows sit on the M axis (rows >= GR hold whatever shared memory holds; MMA rows
-// are independent, so they only produce rows nobody reads).  Warp roles:
-//   warps 0-3  softmax: thread t owns TMEM lane t = grouped row t: reads its S row, keeps the
-//              running max / sum, writes bf16 P into shared memory, rescales its O row only when
-//              the max has grown by more than 2^8 (so P stays within bf16 range), and writes the
-//              partial at the end of a unit;
-//   warp 4     TMA producer for K/V tiles;
-//   warp 5     allocates tensor memory, loads Q by TMA, issues every MMA and commits them to the
-//              mbarriers that hand S, P, O and the K/V stages between the roles.
-// S and P are double-buffered, so the QK^T product of tile n+1 runs under the softmax of tile n.
+// Same work decomposition, TMA ring and partial format as above, but the two products run as
+// tcgen05.mma with accumulators in tensor memory:
+//   S[128 x 64]  = Q[128 x D] K_tile^T      (A = Q in tensor memory, B = K tile, K-major, 128-byte swizzle)
+//   O[128 x D]  += P[128 x 64] V_tile       (A = P in tensor memory, B = V tile, MN-major)
+// Both A operands live in tensor memory (Q is written there once per unit, P once per tile), so
+// shared memory carries nothing but the K/V stream: the tensor core reads each K and V tile once
+// and the ring takes all 227 KB.  The grouped rows sit on the M axis (rows >= GR hold whatever
+// tensor memory holds; MMA rows are independent, so they only produce rows nobody reads).
+//
+// Tiles alternate between two independent softmax streams (even and odd tiles of the CTA).
+// Each stream has its own S buffer, P buffer, O accumulator and running (reference, sum), and
+// emits its own partial, so the streams never exchange anything; the merge kernel sees two
+// partials per CTA and unit.  Warp roles (352 threads):
+//   warps 0-3  softmax of stream 0, warps 4-7 softmax of stream 1: a thread owns the TMEM lane
+//              (= grouped row) 32*(warp%4)+lane: reads its S row, turns it into bf16
+//              probabilities in tensor memory, keeps the running sum, and writes the partial at
+//              the end of a unit; stream 0 also writes the unit's Q rows into tensor memory;
+//   warp 8     TMA producer for K/V tiles;
+//   warp 9     allocates tensor memory and issues the QK^T MMAs;
+//   warp 10    issues the PV MMAs.  (Two issuing threads because a tcgen05.commit costs its
+//              thread about 200 cycles: one thread doing all of a tile's MMAs and commits
+//              would itself be the slowest stage.)
+// A K/V stage goes back to the producer when a softmax warp has seen the tile's PV complete.
+// While one stream works on tile n the tensor core computes QK^T of tile n+1 for the other.
+//
+// Softmax reference.  exp2(s*c - m_ref) is exact for any reference m_ref as long as nothing
+// overflows, so the row maximum is not tracked tile by tile: the reference is the maximum of
+// the stream's first tile and is moved (with a rescale of the O row and the sum) only when a
+// tile's probabilities sum above 2^16.
+//
 // A wait whose outcome is the same for every lane of the warp (needed because the warp goes on
 // to warp-collective TMEM instructions).
 __device__ __forceinline__ bool warp_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     return __all_sync(0xffffffffu, mbar_wait_bounded(bar, parity, abort_flag));
 }
 
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 352;
 constexpr int kTcMaxStages = 8;
-constexpr float kRescaleSlack = 8.f;  // log2 units
+constexpr float kSumLimit = 65536.f;  // a tile sum at or above this moves the softmax reference
 
 struct TcLayout {
-    int rows_pad;   // GR rounded up to 8
-    int nstage;     // K/V stages in the ring
-    int n_active;   // softmax warps that own at least one grouped row
-    uint32_t off_q, off_p0, off_p1, off_stage;  // bytes from the 1024-aligned base
+    int nstage;    // K/V stages in the ring
+    int n_active;  // softmax warps per stream that own at least one grouped row
 };
 
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
-                              const __grid_constant__ CUtensorMap tmV,
-                              const __grid_constant__ CUtensorMap tmQ, const AttnArgs a,
+                              const __grid_constant__ CUtensorMap tmV, const AttnArgs a,
                               const TcLayout lay) {
     constexpr int STAGE = stage_bytes(D);
     constexpr int HALF = kTile * 128;
     constexpr int NHALF = D / 64;
-    constexpr uint32_t TMEM_COLS = 256;
-    constexpr uint32_t COL_S0 = 0, COL_S1 = 64, COL_O = 128;
+    constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t COL_S = 0;    // S of stream s at COL_S + 64 s
+    constexpr uint32_t COL_O = 128;  // O of stream s at COL_O + 128 s
+    constexpr uint32_t COL_Q = 384;  // Q: D/2 columns of bf16 pairs
+    constexpr uint32_t COL_P = 448;  // P of stream s at COL_P + 32 s (64 keys = 32 columns)
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kTcMaxStages];
     __shared__ uint64_t empty_bar[kTcMaxStages];
     __shared__ uint64_t s_full[2], p_full[2], pv_done[2];
-    __shared__ uint64_t q_full, o_free;
+    __shared__ uint64_t q_ready, q_free, o_free;
     __shared__ uint32_t tmem_slot;
     __shared__ Walk s_walk;
     __shared__ int s_abort;
@@ -453,8 +469,9 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             mbar_init(&p_full[i], lay.n_active);
             mbar_init(&pv_done[i], 1);
         }
-        mbar_init(&q_full, 1);
-        mbar_init(&o_free, lay.n_active);
+        mbar_init(&q_ready, lay.n_active);
+        mbar_init(&q_free, 1);
+        mbar_init(&o_free, 2 * lay.n_active);
         fence_mbar_init();
         s_abort = 0;
         Walk w;
@@ -469,7 +486,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
         }
     }
-    if (warp == 5) tmem_alloc(&tmem_slot, TMEM_COLS);
+    if (warp == 9) tmem_alloc(&tmem_slot, TMEM_COLS);  // warp 9 also frees it at the end
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -477,7 +494,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
     Walk w = s_walk;
     volatile int* abort_flag = &s_abort;
 
-    if (warp == 4) {
+    if (warp == 8) {
         // ---------------- TMA producer for K/V tiles ----------------
         if (lane == 0) {
             prefetch_tensormap(&tmK);
@@ -491,7 +508,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                     if (n >= nstage)
                         ok = mbar_wait_bounded(&empty_bar[s], ((n / nstage) - 1) & 1, abort_flag);
                     if (!ok) break;
-                    uint8_t* dst = smem_gen + lay.off_stage + (size_t)s * STAGE;
+                    uint8_t* dst = smem_gen + (size_t)s * STAGE;
                     const int key0 = (w.tile + t) * kTile;
                     mbar_arrive_expect_tx(&full_bar[s], STAGE);
 #pragma unroll
@@ -504,102 +521,134 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 walk_advance(a, w, seg);
             }
         }
-    } else if (warp == 5) {
-        // ---------------- MMA issuer ----------------
+    } else if (warp == 9) {
+        // ---------------- QK^T issuer ----------------
         if (lane == 0) {
-            prefetch_tensormap(&tmQ);
             const uint32_t idesc_qk = umma_idesc_bf16(128, kTile, 0, 0);
-            const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
-            const uint32_t q_base = smem_base + lay.off_q;
-            const uint32_t qhalf = (uint32_t)lay.rows_pad * 128u;
-            const uint32_t p_base[2] = {smem_base + lay.off_p0, smem_base + lay.off_p1};
-            const uint32_t st_base = smem_base + lay.off_stage;
-            const uint32_t tS[2] = {tmem_base + COL_S0, tmem_base + COL_S1};
-            const uint32_t tO = tmem_base + COL_O;
+            // The descriptor is built once; per MMA only a small constant is added to the
+            // start-address field (every address stays below 256 KB: the field never carries).
+            const uint64_t k_desc = umma_smem_desc(smem_base, 16, 1024);
+            const uint32_t tQ = tmem_base + COL_Q;
             bool ok = true;
-
-            auto issue_qk = [&](int n_) {
-                const uint32_t kb = st_base + (uint32_t)(n_ % nstage) * STAGE;
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t half = kk >> 2, ko = (kk & 3) * 32;
-                    umma_bf16_ss(tS[n_ & 1], umma_smem_desc(q_base + half * qhalf + ko, 16, 1024),
-                                 umma_smem_desc(kb + half * HALF + ko, 16, 1024), idesc_qk, kk > 0);
-                }
-                umma_commit(&s_full[n_ & 1]);
-            };
-
             int n = 0, seg_idx = 0;
             while (w.remaining > 0 && ok) {
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
-                // the previous unit's O row has been read out and its MMAs have all completed
-                if (seg_idx > 0) ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, abort_flag);
-                if (!ok) break;
-                mbar_arrive_expect_tx(&q_full, (uint32_t)a.GR * D * 2);
-#pragma unroll
-                for (int h = 0; h < NHALF; ++h)
-                    tma_load_4d(smem_gen + lay.off_q + h * qhalf, &tmQ, &q_full, h * 64, w.kvh * a.G,
-                                0, w.b);
-                ok = mbar_wait_bounded(&q_full, seg_idx & 1, abort_flag);
-                if (ok) ok = mbar_wait_bounded(&full_bar[n % nstage], (n / nstage) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after_sync();
-                issue_qk(n);
+                // the previous unit's O rows have been read out, so all its MMAs have completed
+                // and the Q rows in tensor memory may be replaced: tell stream 0
+                if (seg_idx > 0) {
+                    ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    mbar_arrive(&q_free);
+                }
+                ok = mbar_wait_bounded(&q_ready, seg_idx & 1, abort_flag);
                 for (int t = 0; t < seg && ok; ++t, ++n) {
-                    if (t + 1 < seg) {
-                        ok = mbar_wait_bounded(&full_bar[(n + 1) % nstage], ((n + 1) / nstage) & 1,
-                                               abort_flag);
-                        if (!ok) break;
-                        tc_fence_after_sync();
-                        issue_qk(n + 1);
-                    }
-                    ok = mbar_wait_bounded(&p_full[n & 1], (n >> 1) & 1, abort_flag);
+                    ok = mbar_wait_bounded(&full_bar[n % nstage], (n / nstage) & 1, abort_flag);
+                    // S[n&1] is free once the stream has published the P of its previous tile
+                    if (ok && n >= 2) ok = mbar_wait_bounded(&p_full[n & 1], ((n - 2) >> 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t vb = st_base + (uint32_t)(n % nstage) * STAGE + STAGE / 2;
+                    const uint64_t kd = k_desc + (uint64_t)((uint32_t)(n % nstage) * (STAGE >> 4));
+                    const uint32_t d = tmem_base + COL_S + 64u * (n & 1);
 #pragma unroll
-                    for (int kk = 0; kk < kTile / 16; ++kk)
-                        umma_bf16_ss(tO, umma_smem_desc(p_base[n & 1] + kk * 32, 16, 1024),
-                                     umma_smem_desc(vb + kk * 2048, HALF, 1024), idesc_pv,
-                                     (t > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(&empty_bar[n % nstage]);
-                    umma_commit(&pv_done[n & 1]);
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t half = kk >> 2, ko16 = (kk & 3) * 2;
+                        umma_bf16_ts(d, tQ + 8 * kk, kd + half * (HALF >> 4) + ko16, idesc_qk, kk > 0);
+                    }
+                    umma_commit(&s_full[n & 1]);
                 }
                 walk_advance(a, w, seg);
                 ++seg_idx;
             }
         }
-    } else if (warp < lay.n_active) {
-        // ---------------- softmax warps: thread t owns grouped row t ----------------
-        const int row = tid;
+    } else if (warp == 10) {
+        // ---------------- PV issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
+            const uint64_t v_desc = umma_smem_desc(smem_base + STAGE / 2, HALF, 1024);
+            bool ok = true;
+            int n = 0;
+            while (w.remaining > 0 && ok) {
+                const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+                for (int t = 0; t < seg && ok; ++t, ++n) {
+                    // P(n) is published only after its stream has read the previous unit's O row
+                    ok = mbar_wait_bounded(&p_full[n & 1], (n >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint64_t vd = v_desc + (uint64_t)((uint32_t)(n % nstage) * (STAGE >> 4));
+                    const uint32_t tP = tmem_base + COL_P + 32u * (n & 1);
+                    const uint32_t d = tmem_base + COL_O + 128u * (n & 1);
+#pragma unroll
+                    for (int kk = 0; kk < kTile / 16; ++kk)
+                        umma_bf16_ts(d, tP + 8 * kk, vd + kk * (2048 >> 4), idesc_pv,
+                                     (t >= 2 || kk > 0) ? 1u : 0u);
+                    umma_commit(&pv_done[n & 1]);
+                }
+                walk_advance(a, w, seg);
+            }
+        }
+    } else if ((warp & 3) < lay.n_active) {
+        // ---------------- softmax warps: stream = warp / 4, grouped row = 32 (warp % 4) + lane ----------------
+        const int stream = warp >> 2;
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
         const bool row_valid = row < a.GR;
         const int i_row = row_valid ? row / a.G : 0;
-        const int g_row = row_valid ? row % a.G : 0;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        const uint32_t tS[2] = {tmem_base + lane_base + COL_S0, tmem_base + lane_base + COL_S1};
-        const uint32_t tO = tmem_base + lane_base + COL_O;
-        uint8_t* p_gen[2] = {smem_gen + lay.off_p0, smem_gen + lay.off_p1};
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const uint32_t tS = tmem_base + lane_base + COL_S + 64u * stream;
+        const uint32_t tO = tmem_base + lane_base + COL_O + 128u * stream;
+        const uint32_t tP = tmem_base + lane_base + COL_P + 32u * stream;
+        const uint32_t tQ = tmem_base + lane_base + COL_Q;
+        uint64_t* my_s_full = &s_full[stream];
+        uint64_t* my_p_full = &p_full[stream];
+        uint64_t* my_pv_done = &pv_done[stream];
         const float c = a.scale_log2;
         const int slot_stride = (int)slot_floats(a.GR, D);
-        (void)g_row;
 
-        int n = 0, seg_idx = 0;
+        int n0 = 0, seg_idx = 0;  // n0: CTA-wide index of the unit's first tile
+        int released = -1;        // latest tile of this stream whose K/V stage went back to the producer
         bool ok = true;
         while (w.remaining > 0 && ok) {
             const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
             const int L = w.L;
             const int lim = L - a.R + i_row;
             float m_ref = -INFINITY, l_run = 0.f;
+            int last_n = -1;  // the stream's latest tile of this unit (CTA-wide index)
 
-            for (int t = 0; t < seg && ok; ++t, ++n) {
-                const int sb = n & 1;
-                const int key0 = (w.tile + t) * kTile;
-                ok = warp_wait_bounded(&s_full[sb], (n >> 1) & 1, abort_flag);
+            if (stream == 0) {
+                // this unit's Q rows -> tensor memory (bf16 pairs, as they lie in global memory)
+                if (seg_idx > 0) ok = warp_wait_bounded(&q_free, (seg_idx - 1) & 1, abort_flag);
+                if (!ok) break;
+                const int g_row = row_valid ? row % a.G : 0;
+                const uint4* qrow = reinterpret_cast<const uint4*>(
+                    a.q + (((size_t)w.b * a.R + i_row) * a.Hq + (size_t)w.kvh * a.G + g_row) * D);
+#pragma unroll
+                for (int c4 = 0; c4 < D / 64; ++c4) {
+                    uint32_t qr[32];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const uint4 t4 = row_valid ? __ldg(qrow + c4 * 8 + k) : make_uint4(0, 0, 0, 0);
+                        qr[4 * k] = t4.x;
+                        qr[4 * k + 1] = t4.y;
+                        qr[4 * k + 2] = t4.z;
+                        qr[4 * k + 3] = t4.w;
+                    }
+                    tmem_st_x32(tQ + 32 * c4, qr);
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&q_ready);
+            }
+
+            for (int n = n0 + ((n0 ^ stream) & 1); n < n0 + seg && ok; n += 2) {
+                const int j = n >> 1;  // index of the tile within the stream
+                const int key0 = (w.tile + (n - n0)) * kTile;
+                ok = warp_wait_bounded(my_s_full, j & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
                 uint32_t sr[2][32];
-                tmem_ld_x32(tS[sb], sr[0]);
-                tmem_ld_x32(tS[sb] + 32, sr[1]);
+                tmem_ld_x32(tS, sr[0]);
+                tmem_ld_x32(tS + 32, sr[1]);
                 tmem_wait_ld();
 
                 if (key0 + kTile - 1 > L - a.R) {  // causal rows and the ragged end of the context
@@ -609,92 +658,116 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                         for (int k = 0; k < 32; ++k)
                             if (key0 + h * 32 + k > lim) sr[h][k] = __float_as_uint(-INFINITY);
                 }
-                float mx = -INFINITY;
+
+                uint32_t pk[32];
+                float sum = 0.f;
+                auto exponentials = [&](float m_use) {
+                    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
+                    for (int h = 0; h < 2; ++h)
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(sr[h][k]));
-                const float m_new = row_valid ? fmaxf(m_ref, mx * c) : m_ref;
-                const bool grow = row_valid && (m_new > m_ref + kRescaleSlack);
-                float factor = 1.f;
-                if (grow) {
-                    factor = fast_exp2(m_ref - m_new);
-                    l_run *= factor;
-                    m_ref = m_new;
+                        for (int k = 0; k < 32; k += 2) {
+                            const float p0 = fast_exp2(fmaf(__uint_as_float(sr[h][k]), c, -m_use));
+                            const float p1 = fast_exp2(fmaf(__uint_as_float(sr[h][k + 1]), c, -m_use));
+                            s0 += p0;
+                            s1 += p1;
+                            pk[h * 16 + (k >> 1)] = pack_bf16x2(p0, p1);
+                        }
+                    sum = s0 + s1;
+                };
+                const bool first = last_n < 0;
+                bool redo = row_valid && m_ref == -INFINITY;
+                if (!first) {
+                    exponentials(m_ref == -INFINITY ? 0.f : m_ref);
+                    redo = redo || (row_valid && !(sum < kSumLimit));
                 }
-                // the P buffer of tile n-2 must have been consumed
-                if (n >= 2) ok = warp_wait_bounded(&pv_done[sb], ((n - 2) >> 1) & 1, abort_flag);
-                if (!ok) break;
-                if (t > 0 && __any_sync(0xffffffffu, grow)) {
-                    // O must be at rest (PV of tile n-1 complete) while its rows are rescaled
-                    ok = warp_wait_bounded(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after_sync();
+                if (first || __any_sync(0xffffffffu, redo)) {
+                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int c4 = 0; c4 < D / 32; ++c4) {
-                        uint32_t orow[32];
-                        tmem_ld_x32(tO + 32 * c4, orow);
-                        tmem_wait_ld();
+                    for (int h = 0; h < 2; ++h)
 #pragma unroll
                         for (int k = 0; k < 32; ++k)
-                            orow[k] = __float_as_uint(__uint_as_float(orow[k]) * factor);
-                        tmem_st_x32(tO + 32 * c4, orow);
+                            mx[k & 3] = fmaxf(mx[k & 3], __uint_as_float(sr[h][k]));
+                    const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;
+                    float factor = 1.f;
+                    if (redo && tile_max > m_ref) {
+                        factor = fast_exp2(m_ref - tile_max);  // 0 when there was no reference yet
+                        l_run *= factor;
+                        m_ref = tile_max;
                     }
-                    tmem_wait_st();
+                    if (!first) {
+                        // O must be at rest (the stream's previous PV complete) while rows are rescaled
+                        ok = warp_wait_bounded(my_pv_done, (j - 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+#pragma unroll
+                        for (int c4 = 0; c4 < D / 32; ++c4) {
+                            uint32_t orow[32];
+                            tmem_ld_x32(tO + 32 * c4, orow);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int k = 0; k < 32; ++k)
+                                orow[k] = __float_as_uint(__uint_as_float(orow[k]) * factor);
+                            tmem_st_x32(tO + 32 * c4, orow);
+                        }
+                        tmem_wait_st();
+                    }
+                    exponentials(m_ref == -INFINITY ? 0.f : m_ref);
                 }
-                const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
-                float sum = 0.f;
-                uint32_t pk[32];
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int k = 0; k < 32; k += 2) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[h][k]), c, -m_use));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[h][k + 1]), c, -m_use));
-                        sum += p0 + p1;
-                        pk[h * 16 + (k >> 1)] = pack_bf16x2(p0, p1);
-                    }
                 l_run += sum;
-                if (row < lay.rows_pad) {
-                    uint8_t* prow = p_gen[sb] + row * 128;
-#pragma unroll
-                    for (int ch = 0; ch < 8; ++ch)
-                        *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) =
-                            make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+
+                // the stream's P buffer must have been consumed by its previous PV; that tile's
+                // K/V stage is then free for the producer
+                if (j >= 1) {
+                    ok = warp_wait_bounded(my_pv_done, (j - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    if (quad == 0 && lane == 0 && released < last_n) {
+                        mbar_arrive(&empty_bar[last_n % nstage]);
+                        released = last_n;
+                    }
                 }
+                tmem_st_x32(tP, pk);
                 if (key0 + kTile > L) {
                     // V rows beyond the context may hold any bits: zero them so that 0 * row = 0
                     const int first_bad = L - key0;
-                    uint8_t* vgen = smem_gen + lay.off_stage + (size_t)(n % nstage) * STAGE + STAGE / 2;
+                    uint8_t* vgen = smem_gen + (size_t)(n % nstage) * STAGE + STAGE / 2;
                     const int chunks = (kTile - first_bad) * 8;
                     for (int h = 0; h < NHALF; ++h)
-                        for (int ch = tid; ch < chunks; ch += lay.n_active * 32)
+                        for (int ch = row; ch < chunks; ch += lay.n_active * 32)
                             *reinterpret_cast<uint4*>(vgen + h * HALF + first_bad * 128 + ch * 16) =
                                 make_uint4(0, 0, 0, 0);
+                    fence_proxy_async_smem();
                 }
-                fence_proxy_async_smem();
+                tmem_wait_st();
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&p_full[sb]);
+                if (lane == 0) mbar_arrive(my_p_full);
+                last_n = n;
             }
             if (!ok) break;
 
             // ---- end of the unit: read the O row out of tensor memory and emit the partial ----
-            ok = warp_wait_bounded(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after_sync();
             const int unit = w.b * a.Hkv + w.kvh;
-            float* slot = a.partial + (size_t)(cta + unit) * slot_stride;
+            float* slot = a.partial + ((size_t)(cta + unit) * 2 + stream) * slot_stride;
+            if (last_n >= 0) {
+                ok = warp_wait_bounded(my_pv_done, (last_n >> 1) & 1, abort_flag);
+                if (!ok) break;
+                if (quad == 0 && lane == 0 && released < last_n) {
+                    mbar_arrive(&empty_bar[last_n % nstage]);
+                    released = last_n;
+                }
+                tc_fence_after_sync();
 #pragma unroll
-            for (int c4 = 0; c4 < D / 32; ++c4) {
-                uint32_t orow[32];
-                tmem_ld_x32(tO + 32 * c4, orow);
-                tmem_wait_ld();
-                if (row_valid && m_ref != -INFINITY) {
+                for (int c4 = 0; c4 < D / 32; ++c4) {
+                    uint32_t orow[32];
+                    tmem_ld_x32(tO + 32 * c4, orow);
+                    tmem_wait_ld();
+                    if (row_valid && m_ref != -INFINITY) {
 #pragma unroll
-                    for (int k = 0; k < 32; k += 4)
-                        *reinterpret_cast<uint4*>(slot + (size_t)row * D + 32 * c4 + k) =
-                            make_uint4(orow[k], orow[k + 1], orow[k + 2], orow[k + 3]);
+                        for (int k = 0; k < 32; k += 4)
+                            *reinterpret_cast<uint4*>(slot + (size_t)row * D + 32 * c4 + k) =
+                                make_uint4(orow[k], orow[k + 1], orow[k + 2], orow[k + 3]);
+                    }
                 }
             }
             if (row_valid) {
@@ -704,6 +777,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&o_free);
+            n0 += seg;
             walk_advance(a, w, seg);
             ++seg_idx;
         }
@@ -711,7 +785,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 9) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
@@ -873,52 +947,17 @@ int launch_split(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs&
     return RAPID_OK;
 }
 
-int make_q_map(CUtensorMap* map, const void* q, const rapid_attn_shape& s, int G, int R) {
-    EncodeTiledFn enc = get_encode_fn();
-    if (!enc) {
-        set_error("cuTensorMapEncodeTiled is not available from the CUDA driver");
-        return RAPID_ERR_CUDA;
-    }
-    // q [B, R, Hq, D]: a box of (64 columns, G heads, R rows) lands as G*R rows of 128 bytes,
-    // row index i*G + g: the grouped-row order the kernels use
-    cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.Hq, (cuuint64_t)R, (cuuint64_t)s.B};
-    cuuint64_t strides[3] = {(cuuint64_t)s.D * 2, (cuuint64_t)s.Hq * s.D * 2,
-                             (cuuint64_t)R * s.Hq * s.D * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)G, (cuuint32_t)R, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims, strides,
-                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        set_error("cuTensorMapEncodeTiled (q) failed with CUresult %d", (int)r);
-        return RAPID_ERR_CUDA;
-    }
-    return RAPID_OK;
-}
-
 constexpr int kMaxSmemOptin = 232448 - 1024;  // 227 KB per CTA on sm_100, less the static barriers
 
 template <int D>
-int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
-                    const AttnArgs& a, cudaStream_t stream) {
+int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
+                    cudaStream_t stream) {
     TcLayout lay;
-    lay.rows_pad = (a.GR + 7) / 8 * 8;
     lay.n_active = (a.GR + 31) / 32;
-    const uint32_t qbytes = (uint32_t)(D / 64) * lay.rows_pad * 128;
-    const uint32_t pbytes = (uint32_t)lay.rows_pad * 128;
-    lay.off_q = 0;
-    lay.off_p0 = qbytes;
-    lay.off_p1 = qbytes + pbytes;
-    lay.off_stage = qbytes + 2 * pbytes;
-    int nstage = (kMaxSmemOptin - 1024 - (int)lay.off_stage) / stage_bytes(D);
+    int nstage = (kMaxSmemOptin - 1024) / stage_bytes(D);
     if (nstage > kTcMaxStages) nstage = kTcMaxStages;
     lay.nstage = nstage;
-    // the MMAs read 128 rows of Q and P whatever GR is: those reads must stay inside the allocation
-    const int smem = (int)lay.off_stage + nstage * stage_bytes(D) + 1024;
-    if (nstage < 2 || (int)lay.off_p1 + 128 * 128 > smem - 1024) {
-        set_error("shared-memory layout does not fit");
-        return RAPID_ERR_UNSUPPORTED;
-    }
+    const int smem = nstage * stage_bytes(D) + 1024;
     static bool configured[64] = {};
     int dev = 0;
     RAPID_CUDA_CHECK(cudaGetDevice(&dev));
@@ -928,7 +967,7 @@ int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
                                               kMaxSmemOptin));
         if (dev < 64) configured[dev] = true;
     }
-    verify_attn_splitkv_tc_kernel<D><<<a.num_ctas, kTcThreads, smem, stream>>>(tmK, tmV, tmQ, a, lay);
+    verify_attn_splitkv_tc_kernel<D><<<a.num_ctas, kTcThreads, smem, stream>>>(tmK, tmV, a, lay);
     RAPID_CUDA_CHECK(cudaGetLastError());
     return RAPID_OK;
 }
@@ -975,7 +1014,8 @@ size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma) {
     const int64_t GR = (int64_t)(s->Hq / s->Hkv) * (gamma + 1);
     if (GR > 128) return 0;
     const int MT = (int)((GR + 15) / 16);
-    const int64_t slots = ((int64_t)kMaxCtas + (int64_t)s->B * s->Hkv) * tile_lanes(MT);
+    const int lanes = tile_lanes(MT) > 2 ? tile_lanes(MT) : 2;
+    const int64_t slots = ((int64_t)kMaxCtas + (int64_t)s->B * s->Hkv) * lanes;
     return kWorkspaceHeaderBytes + (size_t)slots * slot_floats((int)GR, s->D) * sizeof(float);
 }
 
@@ -1063,17 +1103,14 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
 
     const int MT = (GR + 15) / 16;
     static const bool legacy = getenv("RAPID_ATTN_LEGACY") != nullptr;
-    int KS = 1;
+    int KS = 2;  // the tensor-memory kernel emits one partial per softmax stream
     if (legacy) {
         KS = tile_lanes(MT);
         rc = s.D == 128 ? dispatch_split<128>(MT, tmK, tmV, a, stream)
                         : dispatch_split<64>(MT, tmK, tmV, a, stream);
     } else {
-        CUtensorMap tmQ;
-        rc = make_q_map(&tmQ, q, s, G, R);
-        if (rc != RAPID_OK) return rc;
-        rc = s.D == 128 ? launch_split_tc<128>(tmK, tmV, tmQ, a, stream)
-                        : launch_split_tc<64>(tmK, tmV, tmQ, a, stream);
+        rc = s.D == 128 ? launch_split_tc<128>(tmK, tmV, a, stream)
+                        : launch_split_tc<64>(tmK, tmV, a, stream);
     }
     if (rc != RAPID_OK) return rc;
 
