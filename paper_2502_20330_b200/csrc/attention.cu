@@ -382,35 +382,43 @@ verify_attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmK,
 // ---------------------------------------------------------------------------------------------
 // Split-KV kernel on the 5th-generation tensor cores.
 //
-// Same work decomposition, TMA ring and partial format as above, but the two products run as
-// tcgen05.mma with accumulators in tensor memory:
-//   S[128 x 64]  = Q[128 x D] K_tile^T      (A = Q in tensor memory, B = K tile, K-major, 128-byte swizzle)
-//   O[128 x D]  += P[128 x 64] V_tile       (A = P in tensor memory, B = V tile, MN-major)
-// Both A operands live in tensor memory (Q is written there once per unit, P once per tile), so
-// shared memory carries nothing but the K/V stream: the tensor core reads each K and V tile once
-// and the ring takes all 227 KB.  The grouped rows sit on the M axis (rows >= GR hold whatever
-// tensor memory holds; MMA rows are independent, so they only produce rows nobody reads).
+// Same work decomposition and partial format as above, but the two products run as tcgen05.mma
+// with accumulators in tensor memory (TMEM):
+//   S[128 x 128] = Q[128 x D] (K_n ; K_n+1)^T   two 64-key tiles per product: A = Q in shared
+//                                                memory, B = the two K tiles, K-major, 128-byte swizzle
+//   O[128 x D]  += P[128 x 64] V_tile            A = P in tensor memory, B = V tile, MN-major
+// The grouped rows sit on the M axis (rows >= GR hold whatever memory holds; MMA rows are
+// independent, so they only produce rows nobody reads).  A tcgen05.mma of 16 reduction steps
+// costs about as much for 64 columns as for 128, and every commit costs its issuing thread
+// about 200 cycles, so scores are produced for pairs of tiles: K tiles live in rings of their
+// own (one per 64-column half) in which consecutive stages are adjacent, which lets one
+// descriptor span the two tiles of a pair (pairs start at even tiles, stage counts are even).
 //
 // Tiles alternate between two independent softmax streams (even and odd tiles of the CTA).
-// Each stream has its own S buffer, P buffer, O accumulator and running (reference, sum), and
-// emits its own partial, so the streams never exchange anything; the merge kernel sees two
-// partials per CTA and unit.  Warp roles (352 threads):
+// Each stream has its own half of the S buffer, O accumulator and running (reference, sum) and
+// emits its own partial; the merge kernel sees two partials per CTA and unit.  Roles (352 threads):
 //   warps 0-3  softmax of stream 0, warps 4-7 softmax of stream 1: a thread owns the TMEM lane
-//              (= grouped row) 32*(warp%4)+lane: reads its S row, turns it into bf16
-//              probabilities in tensor memory, keeps the running sum, and writes the partial at
-//              the end of a unit; stream 0 also writes the unit's Q rows into tensor memory;
+//              (= grouped row) 32*(warp%4)+lane: reads its S row, writes the bf16 probabilities
+//              over the first half of the same columns, keeps the running sum, and writes the
+//              partial at the end of a unit;
 //   warp 8     TMA producer for K/V tiles;
-//   warp 9     allocates tensor memory and issues the QK^T MMAs;
-//   warp 10    issues the PV MMAs.  (Two issuing threads because a tcgen05.commit costs its
-//              thread about 200 cycles: one thread doing all of a tile's MMAs and commits
-//              would itself be the slowest stage.)
-// A K/V stage goes back to the producer when a softmax warp has seen the tile's PV complete.
-// While one stream works on tile n the tensor core computes QK^T of tile n+1 for the other.
+//   warp 9     allocates tensor memory, loads Q by TMA and issues the QK^T MMAs;
+//   warp 10    issues the PV MMAs; the commit of a tile's PV frees its K/V stage, and the same
+//              barrier tells everyone else that the PV is complete.
 //
 // Softmax reference.  exp2(s*c - m_ref) is exact for any reference m_ref as long as nothing
 // overflows, so the row maximum is not tracked tile by tile: the reference is the maximum of
 // the stream's first tile and is moved (with a rescale of the O row and the sum) only when a
 // tile's probabilities sum above 2^16.
+//
+// Barriers and phases.  Every mbarrier wait is a parity wait, which never returns if the
+// barrier gets a whole phase ahead of the waiter.  Each barrier below is therefore one whose
+// next phase cannot complete before all of its waiters have passed the current one:
+//   full/empty[stage]   producer <-> MMA issuers (empty is also the "PV of this tile done" signal;
+//                       with an even stage count a stage's next tile belongs to the same stream)
+//   s_full[b]           scores of group g (b = g & 1) ready; the buffer's next group needs the PVs
+//                       of this one, hence both streams past this wait
+//   p_full[b][h]        probabilities of the tile in half h of buffer b published
 //
 // A wait whose outcome is the same for every lane of the warp (needed because the warp goes on
 // to warp-collective TMEM instructions).
@@ -422,30 +430,56 @@ constexpr int kTcThreads = 352;
 constexpr int kTcMaxStages = 8;
 constexpr float kSumLimit = 65536.f;  // a tile sum at or above this moves the softmax reference
 
+// K/V stages in the rings (even; with the 128-row Q tile they fill the 227 KB of shared memory)
+__host__ __device__ constexpr int tc_stages(int D) { return D == 128 ? 6 : 8; }
+
 struct TcLayout {
-    int nstage;    // K/V stages in the ring
-    int n_active;  // softmax warps per stream that own at least one grouped row
+    int n_active;    // softmax warps per stream that own at least one grouped row
+    uint32_t off_q;  // byte offset of the Q tile (after the K/V rings) from the 1024-aligned base
 };
+
+// Where tile n of a unit lives.  A unit's tiles n0 .. n0+seg-1 (CTA-wide indices) are grouped for
+// the QK^T product: a leading single if n0 is odd, then pairs starting at even tiles, then a
+// trailing single.  `group` counts groups CTA-wide (g0 = count before this unit).
+struct TileSlot {
+    int group;  // CTA-wide group index: S buffer = group & 1, barrier phase = (group >> 1) & 1
+    int half;   // 0 or 1: which 64 columns of the buffer
+};
+__device__ __forceinline__ TileSlot tile_slot(int n, int n0, int g0) {
+    const int lead = n0 & 1;
+    TileSlot t;
+    if (n == n0 && lead) {
+        t.group = g0;
+        t.half = 0;
+    } else {
+        const int m = n - n0 - lead;
+        t.group = g0 + lead + (m >> 1);
+        t.half = m & 1;
+    }
+    return t;
+}
+__device__ __forceinline__ int groups_in_unit(int n0, int seg) {
+    const int lead = n0 & 1;
+    return lead + (seg - lead + 1) / 2;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
-                              const __grid_constant__ CUtensorMap tmV, const AttnArgs a,
+                              const __grid_constant__ CUtensorMap tmV,
+                              const __grid_constant__ CUtensorMap tmQ, const AttnArgs a,
                               const TcLayout lay) {
-    constexpr int STAGE = stage_bytes(D);
-    constexpr int HALF = kTile * 128;
+    constexpr int BLK = kTile * 128;  // bytes of one 64-key x 64-column block
     constexpr int NHALF = D / 64;
     constexpr uint32_t TMEM_COLS = 512;
-    constexpr uint32_t COL_S = 0;    // S of stream s at COL_S + 64 s
-    constexpr uint32_t COL_O = 128;  // O of stream s at COL_O + 128 s
-    constexpr uint32_t COL_Q = 384;  // Q: D/2 columns of bf16 pairs
-    constexpr uint32_t COL_P = 448;  // P of stream s at COL_P + 32 s (64 keys = 32 columns)
+    constexpr uint32_t COL_S = 0;    // S buffer b at COL_S + 128 b; tile in half h at + 64 h; P over its first 32 columns
+    constexpr uint32_t COL_O = 256;  // O of stream s at COL_O + 128 s
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kTcMaxStages];
     __shared__ uint64_t empty_bar[kTcMaxStages];
-    __shared__ uint64_t s_full[2], p_full[2], pv_done[2];
-    __shared__ uint64_t q_ready, q_free, o_free;
+    __shared__ uint64_t s_full[2], p_full[2][2];
+    __shared__ uint64_t q_full, o_free;
     __shared__ uint32_t tmem_slot;
     __shared__ Walk s_walk;
     __shared__ int s_abort;
@@ -457,7 +491,13 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
     const int warp = tid >> 5;
     const int lane = tid & 31;
     const int cta = blockIdx.x;
-    const int nstage = lay.nstage;
+    // The stage count is a compile-time constant: the roles below are single threads whose
+    // index arithmetic (tile -> stage, phase) would otherwise be runtime divisions, and those
+    // cost more than the MMAs they feed.
+    constexpr int nstage = tc_stages(D);
+    // shared-memory map: K rings (one per 64-column half), then V rings, then Q
+    const uint32_t ring = (uint32_t)nstage * BLK;  // bytes of one ring
+    const uint32_t off_k = 0, off_v = NHALF * ring;
 
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) {
@@ -466,11 +506,10 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&s_full[i], 1);
-            mbar_init(&p_full[i], lay.n_active);
-            mbar_init(&pv_done[i], 1);
+            mbar_init(&p_full[i][0], lay.n_active);
+            mbar_init(&p_full[i][1], lay.n_active);
         }
-        mbar_init(&q_ready, lay.n_active);
-        mbar_init(&q_free, 1);
+        mbar_init(&q_full, 1);
         mbar_init(&o_free, 2 * lay.n_active);
         fence_mbar_init();
         s_abort = 0;
@@ -508,53 +547,72 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                     if (n >= nstage)
                         ok = mbar_wait_bounded(&empty_bar[s], ((n / nstage) - 1) & 1, abort_flag);
                     if (!ok) break;
-                    uint8_t* dst = smem_gen + (size_t)s * STAGE;
                     const int key0 = (w.tile + t) * kTile;
-                    mbar_arrive_expect_tx(&full_bar[s], STAGE);
+                    mbar_arrive_expect_tx(&full_bar[s], 2 * NHALF * BLK);
 #pragma unroll
                     for (int h = 0; h < NHALF; ++h) {
-                        tma_load_4d(dst + h * HALF, &tmK, &full_bar[s], h * 64, key0, w.kvh, w.b);
-                        tma_load_4d(dst + STAGE / 2 + h * HALF, &tmV, &full_bar[s], h * 64, key0,
-                                    w.kvh, w.b);
+                        tma_load_4d(smem_gen + off_k + h * ring + s * BLK, &tmK, &full_bar[s], h * 64,
+                                    key0, w.kvh, w.b);
+                        tma_load_4d(smem_gen + off_v + h * ring + s * BLK, &tmV, &full_bar[s], h * 64,
+                                    key0, w.kvh, w.b);
                     }
                 }
                 walk_advance(a, w, seg);
             }
         }
     } else if (warp == 9) {
-        // ---------------- QK^T issuer ----------------
+        // ---------------- Q loader and QK^T issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc_qk = umma_idesc_bf16(128, kTile, 0, 0);
-            // The descriptor is built once; per MMA only a small constant is added to the
+            prefetch_tensormap(&tmQ);
+            const uint32_t idesc_1 = umma_idesc_bf16(128, kTile, 0, 0);
+            const uint32_t idesc_2 = umma_idesc_bf16(128, 2 * kTile, 0, 0);
+            // Descriptors are built once; per MMA only a small constant is added to the
             // start-address field (every address stays below 256 KB: the field never carries).
-            const uint64_t k_desc = umma_smem_desc(smem_base, 16, 1024);
-            const uint32_t tQ = tmem_base + COL_Q;
+            const uint64_t k_desc = umma_smem_desc(smem_base + off_k, 16, 1024);
+            const uint64_t q_desc = umma_smem_desc(smem_base + lay.off_q, 16, 1024);
+            constexpr uint32_t QHALF16 = (128 * 128) >> 4;  // one 64-column half of Q: 128 rows of 128 bytes
             bool ok = true;
-            int n = 0, seg_idx = 0;
+            int n = 0, g = 0, seg_idx = 0;
+            int prev_first[2] = {-1, -1}, prev_cnt[2] = {0, 0};  // tiles of the last group in each S buffer
             while (w.remaining > 0 && ok) {
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 // the previous unit's O rows have been read out, so all its MMAs have completed
-                // and the Q rows in tensor memory may be replaced: tell stream 0
-                if (seg_idx > 0) {
-                    ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    mbar_arrive(&q_free);
-                }
-                ok = mbar_wait_bounded(&q_ready, seg_idx & 1, abort_flag);
-                for (int t = 0; t < seg && ok; ++t, ++n) {
-                    ok = mbar_wait_bounded(&full_bar[n % nstage], (n / nstage) & 1, abort_flag);
-                    // S[n&1] is free once the stream has published the P of its previous tile
-                    if (ok && n >= 2) ok = mbar_wait_bounded(&p_full[n & 1], ((n - 2) >> 1) & 1, abort_flag);
+                // and Q may be replaced
+                if (seg_idx > 0) ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, abort_flag);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&q_full, (uint32_t)a.GR * D * 2);
+#pragma unroll
+                for (int h = 0; h < NHALF; ++h)
+                    tma_load_4d(smem_gen + lay.off_q + h * (128 * 128), &tmQ, &q_full, h * 64,
+                                w.kvh * a.G, 0, w.b);
+                ok = mbar_wait_bounded(&q_full, seg_idx & 1, abort_flag);
+                const int n_end = n + seg;
+                while (n < n_end && ok) {
+                    const int cnt = ((n & 1) || n + 1 >= n_end) ? 1 : 2;  // pairs start at even tiles
+                    const int b = g & 1;
+                    // the S buffer is free once the PVs of the group that used it last have completed
+                    for (int i = 0; i < prev_cnt[b] && ok; ++i) {
+                        const int pn = prev_first[b] + i;
+                        ok = mbar_wait_bounded(&empty_bar[pn % nstage], (pn / nstage) & 1, abort_flag);
+                    }
+                    for (int i = 0; i < cnt && ok; ++i)
+                        ok = mbar_wait_bounded(&full_bar[(n + i) % nstage], ((n + i) / nstage) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint64_t kd = k_desc + (uint64_t)((uint32_t)(n % nstage) * (STAGE >> 4));
-                    const uint32_t d = tmem_base + COL_S + 64u * (n & 1);
+                    const uint64_t kd = k_desc + (uint64_t)((uint32_t)(n % nstage) * (BLK >> 4));
+                    const uint32_t d = tmem_base + COL_S + 128u * b;
+                    const uint32_t idesc = cnt == 2 ? idesc_2 : idesc_1;
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
                         const uint32_t half = kk >> 2, ko16 = (kk & 3) * 2;
-                        umma_bf16_ts(d, tQ + 8 * kk, kd + half * (HALF >> 4) + ko16, idesc_qk, kk > 0);
+                        umma_bf16_ss(d, q_desc + half * QHALF16 + ko16, kd + half * (ring >> 4) + ko16, idesc,
+                                     kk > 0);
                     }
-                    umma_commit(&s_full[n & 1]);
+                    umma_commit(&s_full[b]);
+                    prev_first[b] = n;
+                    prev_cnt[b] = cnt;
+                    n += cnt;
+                    ++g;
                 }
                 walk_advance(a, w, seg);
                 ++seg_idx;
@@ -564,25 +622,34 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
         // ---------------- PV issuer ----------------
         if (lane == 0) {
             const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
-            const uint64_t v_desc = umma_smem_desc(smem_base + STAGE / 2, HALF, 1024);
+            // V tile as MN-major B: 64-column blocks `ring` bytes apart, 8-key groups 1024 bytes apart
+            const uint64_t v_desc = umma_smem_desc(smem_base + off_v, ring, 1024);
             bool ok = true;
-            int n = 0;
+            int n = 0, g0 = 0;
+            // p_full[b][0] completes one phase per group of buffer b, p_full[b][1] only for the
+            // groups that are pairs: its phase is counted here
+            int pairs_seen[2] = {0, 0};
             while (w.remaining > 0 && ok) {
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+                const int n0 = n;
                 for (int t = 0; t < seg && ok; ++t, ++n) {
+                    const TileSlot ts = tile_slot(n, n0, g0);
+                    const int b = ts.group & 1;
                     // P(n) is published only after its stream has read the previous unit's O row
-                    ok = mbar_wait_bounded(&p_full[n & 1], (n >> 1) & 1, abort_flag);
+                    const int phase = ts.half ? pairs_seen[b]++ : (ts.group >> 1);
+                    ok = mbar_wait_bounded(&p_full[b][ts.half], phase & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint64_t vd = v_desc + (uint64_t)((uint32_t)(n % nstage) * (STAGE >> 4));
-                    const uint32_t tP = tmem_base + COL_P + 32u * (n & 1);
+                    const uint64_t vd = v_desc + (uint64_t)((uint32_t)(n % nstage) * (BLK >> 4));
+                    const uint32_t tP = tmem_base + COL_S + 128u * b + 64u * ts.half;
                     const uint32_t d = tmem_base + COL_O + 128u * (n & 1);
 #pragma unroll
                     for (int kk = 0; kk < kTile / 16; ++kk)
                         umma_bf16_ts(d, tP + 8 * kk, vd + kk * (2048 >> 4), idesc_pv,
                                      (t >= 2 || kk > 0) ? 1u : 0u);
-                    umma_commit(&pv_done[n & 1]);
+                    umma_commit(&empty_bar[n % nstage]);  // PV(n) complete: stage free, P/S columns free
                 }
+                g0 += groups_in_unit(n0, seg);
                 walk_advance(a, w, seg);
             }
         }
@@ -594,18 +661,11 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
         const bool row_valid = row < a.GR;
         const int i_row = row_valid ? row / a.G : 0;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        const uint32_t tS = tmem_base + lane_base + COL_S + 64u * stream;
         const uint32_t tO = tmem_base + lane_base + COL_O + 128u * stream;
-        const uint32_t tP = tmem_base + lane_base + COL_P + 32u * stream;
-        const uint32_t tQ = tmem_base + lane_base + COL_Q;
-        uint64_t* my_s_full = &s_full[stream];
-        uint64_t* my_p_full = &p_full[stream];
-        uint64_t* my_pv_done = &pv_done[stream];
         const float c = a.scale_log2;
         const int slot_stride = (int)slot_floats(a.GR, D);
 
-        int n0 = 0, seg_idx = 0;  // n0: CTA-wide index of the unit's first tile
-        int released = -1;        // latest tile of this stream whose K/V stage went back to the producer
+        int n0 = 0, g0 = 0;  // CTA-wide tile / group index of the unit's first tile / group
         bool ok = true;
         while (w.remaining > 0 && ok) {
             const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
@@ -614,36 +674,11 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             float m_ref = -INFINITY, l_run = 0.f;
             int last_n = -1;  // the stream's latest tile of this unit (CTA-wide index)
 
-            if (stream == 0) {
-                // this unit's Q rows -> tensor memory (bf16 pairs, as they lie in global memory)
-                if (seg_idx > 0) ok = warp_wait_bounded(&q_free, (seg_idx - 1) & 1, abort_flag);
-                if (!ok) break;
-                const int g_row = row_valid ? row % a.G : 0;
-                const uint4* qrow = reinterpret_cast<const uint4*>(
-                    a.q + (((size_t)w.b * a.R + i_row) * a.Hq + (size_t)w.kvh * a.G + g_row) * D);
-#pragma unroll
-                for (int c4 = 0; c4 < D / 64; ++c4) {
-                    uint32_t qr[32];
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const uint4 t4 = row_valid ? __ldg(qrow + c4 * 8 + k) : make_uint4(0, 0, 0, 0);
-                        qr[4 * k] = t4.x;
-                        qr[4 * k + 1] = t4.y;
-                        qr[4 * k + 2] = t4.z;
-                        qr[4 * k + 3] = t4.w;
-                    }
-                    tmem_st_x32(tQ + 32 * c4, qr);
-                }
-                tmem_wait_st();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&q_ready);
-            }
-
             for (int n = n0 + ((n0 ^ stream) & 1); n < n0 + seg && ok; n += 2) {
-                const int j = n >> 1;  // index of the tile within the stream
                 const int key0 = (w.tile + (n - n0)) * kTile;
-                ok = warp_wait_bounded(my_s_full, j & 1, abort_flag);
+                const TileSlot ts = tile_slot(n, n0, g0);
+                const uint32_t tS = tmem_base + lane_base + COL_S + 128u * (ts.group & 1) + 64u * ts.half;
+                ok = warp_wait_bounded(&s_full[ts.group & 1], (ts.group >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
                 uint32_t sr[2][32];
@@ -697,7 +732,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                     }
                     if (!first) {
                         // O must be at rest (the stream's previous PV complete) while rows are rescaled
-                        ok = warp_wait_bounded(my_pv_done, (j - 1) & 1, abort_flag);
+                        ok = warp_wait_bounded(&empty_bar[last_n % nstage], (last_n / nstage) & 1, abort_flag);
                         if (!ok) break;
                         tc_fence_after_sync();
 #pragma unroll
@@ -716,32 +751,22 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 }
                 l_run += sum;
 
-                // the stream's P buffer must have been consumed by its previous PV; that tile's
-                // K/V stage is then free for the producer
-                if (j >= 1) {
-                    ok = warp_wait_bounded(my_pv_done, (j - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    if (quad == 0 && lane == 0 && released < last_n) {
-                        mbar_arrive(&empty_bar[last_n % nstage]);
-                        released = last_n;
-                    }
-                }
-                tmem_st_x32(tP, pk);
+                tmem_st_x32(tS, pk);  // P over the first half of the tile's own S columns
                 if (key0 + kTile > L) {
                     // V rows beyond the context may hold any bits: zero them so that 0 * row = 0
                     const int first_bad = L - key0;
-                    uint8_t* vgen = smem_gen + (size_t)(n % nstage) * STAGE + STAGE / 2;
                     const int chunks = (kTile - first_bad) * 8;
-                    for (int h = 0; h < NHALF; ++h)
+                    for (int h = 0; h < NHALF; ++h) {
+                        uint8_t* vgen = smem_gen + off_v + h * ring + (size_t)(n % nstage) * BLK;
                         for (int ch = row; ch < chunks; ch += lay.n_active * 32)
-                            *reinterpret_cast<uint4*>(vgen + h * HALF + first_bad * 128 + ch * 16) =
-                                make_uint4(0, 0, 0, 0);
+                            *reinterpret_cast<uint4*>(vgen + first_bad * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+                    }
                     fence_proxy_async_smem();
                 }
                 tmem_wait_st();
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(my_p_full);
+                if (lane == 0) mbar_arrive(&p_full[ts.group & 1][ts.half]);
                 last_n = n;
             }
             if (!ok) break;
@@ -750,12 +775,8 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             const int unit = w.b * a.Hkv + w.kvh;
             float* slot = a.partial + ((size_t)(cta + unit) * 2 + stream) * slot_stride;
             if (last_n >= 0) {
-                ok = warp_wait_bounded(my_pv_done, (last_n >> 1) & 1, abort_flag);
+                ok = warp_wait_bounded(&empty_bar[last_n % nstage], (last_n / nstage) & 1, abort_flag);
                 if (!ok) break;
-                if (quad == 0 && lane == 0 && released < last_n) {
-                    mbar_arrive(&empty_bar[last_n % nstage]);
-                    released = last_n;
-                }
                 tc_fence_after_sync();
 #pragma unroll
                 for (int c4 = 0; c4 < D / 32; ++c4) {
@@ -777,9 +798,9 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&o_free);
+            g0 += groups_in_unit(n0, seg);
             n0 += seg;
             walk_advance(a, w, seg);
-            ++seg_idx;
         }
     }
 
@@ -947,17 +968,42 @@ int launch_split(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs&
     return RAPID_OK;
 }
 
+int make_q_map(CUtensorMap* map, const void* q, const rapid_attn_shape& s, int G, int R) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) {
+        set_error("cuTensorMapEncodeTiled is not available from the CUDA driver");
+        return RAPID_ERR_CUDA;
+    }
+    // q [B, R, Hq, D]: a box of (64 columns, G heads, R rows) lands as G*R rows of 128 bytes,
+    // row index i*G + g: the grouped-row order the kernels use
+    cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.Hq, (cuuint64_t)R, (cuuint64_t)s.B};
+    cuuint64_t strides[3] = {(cuuint64_t)s.D * 2, (cuuint64_t)s.Hq * s.D * 2,
+                             (cuuint64_t)R * s.Hq * s.D * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)G, (cuuint32_t)R, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled (q) failed with CUresult %d", (int)r);
+        return RAPID_ERR_CUDA;
+    }
+    return RAPID_OK;
+}
+
 constexpr int kMaxSmemOptin = 232448 - 1024;  // 227 KB per CTA on sm_100, less the static barriers
 
 template <int D>
-int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
-                    cudaStream_t stream) {
+int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
+                    const AttnArgs& a, cudaStream_t stream) {
     TcLayout lay;
     lay.n_active = (a.GR + 31) / 32;
-    int nstage = (kMaxSmemOptin - 1024) / stage_bytes(D);
-    if (nstage > kTcMaxStages) nstage = kTcMaxStages;
-    lay.nstage = nstage;
-    const int smem = nstage * stage_bytes(D) + 1024;
+    const int qbytes = (D / 64) * 128 * 128;  // the MMAs read 128 rows of Q whatever GR is
+    constexpr int nstage = tc_stages(D);  // even: pairs of tiles sit in adjacent stages, no wrap
+    static_assert(nstage * stage_bytes(D) + (D / 64) * 128 * 128 + 1024 <= kMaxSmemOptin, "shared memory");
+    static_assert(nstage <= kTcMaxStages && nstage % 2 == 0, "stage count");
+    lay.off_q = (uint32_t)(nstage * stage_bytes(D));
+    const int smem = nstage * stage_bytes(D) + qbytes + 1024;
     static bool configured[64] = {};
     int dev = 0;
     RAPID_CUDA_CHECK(cudaGetDevice(&dev));
@@ -967,7 +1013,7 @@ int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnAr
                                               kMaxSmemOptin));
         if (dev < 64) configured[dev] = true;
     }
-    verify_attn_splitkv_tc_kernel<D><<<a.num_ctas, kTcThreads, smem, stream>>>(tmK, tmV, a, lay);
+    verify_attn_splitkv_tc_kernel<D><<<a.num_ctas, kTcThreads, smem, stream>>>(tmK, tmV, tmQ, a, lay);
     RAPID_CUDA_CHECK(cudaGetLastError());
     return RAPID_OK;
 }
@@ -1109,8 +1155,11 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
         rc = s.D == 128 ? dispatch_split<128>(MT, tmK, tmV, a, stream)
                         : dispatch_split<64>(MT, tmK, tmV, a, stream);
     } else {
-        rc = s.D == 128 ? launch_split_tc<128>(tmK, tmV, a, stream)
-                        : launch_split_tc<64>(tmK, tmV, a, stream);
+        CUtensorMap tmQ;
+        rc = make_q_map(&tmQ, q, s, G, R);
+        if (rc != RAPID_OK) return rc;
+        rc = s.D == 128 ? launch_split_tc<128>(tmK, tmV, tmQ, a, stream)
+                        : launch_split_tc<64>(tmK, tmV, tmQ, a, stream);
     }
     if (rc != RAPID_OK) return rc;
 
