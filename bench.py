@@ -261,9 +261,7 @@ def run_ours(args, cfg):
         step()
     barrier()
 
-    # timed region: K steps between two events on the launching stream; every layer of every
-    # step also gets an event pair around the split kernel
-    timed_pairs = [[(ev.create(), ev.create()) for _ in range(cfg.layers)] for _ in range(args.steps)]
+    # timed region: K steps between two events on the launching stream, nothing else on it
     e_begin, e_end = ev.create(), ev.create()
     sampler = ClockSampler(local_rank)
     R.kernel_launch_count_reset()
@@ -271,12 +269,20 @@ def run_ours(args, cfg):
     barrier()
     ev.record(e_begin, sptr)
     for s in range(args.steps):
-        step(timed_pairs[s])
+        step()
     ev.record(e_end, sptr)
     barrier()
-    clocks = sampler.stop()
     launches = R.kernel_launch_count()
     total_ms = ev.elapsed_ms(e_begin, e_end)
+    # second live pass for the roofline of the dominant kernel: the same steps with an event pair
+    # around every split kernel (the event between split and merge costs the pair their
+    # programmatic overlap, which is why this pass is not the one that gives `value`)
+    k_steps = min(args.steps, 20)
+    timed_pairs = [[(ev.create(), ev.create()) for _ in range(cfg.layers)] for _ in range(k_steps)]
+    for s in range(k_steps):
+        step(timed_pairs[s])
+    barrier()
+    clocks = sampler.stop()
     split_ms = [ev.elapsed_ms(a, b) for pairs in timed_pairs for (a, b) in pairs]
     status = R.workspace_status(aws) | R.workspace_status(cws)
 
@@ -315,8 +321,9 @@ def run_ours(args, cfg):
                               "split_kernel_per_layer": 1e3 * split_avg_ms,
                               "accept": 1e3 * float(np.median(acc_ms)), "step": 1e3 * ms_per_step},
         "frac_of_hbm_peak": {"measured": value / world / peak, "nominal_8TBs": value / world / 8000.0},
-        "roofline": {"bound": "hbm", "kernel": "verify_attn_splitkv_kernel", "achieved": achieved, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None},
+        "roofline": {"bound": "hbm", "kernel": "verify_attn_splitkv_tc_kernel", "achieved": achieved, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                     "timed": f"CUDA events around each of {len(split_ms)} launches in a second pass of {k_steps} steps"},
         "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
     }
 

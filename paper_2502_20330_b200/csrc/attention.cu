@@ -8,14 +8,12 @@
 // The G*R grouped query rows of a KV head (G = Hq/Hkv heads times R = gamma+1 draft rows) ride
 // together, so each K/V tile leaves HBM once.
 //
-// Inside a CTA one producer warp issues TMA tile loads (128-byte swizzle) into a ring of
-// shared-memory stages guarded by full/empty mbarriers; consumer warps are arranged as
-// MT row blocks (16 grouped rows each) x KS tile lanes: lane ks takes every KS-th tile, runs
-// QK^T and PV on the tensor cores with an fp32 online softmax, and keeps its own running
-// (max, sum, O).  Partials go to the workspace; the merge kernel combines them in a fixed
-// order, so results are bit-identical from run to run.
+// The split kernel (tcgen05 / tensor memory, described at its definition) writes fp32 partials
+// (unnormalised O, softmax reference, sum) to the workspace, two per CTA and unit (one per
+// softmax stream); the merge kernel combines them in a fixed order, so results are bit-identical
+// from run to run.  The merge is launched as a programmatic dependent of the split kernel: its
+// blocks are resident and have done their index arithmetic by the time the last partial lands.
 #include <math.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 #include "tcgen05.cuh"
@@ -26,13 +24,7 @@ namespace {
 
 constexpr int kTile = 64;  // keys per pipeline stage
 
-// Tile lanes per row-block count.  The lane that takes tile n also takes tile n + stages (the
-// stage count is a multiple of every lane count), so a lane never looks at a stage's barrier
-// before it has itself consumed that stage's previous fill: parity waits cannot alias.
-__host__ __device__ constexpr int tile_lanes(int MT) {
-    return MT == 1 ? 6 : MT <= 3 ? 3 : MT <= 5 ? 2 : 1;
-}
-__host__ __device__ constexpr int num_stages(int D) { return D == 128 ? 6 : 12; }
+constexpr int kStreams = 2;  // softmax streams per CTA = partials per CTA and unit
 __host__ __device__ constexpr int stage_bytes(int D) { return 2 * kTile * D * 2; }
 // floats per partial slot: GR rows of D, then GR maxima and GR sums; a multiple of 4 so that
 // every row of every slot can be read with 16-byte loads
@@ -114,269 +106,6 @@ __device__ __forceinline__ void walk_advance(const AttnArgs& a, Walk& w, int seg
             }
         }
     }
-}
-
-template <int D, int MT>
-__global__ void __launch_bounds__((MT * tile_lanes(MT) + 1) * 32, 1)
-verify_attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmK,
-                           const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
-    constexpr int KS = tile_lanes(MT);
-    constexpr int NSTAGE = num_stages(D);
-    constexpr int STAGE = stage_bytes(D);
-    constexpr int HALF = kTile * 128;  // bytes of one 64-column box
-    constexpr int NHALF = D / 64;
-    constexpr int KSTEPS = D / 16;
-
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[NSTAGE];
-    __shared__ uint64_t empty_bar[NSTAGE];
-    __shared__ Walk s_walk;
-    __shared__ int s_abort;
-
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-
-    const int tid = threadIdx.x;
-    const int warp = tid >> 5;
-    const int lane = tid & 31;
-    const int cta = blockIdx.x;
-
-    if (tid == 0) {
-        for (int s = 0; s < NSTAGE; ++s) {
-            mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], MT);
-        }
-        fence_mbar_init();
-        s_abort = 0;
-        Walk w;
-        plan_cta(a, cta, w);
-        s_walk = w;
-        if (cta == 0) {
-            bool bad = false;
-            for (int b = 0; b < a.B; ++b) {
-                const int L = a.ctx_lens[b];
-                bad |= (L < a.R) || (L > a.Lmax);
-            }
-            if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
-        }
-    }
-    __syncthreads();
-    Walk w = s_walk;
-    volatile int* abort_flag = &s_abort;
-
-    if (warp == MT * KS) {
-        // ---------------- producer warp: one lane issues the TMA loads ----------------
-        if (lane == 0) {
-            prefetch_tensormap(&tmK);
-            prefetch_tensormap(&tmV);
-            int n = 0;
-            bool ok = true;
-            while (w.remaining > 0 && ok) {
-                const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
-                for (int t = 0; t < seg && ok; ++t, ++n) {
-                    const int s = n % NSTAGE;
-                    if (n >= NSTAGE)
-                        ok = mbar_wait_bounded(&empty_bar[s], ((n / NSTAGE) - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    uint8_t* dst = smem_gen + (size_t)s * STAGE;
-                    const int key0 = (w.tile + t) * kTile;
-                    mbar_arrive_expect_tx(&full_bar[s], STAGE);
-#pragma unroll
-                    for (int h = 0; h < NHALF; ++h) {
-                        tma_load_4d(dst + h * HALF, &tmK, &full_bar[s], h * 64, key0, w.kvh, w.b);
-                        tma_load_4d(dst + STAGE / 2 + h * HALF, &tmV, &full_bar[s], h * 64, key0,
-                                    w.kvh, w.b);
-                    }
-                }
-                walk_advance(a, w, seg);
-            }
-        }
-    } else {
-        // ---------------- consumer warps ----------------
-        const int mt = warp % MT;
-        const int ks = warp / MT;
-        const int gid = lane >> 2;
-        const int tig = lane & 3;
-        const int row0 = mt * 16 + gid;  // grouped rows of this thread: row0 and row0 + 8
-        const int slot_stride = (int)slot_floats(a.GR, D);
-
-        int n = 0;
-        bool ok = true;
-        while (w.remaining > 0) {
-            const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
-            const int L = w.L;
-
-            // A fragments of Q for this row block: grouped row m = i*G + g (i draft row, g head)
-            uint32_t qf[KSTEPS][4];
-            int lim[2];
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const int m = row0 + 8 * r;
-                const bool valid = m < a.GR;
-                const int i = valid ? m / a.G : 0;
-                const int g = valid ? m % a.G : 0;
-                lim[r] = L - a.R + i;
-                const __nv_bfloat16* qrow =
-                    a.q + (((size_t)w.b * a.R + i) * a.Hq + (size_t)w.kvh * a.G + g) * D;
-#pragma unroll
-                for (int kk = 0; kk < KSTEPS; ++kk) {
-                    uint32_t lo = 0, hi = 0;
-                    if (valid) {
-                        lo = *reinterpret_cast<const uint32_t*>(qrow + kk * 16 + 2 * tig);
-                        hi = *reinterpret_cast<const uint32_t*>(qrow + kk * 16 + 8 + 2 * tig);
-                    }
-                    qf[kk][r] = lo;
-                    qf[kk][2 + r] = hi;
-                }
-            }
-
-            float o[D / 8][4];
-#pragma unroll
-            for (int j = 0; j < D / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
-            float mrow[2] = {-INFINITY, -INFINITY};
-            float lrow[2] = {0.f, 0.f};
-
-            for (int t = 0; t < seg; ++t, ++n) {
-                if (n % KS != ks) continue;
-                const int s = n % NSTAGE;
-                if (ok) ok = mbar_wait_bounded(&full_bar[s], (n / NSTAGE) & 1, abort_flag);
-                if (!ok) continue;
-                const uint32_t kbase = smem_base + s * STAGE;
-                const uint32_t vbase = kbase + STAGE / 2;
-                const int key0 = (w.tile + t) * kTile;
-
-                // rows of V beyond the context may hold any bits (NaN included): zero them so
-                // that a zero probability times that row is exactly zero
-                if (key0 + kTile > L) {
-                    const int first_bad = L - key0;
-                    uint8_t* vgen = smem_gen + (size_t)s * STAGE + STAGE / 2;
-                    const int chunks = (kTile - first_bad) * 8;  // 16-byte chunks per half
-                    for (int h = 0; h < NHALF; ++h)
-                        for (int c = lane; c < chunks; c += 32)
-                            *reinterpret_cast<uint4*>(vgen + h * HALF + first_bad * 128 + c * 16) =
-                                make_uint4(0, 0, 0, 0);
-                    __syncwarp();
-                }
-
-                // ---- S = Q K^T ----
-                float sc[kTile / 8][4];
-#pragma unroll
-                for (int j = 0; j < kTile / 8; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
-#pragma unroll
-                for (int kk = 0; kk < KSTEPS; kk += 2) {
-                    const int chunk = 2 * kk + (lane >> 3);  // 16-byte chunk along D
-                    const int half = chunk >> 3;
-                    const int cc = chunk & 7;
-#pragma unroll
-                    for (int j = 0; j < kTile / 8; ++j) {
-                        const int key = 8 * j + (lane & 7);
-                        const uint32_t addr =
-                            kbase + half * HALF + key * 128 + ((cc ^ (key & 7)) << 4);
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4(b0, b1, b2, b3, addr);
-                        mma_bf16_16816(sc[j], qf[kk], b0, b1);
-                        mma_bf16_16816(sc[j], qf[kk + 1], b2, b3);
-                    }
-                }
-
-                // ---- causal mask among the draft rows and the ragged end of the context ----
-                if (key0 + kTile - 1 > L - a.R) {
-#pragma unroll
-                    for (int j = 0; j < kTile / 8; ++j)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int key = key0 + 8 * j + 2 * tig + (e & 1);
-                            if (key > lim[e >> 1]) sc[j][e] = -INFINITY;
-                        }
-                }
-
-                // ---- online softmax (base 2) ----
-#pragma unroll
-                for (int r = 0; r < 2; ++r) {
-                    float mx = -INFINITY;
-#pragma unroll
-                    for (int j = 0; j < kTile / 8; ++j)
-                        mx = fmaxf(mx, fmaxf(sc[j][2 * r], sc[j][2 * r + 1]));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                    const float m_new = fmaxf(mrow[r], mx * a.scale_log2);
-                    const float m_safe = m_new == -INFINITY ? 0.f : m_new;
-                    const float corr = fast_exp2(mrow[r] - m_safe);
-                    mrow[r] = m_new;
-                    float sum = 0.f;
-#pragma unroll
-                    for (int j = 0; j < kTile / 8; ++j) {
-                        const float p0 = fast_exp2(fmaf(sc[j][2 * r], a.scale_log2, -m_safe));
-                        const float p1 = fast_exp2(fmaf(sc[j][2 * r + 1], a.scale_log2, -m_safe));
-                        sc[j][2 * r] = p0;
-                        sc[j][2 * r + 1] = p1;
-                        sum += p0 + p1;
-                    }
-                    lrow[r] = lrow[r] * corr + sum;
-#pragma unroll
-                    for (int j = 0; j < D / 8; ++j) {
-                        o[j][2 * r] *= corr;
-                        o[j][2 * r + 1] *= corr;
-                    }
-                }
-
-                // ---- O += P V ----
-#pragma unroll
-                for (int kk = 0; kk < kTile / 16; ++kk) {
-                    uint32_t pa[4];
-                    pa[0] = pack_bf16x2(sc[2 * kk][0], sc[2 * kk][1]);
-                    pa[1] = pack_bf16x2(sc[2 * kk][2], sc[2 * kk][3]);
-                    pa[2] = pack_bf16x2(sc[2 * kk + 1][0], sc[2 * kk + 1][1]);
-                    pa[3] = pack_bf16x2(sc[2 * kk + 1][2], sc[2 * kk + 1][3]);
-                    const int key = 16 * kk + ((lane >> 3) & 1) * 8 + (lane & 7);
-#pragma unroll
-                    for (int jn = 0; jn < D / 8; jn += 2) {
-                        const int chunk = jn + (lane >> 4);
-                        const int half = chunk >> 3;
-                        const int cc = chunk & 7;
-                        const uint32_t addr =
-                            vbase + half * HALF + key * 128 + ((cc ^ (key & 7)) << 4);
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4_trans(b0, b1, b2, b3, addr);
-                        mma_bf16_16816(o[jn], pa, b0, b1);
-                        mma_bf16_16816(o[jn + 1], pa, b2, b3);
-                    }
-                }
-
-                // hand the stage back to the producer
-                if (key0 + kTile > L) fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty_bar[s]);
-            }
-
-            // ---- write this warp's partial (unnormalised O, running max, running sum) ----
-            const int unit = w.b * a.Hkv + w.kvh;
-            float* slot = a.partial + ((size_t)(cta + unit) * KS + ks) * slot_stride;
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                float l = lrow[r];
-                l += __shfl_xor_sync(0xffffffffu, l, 1);
-                l += __shfl_xor_sync(0xffffffffu, l, 2);
-                const int m = row0 + 8 * r;
-                if (m < a.GR) {
-                    if (tig == 0) {
-                        slot[a.GR * D + m] = mrow[r];
-                        slot[a.GR * D + a.GR + m] = l;
-                    }
-                    if (mrow[r] != -INFINITY) {
-#pragma unroll
-                        for (int j = 0; j < D / 8; ++j)
-                            *reinterpret_cast<float2*>(slot + (size_t)m * D + 8 * j + 2 * tig) =
-                                make_float2(o[j][2 * r], o[j][2 * r + 1]);
-                    }
-                }
-            }
-            walk_advance(a, w, seg);
-        }
-    }
-
-    __syncthreads();
-    if (tid == 0 && s_abort) atomicOr(a.status, RAPID_STATUS_PIPELINE_TIMEOUT);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -525,6 +254,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
         }
     }
+    asm volatile("griddepcontrol.launch_dependents;");  // the merge blocks may take their seats
     if (warp == 9) tmem_alloc(&tmem_slot, TMEM_COLS);  // warp 9 also frees it at the end
     tc_fence_before_sync();
     __syncthreads();
@@ -822,7 +552,7 @@ __global__ void __launch_bounds__(128)
 verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* lse_out,
                          float* out_f32) {
     constexpr int VEC = D / 32;
-    constexpr int UN = 4;
+    constexpr int UN = 8;
     __shared__ float sh_acc[4][D];
     __shared__ float sh_l[4];
     const int m = blockIdx.x;
@@ -848,6 +578,9 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     const int nslots = (c_last - c_first + 1) * KS;
     const size_t slot_stride = (size_t)slot_floats(a.GR, D);
     const float* base = a.partial + (size_t)(c_first + unit) * KS * slot_stride;  // slots are consecutive
+
+    // everything above depends on the call's inputs only; the partials need the split kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     float M = -INFINITY;
     for (int j = lane; j < nslots; j += 32) M = fmaxf(M, base[j * slot_stride + a.GR * D + m]);
@@ -949,25 +682,6 @@ int make_kv_map(CUtensorMap* map, const void* base, const rapid_attn_shape& s, i
     return RAPID_OK;
 }
 
-template <int D, int MT>
-int launch_split(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
-                 cudaStream_t stream) {
-    constexpr int KS = tile_lanes(MT);
-    constexpr int threads = (MT * KS + 1) * 32;
-    constexpr int smem = num_stages(D) * stage_bytes(D) + 1024;
-    static bool configured[64] = {};
-    int dev = 0;
-    RAPID_CUDA_CHECK(cudaGetDevice(&dev));
-    if (dev >= 64 || !configured[dev]) {
-        RAPID_CUDA_CHECK(cudaFuncSetAttribute(verify_attn_splitkv_kernel<D, MT>,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        if (dev < 64) configured[dev] = true;
-    }
-    verify_attn_splitkv_kernel<D, MT><<<a.num_ctas, threads, smem, stream>>>(tmK, tmV, a);
-    RAPID_CUDA_CHECK(cudaGetLastError());
-    return RAPID_OK;
-}
-
 int make_q_map(CUtensorMap* map, const void* q, const rapid_attn_shape& s, int G, int R) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) {
@@ -1018,23 +732,6 @@ int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
     return RAPID_OK;
 }
 
-template <int D>
-int dispatch_split(int MT, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
-                   cudaStream_t stream) {
-    switch (MT) {
-        case 1: return launch_split<D, 1>(tmK, tmV, a, stream);
-        case 2: return launch_split<D, 2>(tmK, tmV, a, stream);
-        case 3: return launch_split<D, 3>(tmK, tmV, a, stream);
-        case 4: return launch_split<D, 4>(tmK, tmV, a, stream);
-        case 5: return launch_split<D, 5>(tmK, tmV, a, stream);
-        case 6: return launch_split<D, 6>(tmK, tmV, a, stream);
-        case 7: return launch_split<D, 7>(tmK, tmV, a, stream);
-        case 8: return launch_split<D, 8>(tmK, tmV, a, stream);
-    }
-    set_error("unsupported number of grouped rows");
-    return RAPID_ERR_UNSUPPORTED;
-}
-
 int sm_count() {
     static int n = 0;
     if (!n) {
@@ -1059,9 +756,7 @@ size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma) {
     if (s->D != 64 && s->D != 128) return 0;
     const int64_t GR = (int64_t)(s->Hq / s->Hkv) * (gamma + 1);
     if (GR > 128) return 0;
-    const int MT = (int)((GR + 15) / 16);
-    const int lanes = tile_lanes(MT) > 2 ? tile_lanes(MT) : 2;
-    const int64_t slots = ((int64_t)kMaxCtas + (int64_t)s->B * s->Hkv) * lanes;
+    const int64_t slots = ((int64_t)kMaxCtas + (int64_t)s->B * s->Hkv) * kStreams;
     return kWorkspaceHeaderBytes + (size_t)slots * slot_floats((int)GR, s->D) * sizeof(float);
 }
 
@@ -1147,20 +842,11 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     a.num_ctas = num_ctas;
     a.scale_log2 = scale * 1.4426950408889634f;
 
-    const int MT = (GR + 15) / 16;
-    static const bool legacy = getenv("RAPID_ATTN_LEGACY") != nullptr;
-    int KS = 2;  // the tensor-memory kernel emits one partial per softmax stream
-    if (legacy) {
-        KS = tile_lanes(MT);
-        rc = s.D == 128 ? dispatch_split<128>(MT, tmK, tmV, a, stream)
-                        : dispatch_split<64>(MT, tmK, tmV, a, stream);
-    } else {
-        CUtensorMap tmQ;
-        rc = make_q_map(&tmQ, q, s, G, R);
-        if (rc != RAPID_OK) return rc;
-        rc = s.D == 128 ? launch_split_tc<128>(tmK, tmV, tmQ, a, stream)
-                        : launch_split_tc<64>(tmK, tmV, tmQ, a, stream);
-    }
+    CUtensorMap tmQ;
+    rc = make_q_map(&tmQ, q, s, G, R);
+    if (rc != RAPID_OK) return rc;
+    rc = s.D == 128 ? launch_split_tc<128>(tmK, tmV, tmQ, a, stream)
+                    : launch_split_tc<64>(tmK, tmV, tmQ, a, stream);
     if (rc != RAPID_OK) return rc;
 
     if (params && params->split_done_event)
@@ -1169,13 +855,23 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     dim3 grid(GR, s.B * s.Hkv);
     float* lse = params ? params->lse_out : nullptr;
     float* o32 = params ? params->out_f32 : nullptr;
+    // programmatic dependent launch: the merge blocks start while the split kernel still runs and
+    // hold at their grid-dependency wait until its partials are complete and visible
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    __nv_bfloat16* out_bf = static_cast<__nv_bfloat16*>(out);
     if (s.D == 128)
-        verify_attn_merge_kernel<128><<<grid, 128, 0, stream>>>(
-            a, KS, static_cast<__nv_bfloat16*>(out), lse, o32);
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<128>, a, (int)kStreams, out_bf, lse, o32));
     else
-        verify_attn_merge_kernel<64><<<grid, 128, 0, stream>>>(
-            a, KS, static_cast<__nv_bfloat16*>(out), lse, o32);
-    RAPID_CUDA_CHECK(cudaGetLastError());
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<64>, a, (int)kStreams, out_bf, lse, o32));
     count_launch(2);
     return RAPID_OK;
 }
