@@ -55,6 +55,26 @@ def ncu_traffic(workload):
         return None
 
 
+def rank_seed(seed: int, rank: int) -> int:
+    """Every rank verifies its own requests (weak scaling, no exchange on the data path)."""
+    return int(seed) + 1000 * int(rank)
+
+
+def max_over_ranks(value: float, device="cpu") -> float:
+    """MAX all-reduce of a scalar over the default process group (identity without one)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput_gbs(bytes_per_rank_step: int, world: int, ms_per_step: float) -> float:
+    """Whole-job KV-read GB/s: all ranks' bytes over the slowest rank's step time."""
+    return bytes_per_rank_step * world / (ms_per_step * 1e-3) / 1e9
+
+
 def kv_bytes_per_layer(cfg, ctx) -> int:
     return int(4 * cfg.Hkv * cfg.D * int(ctx.sum()))
 
@@ -237,7 +257,7 @@ def run_ours(args, cfg):
         dist.init_process_group("nccl", device_id=dev)
 
     R.load_library()
-    seed = args.seed + 1000 * rank   # every rank verifies its own requests (weak scaling, no exchange)
+    seed = rank_seed(args.seed, rank)
     ctx_cpu = wl.context_lengths(cfg, seed)
     Lmax = wl.cache_capacity(cfg, ctx_cpu)
     layers = []
@@ -302,17 +322,39 @@ def run_ours(args, cfg):
     split_ms = [ev.elapsed_ms(a, b) for pairs in timed_pairs for (a, b) in pairs]
     status = R.workspace_status(aws) | R.workspace_status(cws)
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-
+    total_ms = max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = kv_step * world / (ms_per_step * 1e-3) / 1e9
+    value = job_throughput_gbs(kv_step, world, ms_per_step)
     peak, peak_kind = _peaks()
     split_avg_ms = float(np.mean(split_ms))
     achieved = kv_layer / (split_avg_ms * 1e-3) / 1e9
+
+    # the same step captured once in a CUDA graph and replayed (no per-call host work): what the
+    # GPU needs for a step when launch overhead is out of the picture
+    graph_us = None
+    try:
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for (q, k, v, out) in layers:
+                    R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws, stream=side)
+                R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params, stream=side)
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = min(args.steps, 20)
+        for _ in range(3):
+            g.replay()
+        g0.record()
+        for _ in range(reps):
+            g.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        graph_us = 1e3 * g0.elapsed_time(g1) / reps
+        del g
+    except Exception as exc:  # reported, never fatal: the direct calls above are the measurement
+        graph_us = f"unavailable: {exc}"
 
     # accept latency alone (events around the call, L2-warm rows by nature of the step)
     a0, a1 = ev.create(), ev.create()
@@ -335,7 +377,8 @@ def run_ours(args, cfg):
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
         "verify_latency_us": {"attention_per_layer": 1e3 * (ms_per_step - float(np.median(acc_ms))) / cfg.layers,
                               "split_kernel_per_layer": 1e3 * split_avg_ms,
-                              "accept": 1e3 * float(np.median(acc_ms)), "step": 1e3 * ms_per_step},
+                              "accept": 1e3 * float(np.median(acc_ms)), "step": 1e3 * ms_per_step,
+                              "step_cuda_graph_replay": graph_us},
         "frac_of_hbm_peak": {"measured": value / world / peak, "nominal_8TBs": value / world / 8000.0},
         "roofline": {"bound": "hbm", "kernel": "verify_attn_splitkv_tc_kernel", "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": ncu_traffic(cfg.name),

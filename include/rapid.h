@@ -233,7 +233,9 @@ int rapid_accept_static(const float* target_logits, const float* draft_logits,
  * stream, with no host synchronisation in between (Algorithm 1, one iteration
  * of the outer loop after drafting).  The projections and the LM head that turn
  * attention outputs into logits belong to the caller's model, so the logits are
- * inputs here.  Arguments are those of the two calls.
+ * inputs here.  Arguments are those of the two calls.  Because nothing in it
+ * touches the host, the chain can be captured in a CUDA graph and replayed
+ * (device pointers and shapes are frozen at capture; their contents are not).
  */
 int rapid_verify_step(const void* q, const void* k_cache, const void* v_cache,
                       const int32_t* ctx_lens, int gamma, void* out,

@@ -50,3 +50,39 @@ def test_verify_step_host_buffers():
         ref, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx.numpy(), cfg.gamma)
         parity.check_attention(out.float().numpy(), ref)
         parity.check_accept(z.numpy(), d.numpy(), tok.numpy(), u.numpy(), 5.0, 1.0, 0.1, 0, alen.numpy(), ntok.numpy())
+
+
+def test_verify_step_replays_from_a_cuda_graph():
+    """The chained step has no host synchronisation: it can be captured once and replayed."""
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("t", B=2, Hq=32, Hkv=8, D=128, gamma=8, V=32000, ctx_lens=(5000, 3000), target_sigma=1.0)
+    q, k, v, ctx, z, d, tok, u = _inputs(cfg, 23, "cuda")
+    aws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, k.shape[2], cfg.gamma))
+    cws = R.new_workspace(R.accept_workspace_bytes(cfg.B, cfg.gamma, cfg.V))
+    out = torch.zeros_like(q)
+    alen = torch.zeros(cfg.B, dtype=torch.int32, device="cuda"); ntok = torch.zeros_like(alen)
+    # eager reference
+    R.rapid_verify_step(q, k, v, ctx, cfg.gamma, out, aws, z, d, tok, u, 5.0, alen, ntok, cws)
+    torch.cuda.synchronize()
+    ref_out, ref_alen, ref_ntok = out.clone(), alen.clone(), ntok.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            R.rapid_verify_step(q, k, v, ctx, cfg.gamma, out, aws, z, d, tok, u, 5.0, alen, ntok, cws, stream=side)
+    for _ in range(3):
+        out.zero_(); alen.zero_(); ntok.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, ref_out) and torch.equal(alen, ref_alen) and torch.equal(ntok, ref_ntok)
+    # new inputs in the same buffers are picked up by the replay (pointers, not values, are captured)
+    q2, k2, v2, _, z2, d2, tok2, u2 = _inputs(cfg, 24, "cuda")
+    q.copy_(q2); k.copy_(k2); v.copy_(v2); z.copy_(z2); d.copy_(d2); tok.copy_(tok2); u.copy_(u2)
+    g.replay()
+    torch.cuda.synchronize()
+    ref, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx.cpu().numpy(), cfg.gamma)
+    parity.check_attention(out.float().cpu().numpy(), ref)
+    parity.check_accept(z.cpu().numpy(), d.cpu().numpy(), tok.cpu().numpy(), u.cpu().numpy(), 5.0, 1.0, 0.1, 0,
+                        alen.cpu().numpy(), ntok.cpu().numpy())
+    assert R.workspace_status(aws) == 0 and R.workspace_status(cws) == 0
