@@ -228,6 +228,8 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
     const uint32_t ring = (uint32_t)nstage * BLK;  // bytes of one ring
     const uint32_t off_k = 0, off_v = NHALF * ring;
 
+    // Prologue that touches no input: it may overlap the tail of whatever kernel precedes this
+    // one in the stream (the launch is a programmatic dependent).
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) {
             mbar_init(&full_bar[s], 1);
@@ -242,6 +244,16 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
         mbar_init(&o_free, 2 * lay.n_active);
         fence_mbar_init();
         s_abort = 0;
+        prefetch_tensormap(&tmK);
+        prefetch_tensormap(&tmV);
+        prefetch_tensormap(&tmQ);
+    }
+    if (warp == 9) tmem_alloc(&tmem_slot, TMEM_COLS);  // warp 9 also frees it at the end
+    // From here on inputs are read (and, much later, the workspace is written): the preceding
+    // kernel must have completed.  Then the merge blocks of this call may take their seats.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+    if (tid == 0) {
         Walk w;
         plan_cta(a, cta, w);
         s_walk = w;
@@ -254,8 +266,6 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
         }
     }
-    asm volatile("griddepcontrol.launch_dependents;");  // the merge blocks may take their seats
-    if (warp == 9) tmem_alloc(&tmem_slot, TMEM_COLS);  // warp 9 also frees it at the end
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -581,6 +591,7 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
 
     // everything above depends on the call's inputs only; the partials need the split kernel
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");  // a following dependent launch may begin its prologue
 
     float M = -INFINITY;
     for (int j = lane; j < nslots; j += 32) M = fmaxf(M, base[j * slot_stride + a.GR * D + m]);
@@ -727,8 +738,19 @@ int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
                                               kMaxSmemOptin));
         if (dev < 64) configured[dev] = true;
     }
-    verify_attn_splitkv_tc_kernel<D><<<a.num_ctas, kTcThreads, smem, stream>>>(tmK, tmV, tmQ, a, lay);
-    RAPID_CUDA_CHECK(cudaGetLastError());
+    // programmatic dependent launch: the kernel's input-free prologue may overlap the tail of the
+    // preceding kernel; it waits for that kernel's completion before it reads anything
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.num_ctas);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_splitkv_tc_kernel<D>, tmK, tmV, tmQ, a, lay));
     return RAPID_OK;
 }
 
