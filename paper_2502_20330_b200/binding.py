@@ -85,9 +85,14 @@ def load_library():
     global _lib
     if _lib is None:
         if not os.path.exists(_LIB_PATH):
-            raise RuntimeError(
-                f"{_LIB_PATH} is missing: build it with `python -m paper_2502_20330_b200.build` "
-                "(this package has no CPU or PyTorch fallback)")
+            # build in-tree with nvcc if the toolchain is here; otherwise fail loudly
+            try:
+                from . import build as _build
+                _build.build()
+            except Exception as exc:
+                raise RuntimeError(
+                    f"{_LIB_PATH} is missing and could not be built ({exc}): run "
+                    "`python -m paper_2502_20330_b200.build` (this package has no CPU or PyTorch fallback)")
         lib = ctypes.CDLL(_LIB_PATH)
         vp, i32, i64, sz, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t, ctypes.c_float
         lib.rapid_attention_workspace_bytes.restype = sz
