@@ -272,6 +272,34 @@ int rapid_verify_step_host(const void* h_q, const void* h_k_cache, const void* h
 size_t rapid_verify_step_host_arena_bytes(const rapid_attn_shape* attn_shape, int gamma,
                                           const rapid_accept_shape* accept_shape);
 
+/* ---- bookkeeping around the step --------------------------------------------------------------- */
+
+/*
+ * Appends the K/V rows of the R = gamma+1 newest tokens (the last accepted token and the gamma
+ * drafts x'_i .. x'_{i+gamma-1} of Algorithm 1) to every sequence's cache and counts them in
+ * ctx_lens, which is the state rapid_verify_attention expects.
+ *   k_new, v_new : device [B, R, Hkv, D] bf16, dense
+ *   k_cache, v_cache : device, geometry of `shape` (strides honoured)
+ *   ctx_lens : device int32 [B]; on entry the number of cached tokens, on exit that number + R
+ * A sequence whose cache cannot take R more rows (ctx_lens[b] + R > Lmax, or a negative length)
+ * is left untouched and sets RAPID_STATUS_BAD_CTX_LEN in *status_word.
+ *   status_word : device int32 (for instance the first word of an initialised workspace)
+ */
+int rapid_kv_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                    int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
+                    int32_t* status_word, void* cuda_stream);
+
+/*
+ * Closes a verify step (Algorithm 1: accepted drafts become x_j, the rest is discarded): of the R
+ * rows appended before the step the cache keeps the last accepted token and the accept_len[b]
+ * accepted drafts,  ctx_lens[b] -= gamma - accept_len[b].  (The token sampled by the step is
+ * appended, with the next drafts, by the next rapid_kv_append.)  accept_len outside [0, gamma]
+ * is clamped and sets RAPID_STATUS_BAD_CTX_LEN in *status_word.
+ *   ctx_lens : device int32 [B];  accept_len : device int32 [B] (rapid_accept's output)
+ */
+int rapid_step_commit(int32_t* ctx_lens, const int32_t* accept_len, int gamma, int B,
+                      int32_t* status_word, void* cuda_stream);
+
 /* ---- misc ------------------------------------------------------------------------------------ */
 
 /* Description of the last error on this thread ("" if none).  Never NULL. */

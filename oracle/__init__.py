@@ -185,3 +185,37 @@ def accept(target_logits, draft_logits, draft_tokens, uniforms, eta, T=1.0, tail
     if rc != 0:
         raise ValueError(f"oracle_accept failed with {rc}")
     return dict(accept_len=accept_len, next_token=next_token, flags=flags, ratios=ratios)
+
+
+def kv_append(k_cache, v_cache, k_new, v_new, ctx_lens, gamma):
+    """Bookkeeping before a verify step (Algorithm 1: the last accepted token and the gamma drafts join
+    the sequence the target scores): rows [L_b, L_b + R) of sequence b take k_new[b] / v_new[b]
+    ([B, R, Hkv, D] -> cache [B, Hkv, Lmax, D]) and L_b grows by R = gamma + 1.  A sequence without
+    room for R rows is left as it is.  Works on copies; returns (k_cache, v_cache, ctx_lens, overflowed)."""
+    k_cache = np.array(k_cache, copy=True)
+    v_cache = np.array(v_cache, copy=True)
+    ctx = np.array(ctx_lens, dtype=np.int64, copy=True)
+    R = gamma + 1
+    Lmax = k_cache.shape[2]
+    overflowed = False
+    for b in range(k_cache.shape[0]):
+        L = int(ctx[b])
+        if L < 0 or L + R > Lmax:
+            overflowed = True
+            continue
+        for i in range(R):
+            for h in range(k_cache.shape[1]):
+                k_cache[b, h, L + i, :] = k_new[b, i, h, :]
+                v_cache[b, h, L + i, :] = v_new[b, i, h, :]
+        ctx[b] = L + R
+    return k_cache, v_cache, ctx.astype(np.int32), overflowed
+
+
+def step_commit(ctx_lens, accept_len, gamma):
+    """Bookkeeping after a verify step (Algorithm 1: x_j <- x'_j for the accepted drafts, the others are
+    discarded): the cache keeps the last accepted token and the accepted drafts, L_b -= gamma - n_b."""
+    ctx = np.array(ctx_lens, dtype=np.int64, copy=True)
+    for b in range(ctx.size):
+        n = min(max(int(accept_len[b]), 0), gamma)
+        ctx[b] -= gamma - n
+    return ctx.astype(np.int32)

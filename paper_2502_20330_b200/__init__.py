@@ -18,6 +18,8 @@ from .binding import (  # noqa: F401
     new_workspace,
     rapid_accept,
     rapid_accept_static,
+    rapid_kv_append,
+    rapid_step_commit,
     rapid_verify_attention,
     rapid_verify_step,
     rapid_verify_step_host,

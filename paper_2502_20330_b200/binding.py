@@ -22,7 +22,8 @@ EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
     "rapid_workspace_status", "rapid_verify_attention", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
-    "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_last_error",
+    "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_step_commit",
+    "rapid_last_error",
     "rapid_version", "rapid_kernel_launch_count", "rapid_kernel_launch_count_reset",
 ]
 
@@ -117,6 +118,10 @@ def load_library():
         lib.rapid_verify_step_host.argtypes = attn_args + acc_args + [vp, sz, ctypes.POINTER(ctypes.c_int32), vp]
         lib.rapid_verify_step_host_arena_bytes.restype = sz
         lib.rapid_verify_step_host_arena_bytes.argtypes = [ctypes.POINTER(_AttnShape), i32, ctypes.POINTER(_AcceptShape)]
+        lib.rapid_kv_append.restype = i32
+        lib.rapid_kv_append.argtypes = [vp, vp, vp, vp, vp, i32, ctypes.POINTER(_AttnShape), vp, vp]
+        lib.rapid_step_commit.restype = i32
+        lib.rapid_step_commit.argtypes = [vp, vp, i32, i32, vp, vp]
         lib.rapid_last_error.restype = ctypes.c_char_p
         lib.rapid_version.restype = i32
         lib.rapid_kernel_launch_count.restype = i64
@@ -292,6 +297,28 @@ def rapid_verify_step(q, k_cache, v_cache, ctx_lens, gamma, out, attn_workspace,
         _p(target_logits), _p(draft_logits), _p(draft_tokens), _p(uniforms), float(eta), _p(out_accept_len),
         _p(out_next_token), ctypes.byref(cshape), _accept_params(accept_params), _p(accept_workspace),
         _nbytes(accept_workspace), _stream_ptr(stream)))
+
+
+def rapid_kv_append(k_new, v_new, k_cache, v_cache, ctx_lens, gamma, status_word, stream=None) -> None:
+    """Appends k_new/v_new [B, gamma+1, Hkv, D] (bf16) at ctx_lens and adds gamma+1 to ctx_lens (in place)."""
+    if k_new.dtype != torch.bfloat16 or v_new.dtype != torch.bfloat16 or ctx_lens.dtype != torch.int32:
+        raise TypeError("k_new/v_new must be bfloat16 and ctx_lens int32")
+    B, R, Hkv, D = k_new.shape
+    if R != gamma + 1 or not (k_new.is_contiguous() and v_new.is_contiguous()) or k_new.shape != v_new.shape:
+        raise ValueError("k_new and v_new must be dense [B, gamma+1, Hkv, D]")
+    if k_cache.stride() != v_cache.stride() or k_cache.shape != v_cache.shape or k_cache.stride(3) != 1:
+        raise ValueError("k_cache and v_cache must share shape and strides with a contiguous head_dim")
+    shape = _AttnShape(B, Hkv, Hkv, D, k_cache.shape[2], k_cache.stride(0), k_cache.stride(1), k_cache.stride(2))
+    _check(load_library().rapid_kv_append(_p(k_new), _p(v_new), _p(k_cache), _p(v_cache), _p(ctx_lens), gamma,
+                                          ctypes.byref(shape), _p(status_word), _stream_ptr(stream)))
+
+
+def rapid_step_commit(ctx_lens, accept_len, gamma, status_word, stream=None) -> None:
+    """ctx_lens[b] -= gamma - accept_len[b] (in place): drops the rejected drafts' rows from the cache."""
+    if ctx_lens.dtype != torch.int32 or accept_len.dtype != torch.int32:
+        raise TypeError("ctx_lens and accept_len must be int32")
+    _check(load_library().rapid_step_commit(_p(ctx_lens), _p(accept_len), gamma, ctx_lens.numel(),
+                                            _p(status_word), _stream_ptr(stream)))
 
 
 def rapid_verify_step_host(q, k_cache, v_cache, ctx_lens, gamma, out, target_logits, draft_logits, draft_tokens,

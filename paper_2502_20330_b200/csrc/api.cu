@@ -24,11 +24,106 @@ void count_launch(int n) { g_launches += n; }
 size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma);
 size_t accept_workspace_bytes(const rapid_accept_shape* s);
 
+namespace {
+
+// One block per (sequence, new row, KV head): copies D bf16 of K and of V into the cache.
+__global__ void kv_append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                                 __nv_bfloat16* k_cache, __nv_bfloat16* v_cache,
+                                 const int32_t* __restrict__ ctx_lens, int R, int Hkv, int D, long long Lmax,
+                                 long long sb, long long sh, long long sl, int32_t* status) {
+    const int b = blockIdx.z, i = blockIdx.y, h = blockIdx.x;
+    const long long L = ctx_lens[b];
+    if (L < 0 || L + R > Lmax) {
+        if (i == 0 && h == 0 && threadIdx.x == 0) atomicOr(status, RAPID_STATUS_BAD_CTX_LEN);
+        return;
+    }
+    const int chunks = D / 8;  // 16-byte chunks per row
+    const size_t src = (((size_t)b * R + i) * Hkv + h) * chunks;
+    const size_t dst = (size_t)b * sb + (size_t)h * sh + (size_t)(L + i) * sl;
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+        reinterpret_cast<uint4*>(k_cache + dst)[c] = k_new[src + c];
+        reinterpret_cast<uint4*>(v_cache + dst)[c] = v_new[src + c];
+    }
+}
+
+// Runs after the copies (same stream): ctx_lens[b] += R where the rows fitted.
+__global__ void kv_append_lens_kernel(int32_t* ctx_lens, int B, int R, long long Lmax) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const long long L = ctx_lens[b];
+    if (L >= 0 && L + R <= Lmax) ctx_lens[b] = (int32_t)(L + R);
+}
+
+__global__ void step_commit_kernel(int32_t* ctx_lens, const int32_t* __restrict__ accept_len, int gamma, int B,
+                                   int32_t* status) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int n = accept_len[b];
+    if (n < 0 || n > gamma) {
+        atomicOr(status, RAPID_STATUS_BAD_CTX_LEN);
+        n = n < 0 ? 0 : gamma;
+    }
+    ctx_lens[b] -= gamma - n;
+}
+
+}  // namespace
+
 }  // namespace rapid
 
 using namespace rapid;
 
 extern "C" {
+
+int rapid_kv_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                    int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
+                    int32_t* status_word, void* cuda_stream) {
+    clear_error();
+    if (!k_new || !v_new || !k_cache || !v_cache || !ctx_lens || !shape || !status_word) {
+        set_error("rapid_kv_append: NULL argument");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const rapid_attn_shape& s = *shape;
+    if (s.B <= 0 || s.Hkv <= 0 || s.Lmax <= 0 || gamma < 0 || s.B > 65535 || gamma + 1 > 65535) {
+        set_error("rapid_kv_append: invalid shape");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (s.D <= 0 || s.D % 8) {
+        set_error("rapid_kv_append: head_dim must be a positive multiple of 8");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const int64_t sl = s.kv_stride_l ? s.kv_stride_l : s.D;
+    const int64_t sh = s.kv_stride_h ? s.kv_stride_h : s.Lmax * sl;
+    const int64_t sb = s.kv_stride_b ? s.kv_stride_b : s.Hkv * sh;
+    if (sl % 8 || sh % 8 || sb % 8 ||
+        (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache) & 15)) {
+        set_error("rapid_kv_append: strides must be multiples of 8 elements and pointers 16-byte aligned");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const int R = gamma + 1;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    kv_append_kernel<<<dim3(s.Hkv, R, s.B), 32, 0, st>>>(
+        static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
+        static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache), ctx_lens, R, s.Hkv, s.D,
+        (long long)s.Lmax, (long long)sb, (long long)sh, (long long)sl, status_word);
+    kv_append_lens_kernel<<<(s.B + 127) / 128, 128, 0, st>>>(ctx_lens, s.B, R, (long long)s.Lmax);
+    RAPID_CUDA_CHECK(cudaGetLastError());
+    count_launch(2);
+    return RAPID_OK;
+}
+
+int rapid_step_commit(int32_t* ctx_lens, const int32_t* accept_len, int gamma, int B,
+                      int32_t* status_word, void* cuda_stream) {
+    clear_error();
+    if (!ctx_lens || !accept_len || !status_word || B <= 0 || gamma < 0) {
+        set_error("rapid_step_commit: invalid argument");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    step_commit_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        ctx_lens, accept_len, gamma, B, status_word);
+    RAPID_CUDA_CHECK(cudaGetLastError());
+    count_launch(1);
+    return RAPID_OK;
+}
 
 size_t rapid_attention_workspace_bytes(const rapid_attn_shape* shape, int gamma) {
     return attention_workspace_bytes(shape, gamma);
