@@ -161,3 +161,21 @@ def test_ragged_qwen_batch_sampled_rows():
     n_units = cfg.B * cfg.Hq * cfg.R
     units = np.arange(3, n_units, n_units // 9, dtype=np.int64)
     _compare(q, k, v, ctx, cfg.gamma, units=units)
+
+
+def test_random_shapes_and_lengths():
+    """Seeded sweep over head layouts, draft counts, ragged lengths and splits: every combination of
+    odd/even first tiles, single and paired tiles, short units and CTAs that straddle several units."""
+    rng = np.random.default_rng(123)
+    layouts = [(8, 2, 128), (4, 4, 64), (12, 2, 64), (16, 2, 128), (7, 7, 128), (32, 8, 128), (64, 8, 128)]
+    for trial in range(14):
+        Hq, Hkv, D = layouts[trial % len(layouts)]
+        G = Hq // Hkv
+        gamma = int(rng.integers(0, max(1, min(9, 128 // G))))
+        B = int(rng.integers(1, 5))
+        Lmax = int(rng.integers(gamma + 1, 1500))
+        lens = tuple(int(rng.integers(gamma + 1, Lmax + 1)) for _ in range(B))
+        cfg = wl.VerifyConfig("fz", B=B, Hq=Hq, Hkv=Hkv, D=D, gamma=gamma, V=4096, ctx_lens=lens, Lmax=Lmax)
+        q, k, v, ctx = wl.attention_inputs(cfg, seed=200 + trial, device="cuda", poison_padding=True)
+        num_ctas = int(rng.choice([0, 1, 3, 5, 16, 37, 148, 300]))
+        _compare(q, k, v, ctx, gamma, num_ctas=num_ctas)
