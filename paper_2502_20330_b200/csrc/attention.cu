@@ -192,7 +192,10 @@ __device__ __forceinline__ int groups_in_unit(int n0, int seg) {
     return lead + (seg - lead + 1) / 2;
 }
 
-template <int D>
+// MR = rows of the MMAs: 128, or 64 when the grouped rows fit (half the tensor-core work for the
+// same issue cost: less power, higher clocks under the board's power cap).  With 64 rows the
+// accumulator row r sits in TMEM lane 32*(r/16) + r%16: 16 lanes of each 32-lane quadrant.
+template <int D, int MR>
 __global__ void __launch_bounds__(kTcThreads, 1)
 verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                               const __grid_constant__ CUtensorMap tmV,
@@ -304,8 +307,8 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
         // ---------------- Q loader and QK^T issuer ----------------
         if (lane == 0) {
             prefetch_tensormap(&tmQ);
-            const uint32_t idesc_1 = umma_idesc_bf16(128, kTile, 0, 0);
-            const uint32_t idesc_2 = umma_idesc_bf16(128, 2 * kTile, 0, 0);
+            const uint32_t idesc_1 = umma_idesc_bf16(MR, kTile, 0, 0);
+            const uint32_t idesc_2 = umma_idesc_bf16(MR, 2 * kTile, 0, 0);
             // Descriptors are built once; per MMA only a small constant is added to the
             // start-address field (every address stays below 256 KB: the field never carries).
             const uint64_t k_desc = umma_smem_desc(smem_base + off_k, 16, 1024);
@@ -361,7 +364,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
     } else if (warp == 10) {
         // ---------------- PV issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
+            const uint32_t idesc_pv = umma_idesc_bf16(MR, D, 0, 1);
             // V tile as MN-major B: 64-column blocks `ring` bytes apart, 8-key groups 1024 bytes apart
             const uint64_t v_desc = umma_smem_desc(smem_base + off_v, ring, 1024);
             bool ok = true;
@@ -397,8 +400,10 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
         // ---------------- softmax warps: stream = warp / 4, grouped row = 32 (warp % 4) + lane ----------------
         const int stream = warp >> 2;
         const int quad = warp & 3;
-        const int row = quad * 32 + lane;
-        const bool row_valid = row < a.GR;
+        constexpr int RPQ = MR / 4;  // accumulator rows per 32-lane quadrant
+        const int row = quad * RPQ + lane;
+        const bool row_valid = lane < RPQ && row < a.GR;
+        const int sidx = quad * 32 + lane;  // thread index within the stream's warps
         const int i_row = row_valid ? row / a.G : 0;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const uint32_t tO = tmem_base + lane_base + COL_O + 128u * stream;
@@ -498,7 +503,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                     const int chunks = (kTile - first_bad) * 8;
                     for (int h = 0; h < NHALF; ++h) {
                         uint8_t* vgen = smem_gen + off_v + h * ring + (size_t)(n % nstage) * BLK;
-                        for (int ch = row; ch < chunks; ch += lay.n_active * 32)
+                        for (int ch = sidx; ch < chunks; ch += lay.n_active * 32)
                             *reinterpret_cast<uint4*>(vgen + first_bad * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
                     }
                     fence_proxy_async_smem();
@@ -718,11 +723,11 @@ int make_q_map(CUtensorMap* map, const void* q, const rapid_attn_shape& s, int G
 
 constexpr int kMaxSmemOptin = 232448 - 1024;  // 227 KB per CTA on sm_100, less the static barriers
 
-template <int D>
+template <int D, int MR>
 int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
                     const AttnArgs& a, cudaStream_t stream) {
     TcLayout lay;
-    lay.n_active = (a.GR + 31) / 32;
+    lay.n_active = (a.GR + MR / 4 - 1) / (MR / 4);
     const int qbytes = (D / 64) * 128 * 128;  // the MMAs read 128 rows of Q whatever GR is
     constexpr int nstage = tc_stages(D);  // even: pairs of tiles sit in adjacent stages, no wrap
     static_assert(nstage * stage_bytes(D) + (D / 64) * 128 * 128 + 1024 <= kMaxSmemOptin, "shared memory");
@@ -733,7 +738,7 @@ int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
     int dev = 0;
     RAPID_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev >= 64 || !configured[dev]) {
-        RAPID_CUDA_CHECK(cudaFuncSetAttribute(verify_attn_splitkv_tc_kernel<D>,
+        RAPID_CUDA_CHECK(cudaFuncSetAttribute(verify_attn_splitkv_tc_kernel<D, MR>,
                                               cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               kMaxSmemOptin));
         if (dev < 64) configured[dev] = true;
@@ -750,7 +755,7 @@ int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_splitkv_tc_kernel<D>, tmK, tmV, tmQ, a, lay));
+    RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_splitkv_tc_kernel<D, MR>, tmK, tmV, tmQ, a, lay));
     return RAPID_OK;
 }
 
@@ -867,8 +872,12 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     CUtensorMap tmQ;
     rc = make_q_map(&tmQ, q, s, G, R);
     if (rc != RAPID_OK) return rc;
-    rc = s.D == 128 ? launch_split_tc<128>(tmK, tmV, tmQ, a, stream)
-                    : launch_split_tc<64>(tmK, tmV, tmQ, a, stream);
+    if (GR <= 64)
+        rc = s.D == 128 ? launch_split_tc<128, 64>(tmK, tmV, tmQ, a, stream)
+                        : launch_split_tc<64, 64>(tmK, tmV, tmQ, a, stream);
+    else
+        rc = s.D == 128 ? launch_split_tc<128, 128>(tmK, tmV, tmQ, a, stream)
+                        : launch_split_tc<64, 128>(tmK, tmV, tmQ, a, stream);
     if (rc != RAPID_OK) return rc;
 
     if (params && params->split_done_event)
