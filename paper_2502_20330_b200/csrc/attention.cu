@@ -288,7 +288,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 for (int t = 0; t < seg && ok; ++t, ++n) {
                     const int s = n % nstage;
                     if (n >= nstage)
-                        ok = mbar_wait_bounded(&empty_bar[s], ((n / nstage) - 1) & 1, abort_flag);
+                        ok = mbar_wait_bounded_relaxed(&empty_bar[s], ((n / nstage) - 1) & 1, abort_flag);
                     if (!ok) break;
                     const int key0 = (w.tile + t) * kTile;
                     mbar_arrive_expect_tx(&full_bar[s], 2 * NHALF * BLK);

@@ -89,6 +89,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // timeout / abort.
 constexpr long long kWaitCycleLimit = 2000000000LL;
 
+// Same wait for a role that is not on the critical path (the TMA producer runs several stages
+// ahead): it sleeps between polls instead of spinning, which saves power for the clocks.
+__device__ __forceinline__ bool mbar_wait_bounded_relaxed(uint64_t* bar, uint32_t parity,
+                                                          volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        __nanosleep(200);
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycleLimit) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity,
                                                   volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
