@@ -142,6 +142,8 @@ __global__ void __launch_bounds__(kThreads) accept_stats_kernel(const AcceptArgs
     const int b = row / a.R, k = row % a.R;
     const int v0 = c * a.chunk, v1 = min(v0 + a.chunk, a.V);
     const bool draft = k < a.gamma;
+    griddep_wait();  // the logits may come from the kernel just before this one
+    griddep_launch_dependents();
     const Frag fz = load_frag(a.z + (size_t)row * a.zs, v0, v1, -INFINITY);
     Frag fd;
     if (draft) fd = load_frag(a.d + (size_t)(b * a.gamma + k) * a.ds, v0, v1, -INFINITY);
@@ -202,8 +204,12 @@ __global__ void __launch_bounds__(kThreads) accept_shift_stats_kernel(const Acce
     const int b = drow / a.gamma, k = drow % a.gamma;
     const int row = b * a.R + k;
     const int v0 = c * a.chunk, v1 = min(v0 + a.chunk, a.V);
+    // the logits are inputs of the call (pass 1 has waited for their producer): load them while
+    // pass 1 drains, then wait for its statistics
+    griddep_launch_dependents();
     const Frag fz = load_frag(a.z + (size_t)row * a.zs, v0, v1, -INFINITY);
     const Frag fd = load_frag(a.d + (size_t)drow * a.ds, v0, v1, -INFINITY);
+    griddep_wait();
     const RowStats r = load_row_stats(a, row, true);
     float my = -INFINITY, sy = 0.f;
 #pragma unroll
@@ -242,12 +248,14 @@ __global__ void __launch_bounds__(kThreads) accept_residual_kernel(const AcceptA
     const bool draft = k < a.gamma;
     const int v0 = c * a.chunk, v1 = min(v0 + a.chunk, a.V);
     const float* z = a.z + (size_t)row * a.zs;
+    griddep_launch_dependents();
     const Frag fz = load_frag(z, v0, v1, -INFINITY);
     float sw = 0.f, sp = 0.f;
     if (draft) {
         const int drow = b * a.gamma + k;
         const Frag fd = load_frag(a.d + (size_t)drow * a.ds, v0, v1, -INFINITY);
         int tok = a.tokens[drow];
+        griddep_wait();  // statistics of the earlier passes
         const RowStats r = load_row_stats(a, row, true);
         const float* ys = reinterpret_cast<const float*>(a.ystats + (size_t)drow * a.NCH);
         float My, Sy;
@@ -283,6 +291,7 @@ __global__ void __launch_bounds__(kThreads) accept_residual_kernel(const AcceptA
             }
         }
     } else {
+        griddep_wait();
         const RowStats r = load_row_stats(a, row, false);
 #pragma unroll
         for (int g = 0; g < kPerThread; ++g) {
@@ -319,6 +328,8 @@ __global__ void __launch_bounds__(kThreads) accept_select_kernel(const AcceptArg
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
+    griddep_wait();
+    griddep_launch_dependents();
 
     // number of leading accepted drafts
     int n = 0;
@@ -542,16 +553,18 @@ int launch_accept(const float* target_logits, const float* draft_logits,
     a.mode = mode;
 
     int launches = 0;
-    accept_stats_kernel<<<dim3(a.NCH, (unsigned)rows), kThreads, 0, stream>>>(a);
+    // every pass is a programmatic dependent of the one before: it loads its logits while its
+    // predecessor drains and waits for the predecessor's statistics only then
+    RAPID_CUDA_CHECK(launch_dependent(accept_stats_kernel, dim3(a.NCH, (unsigned)rows), dim3(kThreads), 0, stream, a));
     ++launches;
     if (s.gamma > 0) {
-        accept_shift_stats_kernel<<<dim3(a.NCH, (unsigned)drows), kThreads, 0, stream>>>(a);
+        RAPID_CUDA_CHECK(launch_dependent(accept_shift_stats_kernel, dim3(a.NCH, (unsigned)drows), dim3(kThreads), 0,
+                                          stream, a));
         ++launches;
     }
-    accept_residual_kernel<<<dim3(a.NCH, (unsigned)rows), kThreads, 0, stream>>>(a);
-    accept_select_kernel<<<s.B, kThreads, 0, stream>>>(a);
+    RAPID_CUDA_CHECK(launch_dependent(accept_residual_kernel, dim3(a.NCH, (unsigned)rows), dim3(kThreads), 0, stream, a));
+    RAPID_CUDA_CHECK(launch_dependent(accept_select_kernel, dim3(s.B), dim3(kThreads), 0, stream, a));
     launches += 2;
-    RAPID_CUDA_CHECK(cudaGetLastError());
     count_launch(launches);
     return RAPID_OK;
 }
