@@ -14,7 +14,6 @@
 // from run to run.  The merge is launched as a programmatic dependent of the split kernel: its
 // blocks are resident and have done their index arithmetic by the time the last partial lands.
 #include <math.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 #include "tcgen05.cuh"
@@ -41,7 +40,6 @@ struct AttnArgs {
     int B, Hq, Hkv, G, R, GR;
     int Lmax;
     int num_ctas;
-    int tile_keys;     // keys per scheduling tile (what plan, walk and merge count in)
     float scale_log2;  // softmax scale * log2(e)
 };
 
@@ -54,13 +52,13 @@ struct Walk {
 __device__ __forceinline__ int clamp_len(int L, int R, int Lmax) {
     return L < R ? R : (L > Lmax ? Lmax : L);
 }
-__device__ __forceinline__ int tiles_of(int L, int tile_keys) { return (L + tile_keys - 1) / tile_keys; }
+__device__ __forceinline__ int tiles_of(int L) { return (L + kTile - 1) / kTile; }
 
 // Flat tile range of CTA c of n: [c*T/n, (c+1)*T/n).
 __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     long long T = 0;
     for (int b = 0; b < a.B; ++b)
-        T += (long long)a.Hkv * tiles_of(clamp_len(a.ctx_lens[b], a.R, a.Lmax), a.tile_keys);
+        T += (long long)a.Hkv * tiles_of(clamp_len(a.ctx_lens[b], a.R, a.Lmax));
     // with fewer tiles than CTAs only the first T CTAs work, one tile each: no CTA inside the
     // range of a unit is ever empty, which the merge relies on
     const long long nc = T < a.num_ctas ? T : a.num_ctas;
@@ -80,7 +78,7 @@ __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     long long t = t0;
     for (int b = 0; b < a.B; ++b) {
         const int L = clamp_len(a.ctx_lens[b], a.R, a.Lmax);
-        const int nt = tiles_of(L, a.tile_keys);
+        const int nt = tiles_of(L);
         const long long span = (long long)a.Hkv * nt;
         if (t < span) {
             w.b = b;
@@ -104,7 +102,7 @@ __device__ __forceinline__ void walk_advance(const AttnArgs& a, Walk& w, int seg
             ++w.b;
             if (w.b < a.B) {
                 w.L = clamp_len(a.ctx_lens[w.b], a.R, a.Lmax);
-                w.ntiles = tiles_of(w.L, a.tile_keys);
+                w.ntiles = tiles_of(w.L);
             }
         }
     }
@@ -560,8 +558,6 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
     if (tid == 0 && s_abort) atomicOr(a.status, RAPID_STATUS_PIPELINE_TIMEOUT);
 }
 
-#include "attention_kt.cuh"
-
 // Merge: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the partials of a unit.
 // One block of 4 warps per (grouped row, unit): warp w takes the slots j = w, w+4, ... (four
 // loads in flight per lane), lanes span D; the four warp sums are added in warp order, so the
@@ -584,7 +580,7 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     long long T = 0, t0 = 0;
     int nt_b = 0;
     for (int bb = 0; bb < a.B; ++bb) {
-        const int nt = tiles_of(clamp_len(a.ctx_lens[bb], a.R, a.Lmax), a.tile_keys);
+        const int nt = tiles_of(clamp_len(a.ctx_lens[bb], a.R, a.Lmax));
         if (bb < b) t0 += (long long)a.Hkv * nt;
         if (bb == b) nt_b = nt;
         T += (long long)a.Hkv * nt;
@@ -682,7 +678,7 @@ EncodeTiledFn get_encode_fn() {
 }
 
 int make_kv_map(CUtensorMap* map, const void* base, const rapid_attn_shape& s, int64_t sb,
-                int64_t sh, int64_t sl, int box_rows) {
+                int64_t sh, int64_t sl) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) {
         set_error("cuTensorMapEncodeTiled is not available from the CUDA driver");
@@ -690,7 +686,7 @@ int make_kv_map(CUtensorMap* map, const void* base, const rapid_attn_shape& s, i
     }
     cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.Lmax, (cuuint64_t)s.Hkv, (cuuint64_t)s.B};
     cuuint64_t strides[3] = {(cuuint64_t)sl * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+    cuuint32_t box[4] = {64, (cuuint32_t)kTile, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
                      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -761,40 +757,6 @@ int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
     cfg.numAttrs = 1;
     RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_splitkv_tc_kernel<D, MR>, tmK, tmV, tmQ, a, lay));
     return RAPID_OK;
-}
-
-template <int NC>
-int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ, const AttnArgs& a,
-                    cudaStream_t stream) {
-    constexpr int smem = kt::smem_bytes(NC);
-    static_assert(smem <= kMaxSmemOptin - 4096, "shared memory (dynamic + the kernel's static arrays)");
-    static bool configured[64] = {};
-    int dev = 0;
-    RAPID_CUDA_CHECK(cudaGetDevice(&dev));
-    if (dev >= 64 || !configured[dev]) {
-        RAPID_CUDA_CHECK(cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC>,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        if (dev < 64) configured[dev] = true;
-    }
-    RAPID_CUDA_CHECK(launch_dependent(kt::verify_attn_splitkv_kt_kernel<NC>, dim3(a.num_ctas), dim3(kt::kThreads),
-                                      (size_t)smem, stream, tmK, tmV, tmQ, a));
-    return RAPID_OK;
-}
-
-int dispatch_split_kt(int NC, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
-                      const AttnArgs& a, cudaStream_t stream) {
-    switch (NC) {
-        case 1: return launch_split_kt<1>(tmK, tmV, tmQ, a, stream);
-        case 2: return launch_split_kt<2>(tmK, tmV, tmQ, a, stream);
-        case 3: return launch_split_kt<3>(tmK, tmV, tmQ, a, stream);
-        case 4: return launch_split_kt<4>(tmK, tmV, tmQ, a, stream);
-        case 5: return launch_split_kt<5>(tmK, tmV, tmQ, a, stream);
-        case 6: return launch_split_kt<6>(tmK, tmV, tmQ, a, stream);
-        case 7: return launch_split_kt<7>(tmK, tmV, tmQ, a, stream);
-        case 8: return launch_split_kt<8>(tmK, tmV, tmQ, a, stream);
-    }
-    set_error("unsupported number of grouped rows");
-    return RAPID_ERR_UNSUPPORTED;
 }
 
 int sm_count() {
@@ -886,12 +848,10 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
         return RAPID_ERR_UNSUPPORTED;
     }
 
-    static const bool use_kt = getenv("RAPID_ATTN_KT") != nullptr;
-    const bool kt_path = use_kt && s.D == 128;
     CUtensorMap tmK, tmV;
-    int rc = make_kv_map(&tmK, k_cache, s, sb, sh, sl, kt_path ? kt::kKeys : kTile);
+    int rc = make_kv_map(&tmK, k_cache, s, sb, sh, sl);
     if (rc != RAPID_OK) return rc;
-    rc = make_kv_map(&tmV, v_cache, s, sb, sh, sl, kt_path ? kt::kKeys : kTile);
+    rc = make_kv_map(&tmV, v_cache, s, sb, sh, sl);
     if (rc != RAPID_OK) return rc;
 
     AttnArgs a;
@@ -907,17 +867,12 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     a.GR = GR;
     a.Lmax = (int)s.Lmax;
     a.num_ctas = num_ctas;
-    a.tile_keys = kt_path ? kt::kKeys : kTile;
     a.scale_log2 = scale * 1.4426950408889634f;
 
     CUtensorMap tmQ;
     rc = make_q_map(&tmQ, q, s, G, R);
     if (rc != RAPID_OK) return rc;
-    int n_partials = kStreams;
-    if (kt_path) {
-        n_partials = 1;
-        rc = dispatch_split_kt((GR + 15) / 16, tmK, tmV, tmQ, a, stream);
-    } else if (GR <= 64)
+    if (GR <= 64)
         rc = s.D == 128 ? launch_split_tc<128, 64>(tmK, tmV, tmQ, a, stream)
                         : launch_split_tc<64, 64>(tmK, tmV, tmQ, a, stream);
     else
@@ -945,9 +900,9 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     cfg.numAttrs = 1;
     __nv_bfloat16* out_bf = static_cast<__nv_bfloat16*>(out);
     if (s.D == 128)
-        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<128>, a, n_partials, out_bf, lse, o32));
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<128>, a, (int)kStreams, out_bf, lse, o32));
     else
-        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<64>, a, n_partials, out_bf, lse, o32));
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<64>, a, (int)kStreams, out_bf, lse, o32));
     count_launch(2);
     return RAPID_OK;
 }
