@@ -45,13 +45,14 @@ struct AcceptArgs {
     int32_t* status;   // header word 0
     int32_t* done;     // header word 1: clusters that have finished; back to 0 when the call ends
     float* ratio;      // [B*gamma]
-    int32_t* cand;     // [B*R] candidate token of every row
+    int32_t* cand;     // [B*R] candidate token of every row; bit 31 = drawn from p as a fallback
     int B, gamma, R, V;
     int slice;  // entries per CTA (multiple of 4)
     int per;    // consecutive entries per thread in the search (odd: conflict-free shared reads)
     long long zs, ds;  // row strides
     float inv_T_log2;  // log2(e) / T
     float eta_log2;    // eta * log2(e)
+    float alpha;       // tail_alpha, 0 disables the tail rule
     float log2_alpha;  // log2(tail_alpha), -inf disables the tail rule
     int mode;
 };
@@ -67,77 +68,45 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-// Block-wide (max, rescaled sum) reduction of per-thread online-softmax states; fixed order.
-__device__ __forceinline__ void block_reduce_ms(float& m, float& s, float* sh_m, float* sh_s) {
-    const float wm = warp_max(m);
-    s = (m == -INFINITY) ? 0.f : s * exp2f(m - wm);
-    s = warp_sum(s);
+// Block-wide maximum / sum of two values at once, in a fixed order; sh holds 2 * kWarps floats.
+__device__ __forceinline__ void block_max2(float& x, float& y, float* sh) {
+    x = warp_max(x);
+    y = warp_max(y);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __syncthreads();
     if (lane == 0) {
-        sh_m[warp] = wm;
-        sh_s[warp] = s;
+        sh[warp] = x;
+        sh[kWarps + warp] = y;
     }
     __syncthreads();
-    float M = -INFINITY;
+    x = sh[0];
+    y = sh[kWarps];
 #pragma unroll
-    for (int i = 0; i < kWarps; ++i) M = fmaxf(M, sh_m[i]);
-    float S = 0.f;
-#pragma unroll
-    for (int i = 0; i < kWarps; ++i)
-        S += (sh_m[i] == -INFINITY) ? 0.f : sh_s[i] * exp2f(sh_m[i] - M);
-    m = M;
-    s = S;
+    for (int i = 1; i < kWarps; ++i) {
+        x = fmaxf(x, sh[i]);
+        y = fmaxf(y, sh[kWarps + i]);
+    }
 }
-
-__device__ __forceinline__ float block_reduce_sum(float v, float* sh) {
-    v = warp_sum(v);
+__device__ __forceinline__ void block_sum2(float& x, float& y, float* sh) {
+    x = warp_sum(x);
+    y = warp_sum(y);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __syncthreads();
-    if (lane == 0) sh[warp] = v;
+    if (lane == 0) {
+        sh[warp] = x;
+        sh[kWarps + warp] = y;
+    }
     __syncthreads();
-    float S = 0.f;
+    x = 0.f;
+    y = 0.f;
 #pragma unroll
-    for (int i = 0; i < kWarps; ++i) S += sh[i];
-    return S;
-}
-
-__device__ __forceinline__ void online_add(float& m, float& s, float x) {
-    if (x > m) {
-        s = s * exp2f(m - x) + 1.f;  // exp2f(-inf) = 0 covers the first element
-        m = x;
-    } else if (x != -INFINITY) {  // a logit of -inf carries no mass (and -inf - -inf is NaN)
-        s += exp2f(x - m);
+    for (int i = 0; i < kWarps; ++i) {
+        x += sh[i];
+        y += sh[kWarps + i];
     }
 }
 
-struct RowStats {
-    float Mz, inv_Sz, Md, inv_Sd;
-};
-
-// y in base-2 units: (z/T + eta (q - p)) * log2(e)
-__device__ __forceinline__ float shifted_logit2(const AcceptArgs& a, const RowStats& r, float z,
-                                                float d, float& p, float& q) {
-    const float z2 = z * a.inv_T_log2;
-    p = exp2f(z2 - r.Mz) * r.inv_Sz;
-    q = exp2f(d * a.inv_T_log2 - r.Md) * r.inv_Sd;
-    return fmaf(a.eta_log2, q - p, z2);
-}
-
-// Residual weight of one vocabulary entry of a draft row; also returns phat' (tail rule applied).
-__device__ __forceinline__ float residual_weight(const AcceptArgs& a, const RowStats& r, float My,
-                                                 float inv_Sy, float z, float d, float& p,
-                                                 float& q, float& ph) {
-    const float y2 = shifted_logit2(a, r, z, d, p, q);
-    const float rel = y2 - My;
-    ph = (rel < a.log2_alpha) ? p : exp2f(rel) * inv_Sy;
-    float w;
-    if (a.mode == RAPID_RESIDUAL_PHAT)
-        w = ph - q;
-    else
-        w = fmaxf(p - ph, p - q);
-    return fmaxf(w, 0.f);
-}
+__device__ __forceinline__ float max4(const float4& v) { return fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)); }
 
 __device__ __forceinline__ float warp_incl_scan(float v) {
     const int lane = threadIdx.x & 31;
@@ -159,6 +128,7 @@ __device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, flo
     __syncthreads();
 }
 
+// Combine the per-CTA (max, sum relative to that max) pairs of a row, in rank order.
 __device__ __forceinline__ void combine_ms(const float4* g, bool second, float& M, float& S) {
     M = -INFINITY;
 #pragma unroll
@@ -171,11 +141,13 @@ __device__ __forceinline__ void combine_ms(const float4* g, bool second, float& 
     }
 }
 
+// NV4 = float4 groups a thread owns in each array (group i belongs to thread i % kThreads).
+template <int NV4>
 __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptArgs a) {
     extern __shared__ __align__(16) float slice_mem[];
     __shared__ float4 xch[3];
     __shared__ float4 gath[3][kCluster];
-    __shared__ float sh_m[kWarps], sh_s[kWarps];
+    __shared__ float sh_red[2 * kWarps];
     __shared__ int sh_tok, sh_last, sh_final;
 
     cg::cluster_group cluster = cg::this_cluster();
@@ -187,127 +159,175 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
     const int drow = b * a.gamma + k;
     const int v0 = min(c * a.slice, a.V), v1 = min(v0 + a.slice, a.V);
     const int n4 = (v1 - v0) >> 2;
-    float* zc = slice_mem;
-    float* dc = slice_mem + a.slice;
-    const float* z = a.z + (size_t)row * a.zs + v0;
-    const float* d = draft ? a.d + (size_t)drow * a.ds + v0 : nullptr;
+    float4* zc = reinterpret_cast<float4*>(slice_mem);
+    float4* dc = reinterpret_cast<float4*>(slice_mem + a.slice);
+    const float4* z = reinterpret_cast<const float4*>(a.z + (size_t)row * a.zs + v0);
+    const float4* d = draft ? reinterpret_cast<const float4*>(a.d + (size_t)drow * a.ds + v0) : nullptr;
+    const float c2 = a.inv_T_log2;
 
     griddep_wait();  // the logits may come from the kernel just before this one
     griddep_launch_dependents();
 
-    // ---- step 0: the only pass over global memory ----
-    float mz = -INFINITY, sz = 0.f, md = -INFINITY, sd = 0.f;
-    for (int i0 = 0; i0 < n4; i0 += kBatch * kThreads) {
+    // ---- step 0: the only pass over global memory; p = softmax(z/T), q = softmax(d/T) ----
+    float mz = -INFINITY, md = -INFINITY;
+#pragma unroll
+    for (int k0 = 0; k0 < NV4; k0 += kBatch) {
         float4 xz[kBatch], xd[kBatch];
 #pragma unroll
         for (int e = 0; e < kBatch; ++e) {
-            const int i = i0 + e * kThreads + tid;
+            const int i = (k0 + e) * kThreads + tid;
             const bool ok = i < n4;
-            xz[e] = ok ? __ldg(reinterpret_cast<const float4*>(z) + i)
-                       : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-            xd[e] = (ok && draft) ? __ldg(reinterpret_cast<const float4*>(d) + i)
-                                  : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            xz[e] = ok ? __ldg(z + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            xd[e] = (ok && draft) ? __ldg(d + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
         }
 #pragma unroll
         for (int e = 0; e < kBatch; ++e) {
-            const int i = i0 + e * kThreads + tid;
+            const int i = (k0 + e) * kThreads + tid;
             if (i < n4) {
-                reinterpret_cast<float4*>(zc)[i] = xz[e];
-                if (draft) reinterpret_cast<float4*>(dc)[i] = xd[e];
+                zc[i] = xz[e];
+                if (draft) dc[i] = xd[e];
             }
-            online_add(mz, sz, xz[e].x * a.inv_T_log2);
-            online_add(mz, sz, xz[e].y * a.inv_T_log2);
-            online_add(mz, sz, xz[e].z * a.inv_T_log2);
-            online_add(mz, sz, xz[e].w * a.inv_T_log2);
+            mz = fmaxf(mz, max4(xz[e]));
+            md = fmaxf(md, max4(xd[e]));
+        }
+    }
+    block_max2(mz, md, sh_red);
+    // slice maxima in base-2 units (scaling by log2(e)/T > 0 keeps the order); an empty or all -inf
+    // slice contributes (-inf, 0)
+    const float Mzb = mz * c2, Mdb = md * c2;
+    const float refz = (mz == -INFINITY) ? 0.f : Mzb, refd = (md == -INFINITY) ? 0.f : Mdb;
+    float sz = 0.f, sd = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < NV4; ++kk) {
+        const int i = kk * kThreads + tid;
+        if (i < n4) {
+            const float4 x = zc[i];
+            sz += fast_exp2(fmaf(x.x, c2, -refz)) + fast_exp2(fmaf(x.y, c2, -refz)) +
+                  fast_exp2(fmaf(x.z, c2, -refz)) + fast_exp2(fmaf(x.w, c2, -refz));
             if (draft) {
-                online_add(md, sd, xd[e].x * a.inv_T_log2);
-                online_add(md, sd, xd[e].y * a.inv_T_log2);
-                online_add(md, sd, xd[e].z * a.inv_T_log2);
-                online_add(md, sd, xd[e].w * a.inv_T_log2);
+                const float4 y = dc[i];
+                sd += fast_exp2(fmaf(y.x, c2, -refd)) + fast_exp2(fmaf(y.y, c2, -refd)) +
+                      fast_exp2(fmaf(y.z, c2, -refd)) + fast_exp2(fmaf(y.w, c2, -refd));
             }
         }
     }
-    block_reduce_ms(mz, sz, sh_m, sh_s);
-    block_reduce_ms(md, sd, sh_m, sh_s);
-    cluster_exchange(cluster, &xch[0], gath[0], make_float4(mz, sz, md, sd));
-    RowStats r;
-    {
-        float S;
-        combine_ms(gath[0], false, r.Mz, S);
-        r.inv_Sz = 1.f / S;
-        r.Md = 0.f;
-        r.inv_Sd = 0.f;
-        if (draft) {
-            combine_ms(gath[0], true, r.Md, S);
-            r.inv_Sd = 1.f / S;
-        }
-    }
+    block_sum2(sz, sd, sh_red);
+    cluster_exchange(cluster, &xch[0], gath[0], make_float4(mz == -INFINITY ? -INFINITY : Mzb, sz,
+                                                            md == -INFINITY ? -INFINITY : Mdb, sd));
+    // p = 2^(z * c2 - Mz) / Sz, q = 2^(d * c2 - Md) / Sd.  The row maximum is taken off inside the
+    // fused multiply-add, before anything is rounded, and the normaliser is applied as a factor:
+    // at a low temperature the scaled logits are in the hundreds, and a constant folded from
+    // Mz + log2 Sz would be rounded at that magnitude, scaling every p of the row by the same
+    // 1 + 1e-5 -- more than the whole residual mass when p and phat nearly coincide.  This way the
+    // top entry is exactly 1/Sz, and phat's top entry exactly 1/Sy.
+    float Mz, Sz, Md = 0.f, Sd = 1.f;
+    combine_ms(gath[0], false, Mz, Sz);
+    if (draft) combine_ms(gath[0], true, Md, Sd);
+    const float iSz = 1.f / Sz, iSd = 1.f / Sd;
 
-    // ---- step 1: normaliser of phat (draft rows) ----
-    float My = 0.f, inv_Sy = 0.f;
-    if (draft) {
-        float my = -INFINITY, sy = 0.f;
-        for (int i = tid; i < n4; i += kThreads) {
-            const float4 x = reinterpret_cast<const float4*>(zc)[i];
-            const float4 y = reinterpret_cast<const float4*>(dc)[i];
-            float p, q;
-            online_add(my, sy, shifted_logit2(a, r, x.x, y.x, p, q));
-            online_add(my, sy, shifted_logit2(a, r, x.y, y.y, p, q));
-            online_add(my, sy, shifted_logit2(a, r, x.z, y.z, p, q));
-            online_add(my, sy, shifted_logit2(a, r, x.w, y.w, p, q));
-        }
-        block_reduce_ms(my, sy, sh_m, sh_s);
-        cluster_exchange(cluster, &xch[1], gath[1], make_float4(my, sy, 0.f, 0.f));
-        float Sy;
-        combine_ms(gath[1], false, My, Sy);
-        inv_Sy = 1.f / Sy;
-    }
-
-    // ---- step 2: slice sums of the residual weights and of p; the ratio at the draft token ----
     float sw = 0.f, sp = 0.f;
+    float My = 0.f, Sy = 1.f;
     if (draft) {
+        // ---- step 1: y = z/T + eta (q - p) up to the constant Mz, and the normaliser of phat ----
+        // p and q replace the logits in shared memory; y stays in registers
+        float ev[NV4 * 4];
+        float my = -INFINITY, unused = -INFINITY;
+#pragma unroll
+        for (int kk = 0; kk < NV4; ++kk) {
+            const int i = kk * kThreads + tid;
+            if (i < n4) {
+                const float4 x = zc[i], y = dc[i];
+                const float lp[4] = {fmaf(x.x, c2, -Mz), fmaf(x.y, c2, -Mz), fmaf(x.z, c2, -Mz), fmaf(x.w, c2, -Mz)};
+                const float lq[4] = {fmaf(y.x, c2, -Md), fmaf(y.y, c2, -Md), fmaf(y.z, c2, -Md), fmaf(y.w, c2, -Md)};
+                float p[4], q[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    p[e] = fast_exp2(lp[e]) * iSz;
+                    q[e] = fast_exp2(lq[e]) * iSd;
+                    // a logit of -inf has p = 0 and takes no part in phat either
+                    const float y2 = (lp[e] == -INFINITY) ? -INFINITY : fmaf(a.eta_log2, q[e] - p[e], lp[e]);
+                    ev[4 * kk + e] = y2;
+                    my = fmaxf(my, y2);
+                }
+                zc[i] = make_float4(p[0], p[1], p[2], p[3]);
+                dc[i] = make_float4(q[0], q[1], q[2], q[3]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) ev[4 * kk + e] = -INFINITY;
+            }
+        }
+        block_max2(my, unused, sh_red);
+        const float refy = (my == -INFINITY) ? 0.f : my;
+        float sy = 0.f, zero = 0.f;
+#pragma unroll
+        for (int e = 0; e < NV4 * 4; ++e) {
+            ev[e] = fast_exp2(ev[e] - refy);  // phat up to the factor 2^(my - My) / Sy
+            sy += ev[e];
+        }
+        block_sum2(sy, zero, sh_red);
+        cluster_exchange(cluster, &xch[1], gath[1], make_float4(my, sy, 0.f, 0.f));
+        combine_ms(gath[1], false, My, Sy);
+        const float rel = (my == -INFINITY) ? 0.f : exp2f(my - My);  // phat / max(phat) = ev * rel
+        const float to_phat = rel / Sy;
+
+        // ---- step 2: the ratio at the draft token, then the residual weights ----
         int tok = a.tokens[drow];
         if (tok < 0 || tok >= a.V) {
             if (c == 0 && tid == 0) atomicOr(a.status, RAPID_STATUS_BAD_DRAFT_TOKEN);
             tok = tok < 0 ? 0 : a.V - 1;
         }
-        for (int i = tid; i < n4; i += kThreads) {
-            const float4 x = reinterpret_cast<const float4*>(zc)[i];
-            const float4 y = reinterpret_cast<const float4*>(dc)[i];
-            const float xs[4] = {x.x, x.y, x.z, x.w};
-            const float ys[4] = {y.x, y.y, y.z, y.w};
+        const int tl = tok - v0;
+        if (tl >= 0 && tl < v1 - v0 && ((tl >> 2) % kThreads) == tid) {
+            // formed from log-probabilities: a draft token deep in the tail has p, phat and q far
+            // below the fp32 normal range while their ratio is O(1)
+            const float p = slice_mem[tl], q = slice_mem[a.slice + tl];
+            const float az = fmaf(__ldg(a.z + (size_t)row * a.zs + tok), c2, -Mz);
+            const float lq = fmaf(__ldg(a.d + (size_t)drow * a.ds + tok), c2, -Md) - log2f(Sd);
+            const float y2 = fmaf(a.eta_log2, q - p, az);
+            const float lph = (y2 - My < a.log2_alpha) ? az - log2f(Sz) : (y2 - My) - log2f(Sy);
+            const float ratio = (lq == -INFINITY) ? INFINITY : exp2f(lph - lq);
+            a.ratio[drow] = ratio;
+            if (a.ratio_out) a.ratio_out[drow] = ratio;
+        }
+        // the weights replace p in shared memory, p moves to where q was (the fallback draws from it)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                float p, q, ph;
-                sw += residual_weight(a, r, My, inv_Sy, xs[e], ys[e], p, q, ph);
-                sp += p;
-                if (v0 + 4 * i + e == tok) {
-                    // the ratio is formed from log-probabilities: a draft token deep in the tail
-                    // has p, phat and q far below the fp32 normal range while their ratio is O(1)
-                    const float z2 = xs[e] * a.inv_T_log2;
-                    const float lq = (ys[e] * a.inv_T_log2 - r.Md) + log2f(r.inv_Sd);
-                    const float y2 = fmaf(a.eta_log2, q - p, z2);
-                    const float lph = (y2 - My < a.log2_alpha) ? (z2 - r.Mz) + log2f(r.inv_Sz)
-                                                               : (y2 - My) + log2f(inv_Sy);
-                    const float ratio = (lq == -INFINITY) ? INFINITY : exp2f(lph - lq);
-                    a.ratio[drow] = ratio;
-                    if (a.ratio_out) a.ratio_out[drow] = ratio;
+        for (int kk = 0; kk < NV4; ++kk) {
+            const int i = kk * kThreads + tid;
+            if (i < n4) {
+                const float4 p4 = zc[i], q4 = dc[i];
+                const float p[4] = {p4.x, p4.y, p4.z, p4.w};
+                const float q[4] = {q4.x, q4.y, q4.z, q4.w};
+                float w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float en = ev[4 * kk + e];
+                    const float ph = (en * rel < a.alpha) ? p[e] : en * to_phat;  // tail rule
+                    const float r = (a.mode == RAPID_RESIDUAL_PHAT) ? ph - q[e] : fmaxf(p[e] - ph, p[e] - q[e]);
+                    w[e] = fmaxf(r, 0.f);
+                    sw += w[e];
+                    sp += p[e];
                 }
+                zc[i] = make_float4(w[0], w[1], w[2], w[3]);
+                dc[i] = p4;
             }
         }
     } else {
-        for (int i = tid; i < n4; i += kThreads) {
-            const float4 x = reinterpret_cast<const float4*>(zc)[i];
-            sp += exp2f(x.x * a.inv_T_log2 - r.Mz) * r.inv_Sz;
-            sp += exp2f(x.y * a.inv_T_log2 - r.Mz) * r.inv_Sz;
-            sp += exp2f(x.z * a.inv_T_log2 - r.Mz) * r.inv_Sz;
-            sp += exp2f(x.w * a.inv_T_log2 - r.Mz) * r.inv_Sz;
+        // bonus row: the weights are p itself
+#pragma unroll
+        for (int kk = 0; kk < NV4; ++kk) {
+            const int i = kk * kThreads + tid;
+            if (i < n4) {
+                const float4 x = zc[i];
+                const float4 p = make_float4(fast_exp2(fmaf(x.x, c2, -Mz)) * iSz, fast_exp2(fmaf(x.y, c2, -Mz)) * iSz,
+                                             fast_exp2(fmaf(x.z, c2, -Mz)) * iSz, fast_exp2(fmaf(x.w, c2, -Mz)) * iSz);
+                sp += (p.x + p.y) + (p.z + p.w);
+                zc[i] = p;
+            }
         }
         sw = sp;
     }
-    sw = block_reduce_sum(sw, sh_m);
-    sp = block_reduce_sum(sp, sh_s);
-    cluster_exchange(cluster, &xch[2], gath[2], make_float4(sw, sp, 0.f, 0.f));
+    block_sum2(sw, sp, sh_red);
+    cluster_exchange(cluster, &xch[2], gath[2], make_float4(sw, sp, 0.f, 0.f));  // also a CTA barrier
 
     // ---- step 3: the row's candidate token by inverse CDF (every CTA finds the same slice) ----
     const float u = a.uniforms[b * a.R + a.gamma];
@@ -315,8 +335,9 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
     float W = 0.f;
 #pragma unroll
     for (int rr = 0; rr < kCluster; ++rr) W += use_p ? gath[2][rr].y : gath[2][rr].x;
+    int fell_back = 0;  // reported only if this row turns out to be the one Algorithm 1 reaches
     if (!(W > 0.f) || !isfinite(W)) {  // empty residual: defined fallback, draw from p
-        if (!use_p && c == 0 && tid == 0) atomicOr(a.status, RAPID_STATUS_RESIDUAL_FALLBACK);
+        if (!use_p) fell_back = (int)0x80000000;
         use_p = true;
         W = 0.f;
 #pragma unroll
@@ -348,43 +369,26 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
         want_last = true;
     }
     if (owner < 0) {  // nothing has mass at all (non-finite logits): defined output
-        if (c == 0 && tid == 0) a.cand[row] = 0;
+        if (c == 0 && tid == 0) a.cand[row] = fell_back;
     } else if (c == owner) {
         // thread t owns a.per consecutive entries, so the prefix order is the vocabulary order
+        const float* wsrc = (use_p && draft) ? slice_mem + a.slice : slice_mem;
         const int t0 = min(tid * a.per, v1 - v0), t1 = min(t0 + a.per, v1 - v0);
         float mine = 0.f;
-        for (int i = t0; i < t1; ++i) {
-            float w;
-            if (draft) {
-                float p, q, ph;
-                const float rw = residual_weight(a, r, My, inv_Sy, zc[i], dc[i], p, q, ph);
-                w = use_p ? p : rw;
-            } else {
-                w = exp2f(zc[i] * a.inv_T_log2 - r.Mz) * r.inv_Sz;
-            }
-            mine += w;
-        }
+        for (int i = t0; i < t1; ++i) mine += wsrc[i];
         const float incl_w = warp_incl_scan(mine);
         if (tid == 0) {
             sh_tok = 0x7fffffff;
             sh_last = -1;
         }
-        __syncthreads();  // sh_m is free again (block_reduce_sum has been read by everyone)
-        if (lane == 31) sh_m[warp] = incl_w;
+        if (lane == 31) sh_red[warp] = incl_w;
         __syncthreads();
         float cum = before;
-        for (int wdx = 0; wdx < warp; ++wdx) cum += sh_m[wdx];
+        for (int wdx = 0; wdx < warp; ++wdx) cum += sh_red[wdx];
         cum += incl_w - mine;
         int found = 0x7fffffff, last = -1;
         for (int i = t0; i < t1; ++i) {
-            float w;
-            if (draft) {
-                float p, q, ph;
-                const float rw = residual_weight(a, r, My, inv_Sy, zc[i], dc[i], p, q, ph);
-                w = use_p ? p : rw;
-            } else {
-                w = exp2f(zc[i] * a.inv_T_log2 - r.Mz) * r.inv_Sz;
-            }
+            const float w = wsrc[i];
             if (w > 0.f) {
                 cum += w;
                 last = v0 + i;
@@ -394,7 +398,7 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
         if (found != 0x7fffffff) atomicMin(&sh_tok, found);
         if (last >= 0) atomicMax(&sh_last, last);
         __syncthreads();
-        if (tid == 0) a.cand[row] = sh_tok != 0x7fffffff ? sh_tok : (sh_last >= 0 ? sh_last : v0);
+        if (tid == 0) a.cand[row] = (sh_tok != 0x7fffffff ? sh_tok : (sh_last >= 0 ? sh_last : v0)) | fell_back;
     }
 
     // ---- the last cluster to finish settles every sequence ----
@@ -416,8 +420,10 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
             const float us = a.uniforms[s * a.R + n];
             if (!(us <= fminf(1.f, ratio))) break;
         }
+        const int cand = __ldcg(a.cand + s * a.R + n);  // bit 31: the row fell back to p
+        if (cand < 0) atomicOr(a.status, RAPID_STATUS_RESIDUAL_FALLBACK);
         a.accept_len[s] = n;
-        a.next_token[s] = __ldcg(a.cand + s * a.R + n);
+        a.next_token[s] = cand & 0x7fffffff;
     }
     if (tid == 0) *a.done = 0;  // ready for the next call on this workspace
 }
@@ -506,13 +512,16 @@ int launch_accept(const float* target_logits, const float* draft_logits,
     a.ds = ds;
     a.inv_T_log2 = 1.4426950408889634f / T;
     a.eta_log2 = eta * 1.4426950408889634f;
+    a.alpha = alpha;
     a.log2_alpha = alpha > 0.f ? log2f(alpha) : -INFINITY;
     a.mode = mode;
 
     int dev = 0;
     RAPID_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices || !g_smem_opted[dev]) {
-        RAPID_CUDA_CHECK(cudaFuncSetAttribute(accept_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        RAPID_CUDA_CHECK(cudaFuncSetAttribute(accept_fused_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              2 * 8 * 4 * kThreads * (int)sizeof(float)));
+        RAPID_CUDA_CHECK(cudaFuncSetAttribute(accept_fused_kernel<12>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               2 * kMaxSlice * (int)sizeof(float)));
         if (dev >= 0 && dev < kMaxDevices) g_smem_opted[dev] = true;
     }
@@ -531,7 +540,10 @@ int launch_accept(const float* target_logits, const float* draft_logits,
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, accept_fused_kernel, a));
+    if (a.slice <= 8 * 4 * kThreads)
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, accept_fused_kernel<8>, a));
+    else
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, accept_fused_kernel<12>, a));
     count_launch(1);
     return RAPID_OK;
 }
