@@ -199,10 +199,10 @@ int rapid_accept(const float* target_logits, const float* draft_logits,
  * promised not to touch the allocator after warm-up because cudaMalloc and
  * cudaFree stall every stream of the device, or a component whose memory
  * budget is fixed by contract.  Such a caller still owns the logits, tokens,
- * uniforms and the two output arrays, but has nowhere to put the few hundred
- * kilobytes of per-row statistics the accept passes exchange.
+ * uniforms and the two output arrays, but has nowhere to put the per-row
+ * ratios and candidate tokens the accept kernel leaves for its epilogue.
  *
- * Here that scratch is a fixed array inside the library image (about 1.1 MB,
+ * Here that scratch is a fixed array inside the library image (about 5 KB,
  * resident on every GPU that loads the library until the process ends).  The
  * computation, the kernels and the results are those of rapid_accept.
  *
