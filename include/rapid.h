@@ -54,6 +54,7 @@ extern "C" {
 #define RAPID_STATUS_BAD_DRAFT_TOKEN 2    /* draft token outside [0, V): clamped into range           */
 #define RAPID_STATUS_RESIDUAL_FALLBACK 4  /* residual mass was 0 / not finite: token drawn from p    */
 #define RAPID_STATUS_PIPELINE_TIMEOUT 8   /* an on-chip wait hit its time limit: outputs invalid      */
+#define RAPID_STATUS_BAD_BLOCK_TABLE 16  /* a block-table entry outside [0, num_blocks): read as 0s  */
 
 /* residual_mode */
 #define RAPID_RESIDUAL_PAPER 0 /* norm(max(p - phat, p - q, 0)): Algorithm 1, residual step               */
@@ -161,6 +162,45 @@ int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cac
                            const int32_t* ctx_lens, int gamma, void* out,
                            const rapid_attn_shape* shape, const rapid_attn_params* params,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Geometry of a paged KV cache: a pool of fixed-size blocks shared by all
+ * sequences, as serving engines keep it.  (The paper does not say how the
+ * cache is stored; the computation is that of rapid_verify_attention.)
+ *   k_pool / v_pool : [num_blocks, Hkv, block_size, D] bf16 with element
+ *                     strides stride_block / stride_h / stride_l
+ *                     (0 = dense: Hkv*block_size*D, block_size*D, D);
+ *                     [num_blocks, block_size, Hkv, D] is the same pool with
+ *                     stride_h = D and stride_l = Hkv*D
+ *   block_table     : device int32 [B, max_blocks_per_seq]; logical keys
+ *                     [i*block_size, (i+1)*block_size) of sequence b live in
+ *                     physical block block_table[b, i].  Entries past the
+ *                     blocks a sequence uses are never read.
+ *   block_size      : a power of two, at least 64
+ */
+typedef struct rapid_paged_kv {
+    int32_t block_size;
+    int32_t num_blocks;
+    int32_t max_blocks_per_seq;
+    int32_t reserved;
+    int64_t stride_block;
+    int64_t stride_h;
+    int64_t stride_l;
+} rapid_paged_kv;
+
+/*
+ * rapid_verify_attention over a paged cache.  shape->Lmax must equal
+ * max_blocks_per_seq * block_size (the logical capacity); shape's kv strides
+ * are ignored.  A table entry outside [0, num_blocks) sets
+ * RAPID_STATUS_BAD_BLOCK_TABLE and its keys and values read as zeros.  The
+ * pools and the table are only read.  Everything else (arguments, results,
+ * workspace, errors) is as in rapid_verify_attention.
+ */
+int rapid_verify_attention_paged(const void* q, const void* k_pool, const void* v_pool,
+                                 const int32_t* block_table, const rapid_paged_kv* paged,
+                                 const int32_t* ctx_lens, int gamma, void* out,
+                                 const rapid_attn_shape* shape, const rapid_attn_params* params,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
  * Accept / residual (Algorithm 1, validation loop and residual step;

@@ -187,6 +187,26 @@ def accept(target_logits, draft_logits, draft_tokens, uniforms, eta, T=1.0, tail
     return dict(accept_len=accept_len, next_token=next_token, flags=flags, ratios=ratios)
 
 
+def paged_gather(pool, block_table, ctx_lens):
+    """A paged cache written out as the contiguous cache it stands for (storage only; the paper's
+    attention is defined on the logical sequence): pool [num_blocks, Hkv, block_size, D],
+    block_table [B, max_blocks] -> cache [B, Hkv, max_blocks * block_size, D], where logical key j
+    of sequence b is pool[block_table[b, j // block_size], :, j % block_size, :].  Only the
+    ctx_lens[b] keys a sequence holds are looked up; the rest of its rows stay zero."""
+    pool = np.asarray(pool)
+    table = np.asarray(block_table)
+    nb, Hkv, bs, D = pool.shape
+    B, mb = table.shape
+    out = np.zeros((B, Hkv, mb * bs, D), dtype=pool.dtype)
+    for b in range(B):
+        for j in range(int(ctx_lens[b])):
+            blk = int(table[b, j // bs])
+            if not 0 <= blk < nb:
+                raise ValueError(f"block table entry {blk} of sequence {b} outside the pool")
+            out[b, :, j, :] = pool[blk, :, j % bs, :]
+    return out
+
+
 def kv_append(k_cache, v_cache, k_new, v_new, ctx_lens, gamma):
     """Bookkeeping before a verify step (Algorithm 1: the last accepted token and the gamma drafts join
     the sequence the target scores): rows [L_b, L_b + R) of sequence b take k_new[b] / v_new[b]

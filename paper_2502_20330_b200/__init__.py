@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     rapid_kv_append,
     rapid_step_commit,
     rapid_verify_attention,
+    rapid_verify_attention_paged,
     rapid_verify_step,
     rapid_verify_step_host,
     verify_step_host_arena_bytes,
@@ -31,6 +32,7 @@ from .binding import (  # noqa: F401
     STATUS_BAD_DRAFT_TOKEN,
     STATUS_RESIDUAL_FALLBACK,
     STATUS_PIPELINE_TIMEOUT,
+    STATUS_BAD_BLOCK_TABLE,
     RESIDUAL_PAPER,
     RESIDUAL_PHAT,
 )

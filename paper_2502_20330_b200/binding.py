@@ -15,12 +15,13 @@ STATUS_BAD_CTX_LEN = 1
 STATUS_BAD_DRAFT_TOKEN = 2
 STATUS_RESIDUAL_FALLBACK = 4
 STATUS_PIPELINE_TIMEOUT = 8
+STATUS_BAD_BLOCK_TABLE = 16
 RESIDUAL_PAPER = 0
 RESIDUAL_PHAT = 1
 
 EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
-    "rapid_workspace_status", "rapid_verify_attention", "rapid_accept", "rapid_accept_static",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_paged", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
     "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_step_commit",
     "rapid_last_error",
@@ -38,6 +39,12 @@ class _AttnShape(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32),
                 ("D", ctypes.c_int32), ("Lmax", ctypes.c_int64), ("kv_stride_b", ctypes.c_int64),
                 ("kv_stride_h", ctypes.c_int64), ("kv_stride_l", ctypes.c_int64)]
+
+
+class _PagedKv(ctypes.Structure):
+    _fields_ = [("block_size", ctypes.c_int32), ("num_blocks", ctypes.c_int32),
+                ("max_blocks_per_seq", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("stride_block", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_l", ctypes.c_int64)]
 
 
 class _AttnParams(ctypes.Structure):
@@ -108,6 +115,8 @@ def load_library():
         acc_args = [vp, vp, vp, vp, f32, vp, vp, ctypes.POINTER(_AcceptShape), ctypes.POINTER(_AcceptParams)]
         lib.rapid_verify_attention.restype = i32
         lib.rapid_verify_attention.argtypes = attn_args + [vp, sz, vp]
+        lib.rapid_verify_attention_paged.restype = i32
+        lib.rapid_verify_attention_paged.argtypes = [vp, vp, vp, vp, ctypes.POINTER(_PagedKv)] + attn_args[3:] + [vp, sz, vp]
         lib.rapid_accept.restype = i32
         lib.rapid_accept.argtypes = acc_args + [vp, sz, vp]
         lib.rapid_accept_static.restype = i32
@@ -251,6 +260,32 @@ def rapid_verify_attention(q, k_cache, v_cache, ctx_lens, gamma, out, workspace,
     _check(load_library().rapid_verify_attention(_p(q), _p(k_cache), _p(v_cache), _p(ctx_lens), gamma, _p(out),
                                                  ctypes.byref(shape), _attn_params(params), _p(workspace),
                                                  _nbytes(workspace), _stream_ptr(stream)))
+
+
+def rapid_verify_attention_paged(q, k_pool, v_pool, block_table, ctx_lens, gamma, out, workspace,
+                                 params: Optional[AttnParams] = None, stream=None) -> None:
+    """Verify attention over a paged cache: k_pool/v_pool [num_blocks, Hkv, block_size, D] bf16 (any
+    strides with a contiguous head_dim), block_table [B, max_blocks_per_seq] int32."""
+    if q.dtype != torch.bfloat16 or k_pool.dtype != torch.bfloat16 or v_pool.dtype != torch.bfloat16 \
+            or out.dtype != torch.bfloat16 or ctx_lens.dtype != torch.int32 or block_table.dtype != torch.int32:
+        raise TypeError("q/k/v/out must be bfloat16, ctx_lens and block_table int32")
+    if not (q.is_contiguous() and out.is_contiguous()) or q.shape[1] != gamma + 1 or out.shape != q.shape:
+        raise ValueError("q and out must be dense [B, gamma+1, Hq, D]")
+    if k_pool.stride() != v_pool.stride() or k_pool.shape != v_pool.shape or k_pool.stride(3) != 1:
+        raise ValueError("k_pool and v_pool must share shape and strides, with a contiguous head_dim")
+    if not block_table.is_contiguous() or block_table.shape[0] != q.shape[0]:
+        raise ValueError("block_table must be dense [B, max_blocks_per_seq]")
+    B, R, Hq, D = q.shape
+    nb, Hkv, bs, Dk = k_pool.shape
+    if Dk != D:
+        raise ValueError("q and k_pool disagree on head_dim")
+    mb = block_table.shape[1]
+    shape = _AttnShape(B, Hq, Hkv, D, mb * bs, 0, 0, 0)
+    paged = _PagedKv(bs, nb, mb, 0, k_pool.stride(0), k_pool.stride(1), k_pool.stride(2))
+    _check(load_library().rapid_verify_attention_paged(_p(q), _p(k_pool), _p(v_pool), _p(block_table),
+                                                       ctypes.byref(paged), _p(ctx_lens), gamma, _p(out),
+                                                       ctypes.byref(shape), _attn_params(params), _p(workspace),
+                                                       _nbytes(workspace), _stream_ptr(stream)))
 
 
 def rapid_accept(target_logits, draft_logits, draft_tokens, uniforms, eta, out_accept_len, out_next_token,

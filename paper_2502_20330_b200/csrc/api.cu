@@ -167,6 +167,21 @@ int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cac
                                    static_cast<cudaStream_t>(cuda_stream));
 }
 
+int rapid_verify_attention_paged(const void* q, const void* k_pool, const void* v_pool,
+                                 const int32_t* block_table, const rapid_paged_kv* paged,
+                                 const int32_t* ctx_lens, int gamma, void* out,
+                                 const rapid_attn_shape* shape, const rapid_attn_params* params,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    clear_error();
+    if (!paged || !block_table) {
+        set_error("rapid_verify_attention_paged: NULL paged geometry or block table");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    return launch_verify_attention(q, k_pool, v_pool, ctx_lens, gamma, out, shape, params, workspace,
+                                   workspace_bytes, static_cast<cudaStream_t>(cuda_stream), paged,
+                                   block_table);
+}
+
 int rapid_accept(const float* target_logits, const float* draft_logits,
                  const int32_t* draft_tokens, const float* uniforms, float eta,
                  int32_t* out_accept_len, int32_t* out_next_token,

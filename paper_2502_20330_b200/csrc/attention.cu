@@ -41,6 +41,10 @@ struct AttnArgs {
     int Lmax;
     int num_ctas;
     float scale_log2;  // softmax scale * log2(e)
+    // paged cache (block_table != nullptr): logical key tile t of sequence b lives in physical
+    // block block_table[b * max_blocks + (t >> tile_shift)], at tile (t & tile_mask) inside it
+    const int32_t* block_table;
+    int max_blocks, num_blocks, tile_shift;
 };
 
 struct Walk {
@@ -287,17 +291,31 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 for (int t = 0; t < seg && ok; ++t, ++n) {
                     const int s = n % nstage;
+                    // coordinates of the tile: (key, outermost) = (logical position, sequence), or,
+                    // paged, (position inside the block, physical block).  The table entry is
+                    // fetched before the wait for a free stage, so the two overlap.
+                    int key0 = (w.tile + t) * kTile, outer = w.b;
+                    if (a.block_table) {
+                        const int tile = w.tile + t;
+                        outer = __ldg(a.block_table + (size_t)w.b * a.max_blocks + (tile >> a.tile_shift));
+                        key0 = (tile & ((1 << a.tile_shift) - 1)) * kTile;
+                    }
                     if (n >= nstage)
                         ok = mbar_wait_bounded_relaxed(&empty_bar[s], ((n / nstage) - 1) & 1, abort_flag);
                     if (!ok) break;
-                    const int key0 = (w.tile + t) * kTile;
+                    if (a.block_table && (unsigned)outer >= (unsigned)a.num_blocks) {
+                        // the copy below reads zeros for a block outside the pool (the tensor map
+                        // bounds every coordinate); say so in the status word
+                        atomicOr(a.status, RAPID_STATUS_BAD_BLOCK_TABLE);
+                        outer = a.num_blocks;
+                    }
                     mbar_arrive_expect_tx(&full_bar[s], 2 * NHALF * BLK);
 #pragma unroll
                     for (int h = 0; h < NHALF; ++h) {
                         tma_load_4d(smem_gen + off_k + h * ring + s * BLK, &tmK, &full_bar[s], h * 64,
-                                    key0, w.kvh, w.b);
+                                    key0, w.kvh, outer);
                         tma_load_4d(smem_gen + off_v + h * ring + s * BLK, &tmV, &full_bar[s], h * 64,
-                                    key0, w.kvh, w.b);
+                                    key0, w.kvh, outer);
                     }
                 }
                 walk_advance(a, w, seg);
@@ -677,14 +695,16 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-int make_kv_map(CUtensorMap* map, const void* base, const rapid_attn_shape& s, int64_t sb,
-                int64_t sh, int64_t sl) {
+// Tensor map of a cache [outer][Hkv][keys][D] with element strides sb / sh / sl: outer = sequences
+// and keys = Lmax for a contiguous cache, outer = physical blocks and keys = block size for a paged one.
+int make_kv_map(CUtensorMap* map, const void* base, const rapid_attn_shape& s, int64_t outer,
+                int64_t keys, int64_t sb, int64_t sh, int64_t sl) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) {
         set_error("cuTensorMapEncodeTiled is not available from the CUDA driver");
         return RAPID_ERR_CUDA;
     }
-    cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)s.Lmax, (cuuint64_t)s.Hkv, (cuuint64_t)s.B};
+    cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)keys, (cuuint64_t)s.Hkv, (cuuint64_t)outer};
     cuuint64_t strides[3] = {(cuuint64_t)sl * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
     cuuint32_t box[4] = {64, (cuuint32_t)kTile, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -790,9 +810,14 @@ size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma) {
 int launch_verify_attention(const void* q, const void* k_cache, const void* v_cache,
                             const int32_t* ctx_lens, int gamma, void* out,
                             const rapid_attn_shape* shape, const rapid_attn_params* params,
-                            void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+                            void* workspace, size_t workspace_bytes, cudaStream_t stream,
+                            const rapid_paged_kv* paged, const int32_t* block_table) {
     if (!q || !k_cache || !v_cache || !ctx_lens || !out || !shape) {
         set_error("rapid_verify_attention: NULL argument");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (paged && !block_table) {
+        set_error("rapid_verify_attention_paged: NULL block table");
         return RAPID_ERR_INVALID_ARG;
     }
     if (!attn_shape_ok(shape, gamma)) {
@@ -816,9 +841,30 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
         set_error("rapid_verify_attention: Lmax %lld out of range", (long long)s.Lmax);
         return RAPID_ERR_INVALID_ARG;
     }
-    const int64_t sl = s.kv_stride_l ? s.kv_stride_l : s.D;
-    const int64_t sh = s.kv_stride_h ? s.kv_stride_h : s.Lmax * sl;
-    const int64_t sb = s.kv_stride_b ? s.kv_stride_b : s.Hkv * sh;
+    int64_t sl, sh, sb, outer = s.B, keys = s.Lmax;
+    int tile_shift = 0;
+    if (paged) {
+        const int64_t bs = paged->block_size;
+        if (bs < kTile || (bs & (bs - 1)) || paged->num_blocks <= 0 || paged->max_blocks_per_seq <= 0) {
+            set_error("rapid_verify_attention_paged: block_size must be a power of two >= %d, num_blocks and "
+                      "max_blocks_per_seq positive", kTile);
+            return RAPID_ERR_UNSUPPORTED;
+        }
+        if (s.Lmax != (int64_t)paged->max_blocks_per_seq * bs) {
+            set_error("rapid_verify_attention_paged: shape->Lmax must equal max_blocks_per_seq * block_size");
+            return RAPID_ERR_INVALID_ARG;
+        }
+        while ((kTile << tile_shift) < bs) ++tile_shift;
+        sl = paged->stride_l ? paged->stride_l : s.D;
+        sh = paged->stride_h ? paged->stride_h : bs * sl;
+        sb = paged->stride_block ? paged->stride_block : s.Hkv * sh;
+        outer = paged->num_blocks;
+        keys = bs;
+    } else {
+        sl = s.kv_stride_l ? s.kv_stride_l : s.D;
+        sh = s.kv_stride_h ? s.kv_stride_h : s.Lmax * sl;
+        sb = s.kv_stride_b ? s.kv_stride_b : s.Hkv * sh;
+    }
     if (sl < s.D || sl % 8 || sh % 8 || sb % 8 || sh <= 0 || sb <= 0) {
         set_error("rapid_verify_attention: K/V strides must be positive multiples of 8 elements");
         return RAPID_ERR_UNSUPPORTED;
@@ -849,9 +895,9 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     }
 
     CUtensorMap tmK, tmV;
-    int rc = make_kv_map(&tmK, k_cache, s, sb, sh, sl);
+    int rc = make_kv_map(&tmK, k_cache, s, outer, keys, sb, sh, sl);
     if (rc != RAPID_OK) return rc;
-    rc = make_kv_map(&tmV, v_cache, s, sb, sh, sl);
+    rc = make_kv_map(&tmV, v_cache, s, outer, keys, sb, sh, sl);
     if (rc != RAPID_OK) return rc;
 
     AttnArgs a;
@@ -868,6 +914,10 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     a.Lmax = (int)s.Lmax;
     a.num_ctas = num_ctas;
     a.scale_log2 = scale * 1.4426950408889634f;
+    a.block_table = paged ? block_table : nullptr;
+    a.max_blocks = paged ? paged->max_blocks_per_seq : 0;
+    a.num_blocks = paged ? paged->num_blocks : 0;
+    a.tile_shift = tile_shift;
 
     CUtensorMap tmQ;
     rc = make_q_map(&tmQ, q, s, G, R);

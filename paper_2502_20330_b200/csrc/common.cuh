@@ -55,7 +55,8 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 int launch_verify_attention(const void* q, const void* k_cache, const void* v_cache,
                             const int32_t* ctx_lens, int gamma, void* out,
                             const rapid_attn_shape* shape, const rapid_attn_params* params,
-                            void* workspace, size_t workspace_bytes, cudaStream_t stream);
+                            void* workspace, size_t workspace_bytes, cudaStream_t stream,
+                            const rapid_paged_kv* paged = nullptr, const int32_t* block_table = nullptr);
 int launch_accept(const float* target_logits, const float* draft_logits,
                   const int32_t* draft_tokens, const float* uniforms, float eta,
                   int32_t* out_accept_len, int32_t* out_next_token,

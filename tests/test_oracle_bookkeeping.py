@@ -1,5 +1,6 @@
 """Pins for the oracle's step bookkeeping: invariants any correct append / commit must satisfy."""
 import numpy as np
+import pytest
 
 import oracle
 
@@ -31,3 +32,33 @@ def test_commit_keeps_the_accepted_prefix():
     # append then commit with n accepted leaves exactly 1 + n new rows
     for n in range(6):
         assert oracle.step_commit(np.array([100 + 6]), np.array([n]), 5)[0] == 100 + 1 + n
+
+
+def test_paged_gather_identity_table_is_a_reshape():
+    """With block i of sequence 0 stored in physical block i, the gathered cache is the pool's
+    blocks laid end to end."""
+    rng = np.random.default_rng(3)
+    nb, Hkv, bs, D = 5, 2, 4, 3
+    pool = rng.integers(0, 65535, size=(nb, Hkv, bs, D), dtype=np.uint16)
+    table = np.arange(nb, dtype=np.int32)[None, :]
+    got = oracle.paged_gather(pool, table, [nb * bs])
+    want = pool.transpose(1, 0, 2, 3).reshape(1, Hkv, nb * bs, D)
+    np.testing.assert_array_equal(got, want)
+
+
+def test_paged_gather_follows_the_table_and_stops_at_the_length():
+    rng = np.random.default_rng(4)
+    nb, Hkv, bs, D = 7, 1, 2, 2
+    pool = rng.integers(1, 65535, size=(nb, Hkv, bs, D), dtype=np.uint16)
+    table = np.array([[6, 0, 3], [2, 5, -1]], dtype=np.int32)
+    got = oracle.paged_gather(pool, table, [5, 3])
+    # sequence 0: keys 0,1 <- block 6; 2,3 <- block 0; 4 <- block 3 row 0; key 5 is past its length
+    np.testing.assert_array_equal(got[0, 0, 0], pool[6, 0, 0])
+    np.testing.assert_array_equal(got[0, 0, 3], pool[0, 0, 1])
+    np.testing.assert_array_equal(got[0, 0, 4], pool[3, 0, 0])
+    assert (got[0, 0, 5] == 0).all()
+    # sequence 1: key 2 <- block 5 row 0; the -1 entry is never looked up
+    np.testing.assert_array_equal(got[1, 0, 2], pool[5, 0, 0])
+    assert (got[1, 0, 3:] == 0).all()
+    with pytest.raises(ValueError):
+        oracle.paged_gather(pool, np.array([[9]], dtype=np.int32), [1])

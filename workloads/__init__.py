@@ -113,6 +113,39 @@ def attention_inputs(cfg: VerifyConfig, seed: int, device="cpu", layer: int = 0,
     return q, k, v, ctx.to(device)
 
 
+def paged_layout(k: torch.Tensor, v: torch.Tensor, ctx_lens: torch.Tensor, block_size: int, seed: int,
+                 spare_blocks: int = 3, token_major: bool = False):
+    """Scatter contiguous caches k, v [B,Hkv,Lmax,D] into a pool of ``block_size``-key blocks in a
+    seeded random physical order, as a serving engine's allocator would leave them.
+
+    Returns (k_pool, v_pool, block_table): pools [num_blocks, Hkv, block_size, D] (a strided view of
+    [num_blocks, block_size, Hkv, D] storage when ``token_major``), block_table [B, max_blocks] int32.
+    Blocks no sequence uses (``spare_blocks`` of them, and table entries past a sequence's length,
+    which are -1) hold NaN: nothing may read them."""
+    B, Hkv, Lmax, D = k.shape
+    mb = (Lmax + block_size - 1) // block_size
+    used = [(int(ctx_lens[b]) + block_size - 1) // block_size for b in range(B)]
+    nb = sum(used) + spare_blocks
+    g = _gen(seed * 3000017 + 23, "cpu")
+    perm = torch.randperm(nb, generator=g)
+    table = torch.full((B, mb), -1, dtype=torch.int32)
+    if token_major:
+        kp = torch.full((nb, block_size, Hkv, D), float("nan"), dtype=k.dtype, device=k.device).permute(0, 2, 1, 3)
+        vp = torch.full((nb, block_size, Hkv, D), float("nan"), dtype=k.dtype, device=k.device).permute(0, 2, 1, 3)
+    else:
+        kp = torch.full((nb, Hkv, block_size, D), float("nan"), dtype=k.dtype, device=k.device)
+        vp = torch.full((nb, Hkv, block_size, D), float("nan"), dtype=k.dtype, device=k.device)
+    nxt = 0
+    for b in range(B):
+        for i in range(used[b]):
+            blk = int(perm[nxt]); nxt += 1
+            table[b, i] = blk
+            lo, hi = i * block_size, min((i + 1) * block_size, Lmax)
+            kp[blk, :, :hi - lo] = k[b, :, lo:hi]
+            vp[blk, :, :hi - lo] = v[b, :, lo:hi]
+    return kp, vp, table.to(k.device)
+
+
 def accept_inputs(cfg: VerifyConfig, seed: int, device="cpu"):
     """Draw target_logits [B,R,V] f32, draft_logits [B,gamma,V] f32,
     draft_tokens [B,gamma] i32 (each ~ softmax of its draft row, by a library
