@@ -330,6 +330,19 @@ int rapid_kv_append(const void* k_new, const void* v_new, void* k_cache, void* v
                     int32_t* status_word, void* cuda_stream);
 
 /*
+ * rapid_kv_append into a paged cache (see rapid_paged_kv): position ctx_lens[b] + i of sequence b
+ * is row (ctx_lens[b] + i) % block_size of physical block
+ * block_table[b, (ctx_lens[b] + i) / block_size].  The table must already name a block for every
+ * new position (handing out blocks is the caller's allocator's job); a position whose entry is
+ * outside [0, num_blocks) is not written and sets RAPID_STATUS_BAD_BLOCK_TABLE.  The capacity of a
+ * sequence is max_blocks_per_seq * block_size; block_size need not be a power of two here.
+ *   k_new, v_new : device [B, R, Hkv, D] bf16, dense;  k_pool, v_pool, block_table : device
+ */
+int rapid_kv_append_paged(const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                          const int32_t* block_table, const rapid_paged_kv* paged, int32_t* ctx_lens,
+                          int gamma, int B, int Hkv, int D, int32_t* status_word, void* cuda_stream);
+
+/*
  * Closes a verify step (Algorithm 1: accepted drafts become x_j, the rest is discarded): of the R
  * rows appended before the step the cache keeps the last accepted token and the accept_len[b]
  * accepted drafts,  ctx_lens[b] -= gamma - accept_len[b].  (The token sampled by the step is

@@ -231,6 +231,36 @@ def kv_append(k_cache, v_cache, k_new, v_new, ctx_lens, gamma):
     return k_cache, v_cache, ctx.astype(np.int32), overflowed
 
 
+def kv_append_paged(k_pool, v_pool, block_table, k_new, v_new, ctx_lens, gamma):
+    """kv_append for a paged cache: the row for position j of sequence b goes to
+    pool[block_table[b, j // block_size], :, j % block_size, :].  A sequence without room for R rows
+    (capacity = max_blocks * block_size) is left as it is; a position whose table entry is not a
+    block of the pool is skipped.  Works on copies; returns (k_pool, v_pool, ctx_lens, overflowed, bad_table)."""
+    k_pool = np.array(k_pool, copy=True)
+    v_pool = np.array(v_pool, copy=True)
+    table = np.asarray(block_table)
+    ctx = np.array(ctx_lens, dtype=np.int64, copy=True)
+    R = gamma + 1
+    nb, Hkv, bs, _ = k_pool.shape
+    cap = table.shape[1] * bs
+    overflowed = bad_table = False
+    for b in range(table.shape[0]):
+        L = int(ctx[b])
+        if L < 0 or L + R > cap:
+            overflowed = True
+            continue
+        for i in range(R):
+            blk = int(table[b, (L + i) // bs])
+            if not 0 <= blk < nb:
+                bad_table = True
+                continue
+            for h in range(Hkv):
+                k_pool[blk, h, (L + i) % bs, :] = k_new[b, i, h, :]
+                v_pool[blk, h, (L + i) % bs, :] = v_new[b, i, h, :]
+        ctx[b] = L + R
+    return k_pool, v_pool, ctx.astype(np.int32), overflowed, bad_table
+
+
 def step_commit(ctx_lens, accept_len, gamma):
     """Bookkeeping after a verify step (Algorithm 1: x_j <- x'_j for the accepted drafts, the others are
     discarded): the cache keeps the last accepted token and the accepted drafts, L_b -= gamma - n_b."""

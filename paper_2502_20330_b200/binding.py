@@ -23,7 +23,7 @@ EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
     "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_paged", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
-    "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_step_commit",
+    "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_kv_append_paged", "rapid_step_commit",
     "rapid_last_error",
     "rapid_version", "rapid_kernel_launch_count", "rapid_kernel_launch_count_reset",
 ]
@@ -129,6 +129,8 @@ def load_library():
         lib.rapid_verify_step_host_arena_bytes.argtypes = [ctypes.POINTER(_AttnShape), i32, ctypes.POINTER(_AcceptShape)]
         lib.rapid_kv_append.restype = i32
         lib.rapid_kv_append.argtypes = [vp, vp, vp, vp, vp, i32, ctypes.POINTER(_AttnShape), vp, vp]
+        lib.rapid_kv_append_paged.restype = i32
+        lib.rapid_kv_append_paged.argtypes = [vp, vp, vp, vp, vp, ctypes.POINTER(_PagedKv), vp, i32, i32, i32, i32, vp, vp]
         lib.rapid_step_commit.restype = i32
         lib.rapid_step_commit.argtypes = [vp, vp, i32, i32, vp, vp]
         lib.rapid_last_error.restype = ctypes.c_char_p
@@ -346,6 +348,26 @@ def rapid_kv_append(k_new, v_new, k_cache, v_cache, ctx_lens, gamma, status_word
     shape = _AttnShape(B, Hkv, Hkv, D, k_cache.shape[2], k_cache.stride(0), k_cache.stride(1), k_cache.stride(2))
     _check(load_library().rapid_kv_append(_p(k_new), _p(v_new), _p(k_cache), _p(v_cache), _p(ctx_lens), gamma,
                                           ctypes.byref(shape), _p(status_word), _stream_ptr(stream)))
+
+
+def rapid_kv_append_paged(k_new, v_new, k_pool, v_pool, block_table, ctx_lens, gamma, status_word, stream=None) -> None:
+    """rapid_kv_append into pools [num_blocks, Hkv, block_size, D] through block_table [B, max_blocks] (int32)."""
+    if k_new.dtype != torch.bfloat16 or v_new.dtype != torch.bfloat16 or ctx_lens.dtype != torch.int32 \
+            or block_table.dtype != torch.int32 or k_pool.dtype != torch.bfloat16 or v_pool.dtype != torch.bfloat16:
+        raise TypeError("k_new/v_new and the pools must be bfloat16, ctx_lens and block_table int32")
+    B, R, Hkv, D = k_new.shape
+    if R != gamma + 1 or not (k_new.is_contiguous() and v_new.is_contiguous()) or k_new.shape != v_new.shape:
+        raise ValueError("k_new and v_new must be dense [B, gamma+1, Hkv, D]")
+    if k_pool.stride() != v_pool.stride() or k_pool.shape != v_pool.shape or k_pool.stride(3) != 1 \
+            or k_pool.shape[1] != Hkv or k_pool.shape[3] != D:
+        raise ValueError("k_pool and v_pool must be [num_blocks, Hkv, block_size, D] with equal strides")
+    if not block_table.is_contiguous() or block_table.shape[0] != B:
+        raise ValueError("block_table must be dense [B, max_blocks_per_seq]")
+    paged = _PagedKv(k_pool.shape[2], k_pool.shape[0], block_table.shape[1], 0, k_pool.stride(0), k_pool.stride(1),
+                     k_pool.stride(2))
+    _check(load_library().rapid_kv_append_paged(_p(k_new), _p(v_new), _p(k_pool), _p(v_pool), _p(block_table),
+                                                ctypes.byref(paged), _p(ctx_lens), gamma, B, Hkv, D,
+                                                _p(status_word), _stream_ptr(stream)))
 
 
 def rapid_step_commit(ctx_lens, accept_len, gamma, status_word, stream=None) -> None:

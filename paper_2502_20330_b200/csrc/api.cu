@@ -47,6 +47,36 @@ __global__ void kv_append_kernel(const uint4* __restrict__ k_new, const uint4* _
 }
 
 // Runs after the copies (same stream): ctx_lens[b] += R where the rows fitted.
+// The same append into a paged cache: position L + i of sequence b is row (L + i) % block_size of
+// physical block block_table[b][(L + i) / block_size].
+__global__ void kv_append_paged_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                                       __nv_bfloat16* k_pool, __nv_bfloat16* v_pool,
+                                       const int32_t* __restrict__ block_table,
+                                       const int32_t* __restrict__ ctx_lens, int R, int Hkv, int D,
+                                       int block_size, int num_blocks, int max_blocks, long long sblk,
+                                       long long sh, long long sl, int32_t* status) {
+    const int b = blockIdx.z, i = blockIdx.y, h = blockIdx.x;
+    const long long L = ctx_lens[b];
+    const long long Lmax = (long long)max_blocks * block_size;
+    if (L < 0 || L + R > Lmax) {
+        if (i == 0 && h == 0 && threadIdx.x == 0) atomicOr(status, RAPID_STATUS_BAD_CTX_LEN);
+        return;
+    }
+    const long long pos = L + i;
+    const int blk = block_table[(size_t)b * max_blocks + pos / block_size];
+    if (blk < 0 || blk >= num_blocks) {  // no block behind this position: the row is not written
+        if (h == 0 && threadIdx.x == 0) atomicOr(status, RAPID_STATUS_BAD_BLOCK_TABLE);
+        return;
+    }
+    const int chunks = D / 8;
+    const size_t src = (((size_t)b * R + i) * Hkv + h) * chunks;
+    const size_t dst = (size_t)blk * sblk + (size_t)h * sh + (size_t)(pos % block_size) * sl;
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+        reinterpret_cast<uint4*>(k_pool + dst)[c] = k_new[src + c];
+        reinterpret_cast<uint4*>(v_pool + dst)[c] = v_new[src + c];
+    }
+}
+
 __global__ void kv_append_lens_kernel(int32_t* ctx_lens, int B, int R, long long Lmax) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
@@ -106,6 +136,45 @@ int rapid_kv_append(const void* k_new, const void* v_new, void* k_cache, void* v
         static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache), ctx_lens, R, s.Hkv, s.D,
         (long long)s.Lmax, (long long)sb, (long long)sh, (long long)sl, status_word);
     kv_append_lens_kernel<<<(s.B + 127) / 128, 128, 0, st>>>(ctx_lens, s.B, R, (long long)s.Lmax);
+    RAPID_CUDA_CHECK(cudaGetLastError());
+    count_launch(2);
+    return RAPID_OK;
+}
+
+int rapid_kv_append_paged(const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                          const int32_t* block_table, const rapid_paged_kv* paged, int32_t* ctx_lens,
+                          int gamma, int B, int Hkv, int D, int32_t* status_word, void* cuda_stream) {
+    clear_error();
+    if (!k_new || !v_new || !k_pool || !v_pool || !block_table || !paged || !ctx_lens || !status_word) {
+        set_error("rapid_kv_append_paged: NULL argument");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (B <= 0 || Hkv <= 0 || gamma < 0 || B > 65535 || gamma + 1 > 65535 || paged->block_size <= 0 ||
+        paged->num_blocks <= 0 || paged->max_blocks_per_seq <= 0) {
+        set_error("rapid_kv_append_paged: invalid shape");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (D <= 0 || D % 8) {
+        set_error("rapid_kv_append_paged: head_dim must be a positive multiple of 8");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const int64_t sl = paged->stride_l ? paged->stride_l : D;
+    const int64_t sh = paged->stride_h ? paged->stride_h : (int64_t)paged->block_size * sl;
+    const int64_t sblk = paged->stride_block ? paged->stride_block : Hkv * sh;
+    if (sl % 8 || sh % 8 || sblk % 8 ||
+        (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_pool | (uintptr_t)v_pool) & 15)) {
+        set_error("rapid_kv_append_paged: strides must be multiples of 8 elements and pointers 16-byte aligned");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const int R = gamma + 1;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    kv_append_paged_kernel<<<dim3(Hkv, R, B), 32, 0, st>>>(
+        static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
+        static_cast<__nv_bfloat16*>(k_pool), static_cast<__nv_bfloat16*>(v_pool), block_table, ctx_lens, R,
+        Hkv, D, paged->block_size, paged->num_blocks, paged->max_blocks_per_seq, (long long)sblk,
+        (long long)sh, (long long)sl, status_word);
+    kv_append_lens_kernel<<<(B + 127) / 128, 128, 0, st>>>(
+        ctx_lens, B, R, (long long)paged->max_blocks_per_seq * paged->block_size);
     RAPID_CUDA_CHECK(cudaGetLastError());
     count_launch(2);
     return RAPID_OK;

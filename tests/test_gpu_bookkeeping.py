@@ -99,3 +99,32 @@ def test_several_steps_of_the_outer_loop():
         seen.update(alen.cpu().tolist())
     assert int(status.item()) == 0 and len(seen) >= 3
     assert R.workspace_status(aws) == 0 and R.workspace_status(cws) == 0
+
+
+@pytest.mark.parametrize("token_major", [False, True])
+def test_paged_append_matches_the_oracle_bit_for_bit(token_major):
+    import paper_2502_20330_b200 as R
+    B, Hkv, bs, D, gamma, mb = 4, 2, 64, 128, 3, 5
+    nb = B * mb + 3
+    g = torch.Generator(device="cuda").manual_seed(8)
+    if token_major:
+        kp = torch.randn(nb, bs, Hkv, D, generator=g, device="cuda").bfloat16().permute(0, 2, 1, 3)
+        vp = torch.randn(nb, bs, Hkv, D, generator=g, device="cuda").bfloat16().permute(0, 2, 1, 3)
+    else:
+        kp = torch.randn(nb, Hkv, bs, D, generator=g, device="cuda").bfloat16()
+        vp = torch.randn(nb, Hkv, bs, D, generator=g, device="cuda").bfloat16()
+    kn = torch.randn(B, gamma + 1, Hkv, D, generator=g, device="cuda").bfloat16()
+    vn = torch.randn(B, gamma + 1, Hkv, D, generator=g, device="cuda").bfloat16()
+    table = torch.randperm(nb, generator=torch.Generator().manual_seed(9))[:B * mb].reshape(B, mb).to(torch.int32)
+    table[1, 2] = -1                                   # sequence 1 crosses into a block nobody handed out
+    table = table.cuda()
+    ctx = torch.tensor([0, 126, 62, 318], dtype=torch.int32, device="cuda")   # the last has no room (cap 320)
+    rk, rv, rctx, over, bad = oracle.kv_append_paged(_bits(kp), _bits(vp), table.cpu().numpy(), _bits(kn), _bits(vn),
+                                                     ctx.cpu().numpy(), gamma)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    R.rapid_kv_append_paged(kn, vn, kp, vp, table, ctx, gamma, status)
+    torch.cuda.synchronize()
+    assert (_bits(kp) == rk).all() and (_bits(vp) == rv).all()
+    assert ctx.cpu().numpy().tolist() == rctx.tolist()
+    assert over and bad
+    assert int(status.item()) == (R.STATUS_BAD_CTX_LEN | R.STATUS_BAD_BLOCK_TABLE)

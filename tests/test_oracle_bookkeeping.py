@@ -62,3 +62,29 @@ def test_paged_gather_follows_the_table_and_stops_at_the_length():
     assert (got[1, 0, 3:] == 0).all()
     with pytest.raises(ValueError):
         oracle.paged_gather(pool, np.array([[9]], dtype=np.int32), [1])
+
+
+def test_paged_append_commutes_with_gather():
+    """Appending to the paged cache and then writing it out contiguously gives what appending to the
+    written-out cache gives."""
+    rng = np.random.default_rng(5)
+    B, Hkv, bs, D, gamma, mb = 3, 2, 4, 3, 2, 4
+    R = gamma + 1
+    nb = B * mb + 2
+    perm = rng.permutation(nb)[:B * mb].reshape(B, mb).astype(np.int32)
+    kp = rng.integers(1, 60000, (nb, Hkv, bs, D)).astype(np.uint16)
+    vp = rng.integers(1, 60000, (nb, Hkv, bs, D)).astype(np.uint16)
+    ctx = np.array([5, 0, 14], dtype=np.int32)          # the last one has no room for 3 more of 16
+    kn = rng.integers(1, 60000, (B, R, Hkv, D)).astype(np.uint16)
+    vn = rng.integers(1, 60000, (B, R, Hkv, D)).astype(np.uint16)
+    kp2, vp2, ctx2, over, bad = oracle.kv_append_paged(kp, vp, perm, kn, vn, ctx, gamma)
+    assert over and not bad
+    kc, vc, ctx3, over3 = oracle.kv_append(oracle.paged_gather(kp, perm, [mb * bs] * B),
+                                           oracle.paged_gather(vp, perm, [mb * bs] * B), kn, vn, ctx, gamma)
+    np.testing.assert_array_equal(ctx2, ctx3)
+    np.testing.assert_array_equal(ctx2, [8, 3, 14])
+    np.testing.assert_array_equal(oracle.paged_gather(kp2, perm, [mb * bs] * B), kc)
+    np.testing.assert_array_equal(oracle.paged_gather(vp2, perm, [mb * bs] * B), vc)
+    # blocks no table entry names are untouched
+    unused = sorted(set(range(nb)) - set(perm.ravel().tolist()))
+    np.testing.assert_array_equal(kp2[unused], kp[unused])
