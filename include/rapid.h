@@ -93,6 +93,10 @@ typedef struct rapid_attn_params {
     float* out_f32;   /* device [B, R, Hq, D] fp32 output before bf16 rounding, or NULL           */
     void* split_done_event; /* a cudaEvent_t recorded on the stream between the split and the merge
                                kernel (lets a caller time the two separately), or NULL          */
+    int32_t all_keys_visible; /* non-zero: no causal stair, every row sees all ctx_lens[b] keys, and
+                                 ctx_lens[b] >= 1 suffices.  For a shard of the context that does not
+                                 hold the rows' own keys (see rapid_merge_partials)                */
+    int32_t reserved;
 } rapid_attn_params;
 
 /*
@@ -162,6 +166,22 @@ int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cac
                            const int32_t* ctx_lens, int gamma, void* out,
                            const rapid_attn_shape* shape, const rapid_attn_params* params,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Combines P partial attention results of the same rows over disjoint sets of keys -- the context
+ * of a sequence sharded over P GPUs, each of which ran rapid_verify_attention on its keys with
+ * out_f32 and lse_out (all_keys_visible on every shard but the one that holds the R newest keys)
+ * and gathered the others' results.  (Not in the paper, whose runs keep a sequence's cache on one
+ * device or use the serving stack's own parallelism; the identity is the one the split kernels'
+ * merge uses.)
+ *   out[r,:] = sum_p exp(lse_parts[p,r] - LSE_r) * o_parts[p,r,:],  LSE_r = log sum_p exp(lse_parts[p,r])
+ *   o_parts   : device fp32 [P, rows, D], each normalised by its own sum;  lse_parts : device fp32 [P, rows]
+ *   out       : device bf16 [rows, D] or NULL;  out_f32 : device fp32 [rows, D] or NULL (one of the two at least)
+ *   lse_out   : device fp32 [rows] or NULL
+ * A partial with lse = -inf (a shard without keys) takes no part; a row with no keys anywhere is 0.
+ */
+int rapid_merge_partials(const float* o_parts, const float* lse_parts, int P, int64_t rows, int D, void* out,
+                         float* out_f32, float* lse_out, void* cuda_stream);
 
 /*
  * Geometry of a paged KV cache: a pool of fixed-size blocks shared by all

@@ -187,6 +187,24 @@ def accept(target_logits, draft_logits, draft_tokens, uniforms, eta, T=1.0, tail
     return dict(accept_len=accept_len, next_token=next_token, flags=flags, ratios=ratios)
 
 
+def merge_partials(o_parts, lse_parts):
+    """Attention over a union of disjoint key sets from the attentions over each set: with
+    Z_p = sum_j exp(s_j) over set p (lse_p = log Z_p) and o_p = sum_j exp(s_j) v_j / Z_p,
+    the result over the union is sum_p Z_p o_p / sum_p Z_p.  fp64; o_parts [P, ..., D], lse_parts [P, ...].
+    A set without keys has lse = -inf and takes no part.  Returns (out [..., D], lse [...])."""
+    o = np.asarray(o_parts, dtype=np.float64)
+    l = np.asarray(lse_parts, dtype=np.float64)
+    M = l.max(axis=0)
+    safe = np.where(np.isfinite(M), M, 0.0)
+    w = np.exp(l - safe)                      # exp(-inf) = 0 drops the empty sets
+    den = w.sum(axis=0)
+    num = (w[..., None] * np.where(w[..., None] > 0, o, 0.0)).sum(axis=0)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        out = np.where(den[..., None] > 0, num / den[..., None], 0.0)
+        lse = np.where(den > 0, safe + np.log(den), -np.inf)
+    return out, lse
+
+
 def paged_gather(pool, block_table, ctx_lens):
     """A paged cache written out as the contiguous cache it stands for (storage only; the paper's
     attention is defined on the logical sequence): pool [num_blocks, Hkv, block_size, D],

@@ -19,6 +19,7 @@ from .binding import (  # noqa: F401
     rapid_accept,
     rapid_accept_static,
     rapid_kv_append,
+    rapid_merge_partials,
     rapid_kv_append_paged,
     rapid_step_commit,
     rapid_verify_attention,

@@ -21,7 +21,7 @@ RESIDUAL_PHAT = 1
 
 EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
-    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_paged", "rapid_accept", "rapid_accept_static",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
     "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_kv_append_paged", "rapid_step_commit",
     "rapid_last_error",
@@ -50,7 +50,8 @@ class _PagedKv(ctypes.Structure):
 class _AttnParams(ctypes.Structure):
     _fields_ = [("scale", ctypes.c_float), ("num_ctas", ctypes.c_int32),
                 ("lse_out", ctypes.c_void_p), ("out_f32", ctypes.c_void_p),
-                ("split_done_event", ctypes.c_void_p)]
+                ("split_done_event", ctypes.c_void_p), ("all_keys_visible", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
 
 
 class _AcceptShape(ctypes.Structure):
@@ -71,6 +72,7 @@ class AttnParams:
     lse_out: Optional[torch.Tensor] = None   # [B,R,Hq] float32
     out_f32: Optional[torch.Tensor] = None   # [B,R,Hq,D] float32
     split_done_event: Optional[int] = None   # cudaEvent_t handle recorded between split and merge
+    all_keys_visible: bool = False           # no causal stair: a context shard without the rows' own keys
 
 
 @dataclass
@@ -117,6 +119,8 @@ def load_library():
         lib.rapid_verify_attention.argtypes = attn_args + [vp, sz, vp]
         lib.rapid_verify_attention_paged.restype = i32
         lib.rapid_verify_attention_paged.argtypes = [vp, vp, vp, vp, ctypes.POINTER(_PagedKv)] + attn_args[3:] + [vp, sz, vp]
+        lib.rapid_merge_partials.restype = i32
+        lib.rapid_merge_partials.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp]
         lib.rapid_accept.restype = i32
         lib.rapid_accept.argtypes = acc_args + [vp, sz, vp]
         lib.rapid_accept_static.restype = i32
@@ -187,7 +191,7 @@ def _attn_params(p: Optional[AttnParams]):
         return None
     return ctypes.byref(_AttnParams(p.scale, p.num_ctas, p.lse_out.data_ptr() if p.lse_out is not None else None,
                                     p.out_f32.data_ptr() if p.out_f32 is not None else None,
-                                    p.split_done_event))
+                                    p.split_done_event, 1 if p.all_keys_visible else 0, 0))
 
 
 def _accept_shape(target_logits: torch.Tensor, draft_logits: torch.Tensor) -> _AcceptShape:
@@ -288,6 +292,22 @@ def rapid_verify_attention_paged(q, k_pool, v_pool, block_table, ctx_lens, gamma
                                                        ctypes.byref(paged), _p(ctx_lens), gamma, _p(out),
                                                        ctypes.byref(shape), _attn_params(params), _p(workspace),
                                                        _nbytes(workspace), _stream_ptr(stream)))
+
+
+def rapid_merge_partials(o_parts, lse_parts, out=None, out_f32=None, lse_out=None, stream=None) -> None:
+    """Log-sum-exp combination of P partial attention results: o_parts [P, ..., D] float32 (each normalised),
+    lse_parts [P, ...] float32 -> out [..., D] bfloat16 and / or out_f32, lse_out [...]."""
+    if o_parts.dtype != torch.float32 or lse_parts.dtype != torch.float32:
+        raise TypeError("o_parts and lse_parts must be float32")
+    if not (o_parts.is_contiguous() and lse_parts.is_contiguous()) or o_parts.shape[:-1] != lse_parts.shape:
+        raise ValueError("o_parts must be dense [P, ..., D] and lse_parts dense [P, ...]")
+    P, D = o_parts.shape[0], o_parts.shape[-1]
+    rows = lse_parts[0].numel()
+    for t, dt, n in ((out, torch.bfloat16, rows * D), (out_f32, torch.float32, rows * D), (lse_out, torch.float32, rows)):
+        if t is not None and (t.dtype != dt or t.numel() != n or not t.is_contiguous()):
+            raise ValueError("output tensors must be dense, of the rows' shape and of the documented dtype")
+    _check(load_library().rapid_merge_partials(_p(o_parts), _p(lse_parts), P, rows, D, _p(out), _p(out_f32),
+                                               _p(lse_out), _stream_ptr(stream)))
 
 
 def rapid_accept(target_logits, draft_logits, draft_tokens, uniforms, eta, out_accept_len, out_next_token,

@@ -251,6 +251,13 @@ int rapid_verify_attention_paged(const void* q, const void* k_pool, const void* 
                                    block_table);
 }
 
+int rapid_merge_partials(const float* o_parts, const float* lse_parts, int P, int64_t rows, int D, void* out,
+                         float* out_f32, float* lse_out, void* cuda_stream) {
+    clear_error();
+    return launch_merge_partials(o_parts, lse_parts, P, rows, D, out, out_f32, lse_out,
+                                 static_cast<cudaStream_t>(cuda_stream));
+}
+
 int rapid_accept(const float* target_logits, const float* draft_logits,
                  const int32_t* draft_tokens, const float* uniforms, float eta,
                  int32_t* out_accept_len, int32_t* out_next_token,

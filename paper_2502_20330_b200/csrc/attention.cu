@@ -45,6 +45,10 @@ struct AttnArgs {
     // block block_table[b * max_blocks + (t >> tile_shift)], at tile (t & tile_mask) inside it
     const int32_t* block_table;
     int max_blocks, num_blocks, tile_shift;
+    // stair = R: row i sees keys <= L - R + i (the R newest keys are the rows' own, causal among
+    // themselves); stair = 0: every row sees all L keys (a shard of the context without those rows).
+    // Lmin = the shortest admissible length: R resp. 1.
+    int stair, Lmin;
 };
 
 struct Walk {
@@ -62,7 +66,7 @@ __device__ __forceinline__ int tiles_of(int L) { return (L + kTile - 1) / kTile;
 __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     long long T = 0;
     for (int b = 0; b < a.B; ++b)
-        T += (long long)a.Hkv * tiles_of(clamp_len(a.ctx_lens[b], a.R, a.Lmax));
+        T += (long long)a.Hkv * tiles_of(clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax));
     // with fewer tiles than CTAs only the first T CTAs work, one tile each: no CTA inside the
     // range of a unit is ever empty, which the merge relies on
     const long long nc = T < a.num_ctas ? T : a.num_ctas;
@@ -81,7 +85,7 @@ __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     if (w.remaining <= 0) return;
     long long t = t0;
     for (int b = 0; b < a.B; ++b) {
-        const int L = clamp_len(a.ctx_lens[b], a.R, a.Lmax);
+        const int L = clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax);
         const int nt = tiles_of(L);
         const long long span = (long long)a.Hkv * nt;
         if (t < span) {
@@ -105,7 +109,7 @@ __device__ __forceinline__ void walk_advance(const AttnArgs& a, Walk& w, int seg
             w.kvh = 0;
             ++w.b;
             if (w.b < a.B) {
-                w.L = clamp_len(a.ctx_lens[w.b], a.R, a.Lmax);
+                w.L = clamp_len(a.ctx_lens[w.b], a.Lmin, a.Lmax);
                 w.ntiles = tiles_of(w.L);
             }
         }
@@ -268,7 +272,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             bool bad = false;
             for (int b = 0; b < a.B; ++b) {
                 const int L = a.ctx_lens[b];
-                bad |= (L < a.R) || (L > a.Lmax);
+                bad |= (L < a.Lmin) || (L > a.Lmax);
             }
             if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
         }
@@ -433,7 +437,8 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
         while (w.remaining > 0 && ok) {
             const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
             const int L = w.L;
-            const int lim = L - a.R + i_row;
+            const int lim = a.stair ? L - a.R + i_row : L - 1;
+            const int all_see = a.stair ? L - a.R : L - 1;  // the last key every row sees
             float m_ref = -INFINITY, l_run = 0.f;
             int last_n = -1;  // the stream's latest tile of this unit (CTA-wide index)
 
@@ -449,7 +454,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 tmem_ld_x32(tS + 32, sr[1]);
                 tmem_wait_ld();
 
-                if (key0 + kTile - 1 > L - a.R) {  // causal rows and the ragged end of the context
+                if (key0 + kTile - 1 > all_see) {  // causal rows and the ragged end of the context
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -598,7 +603,7 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     long long T = 0, t0 = 0;
     int nt_b = 0;
     for (int bb = 0; bb < a.B; ++bb) {
-        const int nt = tiles_of(clamp_len(a.ctx_lens[bb], a.R, a.Lmax));
+        const int nt = tiles_of(clamp_len(a.ctx_lens[bb], a.Lmin, a.Lmax));
         if (bb < b) t0 += (long long)a.Hkv * nt;
         if (bb == b) nt_b = nt;
         T += (long long)a.Hkv * nt;
@@ -672,6 +677,39 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
         }
         if (lse_out && lane == 0) lse_out[row] = (M + log2f(l)) * 0.69314718055994530942f;
     }
+}
+
+// Combines P partial attention results of the same rows over disjoint key sets (each normalised
+// by its own sum, with the natural-log sum-exp of its scores) into the result over the union:
+//   out = sum_p w_p o_p,  w_p = exp(lse_p - LSE),  LSE = log sum_p exp(lse_p).
+// One warp per row; a partial with lse = -inf (no keys) takes no part.
+__global__ void __launch_bounds__(128) merge_partials_kernel(const float* __restrict__ o_parts,
+                                                             const float* __restrict__ lse_parts, int P,
+                                                             long long rows, int D, __nv_bfloat16* out,
+                                                             float* out_f32, float* lse_out) {
+    const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+    if (row >= rows) return;
+    float M = -INFINITY;
+    for (int p = 0; p < P; ++p) M = fmaxf(M, lse_parts[(size_t)p * rows + row]);
+    float den = 0.f;
+    for (int p = 0; p < P; ++p) {
+        const float l = lse_parts[(size_t)p * rows + row];
+        den += (l == -INFINITY) ? 0.f : __expf(l - M);
+    }
+    for (int d = lane; d < D; d += 32) {
+        float acc = 0.f;
+        for (int p = 0; p < P; ++p) {
+            const float l = lse_parts[(size_t)p * rows + row];
+            if (l != -INFINITY) acc += __expf(l - M) * o_parts[((size_t)p * rows + row) * D + d];
+        }
+        const float val = (M == -INFINITY) ? 0.f : acc / den;
+        if (out) out[row * D + d] = __float2bfloat16_rn(val);
+        if (out_f32) out_f32[row * D + d] = val;
+    }
+    if (lse_out && lane == 0) lse_out[row] = (M == -INFINITY) ? -INFINITY : M + logf(den);
 }
 
 // ---- host side ----------------------------------------------------------------------------
@@ -798,6 +836,24 @@ bool attn_shape_ok(const rapid_attn_shape* s, int gamma) {
 
 }  // namespace
 
+int launch_merge_partials(const float* o_parts, const float* lse_parts, int P, int64_t rows, int D, void* out,
+                          float* out_f32, float* lse_out, cudaStream_t stream) {
+    if (!o_parts || !lse_parts || (!out && !out_f32) || P <= 0 || rows <= 0 || D <= 0) {
+        set_error("rapid_merge_partials: NULL argument or non-positive size");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const int64_t blocks = (rows + 3) / 4;
+    if (blocks > 0x7fffffffLL) {
+        set_error("rapid_merge_partials: too many rows");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    RAPID_CUDA_CHECK(launch_dependent(merge_partials_kernel, dim3((unsigned)blocks), dim3(128), 0, stream, o_parts,
+                                      lse_parts, P, (long long)rows, D, static_cast<__nv_bfloat16*>(out), out_f32,
+                                      lse_out));
+    count_launch(1);
+    return RAPID_OK;
+}
+
 size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma) {
     if (!attn_shape_ok(s, gamma)) return 0;
     if (s->D != 64 && s->D != 128) return 0;
@@ -837,7 +893,8 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
         set_error("rapid_verify_attention: %d grouped rows per KV head exceed 128", GR);
         return RAPID_ERR_UNSUPPORTED;
     }
-    if (s.Lmax < R || s.Lmax > 0x7fffffffLL - kTile) {
+    const bool all_visible = params && params->all_keys_visible;
+    if (s.Lmax < (all_visible ? 1 : R) || s.Lmax > 0x7fffffffLL - kTile) {
         set_error("rapid_verify_attention: Lmax %lld out of range", (long long)s.Lmax);
         return RAPID_ERR_INVALID_ARG;
     }
@@ -918,6 +975,8 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     a.max_blocks = paged ? paged->max_blocks_per_seq : 0;
     a.num_blocks = paged ? paged->num_blocks : 0;
     a.tile_shift = tile_shift;
+    a.stair = all_visible ? 0 : R;
+    a.Lmin = all_visible ? 1 : R;
 
     CUtensorMap tmQ;
     rc = make_q_map(&tmQ, q, s, G, R);

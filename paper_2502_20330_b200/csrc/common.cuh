@@ -57,6 +57,8 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
                             const rapid_attn_shape* shape, const rapid_attn_params* params,
                             void* workspace, size_t workspace_bytes, cudaStream_t stream,
                             const rapid_paged_kv* paged = nullptr, const int32_t* block_table = nullptr);
+int launch_merge_partials(const float* o_parts, const float* lse_parts, int P, int64_t rows, int D, void* out,
+                          float* out_f32, float* lse_out, cudaStream_t stream);
 int launch_accept(const float* target_logits, const float* draft_logits,
                   const int32_t* draft_tokens, const float* uniforms, float eta,
                   int32_t* out_accept_len, int32_t* out_next_token,
