@@ -250,6 +250,22 @@ int rapid_accept(const float* target_logits, const float* draft_logits,
                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Drafter-side sampling (Algorithm 1, the drafting loop: x'_j ~ q = softmax(d/T)), fused with what
+ * the later accept step needs from the drafter: the drawn token's log-probability and the row's
+ * softmax statistics, so that a caller can keep q(x') without another pass over the vocabulary.
+ *   draft_logits : device fp32 [B, V], row stride row_stride elements (0 = V); V % 4 == 0, 16-byte aligned
+ *   uniforms     : device fp32 [B] in [0,1); out_token[b] = the smallest token whose running sum of
+ *                  softmax(d_b/T) exceeds uniforms[b]   (the inverse-CDF rule of rapid_accept)
+ *   out_logq     : device fp32 [B], natural log of q(out_token[b])
+ *   out_row_stats: device fp32 [B, 2] = (max_v d_v/T, log sum_v exp(d_v/T)), or NULL
+ *   workspace    : device, >= rapid_accept_workspace_bytes() of {B, gamma = 0, V}, initialised
+ * Same kernel, limits and error behaviour as rapid_accept with gamma = 0.
+ */
+int rapid_draft_sample(const float* draft_logits, const float* uniforms, float temperature, int32_t* out_token,
+                       float* out_logq, float* out_row_stats, int32_t B, int64_t V, int64_t row_stride,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * rapid_accept without a caller workspace.  (The paper has no counterpart: this
  * entry point exists only for the sake of callers, not of the method.)
  *

@@ -187,6 +187,25 @@ def accept(target_logits, draft_logits, draft_tokens, uniforms, eta, T=1.0, tail
     return dict(accept_len=accept_len, next_token=next_token, flags=flags, ratios=ratios)
 
 
+def draft_sample(draft_logits, uniforms, T=1.0):
+    """Algorithm 1, drafting loop: x' ~ q = softmax(d/T), drawn by the inverse-CDF rule with the given
+    uniform.  fp64.  Returns (token [B] int32, log q(token) [B], row_stats [B,2] = (max d/T, log sum exp d/T))."""
+    d = np.asarray(draft_logits, dtype=np.float32).astype(np.float64)
+    B, V = d.shape
+    tok = np.zeros(B, np.int32)
+    logq = np.zeros(B)
+    stats = np.zeros((B, 2))
+    for b in range(B):
+        x = d[b] / float(T)
+        m = x.max()
+        e = np.exp(x - m)
+        S = e.sum()
+        tok[b] = inverse_cdf(e / S, float(np.float32(uniforms[b])))
+        stats[b] = (m, m + np.log(S))
+        logq[b] = x[tok[b]] - stats[b, 1]
+    return tok, logq, stats
+
+
 def merge_partials(o_parts, lse_parts):
     """Attention over a union of disjoint key sets from the attentions over each set: with
     Z_p = sum_j exp(s_j) over set p (lse_p = log Z_p) and o_p = sum_j exp(s_j) v_j / Z_p,

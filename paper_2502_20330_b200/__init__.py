@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     new_workspace,
     rapid_accept,
     rapid_accept_static,
+    rapid_draft_sample,
     rapid_kv_append,
     rapid_merge_partials,
     rapid_kv_append_paged,

@@ -21,7 +21,7 @@ RESIDUAL_PHAT = 1
 
 EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
-    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_accept", "rapid_accept_static",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
     "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_kv_append_paged", "rapid_step_commit",
     "rapid_last_error",
@@ -119,6 +119,8 @@ def load_library():
         lib.rapid_verify_attention.argtypes = attn_args + [vp, sz, vp]
         lib.rapid_verify_attention_paged.restype = i32
         lib.rapid_verify_attention_paged.argtypes = [vp, vp, vp, vp, ctypes.POINTER(_PagedKv)] + attn_args[3:] + [vp, sz, vp]
+        lib.rapid_draft_sample.restype = i32
+        lib.rapid_draft_sample.argtypes = [vp, vp, f32, vp, vp, vp, i32, i64, i64, vp, sz, vp]
         lib.rapid_merge_partials.restype = i32
         lib.rapid_merge_partials.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp]
         lib.rapid_accept.restype = i32
@@ -292,6 +294,25 @@ def rapid_verify_attention_paged(q, k_pool, v_pool, block_table, ctx_lens, gamma
                                                        ctypes.byref(paged), _p(ctx_lens), gamma, _p(out),
                                                        ctypes.byref(shape), _attn_params(params), _p(workspace),
                                                        _nbytes(workspace), _stream_ptr(stream)))
+
+
+def rapid_draft_sample(draft_logits, uniforms, temperature, out_token, out_logq, workspace, out_row_stats=None,
+                       stream=None) -> None:
+    """x' ~ softmax(draft_logits / T) by inverse CDF with the given uniforms; also log q(x') and, optionally,
+    (max, log-sum-exp) of every row.  draft_logits [B, V] float32 (rows may be strided), uniforms [B]."""
+    if draft_logits.dtype != torch.float32 or uniforms.dtype != torch.float32 or out_logq.dtype != torch.float32:
+        raise TypeError("logits, uniforms and out_logq must be float32")
+    if out_token.dtype != torch.int32 or (out_row_stats is not None and out_row_stats.dtype != torch.float32):
+        raise TypeError("out_token must be int32 and out_row_stats float32")
+    if draft_logits.dim() != 2 or draft_logits.stride(1) != 1:
+        raise ValueError("draft_logits must be [B, V] with a contiguous vocabulary axis")
+    B, V = draft_logits.shape
+    if uniforms.numel() != B or out_token.numel() != B or out_logq.numel() != B or \
+            (out_row_stats is not None and (out_row_stats.numel() != 2 * B or not out_row_stats.is_contiguous())):
+        raise ValueError("uniforms, out_token, out_logq must hold B entries and out_row_stats [B, 2]")
+    _check(load_library().rapid_draft_sample(_p(draft_logits), _p(uniforms), float(temperature), _p(out_token),
+                                             _p(out_logq), _p(out_row_stats), B, V, draft_logits.stride(0),
+                                             _p(workspace), _nbytes(workspace), _stream_ptr(stream)))
 
 
 def rapid_merge_partials(o_parts, lse_parts, out=None, out_f32=None, lse_out=None, stream=None) -> None:

@@ -46,6 +46,8 @@ struct AcceptArgs {
     int32_t* done;     // header word 1: clusters that have finished; back to 0 when the call ends
     float* ratio;      // [B*gamma]
     int32_t* cand;     // [B*R] candidate token of every row; bit 31 = drawn from p as a fallback
+    float* logq_out;   // optional [B]: natural log of the drawn token's probability (gamma = 0 calls)
+    float* stats_out;  // optional [B, 2]: max and log-sum-exp of the row's logits / T (gamma = 0 calls)
     int B, gamma, R, V;
     int slice;  // entries per CTA (multiple of 4)
     int per;    // consecutive entries per thread in the search (odd: conflict-free shared reads)
@@ -398,7 +400,16 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
         if (found != 0x7fffffff) atomicMin(&sh_tok, found);
         if (last >= 0) atomicMax(&sh_last, last);
         __syncthreads();
-        if (tid == 0) a.cand[row] = (sh_tok != 0x7fffffff ? sh_tok : (sh_last >= 0 ? sh_last : v0)) | fell_back;
+        if (tid == 0) {
+            const int tok = sh_tok != 0x7fffffff ? sh_tok : (sh_last >= 0 ? sh_last : v0);
+            a.cand[row] = tok | fell_back;
+            if (a.logq_out && !draft)  // log softmax of the row at the drawn token
+                a.logq_out[b] = (fmaf(__ldg(a.z + (size_t)row * a.zs + tok), c2, -Mz) - log2f(Sz)) * 0.69314718055994530942f;
+        }
+    }
+    if (a.stats_out && !draft && c == 0 && tid == 0) {
+        a.stats_out[2 * b] = Mz * 0.69314718055994530942f;
+        a.stats_out[2 * b + 1] = (Mz + log2f(Sz)) * 0.69314718055994530942f;
     }
 
     // ---- the last cluster to finish settles every sequence ----
@@ -446,6 +457,7 @@ size_t accept_workspace_bytes(const rapid_accept_shape* s) {
     size_t bytes = kWorkspaceHeaderBytes;
     bytes += align_up(drows * sizeof(float) + 4, 256);
     bytes += align_up(rows * sizeof(int32_t), 256);
+    bytes += align_up((size_t)s->B * sizeof(int32_t), 256);  // accept lengths nobody asked for (draft sampling)
     return bytes;
 }
 
@@ -453,13 +465,15 @@ int launch_accept(const float* target_logits, const float* draft_logits,
                   const int32_t* draft_tokens, const float* uniforms, float eta,
                   int32_t* out_accept_len, int32_t* out_next_token,
                   const rapid_accept_shape* shape, const rapid_accept_params* params,
-                  void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+                  void* workspace, size_t workspace_bytes, cudaStream_t stream, float* logq_out,
+                  float* stats_out) {
     if (!accept_shape_ok(shape)) {
         set_error("rapid_accept: invalid shape");
         return RAPID_ERR_INVALID_ARG;
     }
     const rapid_accept_shape& s = *shape;
-    if (!target_logits || !uniforms || !out_accept_len || !out_next_token ||
+    const bool sampling = logq_out || stats_out;  // rapid_draft_sample: gamma = 0, no accept lengths wanted
+    if (!target_logits || !uniforms || (!out_accept_len && !sampling) || !out_next_token ||
         (s.gamma > 0 && (!draft_logits || !draft_tokens))) {
         set_error("rapid_accept: NULL argument");
         return RAPID_ERR_INVALID_ARG;
@@ -499,7 +513,11 @@ int launch_accept(const float* target_logits, const float* draft_logits,
     a.d = draft_logits;
     a.tokens = draft_tokens;
     a.uniforms = uniforms;
-    a.accept_len = out_accept_len;
+    a.accept_len = out_accept_len ? out_accept_len
+                                  : reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + need -
+                                                               align_up((size_t)s.B * sizeof(int32_t), 256));
+    a.logq_out = logq_out;
+    a.stats_out = stats_out;
     a.next_token = out_next_token;
     a.ratio_out = params ? params->ratio_out : nullptr;
     a.B = s.B;
@@ -560,7 +578,7 @@ namespace {
 
 constexpr int kStaticMaxRows = 512;  // B * (gamma + 1) at most
 constexpr size_t kStaticScratchBytes =
-    kWorkspaceHeaderBytes + (size_t)kStaticMaxRows * (sizeof(float) + sizeof(int32_t)) + 2 * 256;
+    kWorkspaceHeaderBytes + (size_t)kStaticMaxRows * (sizeof(float) + 2 * sizeof(int32_t)) + 3 * 256;
 
 static __device__ __align__(256) unsigned char g_accept_scratch[kStaticScratchBytes];
 

@@ -251,6 +251,21 @@ int rapid_verify_attention_paged(const void* q, const void* k_pool, const void* 
                                    block_table);
 }
 
+int rapid_draft_sample(const float* draft_logits, const float* uniforms, float temperature, int32_t* out_token,
+                       float* out_logq, float* out_row_stats, int32_t B, int64_t V, int64_t row_stride,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    clear_error();
+    if (!out_logq) {
+        set_error("rapid_draft_sample: out_logq is required");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    rapid_accept_shape shape = {B, 0, V, row_stride, 0};
+    rapid_accept_params params = {temperature, 0.f, RAPID_RESIDUAL_PAPER, 0, nullptr};
+    return launch_accept(draft_logits, nullptr, nullptr, uniforms, 0.f, nullptr, out_token, &shape, &params,
+                         workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream), out_logq,
+                         out_row_stats);
+}
+
 int rapid_merge_partials(const float* o_parts, const float* lse_parts, int P, int64_t rows, int D, void* out,
                          float* out_f32, float* lse_out, void* cuda_stream) {
     clear_error();

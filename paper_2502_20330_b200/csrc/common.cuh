@@ -63,7 +63,8 @@ int launch_accept(const float* target_logits, const float* draft_logits,
                   const int32_t* draft_tokens, const float* uniforms, float eta,
                   int32_t* out_accept_len, int32_t* out_next_token,
                   const rapid_accept_shape* shape, const rapid_accept_params* params,
-                  void* workspace, size_t workspace_bytes, cudaStream_t stream);
+                  void* workspace, size_t workspace_bytes, cudaStream_t stream, float* logq_out = nullptr,
+                  float* stats_out = nullptr);
 
 // ---- device-side PTX wrappers ---------------------------------------------------------------
 #if defined(__CUDACC__)

@@ -338,3 +338,28 @@ def test_inverse_cdf_skips_zero_weights_and_handles_empty():
     assert oracle.inverse_cdf(w, 0.75) == 4
     assert oracle.inverse_cdf(w, 0.99999999) == 4
     assert oracle.inverse_cdf(np.zeros(4), 0.3) == -1
+
+
+def test_draft_sample_on_a_known_distribution():
+    """Logits = T * log of exact probabilities: the drawn token follows the printed CDF intervals and
+    log q is the log of the printed probability, at any temperature."""
+    probs = np.array([0.1, 0.2, 0.3, 0.4])
+    for T in (1.0, 0.5, 2.0):
+        logits = (T * np.log(probs)).astype(np.float32)[None, :].repeat(6, 0) + 3.0   # a shift changes nothing
+        u = np.array([0.0, 0.05, 0.15, 0.45, 0.75, 0.999], dtype=np.float32)
+        tok, logq, stats = oracle.draft_sample(logits, u, T)
+        assert tok.tolist() == [0, 0, 1, 2, 3, 3]
+        np.testing.assert_allclose(np.exp(logq), probs[tok], rtol=1e-6)
+        np.testing.assert_allclose(stats[:, 0], (logits.astype(np.float64) / T).max(axis=1), rtol=0, atol=1e-12)
+        np.testing.assert_allclose(stats[:, 1] - stats[:, 0], np.log((probs / probs.max()).sum()), atol=1e-6)
+
+
+def test_draft_sample_is_the_gamma_zero_accept():
+    """With no draft rows Algorithm 1's accept step only draws the bonus token from softmax(z/T):
+    the same rule, so the two oracle routines must agree."""
+    rng = np.random.default_rng(11)
+    z = (rng.normal(size=(5, 1, 64)) * 3).astype(np.float32)
+    u = rng.random(size=(5, 1)).astype(np.float32)
+    ref = oracle.accept(z, np.zeros((5, 0, 64), np.float32), np.zeros((5, 0), np.int32), u, eta=0.0, T=0.7)
+    tok, _, _ = oracle.draft_sample(z[:, 0], u[:, 0], 0.7)
+    assert tok.tolist() == ref["next_token"].tolist()
