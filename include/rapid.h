@@ -348,6 +348,26 @@ int rapid_verify_step_host(const void* h_q, const void* h_k_cache, const void* h
 size_t rapid_verify_step_host_arena_bytes(const rapid_attn_shape* attn_shape, int gamma,
                                           const rapid_accept_shape* accept_shape);
 
+/* ---- retrieval for the drafter's context --------------------------------------------------------- */
+
+/*
+ * Retrieval scoring (Section 2.3: chunks of the context are embedded and compared with the query by
+ * cosine similarity; Section 3.1, "RAG Setup": top-k chunks, those below a similarity threshold of
+ * 0.3 filtered out).  The embeddings come from the caller's encoder; this call does the scoring
+ * and the selection for B independent requests.
+ *   chunk_emb : device fp32 [B, Nmax, Dm] (16-byte aligned, Dm % 4 == 0);  query_emb : device fp32 [B, Dm]
+ *   n_chunks  : device int32 [B], chunks request b really has (<= Nmax), or NULL = Nmax for all;
+ *               a count outside [0, Nmax] is clamped and sets RAPID_STATUS_BAD_CTX_LEN
+ *   scores_out: device fp32 [B, Nmax]: e.q / (|e| |q|), 0 for a zero vector and past n_chunks[b]
+ *   sel_idx   : device int32 [B, k]: the chunks with score >= threshold, best first (equal scores:
+ *               lower index first), at most k of them, padded with -1;  sel_count : device int32 [B]
+ *   status_word : device int32 (for instance the first word of an initialised workspace)
+ * Limits: Nmax <= 4096, (Dm + Nmax) * 4 bytes <= 200 KB; otherwise RAPID_ERR_UNSUPPORTED.
+ */
+int rapid_retrieval_select(const float* chunk_emb, const float* query_emb, const int32_t* n_chunks, int32_t B,
+                           int32_t Nmax, int32_t Dm, float threshold, int32_t k, float* scores_out,
+                           int32_t* sel_idx, int32_t* sel_count, int32_t* status_word, void* cuda_stream);
+
 /* ---- bookkeeping around the step --------------------------------------------------------------- */
 
 /*

@@ -187,6 +187,27 @@ def accept(target_logits, draft_logits, draft_tokens, uniforms, eta, T=1.0, tail
     return dict(accept_len=accept_len, next_token=next_token, flags=flags, ratios=ratios)
 
 
+def retrieval_select(chunk_emb, query_emb, k, threshold=0.3, n_chunks=None):
+    """Section 2.3 / Section 3.1 ("RAG Setup"): cosine similarity of every chunk embedding with the
+    query embedding; chunks scoring below the threshold are dropped, of the rest the k best are kept,
+    best first (equal scores: lower index first).  fp64.  chunk_emb [B, N, Dm], query_emb [B, Dm].
+    Returns (scores [B, N] (0 for a zero vector and past n_chunks[b]), list of B index lists)."""
+    E = np.asarray(chunk_emb, dtype=np.float32).astype(np.float64)
+    Q = np.asarray(query_emb, dtype=np.float32).astype(np.float64)
+    B, N, _ = E.shape
+    scores = np.zeros((B, N))
+    chosen = []
+    for b in range(B):
+        n = N if n_chunks is None else int(n_chunks[b])
+        qn = np.sqrt((Q[b] * Q[b]).sum())
+        for i in range(n):
+            den = np.sqrt((E[b, i] * E[b, i]).sum()) * qn
+            scores[b, i] = (E[b, i] * Q[b]).sum() / den if den > 0 else 0.0
+        order = sorted(range(n), key=lambda i: (-scores[b, i], i))
+        chosen.append([i for i in order if scores[b, i] >= threshold][:k])
+    return scores, chosen
+
+
 def draft_sample(draft_logits, uniforms, T=1.0):
     """Algorithm 1, drafting loop: x' ~ q = softmax(d/T), drawn by the inverse-CDF rule with the given
     uniform.  fp64.  Returns (token [B] int32, log q(token) [B], row_stats [B,2] = (max d/T, log sum exp d/T))."""

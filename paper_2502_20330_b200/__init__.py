@@ -20,6 +20,8 @@ from .binding import (  # noqa: F401
     rapid_accept_static,
     rapid_draft_sample,
     rapid_kv_append,
+    rapid_retrieval_select,
+    retrieval_budget_chunks,
     rapid_merge_partials,
     rapid_kv_append_paged,
     rapid_step_commit,

@@ -21,7 +21,7 @@ RESIDUAL_PHAT = 1
 
 EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
-    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_retrieval_select", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
     "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_kv_append_paged", "rapid_step_commit",
     "rapid_last_error",
@@ -121,6 +121,8 @@ def load_library():
         lib.rapid_verify_attention_paged.argtypes = [vp, vp, vp, vp, ctypes.POINTER(_PagedKv)] + attn_args[3:] + [vp, sz, vp]
         lib.rapid_draft_sample.restype = i32
         lib.rapid_draft_sample.argtypes = [vp, vp, f32, vp, vp, vp, i32, i64, i64, vp, sz, vp]
+        lib.rapid_retrieval_select.restype = i32
+        lib.rapid_retrieval_select.argtypes = [vp, vp, vp, i32, i32, i32, f32, i32, vp, vp, vp, vp, vp]
         lib.rapid_merge_partials.restype = i32
         lib.rapid_merge_partials.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp]
         lib.rapid_accept.restype = i32
@@ -313,6 +315,32 @@ def rapid_draft_sample(draft_logits, uniforms, temperature, out_token, out_logq,
     _check(load_library().rapid_draft_sample(_p(draft_logits), _p(uniforms), float(temperature), _p(out_token),
                                              _p(out_logq), _p(out_row_stats), B, V, draft_logits.stride(0),
                                              _p(workspace), _nbytes(workspace), _stream_ptr(stream)))
+
+
+def retrieval_budget_chunks(context_tokens: int, chunk_tokens: int = 512, floor_tokens: int = 4096,
+                            fraction: int = 24) -> int:
+    """Chunks the retrieved context may hold: its length is bounded by max(floor_tokens, context / fraction)."""
+    return max(floor_tokens, context_tokens // fraction) // chunk_tokens
+
+
+def rapid_retrieval_select(chunk_emb, query_emb, k, status_word, threshold=0.3, n_chunks=None, stream=None):
+    """Cosine scores of chunk_emb [B, Nmax, Dm] against query_emb [B, Dm] (float32) and the k best chunks
+    at or above ``threshold``.  Returns (scores [B, Nmax], sel_idx [B, k] padded with -1, sel_count [B])."""
+    if chunk_emb.dtype != torch.float32 or query_emb.dtype != torch.float32:
+        raise TypeError("embeddings must be float32")
+    if chunk_emb.dim() != 3 or not chunk_emb.is_contiguous() or not query_emb.is_contiguous() \
+            or query_emb.shape != (chunk_emb.shape[0], chunk_emb.shape[2]):
+        raise ValueError("chunk_emb must be dense [B, Nmax, Dm] and query_emb dense [B, Dm]")
+    if n_chunks is not None and (n_chunks.dtype != torch.int32 or n_chunks.numel() != chunk_emb.shape[0]):
+        raise ValueError("n_chunks must be int32 [B]")
+    B, Nmax, Dm = chunk_emb.shape
+    scores = torch.empty(B, Nmax, dtype=torch.float32, device=chunk_emb.device)
+    sel = torch.empty(B, k, dtype=torch.int32, device=chunk_emb.device)
+    cnt = torch.empty(B, dtype=torch.int32, device=chunk_emb.device)
+    _check(load_library().rapid_retrieval_select(_p(chunk_emb), _p(query_emb), _p(n_chunks), B, Nmax, Dm,
+                                                 float(threshold), int(k), _p(scores), _p(sel), _p(cnt),
+                                                 _p(status_word), _stream_ptr(stream)))
+    return scores, sel, cnt
 
 
 def rapid_merge_partials(o_parts, lse_parts, out=None, out_f32=None, lse_out=None, stream=None) -> None:

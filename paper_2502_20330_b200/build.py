@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librapid.so")
-SOURCES = ["api.cu", "attention.cu", "accept.cu"]
+SOURCES = ["api.cu", "attention.cu", "accept.cu", "retrieval.cu"]
 
 
 def _stale() -> bool:

@@ -266,6 +266,14 @@ int rapid_draft_sample(const float* draft_logits, const float* uniforms, float t
                          out_row_stats);
 }
 
+int rapid_retrieval_select(const float* chunk_emb, const float* query_emb, const int32_t* n_chunks, int32_t B,
+                           int32_t Nmax, int32_t Dm, float threshold, int32_t k, float* scores_out,
+                           int32_t* sel_idx, int32_t* sel_count, int32_t* status_word, void* cuda_stream) {
+    clear_error();
+    return launch_retrieval_select(chunk_emb, query_emb, n_chunks, B, Nmax, Dm, threshold, k, scores_out, sel_idx,
+                                   sel_count, status_word, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int rapid_merge_partials(const float* o_parts, const float* lse_parts, int P, int64_t rows, int D, void* out,
                          float* out_f32, float* lse_out, void* cuda_stream) {
     clear_error();

@@ -57,6 +57,9 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
                             const rapid_attn_shape* shape, const rapid_attn_params* params,
                             void* workspace, size_t workspace_bytes, cudaStream_t stream,
                             const rapid_paged_kv* paged = nullptr, const int32_t* block_table = nullptr);
+int launch_retrieval_select(const float* chunk_emb, const float* query_emb, const int32_t* n_chunks, int B,
+                            int Nmax, int Dm, float threshold, int k, float* scores_out, int32_t* sel_idx,
+                            int32_t* sel_count, int32_t* status_word, cudaStream_t stream);
 int launch_merge_partials(const float* o_parts, const float* lse_parts, int P, int64_t rows, int D, void* out,
                           float* out_f32, float* lse_out, cudaStream_t stream);
 int launch_accept(const float* target_logits, const float* draft_logits,

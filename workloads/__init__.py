@@ -146,6 +146,22 @@ def paged_layout(k: torch.Tensor, v: torch.Tensor, ctx_lens: torch.Tensor, block
     return kp, vp, table.to(k.device)
 
 
+def retrieval_inputs(B: int, n_chunks: int, dim: int, seed: int, device="cpu", lo: float = 0.05, hi: float = 0.75):
+    """Unit-norm chunk embeddings [B, n_chunks, dim] and query embeddings [B, dim] (float32) whose
+    cosine similarities are spread over roughly [lo, hi], i.e. on both sides of the 0.3 threshold the
+    paper filters at -- the shape of a 128K-token context cut into 512-token chunks (256 of them)
+    embedded in 1024 dimensions.  Each chunk is a mix of the query direction and fresh noise."""
+    g = _gen(seed * 4000037 + 29, device)
+    q = torch.randn(B, dim, generator=g, device=device, dtype=torch.float32)
+    q = q / q.norm(dim=-1, keepdim=True)
+    a = lo + (hi - lo) * torch.rand(B, n_chunks, 1, generator=g, device=device, dtype=torch.float32)
+    noise = torch.randn(B, n_chunks, dim, generator=g, device=device, dtype=torch.float32)
+    noise = noise / noise.norm(dim=-1, keepdim=True)
+    e = a * q[:, None, :] + (1 - a * a).sqrt() * noise
+    e = e * (0.5 + torch.rand(B, n_chunks, 1, generator=g, device=device, dtype=torch.float32))  # norms vary
+    return e.contiguous(), q.contiguous()
+
+
 def accept_inputs(cfg: VerifyConfig, seed: int, device="cpu"):
     """Draw target_logits [B,R,V] f32, draft_logits [B,gamma,V] f32,
     draft_tokens [B,gamma] i32 (each ~ softmax of its draft row, by a library
