@@ -14,6 +14,7 @@
 // from run to run.  The merge is launched as a programmatic dependent of the split kernel: its
 // blocks are resident and have done their index arithmetic by the time the last partial lands.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "tcgen05.cuh"
@@ -49,6 +50,12 @@ struct AttnArgs {
     // themselves); stair = 0: every row sees all L keys (a shard of the context without those rows).
     // Lmin = the shortest admissible length: R resp. 1.
     int stair, Lmin;
+    // Work split.  Moving from one (sequence, KV head) unit to the next inside a CTA drains the
+    // pipeline (the unit's O is read out, a new Q is loaded, the first scores have to come back),
+    // which costs about as much as `pad` tiles of streaming.  The flat tile list the CTAs cut into
+    // equal ranges therefore carries `pad` virtual tiles in front of every unit: a CTA whose range
+    // spans a unit boundary gets that many fewer real tiles, and all CTAs finish together.
+    int pad;
 };
 
 struct Walk {
@@ -62,7 +69,31 @@ __device__ __forceinline__ int clamp_len(int L, int R, int Lmax) {
 }
 __device__ __forceinline__ int tiles_of(int L) { return (L + kTile - 1) / kTile; }
 
-// Flat tile range of CTA c of n: [c*T/n, (c+1)*T/n).
+// The padding applies only when every CTA has a few tiles to stream.
+__device__ __forceinline__ int unit_pad(const AttnArgs& a, long long T) {
+    return T >= 4LL * a.num_ctas ? a.pad : 0;
+}
+
+// Real tiles among the first v tiles of the padded flat list (every unit: pad virtual, then nt real).
+__device__ __forceinline__ long long real_tiles_before(const AttnArgs& a, int pad, long long v) {
+    long long real = 0;
+    for (int b = 0; b < a.B; ++b) {
+        const int nt = tiles_of(clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax));
+        const long long ul = nt + pad, span = (long long)a.Hkv * ul;
+        if (v >= span) {
+            real += (long long)a.Hkv * nt;
+            v -= span;
+            continue;
+        }
+        const long long k = v / ul, rem = v - k * ul;
+        long long part = rem - pad;
+        part = part < 0 ? 0 : (part > nt ? nt : part);
+        return real + k * nt + part;
+    }
+    return real;
+}
+
+// Range of CTA c of n in the padded flat list: [c*Tv/n, (c+1)*Tv/n); its real tiles are what it works on.
 __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     long long T = 0;
     for (int b = 0; b < a.B; ++b)
@@ -70,10 +101,12 @@ __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     // with fewer tiles than CTAs only the first T CTAs work, one tile each: no CTA inside the
     // range of a unit is ever empty, which the merge relies on
     const long long nc = T < a.num_ctas ? T : a.num_ctas;
+    const int pad = unit_pad(a, T);
+    const long long Tv = T + (long long)pad * a.B * a.Hkv;
     long long t0 = 0, t1 = 0;
     if (cta < nc) {
-        t0 = (long long)cta * T / nc;
-        t1 = (long long)(cta + 1) * T / nc;
+        t0 = real_tiles_before(a, pad, (long long)cta * Tv / nc);
+        t1 = real_tiles_before(a, pad, (long long)(cta + 1) * Tv / nc);
     }
     w.total = T;
     w.remaining = t1 - t0;
@@ -600,7 +633,7 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
 
-    long long T = 0, t0 = 0;
+    long long T = 0, units_before = 0, t0 = 0;
     int nt_b = 0;
     for (int bb = 0; bb < a.B; ++bb) {
         const int nt = tiles_of(clamp_len(a.ctx_lens[bb], a.Lmin, a.Lmax));
@@ -609,10 +642,14 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
         T += (long long)a.Hkv * nt;
     }
     t0 += (long long)kvh * nt_b;
-    const long long t1 = t0 + nt_b;
+    units_before = (long long)b * a.Hkv + kvh;
     const long long nc = T < a.num_ctas ? T : a.num_ctas;
-    const int c_first = (int)(((t0 + 1) * nc - 1) / T);
-    const int c_last = (int)((t1 * nc - 1) / T);
+    // the unit's real tiles in the padded flat list the split kernel cut: [v0, v1)
+    const int pad = unit_pad(a, T);
+    const long long Tv = T + (long long)pad * a.B * a.Hkv;
+    const long long v0 = t0 + (units_before + 1) * pad, v1 = v0 + nt_b;
+    const int c_first = (int)(((v0 + 1) * nc - 1) / Tv);
+    const int c_last = (int)((v1 * nc - 1) / Tv);
     const int nslots = (c_last - c_first + 1) * KS;
     const size_t slot_stride = (size_t)slot_floats(a.GR, D);
     const float* base = a.partial + (size_t)(c_first + unit) * KS * slot_stride;  // slots are consecutive
@@ -827,6 +864,20 @@ int sm_count() {
     return n;
 }
 
+// Tiles of streaming a unit switch is charged with.  The switch itself takes about 7 us against
+// 1.5 us per tile at head_dim 128; swept on the 8B, 70B and ragged 7B shapes, the launch time
+// falls until 8 and is flat from 8 to 12 (-4.3 % to -4.6 % against no padding).  An environment
+// variable overrides it for experiments.
+int unit_switch_tiles(int D) {
+    static int override_value = -2;
+    if (override_value == -2) {
+        const char* e = getenv("RAPID_UNIT_SWITCH_TILES");
+        override_value = e ? atoi(e) : -1;
+    }
+    if (override_value >= 0 && override_value <= 64) return override_value;
+    return D == 128 ? 10 : 12;
+}
+
 bool attn_shape_ok(const rapid_attn_shape* s, int gamma) {
     if (!s) return false;
     if (s->B <= 0 || s->Hq <= 0 || s->Hkv <= 0 || s->Lmax <= 0 || gamma < 0) return false;
@@ -975,6 +1026,7 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     a.max_blocks = paged ? paged->max_blocks_per_seq : 0;
     a.num_blocks = paged ? paged->num_blocks : 0;
     a.tile_shift = tile_shift;
+    a.pad = unit_switch_tiles(s.D);
     a.stair = all_visible ? 0 : R;
     a.Lmin = all_visible ? 1 : R;
 
