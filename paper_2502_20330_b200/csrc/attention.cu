@@ -623,7 +623,7 @@ __global__ void __launch_bounds__(128)
 verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* lse_out,
                          float* out_f32) {
     constexpr int VEC = D / 32;
-    constexpr int UN = 8;
+    constexpr int UN = 10;
     __shared__ float sh_acc[4][D];
     __shared__ float sh_l[4];
     const int m = blockIdx.x;
@@ -658,6 +658,27 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");  // a following dependent launch may begin its prologue
 
+    // Warp w takes the slots j = w, w + 4, ...  The O rows of its first UN slots are requested at
+    // once, together with every slot's running maximum: neither depends on the other, so the common
+    // case (at most 4 * UN slots per unit) costs one round trip to the partials, not three.
+    float ov[UN][VEC], ms[UN], lv[UN];
+    auto fetch = [&](int j0) {
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const int j = min(j0 + 4 * u, nslots - 1);  // past the end: any valid slot, never used
+            ms[u] = base[(size_t)j * slot_stride + a.GR * D + m];
+            lv[u] = base[(size_t)j * slot_stride + a.GR * D + a.GR + m];  // garbage in an untouched slot: unused
+            const float* slot = base + (size_t)j * slot_stride + (size_t)m * D + lane * VEC;
+            if (VEC == 4) {
+                const float4 t = *reinterpret_cast<const float4*>(slot);
+                ov[u][0] = t.x; ov[u][1] = t.y; ov[u][2] = t.z; ov[u][VEC - 1] = t.w;
+            } else {
+                const float2 t = *reinterpret_cast<const float2*>(slot);
+                ov[u][0] = t.x; ov[u][1] = t.y;
+            }
+        }
+    };
+    fetch(warp);
     float M = -INFINITY;
     for (int j = lane; j < nslots; j += 32) M = fmaxf(M, base[j * slot_stride + a.GR * D + m]);
 #pragma unroll
@@ -668,32 +689,15 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
     float lsum = 0.f;
     for (int j0 = warp; j0 < nslots; j0 += 4 * UN) {
-        float wgt[UN], lv[UN], ov[UN][VEC];
+        if (j0 != warp) fetch(j0);
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
             const int j = j0 + 4 * u;
-            const float* slot = base + (size_t)j * slot_stride;
-            const float ms = j < nslots ? slot[a.GR * D + m] : -INFINITY;
-            const bool live = ms != -INFINITY;  // an untouched slot holds no O: never read it
-            wgt[u] = live ? exp2f(ms - M) : 0.f;
-            lv[u] = live ? slot[a.GR * D + a.GR + m] : 0.f;
+            if (j >= nslots || ms[u] == -INFINITY) continue;  // an untouched slot holds no O: its bits are never used
+            const float wgt = exp2f(ms[u] - M);
+            lsum += wgt * lv[u];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) ov[u][e] = 0.f;
-            if (live) {
-                if (VEC == 4) {
-                    const float4 t = *reinterpret_cast<const float4*>(slot + (size_t)m * D + lane * 4);
-                    ov[u][0] = t.x; ov[u][1] = t.y; ov[u][2] = t.z; ov[u][VEC - 1] = t.w;
-                } else {
-                    const float2 t = *reinterpret_cast<const float2*>(slot + (size_t)m * D + lane * 2);
-                    ov[u][0] = t.x; ov[u][1] = t.y;
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < UN; ++u) {
-            lsum += wgt[u] * lv[u];
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) acc[e] += wgt[u] * ov[u][e];
+            for (int e = 0; e < VEC; ++e) acc[e] += wgt * ov[u][e];
         }
     }
 #pragma unroll
