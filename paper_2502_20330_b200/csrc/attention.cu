@@ -14,7 +14,6 @@
 // from run to run.  The merge is launched as a programmatic dependent of the split kernel: its
 // blocks are resident and have done their index arithmetic by the time the last partial lands.
 #include <math.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 #include "tcgen05.cuh"
@@ -869,18 +868,9 @@ int sm_count() {
 }
 
 // Tiles of streaming a unit switch is charged with.  The switch itself takes about 7 us against
-// 1.5 us per tile at head_dim 128; swept on the 8B, 70B and ragged 7B shapes, the launch time
-// falls until 8 and is flat from 8 to 12 (-4.3 % to -4.6 % against no padding).  An environment
-// variable overrides it for experiments.
-int unit_switch_tiles(int D) {
-    static int override_value = -2;
-    if (override_value == -2) {
-        const char* e = getenv("RAPID_UNIT_SWITCH_TILES");
-        override_value = e ? atoi(e) : -1;
-    }
-    if (override_value >= 0 && override_value <= 64) return override_value;
-    return D == 128 ? 10 : 12;
-}
+// 0.75 us per tile and SM at head_dim 128; swept on the 8B, 70B and ragged 7B shapes, the launch
+// time falls until 8 and is flat from 8 to 12 (-4.3 % to -4.6 % against no padding).
+int unit_switch_tiles(int D) { return D == 128 ? 10 : 12; }
 
 bool attn_shape_ok(const rapid_attn_shape* s, int gamma) {
     if (!s) return false;

@@ -179,3 +179,21 @@ def test_random_shapes_and_lengths():
         q, k, v, ctx = wl.attention_inputs(cfg, seed=200 + trial, device="cuda", poison_padding=True)
         num_ctas = int(rng.choice([0, 1, 3, 5, 16, 37, 148, 300]))
         _compare(q, k, v, ctx, gamma, num_ctas=num_ctas)
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,D,gamma,lo,hi,num_ctas", [
+    (40, 16, 4, 128, 3, 600, 3000, 0),      # 160 short units: every CTA walks through several of them
+    (24, 8, 8, 64, 1, 64, 900, 0),          # 192 units of 1..15 tiles, head_dim 64
+    (3, 32, 8, 128, 8, 5000, 9000, 37),     # a caller-chosen split, a few dozen tiles per CTA
+    (2, 8, 2, 128, 4, 9400, 9500, 0),       # tiles just above four per CTA: the padded split switches on
+    (2, 8, 2, 128, 4, 9200, 9300, 0),       # ... and just below: the plain equal split
+])
+def test_many_units_per_cta(B, Hq, Hkv, D, gamma, lo, hi, num_ctas):
+    """The work split charges every unit a few virtual tiles; ranges that begin or end inside that
+    padding, hold several whole units, or hold nothing but padding must still cover every real tile
+    exactly once and the merge must find every partial."""
+    cfg = wl.VerifyConfig("mu", B=B, Hq=Hq, Hkv=Hkv, D=D, gamma=gamma, V=4096, ctx_range=(lo, hi), Lmax=hi)
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=300 + B, device="cuda", poison_padding=True)
+    rng = np.random.default_rng(B)
+    units = rng.choice(B * Hq * (gamma + 1), size=min(96, B * Hq * (gamma + 1)), replace=False).astype(np.int64)
+    _compare(q, k, v, ctx, gamma, num_ctas=num_ctas, units=units)
