@@ -14,6 +14,7 @@
 // from run to run.  The merge is launched as a programmatic dependent of the split kernel: its
 // blocks are resident and have done their index arithmetic by the time the last partial lands.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "tcgen05.cuh"
@@ -55,6 +56,7 @@ struct AttnArgs {
     // equal ranges therefore carries `pad` virtual tiles in front of every unit: a CTA whose range
     // spans a unit boundary gets that many fewer real tiles, and all CTAs finish together.
     int pad;
+    int tile_keys;  // keys per scheduling tile: what plan, walk and merge count in (64, or 128 for the keys-on-M kernel)
 };
 
 struct Walk {
@@ -66,7 +68,7 @@ struct Walk {
 __device__ __forceinline__ int clamp_len(int L, int R, int Lmax) {
     return L < R ? R : (L > Lmax ? Lmax : L);
 }
-__device__ __forceinline__ int tiles_of(int L) { return (L + kTile - 1) / kTile; }
+__device__ __forceinline__ int tiles_of(int L, int tile_keys) { return (L + tile_keys - 1) / tile_keys; }
 
 // The padding applies only when every CTA has a few tiles to stream.
 __device__ __forceinline__ int unit_pad(const AttnArgs& a, long long T) {
@@ -77,7 +79,7 @@ __device__ __forceinline__ int unit_pad(const AttnArgs& a, long long T) {
 __device__ __forceinline__ long long real_tiles_before(const AttnArgs& a, int pad, long long v) {
     long long real = 0;
     for (int b = 0; b < a.B; ++b) {
-        const int nt = tiles_of(clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax));
+        const int nt = tiles_of(clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax), a.tile_keys);
         const long long ul = nt + pad, span = (long long)a.Hkv * ul;
         if (v >= span) {
             real += (long long)a.Hkv * nt;
@@ -96,7 +98,7 @@ __device__ __forceinline__ long long real_tiles_before(const AttnArgs& a, int pa
 __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     long long T = 0;
     for (int b = 0; b < a.B; ++b)
-        T += (long long)a.Hkv * tiles_of(clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax));
+        T += (long long)a.Hkv * tiles_of(clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax), a.tile_keys);
     // with fewer tiles than CTAs only the first T CTAs work, one tile each: no CTA inside the
     // range of a unit is ever empty, which the merge relies on
     const long long nc = T < a.num_ctas ? T : a.num_ctas;
@@ -118,7 +120,7 @@ __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     long long t = t0;
     for (int b = 0; b < a.B; ++b) {
         const int L = clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax);
-        const int nt = tiles_of(L);
+        const int nt = tiles_of(L, a.tile_keys);
         const long long span = (long long)a.Hkv * nt;
         if (t < span) {
             w.b = b;
@@ -142,7 +144,7 @@ __device__ __forceinline__ void walk_advance(const AttnArgs& a, Walk& w, int seg
             ++w.b;
             if (w.b < a.B) {
                 w.L = clamp_len(a.ctx_lens[w.b], a.Lmin, a.Lmax);
-                w.ntiles = tiles_of(w.L);
+                w.ntiles = tiles_of(w.L, a.tile_keys);
             }
         }
     }
@@ -613,6 +615,8 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
     if (tid == 0 && s_abort) atomicOr(a.status, RAPID_STATUS_PIPELINE_TIMEOUT);
 }
 
+#include "attention_kt.cuh"
+
 // Merge: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the partials of a unit.
 // One block of 4 warps per (grouped row, unit): warp w takes the slots j = w, w+4, ... (four
 // loads in flight per lane), lanes span D; the four warp sums are added in warp order, so the
@@ -635,7 +639,7 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     long long T = 0, units_before = 0, t0 = 0;
     int nt_b = 0;
     for (int bb = 0; bb < a.B; ++bb) {
-        const int nt = tiles_of(clamp_len(a.ctx_lens[bb], a.Lmin, a.Lmax));
+        const int nt = tiles_of(clamp_len(a.ctx_lens[bb], a.Lmin, a.Lmax), a.tile_keys);
         if (bb < b) t0 += (long long)a.Hkv * nt;
         if (bb == b) nt_b = nt;
         T += (long long)a.Hkv * nt;
@@ -776,7 +780,7 @@ EncodeTiledFn get_encode_fn() {
 // Tensor map of a cache [outer][Hkv][keys][D] with element strides sb / sh / sl: outer = sequences
 // and keys = Lmax for a contiguous cache, outer = physical blocks and keys = block size for a paged one.
 int make_kv_map(CUtensorMap* map, const void* base, const rapid_attn_shape& s, int64_t outer,
-                int64_t keys, int64_t sb, int64_t sh, int64_t sl) {
+                int64_t keys, int64_t sb, int64_t sh, int64_t sl, int box_rows) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) {
         set_error("cuTensorMapEncodeTiled is not available from the CUDA driver");
@@ -784,7 +788,7 @@ int make_kv_map(CUtensorMap* map, const void* base, const rapid_attn_shape& s, i
     }
     cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)keys, (cuuint64_t)s.Hkv, (cuuint64_t)outer};
     cuuint64_t strides[3] = {(cuuint64_t)sl * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)kTile, 1, 1};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
                      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -880,6 +884,40 @@ bool attn_shape_ok(const rapid_attn_shape* s, int gamma) {
 }
 
 }  // namespace
+
+template <int NC>
+int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ, const AttnArgs& a,
+                    cudaStream_t stream) {
+    constexpr int smem = kt::smem_bytes(NC);
+    static_assert(smem <= kMaxSmemOptin - 4096, "shared memory (dynamic + the kernel's static arrays)");
+    static bool configured[64] = {};
+    int dev = 0;
+    RAPID_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev >= 64 || !configured[dev]) {
+        RAPID_CUDA_CHECK(cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        if (dev < 64) configured[dev] = true;
+    }
+    RAPID_CUDA_CHECK(launch_dependent(kt::verify_attn_splitkv_kt_kernel<NC>, dim3(a.num_ctas), dim3(kt::kThreads),
+                                      (size_t)smem, stream, tmK, tmV, tmQ, a));
+    return RAPID_OK;
+}
+
+int dispatch_split_kt(int NC, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
+                      const AttnArgs& a, cudaStream_t stream) {
+    switch (NC) {
+        case 1: return launch_split_kt<1>(tmK, tmV, tmQ, a, stream);
+        case 2: return launch_split_kt<2>(tmK, tmV, tmQ, a, stream);
+        case 3: return launch_split_kt<3>(tmK, tmV, tmQ, a, stream);
+        case 4: return launch_split_kt<4>(tmK, tmV, tmQ, a, stream);
+        case 5: return launch_split_kt<5>(tmK, tmV, tmQ, a, stream);
+        case 6: return launch_split_kt<6>(tmK, tmV, tmQ, a, stream);
+        case 7: return launch_split_kt<7>(tmK, tmV, tmQ, a, stream);
+        case 8: return launch_split_kt<8>(tmK, tmV, tmQ, a, stream);
+    }
+    set_error("unsupported number of grouped rows");
+    return RAPID_ERR_UNSUPPORTED;
+}
 
 int launch_merge_partials(const float* o_parts, const float* lse_parts, int P, int64_t rows, int D, void* out,
                           float* out_f32, float* lse_out, cudaStream_t stream) {
@@ -997,9 +1035,13 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     }
 
     CUtensorMap tmK, tmV;
-    int rc = make_kv_map(&tmK, k_cache, s, outer, keys, sb, sh, sl);
+    // bring-up switch for the keys-on-M kernel (head_dim 128; paged caches need blocks of >= 128 keys)
+    static const bool use_kt = getenv("RAPID_ATTN_KT") != nullptr;
+    const bool kt_path = use_kt && s.D == 128 && (!paged || paged->block_size >= kt::kKeys);
+    if (kt_path && paged) --tile_shift;  // blocks are counted in 128-key tiles
+    int rc = make_kv_map(&tmK, k_cache, s, outer, keys, sb, sh, sl, kt_path ? kt::kKeys : kTile);
     if (rc != RAPID_OK) return rc;
-    rc = make_kv_map(&tmV, v_cache, s, outer, keys, sb, sh, sl);
+    rc = make_kv_map(&tmV, v_cache, s, outer, keys, sb, sh, sl, kt_path ? kt::kKeys : kTile);
     if (rc != RAPID_OK) return rc;
 
     AttnArgs a;
@@ -1020,14 +1062,19 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     a.max_blocks = paged ? paged->max_blocks_per_seq : 0;
     a.num_blocks = paged ? paged->num_blocks : 0;
     a.tile_shift = tile_shift;
-    a.pad = unit_switch_tiles(s.D);
+    a.tile_keys = kt_path ? kt::kKeys : kTile;
+    a.pad = kt_path ? 5 : unit_switch_tiles(s.D);
     a.stair = all_visible ? 0 : R;
     a.Lmin = all_visible ? 1 : R;
 
     CUtensorMap tmQ;
     rc = make_q_map(&tmQ, q, s, G, R);
     if (rc != RAPID_OK) return rc;
-    if (GR <= 64)
+    int n_partials = kStreams;
+    if (kt_path) {
+        n_partials = 1;
+        rc = dispatch_split_kt((GR + 15) / 16, tmK, tmV, tmQ, a, stream);
+    } else if (GR <= 64)
         rc = s.D == 128 ? launch_split_tc<128, 64>(tmK, tmV, tmQ, a, stream)
                         : launch_split_tc<64, 64>(tmK, tmV, tmQ, a, stream);
     else
@@ -1055,9 +1102,9 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     cfg.numAttrs = 1;
     __nv_bfloat16* out_bf = static_cast<__nv_bfloat16*>(out);
     if (s.D == 128)
-        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<128>, a, (int)kStreams, out_bf, lse, o32));
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<128>, a, n_partials, out_bf, lse, o32));
     else
-        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<64>, a, (int)kStreams, out_bf, lse, o32));
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<64>, a, n_partials, out_bf, lse, o32));
     count_launch(2);
     return RAPID_OK;
 }

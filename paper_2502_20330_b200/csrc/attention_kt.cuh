@@ -1,0 +1,423 @@
+// Split-KV verify attention with the KEYS on the M axis of the MMAs (head_dim 128).
+//
+//   S^T[128 keys x N] = K_tile[128 x D] Q^T        A = K tile (K-major), B = Q (N grouped rows, K-major)
+//   O^T[D x N]       += V_tile^T[D x 128] P^T      A = V tile (MN-major), B = P^T (K-major, written by the
+//                                                   softmax threads into shared memory)
+// N = grouped rows padded to a multiple of 16.  One softmax thread per KEY (TMEM lane = key), so all
+// 128 softmax threads work whatever the number of grouped rows is, each on N values per tile instead
+// of a few threads on 64 each; the MMAs cost the same ~46 cycles per 16-deep step for any N <= 64.
+// This is the shape of the problem when there are few grouped rows per KV head (the drafter's
+// one-row decode: 4 rows) and it keeps the tensor-core work proportional to the rows that exist.
+//
+// A tile is 128 keys; a stage holds one tile of K and of V (one TMA box of 128 rows per 64-column
+// half).  Work split, partial format (one partial per CTA and unit) and merge are shared with the
+// row-major kernel.  Roles (224 threads): warps 0-3 softmax (thread t = key t of the tile), warp 4
+// TMA producer, warp 5 TMEM allocation + Q load + QK^T issue, warp 6 PV issue.
+//
+// Softmax reference.  As in the row-major kernel the probabilities are taken against a reference
+// m_ref[row] that need not be the running maximum.  It lives in shared memory (every key thread
+// needs every row's value).  It is set from the unit's first tile (a maximum over the 128 key
+// threads: warp shuffles, then the four warps through shared memory) and moved, with a rescale of
+// the O^T columns and of the sums, when a tile holds a score more than 16 (log2 units) above it.
+// The row sums are kept per thread (its keys' share of every row) and added up at the end of a unit
+// in a fixed order.
+//
+// Barriers: every parity wait is on a barrier whose next phase cannot complete before the waiter has
+// passed the current one (per-buffer s_full / p_full, per-stage full / empty; empty doubles as
+// "the PV of this tile has completed").
+#pragma once
+
+namespace kt {
+
+constexpr int kKeys = 128;                 // keys per tile
+constexpr int kThreads = 224;
+constexpr int kBlk = kKeys * 128;          // bytes of one tile x 64-column half
+constexpr float kJump = 16.f;              // a score this far (log2) above the reference moves it
+
+__host__ __device__ constexpr int stages(int NC) { return NC <= 3 ? 3 : 2; }
+__host__ __device__ constexpr int p_blocks(int NC) { return (NC * 16 + 63) / 64; }  // 64-row blocks of P^T
+__host__ __device__ constexpr int smem_bytes(int NC) {
+    // K ring + V ring (two halves each) + Q (two halves) + P^T (128 keys x 128 bytes per 64 grouped rows)
+    return 4 * stages(NC) * kBlk + 2 * (NC * 16) * 128 + p_blocks(NC) * kBlk + 1024;
+}
+
+__device__ __forceinline__ void bar_softmax() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ bool bar_softmax_or(bool flag) {
+    uint32_t res;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(res)
+        : "r"((uint32_t)flag)
+        : "memory");
+    return res != 0;
+}
+__device__ __forceinline__ float warp_max32(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum32(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// NC = N / 16 column chunks (N = grouped rows padded to 16).
+template <int NC>
+__global__ void __launch_bounds__(kThreads, 1)
+verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
+                              const __grid_constant__ CUtensorMap tmV,
+                              const __grid_constant__ CUtensorMap tmQ, const AttnArgs a) {
+    constexpr int D = 128;
+    constexpr int N = NC * 16;
+    constexpr int NST = stages(NC);
+    constexpr int STAGE_TX = 4 * kBlk;  // K and V, two halves each
+    constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t COL_S = 0;    // S^T buffer b at COL_S + 128 b
+    constexpr uint32_t COL_O = 256;  // O^T: N columns
+    // shared-memory map (bytes from the 1024-aligned base)
+    constexpr uint32_t OFF_K = 0, OFF_V = 2 * NST * kBlk, OFF_Q = 4 * NST * kBlk, OFF_P = OFF_Q + 2 * N * 128;
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[NST], empty_bar[NST];
+    __shared__ uint64_t s_full[2], p_full[2];
+    __shared__ uint64_t q_full, o_free;
+    __shared__ uint32_t tmem_slot;
+    __shared__ Walk s_walk;
+    __shared__ int s_abort;
+    __shared__ float sh_mref[128], sh_fac[128], sh_w[4][128];
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int cta = blockIdx.x;
+
+    if (tid == 0) {
+        for (int s = 0; s < NST; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s_full[i], 1);
+            mbar_init(&p_full[i], 4);
+        }
+        mbar_init(&q_full, 1);
+        mbar_init(&o_free, 4);
+        fence_mbar_init();
+        s_abort = 0;
+        prefetch_tensormap(&tmK);
+        prefetch_tensormap(&tmV);
+        prefetch_tensormap(&tmQ);
+    }
+    if (warp == 5) tmem_alloc(&tmem_slot, TMEM_COLS);  // warp 5 also frees it at the end
+    griddep_wait();               // inputs are read from here on
+    griddep_launch_dependents();  // the merge blocks may take their seats
+    if (tid == 0) {
+        Walk w;
+        plan_cta(a, cta, w);
+        s_walk = w;
+        if (cta == 0) {
+            bool bad = false;
+            for (int b = 0; b < a.B; ++b) {
+                const int L = a.ctx_lens[b];
+                bad |= (L < a.Lmin) || (L > a.Lmax);
+            }
+            if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+    Walk w = s_walk;
+    volatile int* abort_flag = &s_abort;
+
+    if (warp == 4) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int jj = 0;
+            bool ok = true;
+            while (w.remaining > 0 && ok) {
+                const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+                for (int t = 0; t < seg && ok; ++t, ++jj) {
+                    const int s = jj % NST;
+                    if (jj >= NST) ok = mbar_wait_bounded_relaxed(&empty_bar[s], ((jj / NST) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    int key0 = (w.tile + t) * kKeys, outer = w.b;
+                    if (a.block_table) {  // paged: (position inside the block, physical block)
+                        const int tile = w.tile + t;
+                        outer = __ldg(a.block_table + (size_t)w.b * a.max_blocks + (tile >> a.tile_shift));
+                        key0 = (tile & ((1 << a.tile_shift) - 1)) * kKeys;
+                        if ((unsigned)outer >= (unsigned)a.num_blocks) {
+                            atomicOr(a.status, RAPID_STATUS_BAD_BLOCK_TABLE);
+                            outer = a.num_blocks;  // outside the pool: the copy reads zeros
+                        }
+                    }
+                    mbar_arrive_expect_tx(&full_bar[s], STAGE_TX);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        tma_load_4d(smem_gen + OFF_K + (h * NST + s) * kBlk, &tmK, &full_bar[s], h * 64, key0, w.kvh, outer);
+                        tma_load_4d(smem_gen + OFF_V + (h * NST + s) * kBlk, &tmV, &full_bar[s], h * 64, key0, w.kvh, outer);
+                    }
+                }
+                walk_advance(a, w, seg);
+            }
+        }
+    } else if (warp == 5) {
+        // ---------------- Q loader and QK^T issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(128, N, 0, 0);
+            const uint64_t k_desc = umma_smem_desc(smem_base + OFF_K, 16, 1024);
+            const uint64_t q_desc = umma_smem_desc(smem_base + OFF_Q, 16, 1024);
+            bool ok = true;
+            int jj = 0, seg_idx = 0;
+            while (w.remaining > 0 && ok) {
+                const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+                // the previous unit has been read out of tensor memory: every MMA of it is complete
+                if (seg_idx > 0) ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, abort_flag);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&q_full, (uint32_t)a.GR * D * 2);
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                    tma_load_4d(smem_gen + OFF_Q + h * (N * 128), &tmQ, &q_full, h * 64, w.kvh * a.G, 0, w.b);
+                ok = mbar_wait_bounded(&q_full, seg_idx & 1, abort_flag);
+                for (int t = 0; t < seg && ok; ++t, ++jj) {
+                    const int s = jj % NST, b = jj & 1;
+                    ok = mbar_wait_bounded(&full_bar[s], (jj / NST) & 1, abort_flag);
+                    // S^T buffer b is free once the probabilities of tile jj-2 have been published
+                    if (ok && jj >= 2) ok = mbar_wait_bounded(&p_full[b], ((jj - 2) >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t d = tmem_base + COL_S + 128u * b;
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t half = kk >> 2, ko16 = (kk & 3) * 2;
+                        umma_bf16_ss(d, k_desc + ((half * NST + s) * kBlk >> 4) + ko16,
+                                     q_desc + (half * (N * 128) >> 4) + ko16, idesc, kk > 0);
+                    }
+                    umma_commit(&s_full[b]);
+                }
+                walk_advance(a, w, seg);
+                ++seg_idx;
+            }
+        }
+    } else if (warp == 6) {
+        // ---------------- PV issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(D, N, 1, 1);
+            // V tile as MN-major A: 64-column blocks NST*kBlk bytes apart, 8-key groups 1024 bytes apart
+            const uint64_t v_desc = umma_smem_desc(smem_base + OFF_V, NST * kBlk, 1024);
+            // P^T as MN-major B: one 128-byte row per key (64 grouped rows), 64-row blocks kBlk bytes apart
+            const uint64_t p_desc = umma_smem_desc(smem_base + OFF_P, kBlk, 1024);
+            const uint32_t d = tmem_base + COL_O;
+            bool ok = true;
+            int jj = 0;
+            while (w.remaining > 0 && ok) {
+                const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+                for (int t = 0; t < seg && ok; ++t, ++jj) {
+                    const int s = jj % NST;
+                    ok = mbar_wait_bounded(&p_full[jj & 1], (jj >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int kk = 0; kk < kKeys / 16; ++kk)
+                        umma_bf16_ss(d, v_desc + (s * kBlk >> 4) + kk * (2048 >> 4), p_desc + kk * (2048 >> 4), idesc,
+                                     (t > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(&empty_bar[s]);  // PV complete: the stage and the P^T buffer are free
+                }
+                walk_advance(a, w, seg);
+            }
+        }
+    } else if (warp < 4) {
+        // ---------------- softmax: thread t = key t of the tile = TMEM lane t ----------------
+        const int t = tid;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const uint32_t tO = tmem_base + lane_base + COL_O;
+        const float c = a.scale_log2;
+        const int slot_stride = (int)slot_floats(a.GR, D);
+        // this key's row of P^T (MN-major: 128 bytes = 64 grouped rows per key, 128-byte swizzle)
+        uint8_t* p_gen = smem_gen + OFF_P + t * 128;
+        const int p_swz = t & 7;
+
+        float lsum[N];  // this key slot's share of every row's sum
+        int jj = 0;
+        bool ok = true;
+        while (w.remaining > 0 && ok) {
+            const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+            const int L = w.L;
+#pragma unroll
+            for (int col = 0; col < N; ++col) lsum[col] = 0.f;
+
+            for (int ti = 0; ti < seg && ok; ++ti, ++jj) {
+                const int b = jj & 1;
+                const uint32_t tS = tmem_base + lane_base + COL_S + 128u * b;
+                const int key = (w.tile + ti) * kKeys + t;
+                // row i sees keys <= L-R+i; rows are column i*G+g: the masked columns are a prefix
+                // (no stair: every row sees every key below L)
+                const int over_ctx = a.stair ? key - (L - a.R) : 0;
+                const int cmin = key >= L ? N : (over_ctx > 0 ? over_ctx * a.G : 0);
+                ok = warp_wait_bounded(&s_full[b], (jj >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+
+                // One pass over the scores: probabilities against the current references, kept in
+                // registers until it is known that no visible score sits far above its reference.
+                float pv[N];
+                bool move = ti == 0;
+                if (ti > 0) {
+#pragma unroll
+                    for (int ch = 0; ch < NC; ++ch) {
+                        uint32_t sr[16];
+                        tmem_ld_x16(tS + 16 * ch, sr);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const int col = 16 * ch + e;
+                            const float x = fmaf(__uint_as_float(sr[e]), c, -sh_mref[col]);
+                            const bool vis = col >= cmin;
+                            move = move || (vis && col < a.GR && x > kJump);
+                            pv[col] = fast_exp2(vis ? x : -INFINITY);
+                        }
+                    }
+                    move = bar_softmax_or(move);
+                }
+                // PV of the previous tile must be complete: it reads P^T, and O^T may be rescaled now
+                if (jj >= 1) {
+                    ok = warp_wait_bounded(&empty_bar[(jj - 1) % NST], ((jj - 1) / NST) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                }
+                if (move) {
+                    // new reference = max(old, this tile's row maxima over the 128 keys)
+#pragma unroll
+                    for (int ch = 0; ch < NC; ++ch) {
+                        uint32_t sr[16];
+                        tmem_ld_x16(tS + 16 * ch, sr);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const int col = 16 * ch + e;
+                            const float v = (col >= cmin && col < a.GR) ? __uint_as_float(sr[e]) * c : -INFINITY;
+                            const float wm = warp_max32(v);
+                            if (lane == 0) sh_w[warp][col] = wm;
+                        }
+                    }
+                    bar_softmax();
+                    if (t < N) {
+                        const float old = ti == 0 ? -INFINITY : sh_mref[t];
+                        const float nm = fmaxf(fmaxf(old, fmaxf(sh_w[0][t], sh_w[1][t])), fmaxf(sh_w[2][t], sh_w[3][t]));
+                        sh_fac[t] = (nm == old) ? 1.f : fast_exp2(old - nm);  // old = -inf gives 0
+                        sh_mref[t] = nm;
+                    }
+                    bar_softmax();
+                    if (ti > 0) {
+#pragma unroll
+                        for (int col = 0; col < N; ++col) lsum[col] *= sh_fac[col];
+                        // thread t is lane t of O^T (= output column d): rescale its N row entries
+#pragma unroll
+                        for (int ch = 0; ch < NC; ++ch) {
+                            uint32_t orow[16];
+                            tmem_ld_x16(tO + 16 * ch, orow);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e)
+                                orow[e] = __float_as_uint(__uint_as_float(orow[e]) * sh_fac[16 * ch + e]);
+                            tmem_st_x16(tO + 16 * ch, orow);
+                        }
+                        tmem_wait_st();
+                    }
+                    // the probabilities again, against the new references
+#pragma unroll
+                    for (int ch = 0; ch < NC; ++ch) {
+                        uint32_t sr[16];
+                        tmem_ld_x16(tS + 16 * ch, sr);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const int col = 16 * ch + e;
+                            const float mr = sh_mref[col];
+                            const float x = col >= cmin ? fmaf(__uint_as_float(sr[e]), c, mr == -INFINITY ? 0.f : -mr) : -INFINITY;
+                            pv[col] = fast_exp2(x);
+                        }
+                    }
+                }
+                // this key's row of P^T: 16-byte chunks of 8 grouped rows each
+#pragma unroll
+                for (int c8 = 0; c8 < N / 8; ++c8) {
+                    uint4 pk;
+                    pk.x = pack_bf16x2(pv[8 * c8 + 0], pv[8 * c8 + 1]);
+                    pk.y = pack_bf16x2(pv[8 * c8 + 2], pv[8 * c8 + 3]);
+                    pk.z = pack_bf16x2(pv[8 * c8 + 4], pv[8 * c8 + 5]);
+                    pk.w = pack_bf16x2(pv[8 * c8 + 6], pv[8 * c8 + 7]);
+                    *reinterpret_cast<uint4*>(p_gen + (c8 >> 3) * kBlk + (((c8 & 7) ^ p_swz) << 4)) = pk;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) lsum[8 * c8 + e] += pv[8 * c8 + e];
+                }
+                if (key - t + kKeys > L) {
+                    // V rows beyond the context may hold any bits: zero them so that 0 * row = 0
+                    const int first_bad = L - (key - t);
+                    const int chunks = (kKeys - first_bad) * 8;
+                    for (int h = 0; h < 2; ++h) {
+                        uint8_t* vgen = smem_gen + OFF_V + (h * NST + jj % NST) * kBlk;
+                        for (int chk = t; chk < chunks; chk += 128)
+                            *reinterpret_cast<uint4*>(vgen + first_bad * 128 + chk * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_full[b]);
+            }
+            if (!ok) break;
+
+            // ---- end of the unit: O^T out of tensor memory, row sums added up, partial written ----
+            ok = warp_wait_bounded(&empty_bar[(jj - 1) % NST], ((jj - 1) / NST) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int unit = w.b * a.Hkv + w.kvh;
+            float* slot = a.partial + (size_t)(cta + unit) * slot_stride;
+#pragma unroll
+            for (int ch = 0; ch < NC; ++ch) {
+                uint32_t orow[16];
+                tmem_ld_x16(tO + 16 * ch, orow);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const int col = 16 * ch + e;
+                    if (col < a.GR && sh_mref[col] != -INFINITY) slot[(size_t)col * D + t] = __uint_as_float(orow[e]);
+                }
+            }
+#pragma unroll
+            for (int col = 0; col < N; ++col) {
+                const float ws = warp_sum32(lsum[col]);
+                if (lane == 0) sh_w[warp][col] = ws;
+            }
+            bar_softmax();
+            if (t < a.GR) {
+                slot[a.GR * D + t] = sh_mref[t];
+                slot[a.GR * D + a.GR + t] = ((sh_w[0][t] + sh_w[1][t]) + sh_w[2][t]) + sh_w[3][t];
+            }
+            bar_softmax();  // sh_w / sh_mref are reused by the next unit
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&o_free);
+            walk_advance(a, w, seg);
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+    if (tid == 0 && s_abort) atomicOr(a.status, RAPID_STATUS_PIPELINE_TIMEOUT);
+}
+
+}  // namespace kt
