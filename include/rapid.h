@@ -85,6 +85,12 @@ typedef struct rapid_attn_shape {
     int64_t kv_stride_l;
 } rapid_attn_shape;
 
+/* Which split kernel rapid_verify_attention uses (rapid_attn_params.kernel). */
+#define RAPID_ATTN_KERNEL_AUTO 0      /* keys on M where it applies, rows on M otherwise                 */
+#define RAPID_ATTN_KERNEL_ROWS_ON_M 1 /* grouped rows on the MMA's M axis: any supported shape           */
+#define RAPID_ATTN_KERNEL_KEYS_ON_M 2 /* keys on the M axis: head_dim 128, <= 48 grouped rows per KV head,
+                                         paged blocks of >= 128 keys; RAPID_ERR_UNSUPPORTED otherwise   */
+
 /* Optional knobs and extra outputs of the attention call (NULL = defaults). */
 typedef struct rapid_attn_params {
     float scale;      /* softmax scale; 0 = 1/sqrt(D)                                             */
@@ -96,7 +102,7 @@ typedef struct rapid_attn_params {
     int32_t all_keys_visible; /* non-zero: no causal stair, every row sees all ctx_lens[b] keys, and
                                  ctx_lens[b] >= 1 suffices.  For a shard of the context that does not
                                  hold the rows' own keys (see rapid_merge_partials)                */
-    int32_t reserved;
+    int32_t kernel;           /* RAPID_ATTN_KERNEL_*: 0 lets the library choose                        */
 } rapid_attn_params;
 
 /*

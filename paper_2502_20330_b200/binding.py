@@ -16,6 +16,7 @@ STATUS_BAD_DRAFT_TOKEN = 2
 STATUS_RESIDUAL_FALLBACK = 4
 STATUS_PIPELINE_TIMEOUT = 8
 STATUS_BAD_BLOCK_TABLE = 16
+ATTN_KERNEL_AUTO, ATTN_KERNEL_ROWS_ON_M, ATTN_KERNEL_KEYS_ON_M = 0, 1, 2
 RESIDUAL_PAPER = 0
 RESIDUAL_PHAT = 1
 
@@ -51,7 +52,7 @@ class _AttnParams(ctypes.Structure):
     _fields_ = [("scale", ctypes.c_float), ("num_ctas", ctypes.c_int32),
                 ("lse_out", ctypes.c_void_p), ("out_f32", ctypes.c_void_p),
                 ("split_done_event", ctypes.c_void_p), ("all_keys_visible", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("kernel", ctypes.c_int32)]
 
 
 class _AcceptShape(ctypes.Structure):
@@ -73,6 +74,7 @@ class AttnParams:
     out_f32: Optional[torch.Tensor] = None   # [B,R,Hq,D] float32
     split_done_event: Optional[int] = None   # cudaEvent_t handle recorded between split and merge
     all_keys_visible: bool = False           # no causal stair: a context shard without the rows' own keys
+    kernel: int = 0                          # 0 automatic, 1 rows on the MMA's M axis, 2 keys on the M axis
 
 
 @dataclass
@@ -195,7 +197,7 @@ def _attn_params(p: Optional[AttnParams]):
         return None
     return ctypes.byref(_AttnParams(p.scale, p.num_ctas, p.lse_out.data_ptr() if p.lse_out is not None else None,
                                     p.out_f32.data_ptr() if p.out_f32 is not None else None,
-                                    p.split_done_event, 1 if p.all_keys_visible else 0, 0))
+                                    p.split_done_event, 1 if p.all_keys_visible else 0, int(p.kernel)))
 
 
 def _accept_shape(target_logits: torch.Tensor, draft_logits: torch.Tensor) -> _AcceptShape:

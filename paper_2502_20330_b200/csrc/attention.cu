@@ -14,7 +14,6 @@
 // from run to run.  The merge is launched as a programmatic dependent of the split kernel: its
 // blocks are resident and have done their index arithmetic by the time the last partial lands.
 #include <math.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 #include "tcgen05.cuh"
@@ -909,11 +908,6 @@ int dispatch_split_kt(int NC, const CUtensorMap& tmK, const CUtensorMap& tmV, co
         case 1: return launch_split_kt<1>(tmK, tmV, tmQ, a, stream);
         case 2: return launch_split_kt<2>(tmK, tmV, tmQ, a, stream);
         case 3: return launch_split_kt<3>(tmK, tmV, tmQ, a, stream);
-        case 4: return launch_split_kt<4>(tmK, tmV, tmQ, a, stream);
-        case 5: return launch_split_kt<5>(tmK, tmV, tmQ, a, stream);
-        case 6: return launch_split_kt<6>(tmK, tmV, tmQ, a, stream);
-        case 7: return launch_split_kt<7>(tmK, tmV, tmQ, a, stream);
-        case 8: return launch_split_kt<8>(tmK, tmV, tmQ, a, stream);
     }
     set_error("unsupported number of grouped rows");
     return RAPID_ERR_UNSUPPORTED;
@@ -1035,9 +1029,21 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     }
 
     CUtensorMap tmK, tmV;
-    // bring-up switch for the keys-on-M kernel (head_dim 128; paged caches need blocks of >= 128 keys)
-    static const bool use_kt = getenv("RAPID_ATTN_KT") != nullptr;
-    const bool kt_path = use_kt && s.D == 128 && (!paged || paged->block_size >= kt::kKeys);
+    // Which split kernel: keys on the MMA's M axis (a softmax thread per key, probabilities through
+    // shared memory) when the grouped rows fit 48 columns -- faster and cheaper per byte there --,
+    // rows on the M axis otherwise (more rows, head_dim 64, paged blocks of 64 keys).
+    const int want = params ? params->kernel : RAPID_ATTN_KERNEL_AUTO;
+    const bool kt_ok = s.D == 128 && (GR + 15) / 16 <= kt::kMaxNC && (!paged || paged->block_size >= kt::kKeys);
+    if (want != RAPID_ATTN_KERNEL_AUTO && want != RAPID_ATTN_KERNEL_ROWS_ON_M && want != RAPID_ATTN_KERNEL_KEYS_ON_M) {
+        set_error("rapid_verify_attention: unknown kernel choice %d", want);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (want == RAPID_ATTN_KERNEL_KEYS_ON_M && !kt_ok) {
+        set_error("rapid_verify_attention: the keys-on-M kernel needs head_dim 128, at most %d grouped rows and, "
+                  "paged, blocks of at least %d keys", 16 * kt::kMaxNC, kt::kKeys);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const bool kt_path = want == RAPID_ATTN_KERNEL_KEYS_ON_M || (want == RAPID_ATTN_KERNEL_AUTO && kt_ok);
     if (kt_path && paged) --tile_shift;  // blocks are counted in 128-key tiles
     int rc = make_kv_map(&tmK, k_cache, s, outer, keys, sb, sh, sl, kt_path ? kt::kKeys : kTile);
     if (rc != RAPID_OK) return rc;

@@ -30,11 +30,12 @@
 namespace kt {
 
 constexpr int kKeys = 128;                 // keys per tile
+constexpr int kMaxNC = 3;                  // up to 48 grouped rows: three K/V stages fit beside Q and P^T
 constexpr int kThreads = 224;
 constexpr int kBlk = kKeys * 128;          // bytes of one tile x 64-column half
 constexpr float kJump = 16.f;              // a score this far (log2) above the reference moves it
 
-__host__ __device__ constexpr int stages(int NC) { return NC <= 3 ? 3 : 2; }
+__host__ __device__ constexpr int stages(int NC) { return 3; }
 __host__ __device__ constexpr int p_blocks(int NC) { return (NC * 16 + 63) / 64; }  // 64-row blocks of P^T
 __host__ __device__ constexpr int smem_bytes(int NC) {
     // K ring + V ring (two halves each) + Q (two halves) + P^T (128 keys x 128 bytes per 64 grouped rows)

@@ -11,7 +11,7 @@ import workloads as wl
 from workloads import bf16_bits
 
 
-def _run(q, k, v, ctx, gamma, num_ctas=0, scale=0.0):
+def _run(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, kernel=0):
     import paper_2502_20330_b200 as R
     B, Rr, Hq, D = q.shape
     Hkv, Lmax = k.shape[1], k.shape[2]
@@ -20,7 +20,7 @@ def _run(q, k, v, ctx, gamma, num_ctas=0, scale=0.0):
     lse = torch.empty(B, Rr, Hq, dtype=torch.float32, device=q.device)
     o32 = torch.empty(B, Rr, Hq, D, dtype=torch.float32, device=q.device)
     R.rapid_verify_attention(q, k, v, ctx, gamma, out, ws,
-                             R.AttnParams(scale=scale, num_ctas=num_ctas, lse_out=lse, out_f32=o32))
+                             R.AttnParams(scale=scale, num_ctas=num_ctas, lse_out=lse, out_f32=o32, kernel=kernel))
     torch.cuda.synchronize()
     return out, lse, o32, R.workspace_status(ws)
 
@@ -30,8 +30,8 @@ def _oracle(q, k, v, ctx, gamma, scale=0.0, units=None):
                                    scale=scale, units=units)
 
 
-def _compare(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, units=None):
-    out, lse, o32, status = _run(q, k, v, ctx, gamma, num_ctas, scale)
+def _compare(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, units=None, kernel=0):
+    out, lse, o32, status = _run(q, k, v, ctx, gamma, num_ctas, scale, kernel)
     assert status == 0
     ref, ref_lse = _oracle(q, k, v, ctx, gamma, scale, units)
     rows = ~np.isnan(ref_lse)
@@ -58,18 +58,21 @@ def test_tiny_config():
     (4, 4, 128, 2, 70),             # G = 1
 ])
 def test_shapes_against_oracle(Hq, Hkv, D, gamma, L):
+    """The library's own choice of kernel, and the rows-on-M kernel forced (it serves every shape)."""
     cfg = wl.VerifyConfig("t", B=2, Hq=Hq, Hkv=Hkv, D=D, gamma=gamma, V=4096, ctx_lens=(L, max(gamma + 1, L // 3)))
     q, k, v, ctx = wl.attention_inputs(cfg, seed=2, device="cuda", poison_padding=True)
     _compare(q, k, v, ctx, gamma)
+    _compare(q, k, v, ctx, gamma, kernel=1)
 
 
+@pytest.mark.parametrize("kernel", [1, 2])
 @pytest.mark.parametrize("num_ctas", [1, 2, 7, 148, 509])
-def test_split_invariance(num_ctas):
+def test_split_invariance(num_ctas, kernel):
     """Any split of the KV length gives the oracle's answer, and fp32 results agree across splits."""
     cfg = wl.VerifyConfig("t", B=3, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(4100, 9, 1111), Lmax=4200)
     q, k, v, ctx = wl.attention_inputs(cfg, seed=3, device="cuda", poison_padding=True)
-    _, _, o32 = _compare(q, k, v, ctx, cfg.gamma, num_ctas=num_ctas)
-    _, _, base, _ = _run(q, k, v, ctx, cfg.gamma, num_ctas=1)
+    _, _, o32 = _compare(q, k, v, ctx, cfg.gamma, num_ctas=num_ctas, kernel=kernel)
+    _, _, base, _ = _run(q, k, v, ctx, cfg.gamma, num_ctas=1, kernel=kernel)
     # splits differ only through where the bf16 rounding of the probabilities falls
     rel = (o32 - base).norm(dim=-1) / base.norm(dim=-1)
     assert rel.max().item() < 5e-3
@@ -103,11 +106,12 @@ def test_explicit_scale_and_strided_cache():
     parity.check_attention(o32.cpu().numpy(), ref)
 
 
-def test_run_to_run_bit_identity():
+@pytest.mark.parametrize("kernel", [1, 2])
+def test_run_to_run_bit_identity(kernel):
     cfg = wl.VerifyConfig("t", B=2, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(6000, 3000))
     q, k, v, ctx = wl.attention_inputs(cfg, seed=7, device="cuda")
-    a = _run(q, k, v, ctx, cfg.gamma)
-    b = _run(q, k, v, ctx, cfg.gamma)
+    a = _run(q, k, v, ctx, cfg.gamma, kernel=kernel)
+    b = _run(q, k, v, ctx, cfg.gamma, kernel=kernel)
     assert torch.equal(a[0], b[0]) and torch.equal(a[2], b[2]) and torch.equal(a[1], b[1])
 
 
@@ -133,6 +137,12 @@ def test_argument_errors():
     with pytest.raises(R.RapidError) as e:
         R.rapid_verify_attention(q, k, v, ctx, 2, out, ws, R.AttnParams(num_ctas=100000))
     assert e.value.code == 1
+    with pytest.raises(R.RapidError) as e:                                # head_dim 64 has no keys-on-M kernel
+        R.rapid_verify_attention(q, k, v, ctx, 2, out, ws, R.AttnParams(kernel=2))
+    assert e.value.code == 2
+    with pytest.raises(R.RapidError) as e:
+        R.rapid_verify_attention(q, k, v, ctx, 2, out, ws, R.AttnParams(kernel=7))
+    assert e.value.code == 1
     assert R.attention_workspace_bytes(1, 8, 2, 96, 128, 2) == 0          # unsupported head_dim
     assert R.attention_workspace_bytes(1, 64, 1, 128, 128, 8) == 0        # 576 grouped rows
 
@@ -152,6 +162,8 @@ def test_llama8b_128k_and_70b_sampled_rows():
         n_units = cfg.B * cfg.Hq * cfg.R
         units = np.array([0, 8, n_units // 2 + 3, n_units - 1], dtype=np.int64)
         _compare(q, k, v, ctx, cfg.gamma, units=units)
+        if name == "llama8b_128k":
+            _compare(q, k, v, ctx, cfg.gamma, units=units, kernel=1)
         del q, k, v
 
 
@@ -179,6 +191,8 @@ def test_random_shapes_and_lengths():
         q, k, v, ctx = wl.attention_inputs(cfg, seed=200 + trial, device="cuda", poison_padding=True)
         num_ctas = int(rng.choice([0, 1, 3, 5, 16, 37, 148, 300]))
         _compare(q, k, v, ctx, gamma, num_ctas=num_ctas)
+        if D == 128 and G * (gamma + 1) <= 48:      # the automatic choice was keys-on-M: rows-on-M too
+            _compare(q, k, v, ctx, gamma, num_ctas=num_ctas, kernel=1)
 
 
 @pytest.mark.parametrize("B,Hq,Hkv,D,gamma,lo,hi,num_ctas", [
