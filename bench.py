@@ -39,16 +39,16 @@ def _peaks():
     return 6650.0, "fallback"
 
 
-def ncu_traffic(workload):
+def ncu_traffic(workload, kernel="verify_attn_splitkv_tc_kernel"):
     """DRAM bytes per split-kernel launch from the committed ncu capture, or None if the kernel
-    sources have changed since the counters were taken."""
+    sources have changed since the counters were taken (or the capture is of the other kernel)."""
     import hashlib
     try:
         rec = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
         h = hashlib.sha256()
-        for f in ("attention.cu", "tcgen05.cuh", "common.cuh"):
+        for f in ("attention.cu", "attention_kt.cuh", "tcgen05.cuh", "common.cuh"):
             h.update(open(os.path.join(ROOT, "paper_2502_20330_b200", "csrc", f), "rb").read())
-        if h.hexdigest() != rec["kernel_sha256"] or workload not in rec:
+        if h.hexdigest() != rec["kernel_sha256"] or workload not in rec or rec.get("kernel") != kernel:
             return None
         return int(rec[workload]["dram_bytes_read"] + rec[workload]["dram_bytes_write"])
     except Exception:
@@ -270,6 +270,9 @@ def run_ours(args, cfg):
     aws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma), device=dev)
     cws = R.new_workspace(R.accept_workspace_bytes(cfg.B, cfg.gamma, cfg.V), device=dev)
     acc_params = R.AcceptParams(temperature=cfg.temperature, tail_alpha=cfg.tail_alpha)
+    attn_params = R.AttnParams(kernel=args.kernel)
+    keys_on_m = args.kernel == 2 or (args.kernel == 0 and cfg.D == 128 and cfg.G * cfg.R <= 48)
+    split_kernel = "verify_attn_splitkv_kt_kernel" if keys_on_m else "verify_attn_splitkv_tc_kernel"
     stream = torch.cuda.current_stream()
     sptr = int(stream.cuda_stream)
     ev = RawEvents()
@@ -282,9 +285,10 @@ def run_ours(args, cfg):
             if split_events is not None:
                 e0, e1 = split_events[li]
                 ev.record(e0, sptr)
-                R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws, R.AttnParams(split_done_event=e1))
+                R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws,
+                                         R.AttnParams(split_done_event=e1, kernel=args.kernel))
             else:
-                R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws)
+                R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws, attn_params)
         R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params)
 
     def barrier():
@@ -308,7 +312,7 @@ def run_ours(args, cfg):
     with torch.cuda.stream(side):
         with torch.cuda.graph(graph, stream=side):
             for (q, k, v, out) in layers:
-                R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws, stream=side)
+                R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws, attn_params, stream=side)
             R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params, stream=side)
     launches_per_step = R.kernel_launch_count()
     torch.cuda.synchronize()
@@ -381,8 +385,8 @@ def run_ours(args, cfg):
                               "accept": 1e3 * float(np.median(acc_ms)), "step": 1e3 * ms_per_step,
                               "step_stream_launches": stream_us},
         "frac_of_hbm_peak": {"measured": value / world / peak, "nominal_8TBs": value / world / 8000.0},
-        "roofline": {"bound": "hbm", "kernel": "verify_attn_splitkv_tc_kernel", "achieved": achieved, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": ncu_traffic(cfg.name),
+        "roofline": {"bound": "hbm", "kernel": split_kernel, "achieved": achieved, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": ncu_traffic(cfg.name, split_kernel),
                      "algorithmic_bytes": kv_layer,
                      "timed": f"CUDA events around each of {len(split_ms)} launches in a second pass of {k_steps} steps"},
         "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
@@ -441,6 +445,8 @@ def main():
     ap.add_argument("--workload", default="llama8b_128k", choices=sorted(wl.CONFIGS))
     ap.add_argument("--layers", type=int, default=0, help="override the number of resident layers")
     ap.add_argument("--seed", type=int, default=2025)
+    ap.add_argument("--kernel", type=int, default=0, choices=[0, 1, 2],
+                    help="split kernel: 0 the library's choice, 1 rows on the MMA's M axis, 2 keys on the M axis")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
