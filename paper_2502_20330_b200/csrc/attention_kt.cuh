@@ -1,26 +1,32 @@
-// Split-KV verify attention with the KEYS on the M axis of the MMAs (head_dim 128).
+// Split-KV verify attention with the KEYS on the M axis of the MMAs (head_dim 128, up to 48 grouped rows).
 //
 //   S^T[128 keys x N] = K_tile[128 x D] Q^T        A = K tile (K-major), B = Q (N grouped rows, K-major)
-//   O^T[D x N]       += V_tile^T[D x 128] P^T      A = V tile (MN-major), B = P^T (K-major, written by the
+//   O^T[D x N]       += V_tile^T[D x 128] P^T      A = V tile (MN-major), B = P^T (MN-major, written by the
 //                                                   softmax threads into shared memory)
 // N = grouped rows padded to a multiple of 16.  One softmax thread per KEY (TMEM lane = key), so all
-// 128 softmax threads work whatever the number of grouped rows is, each on N values per tile instead
-// of a few threads on 64 each; the MMAs cost the same ~46 cycles per 16-deep step for any N <= 64.
-// This is the shape of the problem when there are few grouped rows per KV head (the drafter's
-// one-row decode: 4 rows) and it keeps the tensor-core work proportional to the rows that exist.
+// 128 softmax threads work whatever the number of grouped rows is, one exponential per (key, row)
+// that exists, and the tensor-core work is proportional to N instead of to a 64- or 128-row tile.
 //
 // A tile is 128 keys; a stage holds one tile of K and of V (one TMA box of 128 rows per 64-column
 // half).  Work split, partial format (one partial per CTA and unit) and merge are shared with the
-// row-major kernel.  Roles (224 threads): warps 0-3 softmax (thread t = key t of the tile), warp 4
+// rows-on-M kernel.  Roles (224 threads): warps 0-3 softmax (thread t = key t of the tile), warp 4
 // TMA producer, warp 5 TMEM allocation + Q load + QK^T issue, warp 6 PV issue.
 //
-// Softmax reference.  As in the row-major kernel the probabilities are taken against a reference
+// P^T in shared memory has the layout of a V tile half: one 128-byte row per key holding that key's
+// probabilities for 64 grouped rows, 128-byte swizzle (16-byte chunk index XOR key & 7), 8-key groups
+// 1024 bytes apart.  A softmax thread writes its row with one 16-byte store per 8 grouped rows.
+//
+// Softmax reference.  As in the rows-on-M kernel the probabilities are taken against a reference
 // m_ref[row] that need not be the running maximum.  It lives in shared memory (every key thread
 // needs every row's value).  It is set from the unit's first tile (a maximum over the 128 key
 // threads: warp shuffles, then the four warps through shared memory) and moved, with a rescale of
 // the O^T columns and of the sums, when a tile holds a score more than 16 (log2 units) above it.
-// The row sums are kept per thread (its keys' share of every row) and added up at the end of a unit
-// in a fixed order.
+// That is found in the one pass that forms the probabilities (a block-wide OR per tile); only then
+// are they formed again against the new references.  The row sums are kept per thread (its keys'
+// share of every row) and added up at the end of a unit in a fixed order.
+//
+// Pipeline: S^T is double-buffered in tensor memory, so QK^T(n+1) runs during softmax(n); P^T is
+// single-buffered, so the P^T stores of tile n wait for PV(n-1), the arithmetic before them does not.
 //
 // Barriers: every parity wait is on a barrier whose next phase cannot complete before the waiter has
 // passed the current one (per-buffer s_full / p_full, per-stage full / empty; empty doubles as
