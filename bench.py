@@ -271,7 +271,7 @@ def run_ours(args, cfg):
     cws = R.new_workspace(R.accept_workspace_bytes(cfg.B, cfg.gamma, cfg.V), device=dev)
     acc_params = R.AcceptParams(temperature=cfg.temperature, tail_alpha=cfg.tail_alpha)
     attn_params = R.AttnParams(kernel=args.kernel)
-    keys_on_m = args.kernel == 2 or (args.kernel == 0 and cfg.D == 128 and cfg.G * cfg.R <= 48)
+    keys_on_m = args.kernel == 2 or (args.kernel == 0 and cfg.D == 128 and cfg.G * cfg.R <= 64)
     split_kernel = "verify_attn_splitkv_kt_kernel" if keys_on_m else "verify_attn_splitkv_tc_kernel"
     stream = torch.cuda.current_stream()
     sptr = int(stream.cuda_stream)

@@ -88,7 +88,7 @@ typedef struct rapid_attn_shape {
 /* Which split kernel rapid_verify_attention uses (rapid_attn_params.kernel). */
 #define RAPID_ATTN_KERNEL_AUTO 0      /* keys on M where it applies, rows on M otherwise                 */
 #define RAPID_ATTN_KERNEL_ROWS_ON_M 1 /* grouped rows on the MMA's M axis: any supported shape           */
-#define RAPID_ATTN_KERNEL_KEYS_ON_M 2 /* keys on the M axis: head_dim 128, <= 48 grouped rows per KV head,
+#define RAPID_ATTN_KERNEL_KEYS_ON_M 2 /* keys on the M axis: head_dim 128, <= 64 grouped rows per KV head,
                                          paged blocks of >= 128 keys; RAPID_ERR_UNSUPPORTED otherwise   */
 
 /* Optional knobs and extra outputs of the attention call (NULL = defaults). */

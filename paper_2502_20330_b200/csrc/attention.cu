@@ -908,6 +908,7 @@ int dispatch_split_kt(int NC, const CUtensorMap& tmK, const CUtensorMap& tmV, co
         case 1: return launch_split_kt<1>(tmK, tmV, tmQ, a, stream);
         case 2: return launch_split_kt<2>(tmK, tmV, tmQ, a, stream);
         case 3: return launch_split_kt<3>(tmK, tmV, tmQ, a, stream);
+        case 4: return launch_split_kt<4>(tmK, tmV, tmQ, a, stream);
     }
     set_error("unsupported number of grouped rows");
     return RAPID_ERR_UNSUPPORTED;
@@ -1030,7 +1031,7 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
 
     CUtensorMap tmK, tmV;
     // Which split kernel: keys on the MMA's M axis (a softmax thread per key, probabilities through
-    // shared memory) when the grouped rows fit 48 columns -- faster and cheaper per byte there --,
+    // shared memory) when the grouped rows fit 64 columns -- faster and cheaper per byte there --,
     // rows on the M axis otherwise (more rows, head_dim 64, paged blocks of 64 keys).
     const int want = params ? params->kernel : RAPID_ATTN_KERNEL_AUTO;
     const bool kt_ok = s.D == 128 && (GR + 15) / 16 <= kt::kMaxNC && (!paged || paged->block_size >= kt::kKeys);

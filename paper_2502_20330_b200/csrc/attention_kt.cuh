@@ -1,4 +1,4 @@
-// Split-KV verify attention with the KEYS on the M axis of the MMAs (head_dim 128, up to 48 grouped rows).
+// Split-KV verify attention with the KEYS on the M axis of the MMAs (head_dim 128, up to 64 grouped rows).
 //
 //   S^T[128 keys x N] = K_tile[128 x D] Q^T        A = K tile (K-major), B = Q (N grouped rows, K-major)
 //   O^T[D x N]       += V_tile^T[D x 128] P^T      A = V tile (MN-major), B = P^T (MN-major, written by the
@@ -7,8 +7,9 @@
 // 128 softmax threads work whatever the number of grouped rows is, one exponential per (key, row)
 // that exists, and the tensor-core work is proportional to N instead of to a 64- or 128-row tile.
 //
-// A tile is 128 keys; a stage holds one tile of K and of V (one TMA box of 128 rows per 64-column
-// half).  Work split, partial format (one partial per CTA and unit) and merge are shared with the
+// A tile is 128 keys (one TMA box of 128 rows per 64-column half).  K tiles and V tiles live in
+// rings of their own (three slots each; two K slots for more than 48 rows): a K slot is free once
+// QK^T of its tile has completed, a V slot only after PV.  Work split, partial format (one partial per CTA and unit) and merge are shared with the
 // rows-on-M kernel.  Roles (224 threads): warps 0-3 softmax (thread t = key t of the tile), warp 4
 // TMA producer, warp 5 TMEM allocation + Q load + QK^T issue, warp 6 PV issue.
 //
@@ -36,16 +37,19 @@
 namespace kt {
 
 constexpr int kKeys = 128;                 // keys per tile
-constexpr int kMaxNC = 3;                  // up to 48 grouped rows: three K/V stages fit beside Q and P^T
+constexpr int kMaxNC = 4;                  // up to 64 grouped rows: beyond that the rows-on-M kernel is faster
 constexpr int kThreads = 224;
 constexpr int kBlk = kKeys * 128;          // bytes of one tile x 64-column half
 constexpr float kJump = 16.f;              // a score this far (log2) above the reference moves it
 
-__host__ __device__ constexpr int stages(int NC) { return 3; }
+// K and V tiles live in rings of their own: a K slot is free as soon as QK^T of its tile has
+// completed, a V slot only after PV, so K needs fewer slots than V when space is short.
+__host__ __device__ constexpr int k_slots(int NC) { return NC <= 3 ? 3 : 2; }
+__host__ __device__ constexpr int v_slots(int NC) { return 3; }
 __host__ __device__ constexpr int p_blocks(int NC) { return (NC * 16 + 63) / 64; }  // 64-row blocks of P^T
 __host__ __device__ constexpr int smem_bytes(int NC) {
     // K ring + V ring (two halves each) + Q (two halves) + P^T (128 keys x 128 bytes per 64 grouped rows)
-    return 4 * stages(NC) * kBlk + 2 * (NC * 16) * 128 + p_blocks(NC) * kBlk + 1024;
+    return 2 * (k_slots(NC) + v_slots(NC)) * kBlk + 2 * (NC * 16) * 128 + p_blocks(NC) * kBlk + 1024;
 }
 
 __device__ __forceinline__ void bar_softmax() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -80,16 +84,16 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                               const __grid_constant__ CUtensorMap tmQ, const AttnArgs a) {
     constexpr int D = 128;
     constexpr int N = NC * 16;
-    constexpr int NST = stages(NC);
-    constexpr int STAGE_TX = 4 * kBlk;  // K and V, two halves each
+    constexpr int NK = k_slots(NC), NV = v_slots(NC);
+    constexpr int TILE_TX = 2 * kBlk;  // one tile of K or of V: two 64-column halves
     constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t COL_S = 0;    // S^T buffer b at COL_S + 128 b
     constexpr uint32_t COL_O = 256;  // O^T: N columns
     // shared-memory map (bytes from the 1024-aligned base)
-    constexpr uint32_t OFF_K = 0, OFF_V = 2 * NST * kBlk, OFF_Q = 4 * NST * kBlk, OFF_P = OFF_Q + 2 * N * 128;
+    constexpr uint32_t OFF_K = 0, OFF_V = 2 * NK * kBlk, OFF_Q = 2 * (NK + NV) * kBlk, OFF_P = OFF_Q + 2 * N * 128;
 
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[NST], empty_bar[NST];
+    __shared__ uint64_t k_full[NK], k_empty[NK], v_full[NV], v_empty[NV];
     __shared__ uint64_t s_full[2], p_full[2];
     __shared__ uint64_t q_full, o_free;
     __shared__ uint32_t tmem_slot;
@@ -106,9 +110,13 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
     const int cta = blockIdx.x;
 
     if (tid == 0) {
-        for (int s = 0; s < NST; ++s) {
-            mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], 1);
+        for (int s = 0; s < NK; ++s) {
+            mbar_init(&k_full[s], 1);
+            mbar_init(&k_empty[s], 1);
+        }
+        for (int s = 0; s < NV; ++s) {
+            mbar_init(&v_full[s], 1);
+            mbar_init(&v_empty[s], 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&s_full[i], 1);
@@ -153,9 +161,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
             while (w.remaining > 0 && ok) {
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 for (int t = 0; t < seg && ok; ++t, ++jj) {
-                    const int s = jj % NST;
-                    if (jj >= NST) ok = mbar_wait_bounded_relaxed(&empty_bar[s], ((jj / NST) - 1) & 1, abort_flag);
-                    if (!ok) break;
+                    const int ks = jj % NK, vs = jj % NV;
                     int key0 = (w.tile + t) * kKeys, outer = w.b;
                     if (a.block_table) {  // paged: (position inside the block, physical block)
                         const int tile = w.tile + t;
@@ -166,12 +172,18 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                             outer = a.num_blocks;  // outside the pool: the copy reads zeros
                         }
                     }
-                    mbar_arrive_expect_tx(&full_bar[s], STAGE_TX);
+                    if (jj >= NK) ok = mbar_wait_bounded_relaxed(&k_empty[ks], ((jj / NK) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(&k_full[ks], TILE_TX);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        tma_load_4d(smem_gen + OFF_K + (h * NST + s) * kBlk, &tmK, &full_bar[s], h * 64, key0, w.kvh, outer);
-                        tma_load_4d(smem_gen + OFF_V + (h * NST + s) * kBlk, &tmV, &full_bar[s], h * 64, key0, w.kvh, outer);
-                    }
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_4d(smem_gen + OFF_K + (h * NK + ks) * kBlk, &tmK, &k_full[ks], h * 64, key0, w.kvh, outer);
+                    if (jj >= NV) ok = mbar_wait_bounded_relaxed(&v_empty[vs], ((jj / NV) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(&v_full[vs], TILE_TX);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_4d(smem_gen + OFF_V + (h * NV + vs) * kBlk, &tmV, &v_full[vs], h * 64, key0, w.kvh, outer);
                 }
                 walk_advance(a, w, seg);
             }
@@ -195,8 +207,8 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                     tma_load_4d(smem_gen + OFF_Q + h * (N * 128), &tmQ, &q_full, h * 64, w.kvh * a.G, 0, w.b);
                 ok = mbar_wait_bounded(&q_full, seg_idx & 1, abort_flag);
                 for (int t = 0; t < seg && ok; ++t, ++jj) {
-                    const int s = jj % NST, b = jj & 1;
-                    ok = mbar_wait_bounded(&full_bar[s], (jj / NST) & 1, abort_flag);
+                    const int s = jj % NK, b = jj & 1;
+                    ok = mbar_wait_bounded(&k_full[s], (jj / NK) & 1, abort_flag);
                     // S^T buffer b is free once the probabilities of tile jj-2 have been published
                     if (ok && jj >= 2) ok = mbar_wait_bounded(&p_full[b], ((jj - 2) >> 1) & 1, abort_flag);
                     if (!ok) break;
@@ -205,10 +217,11 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
                         const uint32_t half = kk >> 2, ko16 = (kk & 3) * 2;
-                        umma_bf16_ss(d, k_desc + ((half * NST + s) * kBlk >> 4) + ko16,
+                        umma_bf16_ss(d, k_desc + ((half * NK + s) * kBlk >> 4) + ko16,
                                      q_desc + (half * (N * 128) >> 4) + ko16, idesc, kk > 0);
                     }
                     umma_commit(&s_full[b]);
+                    umma_commit(&k_empty[s]);  // QK^T complete: the K slot is free
                 }
                 walk_advance(a, w, seg);
                 ++seg_idx;
@@ -218,8 +231,8 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
         // ---------------- PV issuer ----------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(D, N, 1, 1);
-            // V tile as MN-major A: 64-column blocks NST*kBlk bytes apart, 8-key groups 1024 bytes apart
-            const uint64_t v_desc = umma_smem_desc(smem_base + OFF_V, NST * kBlk, 1024);
+            // V tile as MN-major A: 64-column blocks NV*kBlk bytes apart, 8-key groups 1024 bytes apart
+            const uint64_t v_desc = umma_smem_desc(smem_base + OFF_V, NV * kBlk, 1024);
             // P^T as MN-major B: one 128-byte row per key (64 grouped rows), 64-row blocks kBlk bytes apart
             const uint64_t p_desc = umma_smem_desc(smem_base + OFF_P, kBlk, 1024);
             const uint32_t d = tmem_base + COL_O;
@@ -228,15 +241,16 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
             while (w.remaining > 0 && ok) {
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 for (int t = 0; t < seg && ok; ++t, ++jj) {
-                    const int s = jj % NST;
+                    const int s = jj % NV;
                     ok = mbar_wait_bounded(&p_full[jj & 1], (jj >> 1) & 1, abort_flag);
+                    if (ok) ok = mbar_wait_bounded(&v_full[s], (jj / NV) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < kKeys / 16; ++kk)
                         umma_bf16_ss(d, v_desc + (s * kBlk >> 4) + kk * (2048 >> 4), p_desc + kk * (2048 >> 4), idesc,
                                      (t > 0 || kk > 0) ? 1u : 0u);
-                    umma_commit(&empty_bar[s]);  // PV complete: the stage and the P^T buffer are free
+                    umma_commit(&v_empty[s]);  // PV complete: the V slot and the P^T buffer are free
                 }
                 walk_advance(a, w, seg);
             }
@@ -275,7 +289,10 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
 
                 // One pass over the scores: probabilities against the current references, kept in
                 // registers until it is known that no visible score sits far above its reference.
-                float pv[N];
+                // (Kept as fp32 up to 48 columns; beyond that as packed bf16 pairs, to stay in registers.)
+                constexpr bool kPacked = NC > 3;
+                float pv[kPacked ? 2 : N];
+                uint32_t pq[kPacked ? N / 2 : 1];
                 bool move = ti == 0;
                 if (ti > 0) {
 #pragma unroll
@@ -284,19 +301,26 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         tmem_ld_x16(tS + 16 * ch, sr);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {
+                        for (int e = 0; e < 16; e += 2) {
                             const int col = 16 * ch + e;
-                            const float x = fmaf(__uint_as_float(sr[e]), c, -sh_mref[col]);
-                            const bool vis = col >= cmin;
-                            move = move || (vis && col < a.GR && x > kJump);
-                            pv[col] = fast_exp2(vis ? x : -INFINITY);
+                            const float x0 = fmaf(__uint_as_float(sr[e]), c, -sh_mref[col]);
+                            const float x1 = fmaf(__uint_as_float(sr[e + 1]), c, -sh_mref[col + 1]);
+                            const bool v0 = col >= cmin, v1 = col + 1 >= cmin;
+                            move = move || (v0 && col < a.GR && x0 > kJump) || (v1 && col + 1 < a.GR && x1 > kJump);
+                            const float p0 = fast_exp2(v0 ? x0 : -INFINITY), p1 = fast_exp2(v1 ? x1 : -INFINITY);
+                            if (kPacked) {
+                                pq[col >> 1] = pack_bf16x2(p0, p1);
+                            } else {
+                                pv[kPacked ? 0 : col] = p0;
+                                pv[kPacked ? 1 : col + 1] = p1;
+                            }
                         }
                     }
                     move = bar_softmax_or(move);
                 }
                 // PV of the previous tile must be complete: it reads P^T, and O^T may be rescaled now
                 if (jj >= 1) {
-                    ok = warp_wait_bounded(&empty_bar[(jj - 1) % NST], ((jj - 1) / NST) & 1, abort_flag);
+                    ok = warp_wait_bounded(&v_empty[(jj - 1) % NV], ((jj - 1) / NV) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
                 }
@@ -346,11 +370,18 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         tmem_ld_x16(tS + 16 * ch, sr);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {
+                        for (int e = 0; e < 16; e += 2) {
                             const int col = 16 * ch + e;
-                            const float mr = sh_mref[col];
-                            const float x = col >= cmin ? fmaf(__uint_as_float(sr[e]), c, mr == -INFINITY ? 0.f : -mr) : -INFINITY;
-                            pv[col] = fast_exp2(x);
+                            const float m0 = sh_mref[col], m1 = sh_mref[col + 1];
+                            const float x0 = col >= cmin ? fmaf(__uint_as_float(sr[e]), c, m0 == -INFINITY ? 0.f : -m0) : -INFINITY;
+                            const float x1 = col + 1 >= cmin ? fmaf(__uint_as_float(sr[e + 1]), c, m1 == -INFINITY ? 0.f : -m1) : -INFINITY;
+                            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                            if (kPacked) {
+                                pq[col >> 1] = pack_bf16x2(p0, p1);
+                            } else {
+                                pv[kPacked ? 0 : col] = p0;
+                                pv[kPacked ? 1 : col + 1] = p1;
+                            }
                         }
                     }
                 }
@@ -358,20 +389,34 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
                 for (int c8 = 0; c8 < N / 8; ++c8) {
                     uint4 pk;
-                    pk.x = pack_bf16x2(pv[8 * c8 + 0], pv[8 * c8 + 1]);
-                    pk.y = pack_bf16x2(pv[8 * c8 + 2], pv[8 * c8 + 3]);
-                    pk.z = pack_bf16x2(pv[8 * c8 + 4], pv[8 * c8 + 5]);
-                    pk.w = pack_bf16x2(pv[8 * c8 + 6], pv[8 * c8 + 7]);
-                    *reinterpret_cast<uint4*>(p_gen + (c8 >> 3) * kBlk + (((c8 & 7) ^ p_swz) << 4)) = pk;
+                    if (kPacked) {
+                        pk = make_uint4(pq[4 * c8], pq[4 * c8 + 1], pq[4 * c8 + 2], pq[4 * c8 + 3]);
+                        // the sums take the probabilities as the tensor cores will see them
+                        const uint32_t u[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) lsum[8 * c8 + e] += pv[8 * c8 + e];
+                        for (int e = 0; e < 4; ++e) {
+                            lsum[8 * c8 + 2 * e] += __uint_as_float(u[e] << 16);
+                            lsum[8 * c8 + 2 * e + 1] += __uint_as_float(u[e] & 0xffff0000u);
+                        }
+                    } else {
+                        const int o = kPacked ? 0 : 8 * c8;
+                        pk.x = pack_bf16x2(pv[o + 0], pv[o + 1]);
+                        pk.y = pack_bf16x2(pv[kPacked ? 0 : o + 2], pv[kPacked ? 1 : o + 3]);
+                        pk.z = pack_bf16x2(pv[kPacked ? 0 : o + 4], pv[kPacked ? 1 : o + 5]);
+                        pk.w = pack_bf16x2(pv[kPacked ? 0 : o + 6], pv[kPacked ? 1 : o + 7]);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) lsum[8 * c8 + e] += pv[kPacked ? 0 : o + e];
+                    }
+                    *reinterpret_cast<uint4*>(p_gen + (c8 >> 3) * kBlk + (((c8 & 7) ^ p_swz) << 4)) = pk;
                 }
                 if (key - t + kKeys > L) {
                     // V rows beyond the context may hold any bits: zero them so that 0 * row = 0
+                    ok = warp_wait_bounded(&v_full[jj % NV], (jj / NV) & 1, abort_flag);  // the V tile has landed
+                    if (!ok) break;
                     const int first_bad = L - (key - t);
                     const int chunks = (kKeys - first_bad) * 8;
                     for (int h = 0; h < 2; ++h) {
-                        uint8_t* vgen = smem_gen + OFF_V + (h * NST + jj % NST) * kBlk;
+                        uint8_t* vgen = smem_gen + OFF_V + (h * NV + jj % NV) * kBlk;
                         for (int chk = t; chk < chunks; chk += 128)
                             *reinterpret_cast<uint4*>(vgen + first_bad * 128 + chk * 16) = make_uint4(0, 0, 0, 0);
                     }
@@ -384,7 +429,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
             if (!ok) break;
 
             // ---- end of the unit: O^T out of tensor memory, row sums added up, partial written ----
-            ok = warp_wait_bounded(&empty_bar[(jj - 1) % NST], ((jj - 1) / NST) & 1, abort_flag);
+            ok = warp_wait_bounded(&v_empty[(jj - 1) % NV], ((jj - 1) / NV) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
             const int unit = w.b * a.Hkv + w.kvh;
