@@ -89,7 +89,7 @@ typedef struct rapid_attn_shape {
 #define RAPID_ATTN_KERNEL_AUTO 0      /* keys on M where it applies, rows on M otherwise                 */
 #define RAPID_ATTN_KERNEL_ROWS_ON_M 1 /* grouped rows on the MMA's M axis: any supported shape           */
 #define RAPID_ATTN_KERNEL_KEYS_ON_M 2 /* keys on the M axis: head_dim 128, <= 64 grouped rows per KV head,
-                                         paged blocks of >= 128 keys; RAPID_ERR_UNSUPPORTED otherwise   */
+                                         any paged block size the call accepts; RAPID_ERR_UNSUPPORTED otherwise   */
 
 /* Optional knobs and extra outputs of the attention call (NULL = defaults). */
 typedef struct rapid_attn_params {

@@ -55,6 +55,7 @@ struct AttnArgs {
     // equal ranges therefore carries `pad` virtual tiles in front of every unit: a CTA whose range
     // spans a unit boundary gets that many fewer real tiles, and all CTAs finish together.
     int pad;
+    int kt_half_blocks;  // keys-on-M kernel over a paged cache with 64-key blocks: two boxes per tile
     int tile_keys;  // keys per scheduling tile: what plan, walk and merge count in (64, or 128 for the keys-on-M kernel)
 };
 
@@ -1034,21 +1035,23 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     // shared memory) when the grouped rows fit 64 columns -- faster and cheaper per byte there --,
     // rows on the M axis otherwise (more rows, head_dim 64, paged blocks of 64 keys).
     const int want = params ? params->kernel : RAPID_ATTN_KERNEL_AUTO;
-    const bool kt_ok = s.D == 128 && (GR + 15) / 16 <= kt::kMaxNC && (!paged || paged->block_size >= kt::kKeys);
+    const bool kt_ok = s.D == 128 && (GR + 15) / 16 <= kt::kMaxNC && (!paged || paged->block_size >= kTile);
     if (want != RAPID_ATTN_KERNEL_AUTO && want != RAPID_ATTN_KERNEL_ROWS_ON_M && want != RAPID_ATTN_KERNEL_KEYS_ON_M) {
         set_error("rapid_verify_attention: unknown kernel choice %d", want);
         return RAPID_ERR_INVALID_ARG;
     }
     if (want == RAPID_ATTN_KERNEL_KEYS_ON_M && !kt_ok) {
         set_error("rapid_verify_attention: the keys-on-M kernel needs head_dim 128, at most %d grouped rows and, "
-                  "paged, blocks of at least %d keys", 16 * kt::kMaxNC, kt::kKeys);
+                  "paged, blocks of at least %d keys", 16 * kt::kMaxNC, kTile);
         return RAPID_ERR_UNSUPPORTED;
     }
     const bool kt_path = want == RAPID_ATTN_KERNEL_KEYS_ON_M || (want == RAPID_ATTN_KERNEL_AUTO && kt_ok);
-    if (kt_path && paged) --tile_shift;  // blocks are counted in 128-key tiles
-    int rc = make_kv_map(&tmK, k_cache, s, outer, keys, sb, sh, sl, kt_path ? kt::kKeys : kTile);
+    const bool kt_half_blocks = kt_path && paged && paged->block_size == kTile;
+    if (kt_path && paged && !kt_half_blocks) --tile_shift;  // blocks are counted in 128-key tiles
+    const int box_rows = kt_path && !kt_half_blocks ? kt::kKeys : kTile;
+    int rc = make_kv_map(&tmK, k_cache, s, outer, keys, sb, sh, sl, box_rows);
     if (rc != RAPID_OK) return rc;
-    rc = make_kv_map(&tmV, v_cache, s, outer, keys, sb, sh, sl, kt_path ? kt::kKeys : kTile);
+    rc = make_kv_map(&tmV, v_cache, s, outer, keys, sb, sh, sl, box_rows);
     if (rc != RAPID_OK) return rc;
 
     AttnArgs a;
@@ -1069,6 +1072,7 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     a.max_blocks = paged ? paged->max_blocks_per_seq : 0;
     a.num_blocks = paged ? paged->num_blocks : 0;
     a.tile_shift = tile_shift;
+    a.kt_half_blocks = kt_half_blocks ? 1 : 0;
     a.tile_keys = kt_path ? kt::kKeys : kTile;
     a.pad = kt_path ? 5 : unit_switch_tiles(s.D);
     a.stair = all_visible ? 0 : R;

@@ -162,28 +162,43 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 for (int t = 0; t < seg && ok; ++t, ++jj) {
                     const int ks = jj % NK, vs = jj % NV;
-                    int key0 = (w.tile + t) * kKeys, outer = w.b;
-                    if (a.block_table) {  // paged: (position inside the block, physical block)
+                    // a tile is one box of 128 keys, or, for a paged cache with 64-key blocks, two
+                    // boxes of 64 keys from two physical blocks (parts = 2)
+                    const int parts = a.kt_half_blocks ? 2 : 1;
+                    int key0[2] = {(w.tile + t) * kKeys, 0}, outer[2] = {w.b, w.b};
+                    if (a.block_table) {
                         const int tile = w.tile + t;
-                        outer = __ldg(a.block_table + (size_t)w.b * a.max_blocks + (tile >> a.tile_shift));
-                        key0 = (tile & ((1 << a.tile_shift) - 1)) * kKeys;
-                        if ((unsigned)outer >= (unsigned)a.num_blocks) {
-                            atomicOr(a.status, RAPID_STATUS_BAD_BLOCK_TABLE);
-                            outer = a.num_blocks;  // outside the pool: the copy reads zeros
+                        for (int p = 0; p < parts; ++p) {
+                            const int lb = a.kt_half_blocks ? 2 * tile + p : (tile >> a.tile_shift);
+                            key0[p] = a.kt_half_blocks ? 0 : (tile & ((1 << a.tile_shift) - 1)) * kKeys;
+                            if (a.kt_half_blocks && lb * 64 >= w.L) {
+                                outer[p] = a.num_blocks;  // wholly past the context: zeros, no table entry is read
+                                continue;
+                            }
+                            outer[p] = __ldg(a.block_table + (size_t)w.b * a.max_blocks + lb);
+                            if ((unsigned)outer[p] >= (unsigned)a.num_blocks) {
+                                atomicOr(a.status, RAPID_STATUS_BAD_BLOCK_TABLE);
+                                outer[p] = a.num_blocks;  // outside the pool: the copy reads zeros
+                            }
                         }
                     }
+                    const uint32_t part_bytes = kBlk / parts;
                     if (jj >= NK) ok = mbar_wait_bounded_relaxed(&k_empty[ks], ((jj / NK) - 1) & 1, abort_flag);
                     if (!ok) break;
                     mbar_arrive_expect_tx(&k_full[ks], TILE_TX);
+                    for (int p = 0; p < parts; ++p)
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_4d(smem_gen + OFF_K + (h * NK + ks) * kBlk, &tmK, &k_full[ks], h * 64, key0, w.kvh, outer);
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_4d(smem_gen + OFF_K + (h * NK + ks) * kBlk + p * part_bytes, &tmK, &k_full[ks],
+                                        h * 64, key0[p], w.kvh, outer[p]);
                     if (jj >= NV) ok = mbar_wait_bounded_relaxed(&v_empty[vs], ((jj / NV) - 1) & 1, abort_flag);
                     if (!ok) break;
                     mbar_arrive_expect_tx(&v_full[vs], TILE_TX);
+                    for (int p = 0; p < parts; ++p)
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_4d(smem_gen + OFF_V + (h * NV + vs) * kBlk, &tmV, &v_full[vs], h * 64, key0, w.kvh, outer);
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_4d(smem_gen + OFF_V + (h * NV + vs) * kBlk + p * part_bytes, &tmV, &v_full[vs],
+                                        h * 64, key0[p], w.kvh, outer[p]);
                 }
                 walk_advance(a, w, seg);
             }
