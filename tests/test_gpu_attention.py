@@ -56,6 +56,8 @@ def test_tiny_config():
     (8, 2, 64, 4, 1000),            # head_dim 64
     (16, 1, 64, 7, 513),            # 128 grouped rows: the maximum
     (4, 4, 128, 2, 70),             # G = 1
+    (64, 8, 128, 6, 2900),          # 56 grouped rows: keys-on-M with packed probabilities, two K slots
+    (64, 8, 128, 7, 1333),          # 64 grouped rows: the most the keys-on-M kernel takes
 ])
 def test_shapes_against_oracle(Hq, Hkv, D, gamma, L):
     """The library's own choice of kernel, and the rows-on-M kernel forced (it serves every shape)."""
