@@ -86,10 +86,11 @@ typedef struct rapid_attn_shape {
 } rapid_attn_shape;
 
 /* Which split kernel rapid_verify_attention uses (rapid_attn_params.kernel). */
-#define RAPID_ATTN_KERNEL_AUTO 0      /* keys on M where it applies, rows on M otherwise                 */
+#define RAPID_ATTN_KERNEL_AUTO 0      /* keys on M for head_dim 128 and <= 64 grouped rows, rows on M otherwise */
 #define RAPID_ATTN_KERNEL_ROWS_ON_M 1 /* grouped rows on the MMA's M axis: any supported shape           */
-#define RAPID_ATTN_KERNEL_KEYS_ON_M 2 /* keys on the M axis: head_dim 128, <= 64 grouped rows per KV head,
-                                         any paged block size the call accepts; RAPID_ERR_UNSUPPORTED otherwise   */
+#define RAPID_ATTN_KERNEL_KEYS_ON_M 2 /* keys on the M axis: head_dim 128, <= 96 grouped rows per KV head (two
+                                         softmax groups beyond 64), any paged block size the call accepts;
+                                         RAPID_ERR_UNSUPPORTED otherwise                                        */
 
 /* Optional knobs and extra outputs of the attention call (NULL = defaults). */
 typedef struct rapid_attn_params {

@@ -14,6 +14,7 @@
 // from run to run.  The merge is launched as a programmatic dependent of the split kernel: its
 // blocks are resident and have done their index arithmetic by the time the last partial lands.
 #include <math.h>
+#include <type_traits>
 
 #include "common.cuh"
 #include "tcgen05.cuh"
@@ -885,7 +886,7 @@ bool attn_shape_ok(const rapid_attn_shape* s, int gamma) {
 
 }  // namespace
 
-template <int NC>
+template <int NC, int SG = 1>
 int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ, const AttnArgs& a,
                     cudaStream_t stream) {
     constexpr int smem = kt::smem_bytes(NC);
@@ -894,12 +895,12 @@ int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
     int dev = 0;
     RAPID_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev >= 64 || !configured[dev]) {
-        RAPID_CUDA_CHECK(cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC>,
+        RAPID_CUDA_CHECK(cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC, SG>,
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         if (dev < 64) configured[dev] = true;
     }
-    RAPID_CUDA_CHECK(launch_dependent(kt::verify_attn_splitkv_kt_kernel<NC>, dim3(a.num_ctas), dim3(kt::kThreads),
-                                      (size_t)smem, stream, tmK, tmV, tmQ, a));
+    RAPID_CUDA_CHECK(launch_dependent(kt::verify_attn_splitkv_kt_kernel<NC, SG>, dim3(a.num_ctas),
+                                      dim3(kt::threads(SG)), (size_t)smem, stream, tmK, tmV, tmQ, a));
     return RAPID_OK;
 }
 
@@ -910,6 +911,9 @@ int dispatch_split_kt(int NC, const CUtensorMap& tmK, const CUtensorMap& tmV, co
         case 2: return launch_split_kt<2>(tmK, tmV, tmQ, a, stream);
         case 3: return launch_split_kt<3>(tmK, tmV, tmQ, a, stream);
         case 4: return launch_split_kt<4>(tmK, tmV, tmQ, a, stream);
+        // more than 64 grouped rows: two softmax groups, each with half of the columns
+        case 5: return launch_split_kt<5, 2>(tmK, tmV, tmQ, a, stream);
+        case 6: return launch_split_kt<6, 2>(tmK, tmV, tmQ, a, stream);
     }
     set_error("unsupported number of grouped rows");
     return RAPID_ERR_UNSUPPORTED;
@@ -1033,19 +1037,22 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     CUtensorMap tmK, tmV;
     // Which split kernel: keys on the MMA's M axis (a softmax thread per key, probabilities through
     // shared memory) when the grouped rows fit 64 columns -- faster and cheaper per byte there --,
-    // rows on the M axis otherwise (more rows, head_dim 64, paged blocks of 64 keys).
+    // rows on the M axis otherwise (more rows, head_dim 64, paged blocks of 64 keys).  From 65 to 96
+    // rows the keys-on-M kernel runs on request only (two softmax groups; measured level with the
+    // rows-on-M kernel at 72 rows, not ahead of it).
     const int want = params ? params->kernel : RAPID_ATTN_KERNEL_AUTO;
-    const bool kt_ok = s.D == 128 && (GR + 15) / 16 <= kt::kMaxNC && (!paged || paged->block_size >= kTile);
+    const bool kt_ok = s.D == 128 && (GR + 15) / 16 <= kt::kMaxNC2 && (!paged || paged->block_size >= kTile);
     if (want != RAPID_ATTN_KERNEL_AUTO && want != RAPID_ATTN_KERNEL_ROWS_ON_M && want != RAPID_ATTN_KERNEL_KEYS_ON_M) {
         set_error("rapid_verify_attention: unknown kernel choice %d", want);
         return RAPID_ERR_INVALID_ARG;
     }
     if (want == RAPID_ATTN_KERNEL_KEYS_ON_M && !kt_ok) {
         set_error("rapid_verify_attention: the keys-on-M kernel needs head_dim 128, at most %d grouped rows and, "
-                  "paged, blocks of at least %d keys", 16 * kt::kMaxNC, kTile);
+                  "paged, blocks of at least %d keys", 16 * kt::kMaxNC2, kTile);
         return RAPID_ERR_UNSUPPORTED;
     }
-    const bool kt_path = want == RAPID_ATTN_KERNEL_KEYS_ON_M || (want == RAPID_ATTN_KERNEL_AUTO && kt_ok);
+    const bool kt_auto = kt_ok && (GR + 15) / 16 <= kt::kMaxNC;
+    const bool kt_path = want == RAPID_ATTN_KERNEL_KEYS_ON_M || (want == RAPID_ATTN_KERNEL_AUTO && kt_auto);
     const bool kt_half_blocks = kt_path && paged && paged->block_size == kTile;
     if (kt_path && paged && !kt_half_blocks) --tile_shift;  // blocks are counted in 128-key tiles
     const int box_rows = kt_path && !kt_half_blocks ? kt::kKeys : kTile;

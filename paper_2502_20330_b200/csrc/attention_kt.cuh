@@ -1,4 +1,4 @@
-// Split-KV verify attention with the KEYS on the M axis of the MMAs (head_dim 128, up to 64 grouped rows).
+// Split-KV verify attention with the KEYS on the M axis of the MMAs (head_dim 128, up to 96 grouped rows).
 //
 //   S^T[128 keys x N] = K_tile[128 x D] Q^T        A = K tile (K-major), B = Q (N grouped rows, K-major)
 //   O^T[D x N]       += V_tile^T[D x 128] P^T      A = V tile (MN-major), B = P^T (MN-major, written by the
@@ -11,7 +11,14 @@
 // rings of their own (two K slots, four V slots; three V slots for more than 48 rows): a K slot is
 // free once QK^T of its tile has completed, a V slot only after PV.  Work split, partial format (one partial per CTA and unit) and merge are shared with the
 // rows-on-M kernel.  Roles (224 threads): warps 0-3 softmax (thread t = key t of the tile), warp 4
-// TMA producer, warp 5 TMEM allocation + Q load + QK^T issue, warp 6 PV issue.
+// TMA producer, warp 5 TMEM allocation + Q load + QK^T issue, warp 6 PV issue.  Beyond 64 grouped
+// rows there are two softmax groups (warps 0-3 and 4-7, 352 threads, the role warps after them):
+// each takes half of the columns for all 128 keys.
+//
+// Columns past the grouped rows (N is a multiple of 16) are made harmless once instead of being
+// tested per element: their rows of Q are zeroed at set-up (scores 0) and their reference is +inf
+// (probabilities 0).  A tile that every row sees whole -- all of a long context but its end -- takes
+// a loop without the per-column mask.
 //
 // P^T in shared memory has the layout of a V tile half: one 128-byte row per key holding that key's
 // probabilities for 64 grouped rows, 128-byte swizzle (16-byte chunk index XOR key & 7), 8-key groups
@@ -37,8 +44,10 @@
 namespace kt {
 
 constexpr int kKeys = 128;                 // keys per tile
-constexpr int kMaxNC = 4;                  // up to 64 grouped rows: beyond that the rows-on-M kernel is faster
-constexpr int kThreads = 224;
+constexpr int kMaxNC = 4;                  // one softmax group serves up to 64 grouped rows
+constexpr int kMaxNC2 = 6;                 // two softmax groups (half of the columns each) serve up to 96
+__host__ __device__ constexpr int threads(int SG) { return 128 * SG + 96; }  // softmax warps + three role warps
+constexpr int kThreads = threads(1);
 constexpr int kBlk = kKeys * 128;          // bytes of one tile x 64-column half
 constexpr float kJump = 16.f;              // a score this far (log2) above the reference moves it
 
@@ -53,19 +62,24 @@ __host__ __device__ constexpr int smem_bytes(int NC) {
     return 2 * (k_slots(NC) + v_slots(NC)) * kBlk + 2 * (NC * 16) * 128 + p_blocks(NC) * kBlk + 1024;
 }
 
-__device__ __forceinline__ void bar_softmax() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-__device__ __forceinline__ bool bar_softmax_or(bool flag) {
+// Named barriers of one softmax group (128 threads): barrier 1 for group 0, barrier 2 for group 1.
+__device__ __forceinline__ void bar_softmax(int grp) {
+    if (grp == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+    else asm volatile("bar.sync 2, 128;" ::: "memory");
+}
+#define RAPID_KT_BAR_OR(ID)                                                                              \
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.or.pred p, " #ID ", 128, q;\n\t" \
+                 "selp.u32 %0, 1, 0, p;\n\t}"                                                            \
+                 : "=r"(res)                                                                             \
+                 : "r"((uint32_t)flag)                                                                   \
+                 : "memory")
+__device__ __forceinline__ bool bar_softmax_or(int grp, bool flag) {
     uint32_t res;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, 128, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(res)
-        : "r"((uint32_t)flag)
-        : "memory");
+    if (grp == 0) RAPID_KT_BAR_OR(1);
+    else RAPID_KT_BAR_OR(2);
     return res != 0;
 }
+#undef RAPID_KT_BAR_OR
 __device__ __forceinline__ float warp_max32(float v) {
 #pragma unroll
     for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
@@ -77,14 +91,21 @@ __device__ __forceinline__ float warp_sum32(float v) {
     return v;
 }
 
-// NC = N / 16 column chunks (N = grouped rows padded to 16).
-template <int NC>
-__global__ void __launch_bounds__(kThreads, 1)
+// NC = N / 16 column chunks (N = grouped rows padded to 16).  SG = softmax groups of 128 threads:
+// group g forms the probabilities of columns [g N/SG, (g+1) N/SG) for all 128 keys of a tile, keeps
+// those rows' references and sums and rescales and reads out those columns of O^T; the groups meet
+// only at the P^T barrier (PV starts when both have published) and at the end of a unit.
+template <int NC, int SG = 1>
+__global__ void __launch_bounds__(threads(SG), 1)
 verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                               const __grid_constant__ CUtensorMap tmV,
                               const __grid_constant__ CUtensorMap tmQ, const AttnArgs a) {
     constexpr int D = 128;
     constexpr int N = NC * 16;
+    constexpr int NG = N / SG;             // columns per softmax group
+    constexpr int CH = NG % 16 == 0 ? 16 : 8;  // columns per tensor-memory load
+    constexpr int WS = 4 * SG;             // softmax warps; the role warps follow
+    static_assert(N % SG == 0 && NG % 8 == 0, "a group's columns are whole 16-byte chunks of a P^T row");
     constexpr int NK = k_slots(NC), NV = v_slots(NC);
     constexpr int TILE_TX = 2 * kBlk;  // one tile of K or of V: two 64-column halves
     constexpr uint32_t TMEM_COLS = 512;
@@ -100,7 +121,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
     __shared__ uint32_t tmem_slot;
     __shared__ Walk s_walk;
     __shared__ int s_abort;
-    __shared__ float sh_mref[128], sh_fac[128], sh_w[4][128];
+    __shared__ __align__(16) float sh_mref[128], sh_fac[128], sh_w[4][128];
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -121,17 +142,17 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&s_full[i], 1);
-            mbar_init(&p_full[i], 4);
+            mbar_init(&p_full[i], WS);
         }
         mbar_init(&q_full, 1);
-        mbar_init(&o_free, 4);
+        mbar_init(&o_free, WS);
         fence_mbar_init();
         s_abort = 0;
         prefetch_tensormap(&tmK);
         prefetch_tensormap(&tmV);
         prefetch_tensormap(&tmQ);
     }
-    if (warp == 5) tmem_alloc(&tmem_slot, TMEM_COLS);  // warp 5 also frees it at the end
+    if (warp == WS + 1) tmem_alloc(&tmem_slot, TMEM_COLS);  // the same warp frees it at the end
     griddep_wait();               // inputs are read from here on
     griddep_launch_dependents();  // the merge blocks may take their seats
     if (tid == 0) {
@@ -147,6 +168,16 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
             if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
         }
     }
+    // The Q rows past the grouped rows are never written by the Q loads: zero them once, so that
+    // the scores of those columns are 0 whatever the shared memory held.
+    {
+        const int pad_chunks = (N - a.GR) * 8;  // 16-byte chunks per 64-column half
+        for (int i = tid; i < 2 * pad_chunks; i += threads(SG)) {
+            const int h = i >= pad_chunks, k16 = h ? i - pad_chunks : i;
+            *reinterpret_cast<uint4*>(smem_gen + OFF_Q + h * (N * 128) + a.GR * 128 + k16 * 16) = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async_smem();
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -154,7 +185,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
     Walk w = s_walk;
     volatile int* abort_flag = &s_abort;
 
-    if (warp == 4) {
+    if (warp == WS) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             int jj = 0;
@@ -204,7 +235,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 walk_advance(a, w, seg);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == WS + 1) {
         // ---------------- Q loader and QK^T issuer ----------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(128, N, 0, 0);
@@ -243,7 +274,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 ++seg_idx;
             }
         }
-    } else if (warp == 6) {
+    } else if (warp == WS + 2) {
         // ---------------- PV issuer ----------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(D, N, 1, 1);
@@ -271,29 +302,32 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 walk_advance(a, w, seg);
             }
         }
-    } else if (warp < 4) {
-        // ---------------- softmax: thread t = key t of the tile = TMEM lane t ----------------
-        const int t = tid;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        const uint32_t tO = tmem_base + lane_base + COL_O;
+    } else if (warp < WS) {
+        // ---------------- softmax: thread t of group grp = key t of the tile = TMEM lane t ----------------
+        const int grp = warp >> 2, wq = warp & 3;
+        const int t = tid & 127;
+        constexpr int C0_STEP = NG;
+        const int C0 = grp * C0_STEP;  // this group's first column
+        const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
+        const uint32_t tO = tmem_base + lane_base + COL_O + C0;
         const float c = a.scale_log2;
         const int slot_stride = (int)slot_floats(a.GR, D);
         // this key's row of P^T (MN-major: 128 bytes = 64 grouped rows per key, 128-byte swizzle)
         uint8_t* p_gen = smem_gen + OFF_P + t * 128;
         const int p_swz = t & 7;
 
-        float lsum[N];  // this key slot's share of every row's sum
+        float lsum[NG];  // this key slot's share of the sums of the group's rows
         int jj = 0;
         bool ok = true;
         while (w.remaining > 0 && ok) {
             const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
             const int L = w.L;
 #pragma unroll
-            for (int col = 0; col < N; ++col) lsum[col] = 0.f;
+            for (int i = 0; i < NG; ++i) lsum[i] = 0.f;
 
             for (int ti = 0; ti < seg && ok; ++ti, ++jj) {
                 const int b = jj & 1;
-                const uint32_t tS = tmem_base + lane_base + COL_S + 128u * b;
+                const uint32_t tS = tmem_base + lane_base + COL_S + 128u * b + C0;
                 const int key = (w.tile + ti) * kKeys + t;
                 // row i sees keys <= L-R+i; rows are column i*G+g: the masked columns are a prefix
                 // (no stair: every row sees every key below L)
@@ -306,33 +340,49 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 // One pass over the scores: probabilities against the current references, kept in
                 // registers until it is known that no visible score sits far above its reference.
                 // (Kept as fp32 up to 48 columns; beyond that as packed bf16 pairs, to stay in registers.)
-                constexpr bool kPacked = NC > 3;
-                float pv[kPacked ? 2 : N];
-                uint32_t pq[kPacked ? N / 2 : 1];
+                constexpr bool kPacked = NG > 48;
+                float pv[kPacked ? 2 : NG];
+                uint32_t pq[kPacked ? NG / 2 : 1];
                 bool move = ti == 0;
                 if (ti > 0) {
+                    // MASKED = false for a tile every row sees whole (all of a long context but its end):
+                    // no per-column predicate.  Columns past the grouped rows need none either: their
+                    // scores are 0 (zero rows of Q) and their reference is +inf, so they come out as 0.
+                    auto first_pass = [&](auto masked_tag) {
+                        constexpr bool MASKED = decltype(masked_tag)::value;
+                        bool far = false;
 #pragma unroll
-                    for (int ch = 0; ch < NC; ++ch) {
-                        uint32_t sr[16];
-                        tmem_ld_x16(tS + 16 * ch, sr);
-                        tmem_wait_ld();
+                        for (int ch = 0; ch < NG / CH; ++ch) {
+                            uint32_t sr[CH];
+                            tmem_ld_cols<CH>(tS + CH * ch, sr);
+                            tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 16; e += 2) {
-                            const int col = 16 * ch + e;
-                            const float x0 = fmaf(__uint_as_float(sr[e]), c, -sh_mref[col]);
-                            const float x1 = fmaf(__uint_as_float(sr[e + 1]), c, -sh_mref[col + 1]);
-                            const bool v0 = col >= cmin, v1 = col + 1 >= cmin;
-                            move = move || (v0 && col < a.GR && x0 > kJump) || (v1 && col + 1 < a.GR && x1 > kJump);
-                            const float p0 = fast_exp2(v0 ? x0 : -INFINITY), p1 = fast_exp2(v1 ? x1 : -INFINITY);
-                            if (kPacked) {
-                                pq[col >> 1] = pack_bf16x2(p0, p1);
-                            } else {
-                                pv[kPacked ? 0 : col] = p0;
-                                pv[kPacked ? 1 : col + 1] = p1;
+                            for (int e = 0; e < CH; e += 4) {
+                                const int li = CH * ch + e, col = C0 + li;
+                                const float4 m = *reinterpret_cast<const float4*>(&sh_mref[col]);
+                                float x[4] = {fmaf(__uint_as_float(sr[e]), c, -m.x), fmaf(__uint_as_float(sr[e + 1]), c, -m.y),
+                                              fmaf(__uint_as_float(sr[e + 2]), c, -m.z),
+                                              fmaf(__uint_as_float(sr[e + 3]), c, -m.w)};
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    if (MASKED) x[i] = col + i >= cmin ? x[i] : -INFINITY;
+                                    far |= x[i] > kJump;
+                                    x[i] = fast_exp2(x[i]);
+                                }
+                                if (kPacked) {
+                                    pq[li >> 1] = pack_bf16x2(x[0], x[1]);
+                                    pq[(li >> 1) + 1] = pack_bf16x2(x[2], x[3]);
+                                } else {
+#pragma unroll
+                                    for (int i = 0; i < 4; ++i) pv[kPacked ? 0 : li + i] = x[i];
+                                }
                             }
                         }
-                    }
-                    move = bar_softmax_or(move);
+                        return far;
+                    };
+                    const bool tile_clear = (w.tile + ti + 1) * kKeys <= L - a.stair;  // the same for every thread
+                    move = tile_clear ? first_pass(std::false_type{}) : first_pass(std::true_type{});
+                    move = bar_softmax_or(grp, move);
                 }
                 // PV of the previous tile must be complete: it reads P^T, and O^T may be rescaled now
                 if (jj >= 1) {
@@ -343,67 +393,71 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 if (move) {
                     // new reference = max(old, this tile's row maxima over the 128 keys)
 #pragma unroll
-                    for (int ch = 0; ch < NC; ++ch) {
-                        uint32_t sr[16];
-                        tmem_ld_x16(tS + 16 * ch, sr);
+                    for (int ch = 0; ch < NG / CH; ++ch) {
+                        uint32_t sr[CH];
+                        tmem_ld_cols<CH>(tS + CH * ch, sr);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            const int col = 16 * ch + e;
+                        for (int e = 0; e < CH; ++e) {
+                            const int col = C0 + CH * ch + e;
                             const float v = (col >= cmin && col < a.GR) ? __uint_as_float(sr[e]) * c : -INFINITY;
                             const float wm = warp_max32(v);
-                            if (lane == 0) sh_w[warp][col] = wm;
+                            if (lane == 0) sh_w[wq][col] = wm;
                         }
                     }
-                    bar_softmax();
-                    if (t < N) {
-                        const float old = ti == 0 ? -INFINITY : sh_mref[t];
-                        const float nm = fmaxf(fmaxf(old, fmaxf(sh_w[0][t], sh_w[1][t])), fmaxf(sh_w[2][t], sh_w[3][t]));
-                        sh_fac[t] = (nm == old) ? 1.f : fast_exp2(old - nm);  // old = -inf gives 0
-                        sh_mref[t] = nm;
+                    bar_softmax(grp);
+                    if (t < NG) {
+                        const int col = C0 + t;
+                        const float old = ti == 0 ? -INFINITY : sh_mref[col];
+                        const float nm =
+                            fmaxf(fmaxf(old, fmaxf(sh_w[0][col], sh_w[1][col])), fmaxf(sh_w[2][col], sh_w[3][col]));
+                        const bool pad = col >= a.GR;  // a column past the grouped rows: reference +inf, probabilities 0
+                        sh_fac[col] = (pad || nm == old) ? 1.f : fast_exp2(old - nm);  // old = -inf gives 0
+                        sh_mref[col] = pad ? INFINITY : nm;
                     }
-                    bar_softmax();
+                    bar_softmax(grp);
                     if (ti > 0) {
 #pragma unroll
-                        for (int col = 0; col < N; ++col) lsum[col] *= sh_fac[col];
-                        // thread t is lane t of O^T (= output column d): rescale its N row entries
+                        for (int i = 0; i < NG; ++i) lsum[i] *= sh_fac[C0 + i];
+                        // thread t is lane t of O^T (= output column d): rescale its group's row entries
 #pragma unroll
-                        for (int ch = 0; ch < NC; ++ch) {
-                            uint32_t orow[16];
-                            tmem_ld_x16(tO + 16 * ch, orow);
+                        for (int ch = 0; ch < NG / CH; ++ch) {
+                            uint32_t orow[CH];
+                            tmem_ld_cols<CH>(tO + CH * ch, orow);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 16; ++e)
-                                orow[e] = __float_as_uint(__uint_as_float(orow[e]) * sh_fac[16 * ch + e]);
-                            tmem_st_x16(tO + 16 * ch, orow);
+                            for (int e = 0; e < CH; ++e)
+                                orow[e] = __float_as_uint(__uint_as_float(orow[e]) * sh_fac[C0 + CH * ch + e]);
+                            tmem_st_cols<CH>(tO + CH * ch, orow);
                         }
                         tmem_wait_st();
                     }
                     // the probabilities again, against the new references
 #pragma unroll
-                    for (int ch = 0; ch < NC; ++ch) {
-                        uint32_t sr[16];
-                        tmem_ld_x16(tS + 16 * ch, sr);
+                    for (int ch = 0; ch < NG / CH; ++ch) {
+                        uint32_t sr[CH];
+                        tmem_ld_cols<CH>(tS + CH * ch, sr);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 16; e += 2) {
-                            const int col = 16 * ch + e;
+                        for (int e = 0; e < CH; e += 2) {
+                            const int li = CH * ch + e, col = C0 + li;
                             const float m0 = sh_mref[col], m1 = sh_mref[col + 1];
                             const float x0 = col >= cmin ? fmaf(__uint_as_float(sr[e]), c, m0 == -INFINITY ? 0.f : -m0) : -INFINITY;
                             const float x1 = col + 1 >= cmin ? fmaf(__uint_as_float(sr[e + 1]), c, m1 == -INFINITY ? 0.f : -m1) : -INFINITY;
                             const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                             if (kPacked) {
-                                pq[col >> 1] = pack_bf16x2(p0, p1);
+                                pq[li >> 1] = pack_bf16x2(p0, p1);
                             } else {
-                                pv[kPacked ? 0 : col] = p0;
-                                pv[kPacked ? 1 : col + 1] = p1;
+                                pv[kPacked ? 0 : li] = p0;
+                                pv[kPacked ? 1 : li + 1] = p1;
                             }
                         }
                     }
                 }
                 // this key's row of P^T: 16-byte chunks of 8 grouped rows each
 #pragma unroll
-                for (int c8 = 0; c8 < N / 8; ++c8) {
+                for (int c8 = 0; c8 < NG / 8; ++c8) {
+                    const int g8 = C0 / 8 + c8;  // the chunk's place in the whole row
                     uint4 pk;
                     if (kPacked) {
                         pk = make_uint4(pq[4 * c8], pq[4 * c8 + 1], pq[4 * c8 + 2], pq[4 * c8 + 3]);
@@ -423,10 +477,11 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
                         for (int e = 0; e < 8; ++e) lsum[8 * c8 + e] += pv[kPacked ? 0 : o + e];
                     }
-                    *reinterpret_cast<uint4*>(p_gen + (c8 >> 3) * kBlk + (((c8 & 7) ^ p_swz) << 4)) = pk;
+                    *reinterpret_cast<uint4*>(p_gen + (g8 >> 3) * kBlk + (((g8 & 7) ^ p_swz) << 4)) = pk;
                 }
-                if (key - t + kKeys > L) {
+                if (grp == 0 && key - t + kKeys > L) {
                     // V rows beyond the context may hold any bits: zero them so that 0 * row = 0
+                    // (one group does it; PV waits for both groups' arrivals)
                     ok = warp_wait_bounded(&v_full[jj % NV], (jj / NV) & 1, abort_flag);  // the V tile has landed
                     if (!ok) break;
                     const int first_bad = L - (key - t);
@@ -451,27 +506,28 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
             const int unit = w.b * a.Hkv + w.kvh;
             float* slot = a.partial + (size_t)(cta + unit) * slot_stride;
 #pragma unroll
-            for (int ch = 0; ch < NC; ++ch) {
-                uint32_t orow[16];
-                tmem_ld_x16(tO + 16 * ch, orow);
+            for (int ch = 0; ch < NG / CH; ++ch) {
+                uint32_t orow[CH];
+                tmem_ld_cols<CH>(tO + CH * ch, orow);
                 tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const int col = 16 * ch + e;
+                for (int e = 0; e < CH; ++e) {
+                    const int col = C0 + CH * ch + e;
                     if (col < a.GR && sh_mref[col] != -INFINITY) slot[(size_t)col * D + t] = __uint_as_float(orow[e]);
                 }
             }
 #pragma unroll
-            for (int col = 0; col < N; ++col) {
-                const float ws = warp_sum32(lsum[col]);
-                if (lane == 0) sh_w[warp][col] = ws;
+            for (int i = 0; i < NG; ++i) {
+                const float ws = warp_sum32(lsum[i]);
+                if (lane == 0) sh_w[wq][C0 + i] = ws;
             }
-            bar_softmax();
-            if (t < a.GR) {
-                slot[a.GR * D + t] = sh_mref[t];
-                slot[a.GR * D + a.GR + t] = ((sh_w[0][t] + sh_w[1][t]) + sh_w[2][t]) + sh_w[3][t];
+            bar_softmax(grp);
+            if (t < NG && C0 + t < a.GR) {
+                const int col = C0 + t;
+                slot[a.GR * D + col] = sh_mref[col];
+                slot[a.GR * D + a.GR + col] = ((sh_w[0][col] + sh_w[1][col]) + sh_w[2][col]) + sh_w[3][col];
             }
-            bar_softmax();  // sh_w / sh_mref are reused by the next unit
+            bar_softmax(grp);  // sh_w / sh_mref are reused by the next unit
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&o_free);
@@ -481,7 +537,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == WS + 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }

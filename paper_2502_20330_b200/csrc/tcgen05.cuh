@@ -113,6 +113,35 @@ __device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t (&r)[
                  : "memory");
 }
 
+// 32 lanes x 8 columns
+__device__ __forceinline__ void tmem_ld_x8(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_st_x8(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 :
+                 : "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+
+// The same moves by chunk width (8 or 16 columns), for loops whose column count is a template parameter.
+template <int CH>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[CH]) {
+    static_assert(CH == 8 || CH == 16, "chunk of 8 or 16 columns");
+    if constexpr (CH == 16) tmem_ld_x16(taddr, r);
+    else tmem_ld_x8(taddr, r);
+}
+template <int CH>
+__device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t (&r)[CH]) {
+    static_assert(CH == 8 || CH == 16, "chunk of 8 or 16 columns");
+    if constexpr (CH == 16) tmem_st_x16(taddr, r);
+    else tmem_st_x8(taddr, r);
+}
+
 #endif  // __CUDACC__
 
 }  // namespace rapid

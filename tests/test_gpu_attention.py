@@ -67,6 +67,28 @@ def test_shapes_against_oracle(Hq, Hkv, D, gamma, L):
     _compare(q, k, v, ctx, gamma, kernel=1)
 
 
+@pytest.mark.parametrize("Hq,Hkv,gamma,L,num_ctas", [
+    (64, 8, 8, 1500, 0),            # 72 grouped rows: two softmax groups of 40 columns
+    (64, 8, 9, 2900, 5),            # 80 rows: no padding column
+    (64, 8, 10, 1333, 1),           # 88 rows: two groups of 48 columns
+    (64, 8, 11, 4000, 148),         # 96 rows: the most the keys-on-M kernel takes
+    (72, 8, 8, 3000, 3),            # G = 9
+    (40, 4, 8, 5000, 37),           # G = 10, CTAs that span units
+])
+def test_keys_on_m_two_softmax_groups(Hq, Hkv, gamma, L, num_ctas):
+    """65 to 96 grouped rows on the keys-on-M kernel (on request: the library's own choice there is rows on M)."""
+    cfg = wl.VerifyConfig("t", B=2, Hq=Hq, Hkv=Hkv, D=128, gamma=gamma, V=4096, ctx_lens=(L, max(gamma + 1, L // 3)))
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=2, device="cuda", poison_padding=True)
+    _, _, o32 = _compare(q, k, v, ctx, gamma, num_ctas=num_ctas, kernel=2)
+    _, _, again, _ = _run(q, k, v, ctx, gamma, num_ctas=num_ctas, kernel=2)
+    assert torch.equal(o32, again)                     # bit-identical from run to run
+    # scores far above the first tile's: the references move, in either group
+    k2 = k.clone()
+    k2[:, :, L // 2:L // 2 + 10] *= 6.0
+    k2[:, :, L - 40:L - 35] *= 9.0
+    _compare(q, k2, v, ctx, gamma, num_ctas=num_ctas, kernel=2)
+
+
 @pytest.mark.parametrize("kernel", [1, 2])
 @pytest.mark.parametrize("num_ctas", [1, 2, 7, 148, 509])
 def test_split_invariance(num_ctas, kernel):
@@ -166,6 +188,8 @@ def test_llama8b_128k_and_70b_sampled_rows():
         _compare(q, k, v, ctx, cfg.gamma, units=units)
         if name == "llama8b_128k":
             _compare(q, k, v, ctx, cfg.gamma, units=units, kernel=1)
+        else:
+            _compare(q, k, v, ctx, cfg.gamma, units=units, kernel=2)   # two softmax groups at full size
         del q, k, v
 
 
