@@ -30,6 +30,17 @@ def _oracle(q, k, v, ctx, gamma, scale=0.0, units=None):
                                    scale=scale, units=units)
 
 
+def _lse_tolerance(q, k, kernel):
+    """Absolute tolerance of the natural-log sum-exp.  The row sums add fp32 probabilities (1e-3 covers
+    their rounding over 128K keys), except on the keys-on-M kernel from 49 to 64 grouped rows, whose
+    threads have no registers for a tile of fp32 probabilities and add the bf16 values the tensor
+    cores multiply: where one key dominates a row, its rounding (bf16 keeps 8 significant bits, so up
+    to 2^-8 relative) shows in full."""
+    grouped_rows = q.shape[2] // k.shape[1] * q.shape[1]
+    wide_keys_on_m = kernel != 1 and q.shape[3] == 128 and 48 < grouped_rows <= 64
+    return 2.0 ** -8 + 5e-4 if wide_keys_on_m else 1e-3
+
+
 def _compare(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, units=None, kernel=0):
     out, lse, o32, status = _run(q, k, v, ctx, gamma, num_ctas, scale, kernel)
     assert status == 0
@@ -37,7 +48,7 @@ def _compare(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, units=None, kernel=0):
     rows = ~np.isnan(ref_lse)
     rep = parity.check_attention(out.float().cpu().numpy(), ref, rows)
     parity.check_attention(o32.cpu().numpy(), ref, rows)
-    assert np.abs(lse.cpu().numpy()[rows] - ref_lse[rows]).max() < 1e-3
+    assert np.abs(lse.cpu().numpy()[rows] - ref_lse[rows]).max() < _lse_tolerance(q, k, kernel)
     return rep, out, o32
 
 
@@ -219,6 +230,29 @@ def test_random_shapes_and_lengths():
         _compare(q, k, v, ctx, gamma, num_ctas=num_ctas)
         if D == 128 and G * (gamma + 1) <= 64:      # the automatic choice was keys-on-M: rows-on-M too
             _compare(q, k, v, ctx, gamma, num_ctas=num_ctas, kernel=1)
+
+
+def test_keys_on_m_random_sweep():
+    """Seeded sweep of the keys-on-M kernel over 1 to 96 grouped rows (every column count, one and two
+    softmax groups, numbers of rows that are no multiple of 8), ragged batches with poisoned padding,
+    splits from 1 to 512 CTAs, and, in a third of the cases, a few keys whose scores sit far above the
+    rest, so that the softmax references move in the middle of a unit."""
+    rng = np.random.default_rng(7)
+    layouts = [(8, 2), (16, 2), (7, 7), (32, 8), (64, 8), (28, 4), (40, 4), (72, 8), (12, 12), (96, 8), (5, 1), (48, 8)]
+    for trial in range(150):
+        Hq, Hkv = layouts[int(rng.integers(len(layouts)))]
+        G = Hq // Hkv
+        gamma = int(rng.integers(0, min(11, 96 // G - 1) + 1))
+        B = int(rng.integers(1, 4))
+        Lmax = int(rng.integers(gamma + 1, 2600))
+        lens = tuple(int(rng.integers(gamma + 1, Lmax + 1)) for _ in range(B))
+        cfg = wl.VerifyConfig("sweep", B=B, Hq=Hq, Hkv=Hkv, D=128, gamma=gamma, V=4096, ctx_lens=lens, Lmax=Lmax)
+        q, k, v, ctx = wl.attention_inputs(cfg, seed=1000 + trial, device="cuda", poison_padding=True)
+        if rng.random() < 0.3:
+            j = int(rng.integers(0, max(1, min(lens) - 1)))
+            k[:, :, j:j + 3] *= float(rng.choice([4.0, 8.0]))
+        num_ctas = int(rng.choice([0, 1, 2, 3, 5, 16, 37, 148, 300, 512]))
+        _compare(q, k, v, ctx, gamma, num_ctas=num_ctas, kernel=2)
 
 
 @pytest.mark.parametrize("B,Hq,Hkv,D,gamma,lo,hi,num_ctas", [
