@@ -59,6 +59,11 @@ def _load():
             vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, c_i64,
             ctypes.c_int, c_i64, c_i64, c_i64, c_dbl, vp, c_i64, vp, vp,
         ]
+        lib.oracle_verify_attention_window.restype = ctypes.c_int
+        lib.oracle_verify_attention_window.argtypes = [
+            vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, c_i64,
+            ctypes.c_int, c_i64, c_i64, c_i64, c_dbl, c_i64, c_i64, vp, c_i64, vp, vp,
+        ]
         lib.oracle_rapid_distributions.restype = None
         lib.oracle_rapid_distributions.argtypes = [vp, vp, c_i64, c_dbl, c_dbl, c_dbl, vp, vp, vp, vp]
         lib.oracle_residual_weights.restype = None
@@ -88,8 +93,11 @@ def _c(a, dtype):
 
 
 def verify_attention(q_bits, k_bits, v_bits, ctx_lens, gamma, scale=0.0, units=None,
-                     kv_strides=None):
+                     kv_strides=None, sink=0, window=0):
     """Definition of verify attention.
+
+    ``window > 0`` applies the sink + window visibility of the streaming drafter of Section 3.2
+    (row i with own key lim sees key j iff j <= lim and (j < sink or j > lim - window)).
 
     q_bits [B,R,Hq,D] uint16 (bf16 bits); k_bits, v_bits [B,Hkv,Lmax,D] uint16
     (or flat arrays when ``kv_strides=(stride_b, stride_h, stride_l, Lmax, Hkv)``
@@ -119,9 +127,16 @@ def verify_attention(q_bits, k_bits, v_bits, ctx_lens, gamma, scale=0.0, units=N
         n_units = units.size
     else:
         n_units = 0
-    rc = lib.oracle_verify_attention(
-        _ptr(q_bits), _ptr(k_bits), _ptr(v_bits), _ptr(ctx_lens), B, Hq, Hkv, D, Lmax, gamma,
-        sb, sh, sl, float(scale), _ptr(units), n_units, _ptr(out), _ptr(lse))
+    if window > 0:
+        rc = lib.oracle_verify_attention_window(
+            _ptr(q_bits), _ptr(k_bits), _ptr(v_bits), _ptr(ctx_lens), B, Hq, Hkv, D, Lmax, gamma,
+            sb, sh, sl, float(scale), int(sink), int(window), _ptr(units), n_units, _ptr(out), _ptr(lse))
+    else:
+        if sink:
+            raise ValueError("sink keys need a window")
+        rc = lib.oracle_verify_attention(
+            _ptr(q_bits), _ptr(k_bits), _ptr(v_bits), _ptr(ctx_lens), B, Hq, Hkv, D, Lmax, gamma,
+            sb, sh, sl, float(scale), _ptr(units), n_units, _ptr(out), _ptr(lse))
     if rc != 0:
         raise ValueError(f"oracle_verify_attention failed with {rc}")
     return out, lse

@@ -7,10 +7,10 @@
  * Only the tests, the smoke check and the benchmark's CPU-baseline leg use it.
  *
  * Two parts:
- *   - verify attention: the target model's single validation pass over the full
- *     context (Algorithm 1, the LogitsOf step; Section 2.1 "single forward
- *     pass").  The paper prints no attention formula, so this is the textbook
- *     definition: masked softmax(scale * q k^T) v, causal among the draft rows.
+ *   - verify attention: the target model scores all draft positions in one pass
+ *     over the full context (Algorithm 1, the LogitsOf step; Section 2.1).  The
+ *     paper prints no attention formula, so this is the textbook definition:
+ *     masked softmax(scale * q k^T) v, causal among the draft rows.
  *   - accept / residual: Algorithm 1's validation loop with the
  *     retrieval-augmented target of Eq. (new_target) / Eq. (delta), the tail
  *     rule of Section 2.4 and the residual of Algorithm 1's last step.
@@ -124,6 +124,89 @@ int oracle_verify_attention(const uint16_t* q, const uint16_t* k, const uint16_t
         for (int d = 0; d < D; ++d) orow[d] = acc[d] / denom;
         if (lse) lse[((int64_t)b * R + i) * Hq + h] = m + log(denom);
         free(s);
+        free(acc);
+        free(qd);
+    }
+    return failed ? -2 : 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Verify attention under a sink + window mask.                              */
+/*                                                                           */
+/* Section 3.2 describes the streaming drafter the paper compares with       */
+/* (MagicDec / StreamingLLM): a KV budget of 4,096 entries of which 4 are     */
+/* "sink" tokens at the start of the sequence, the rest the most recent      */
+/* ones.  Laid over a full cache that is a visibility rule: row i, whose own */
+/* key is own = L_b - R + i, sees key j iff                                   */
+/*     j <= own   and   ( j < sink   or   j > own - window ).                 */
+/* Everything else is the definition above: masked softmax over the visible  */
+/* keys, fp64.  Hidden keys are never read.  window >= 1 (a row always sees   */
+/* its own key); sink >= 0.  Same layouts, unit_list and return codes as     */
+/* oracle_verify_attention.                                                  */
+/* ------------------------------------------------------------------------ */
+int oracle_verify_attention_window(const uint16_t* q, const uint16_t* k, const uint16_t* v,
+                                   const int32_t* ctx_lens, int B, int Hq, int Hkv, int D,
+                                   int64_t Lmax, int gamma, int64_t kv_stride_b,
+                                   int64_t kv_stride_h, int64_t kv_stride_l, double scale,
+                                   int64_t sink, int64_t window, const int64_t* unit_list,
+                                   int64_t n_units, double* out, double* lse) {
+    const int R = gamma + 1;
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || gamma < 0 || Hq % Hkv != 0) return -1;
+    if (sink < 0 || window < 1) return -1;
+    const int G = Hq / Hkv;
+    for (int b = 0; b < B; ++b)
+        if (ctx_lens[b] < R || (int64_t)ctx_lens[b] > Lmax) return -1;
+    if (scale == 0.0) scale = 1.0 / sqrt((double)D);
+    const int64_t all_units = (int64_t)B * Hq * R;
+    if (!unit_list) n_units = all_units;
+    for (int64_t t = 0; unit_list && t < n_units; ++t)
+        if (unit_list[t] < 0 || unit_list[t] >= all_units) return -1;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t t = 0; t < n_units; ++t) {
+        const int64_t unit = unit_list ? unit_list[t] : t;
+        const int b = (int)(unit / ((int64_t)Hq * R));
+        const int h = (int)((unit / R) % Hq);
+        const int i = (int)(unit % R);
+        const int kv_head = h / G;
+        const int64_t L = ctx_lens[b];
+        const int64_t own = L - R + i; /* the row's own key */
+        const uint16_t* qrow = q + (((int64_t)b * R + i) * Hq + h) * D;
+        const uint16_t* kbase = k + b * kv_stride_b + kv_head * kv_stride_h;
+        const uint16_t* vbase = v + b * kv_stride_b + kv_head * kv_stride_h;
+        double* score = (double*)malloc((size_t)(own + 1) * sizeof(double));
+        double* acc = (double*)calloc((size_t)D, sizeof(double));
+        double* qd = (double*)malloc((size_t)D * sizeof(double));
+        if (!score || !acc || !qd) {
+#pragma omp atomic write
+            failed = 1;
+            free(score);
+            free(acc);
+            free(qd);
+            continue;
+        }
+        for (int d = 0; d < D; ++d) qd[d] = bf16_bits_to_double(qrow[d]);
+        double m = -INFINITY;
+        for (int64_t j = 0; j <= own; ++j) {
+            if (!(j < sink || j > own - window)) continue; /* hidden */
+            const uint16_t* krow = kbase + j * kv_stride_l;
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += qd[d] * bf16_bits_to_double(krow[d]);
+            score[j] = scale * dot;
+            if (score[j] > m) m = score[j];
+        }
+        double denom = 0.0;
+        for (int64_t j = 0; j <= own; ++j) {
+            if (!(j < sink || j > own - window)) continue;
+            const double e = exp(score[j] - m);
+            denom += e;
+            const uint16_t* value_row = vbase + j * kv_stride_l;
+            for (int d = 0; d < D; ++d) acc[d] += e * bf16_bits_to_double(value_row[d]);
+        }
+        double* orow = out + (((int64_t)b * R + i) * Hq + h) * D;
+        for (int d = 0; d < D; ++d) orow[d] = acc[d] / denom;
+        if (lse) lse[((int64_t)b * R + i) * Hq + h] = m + log(denom);
+        free(score);
         free(acc);
         free(qd);
     }

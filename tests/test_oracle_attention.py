@@ -178,3 +178,80 @@ def test_invalid_lengths_are_rejected():
         oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(k), np.array([2], np.int32), 2)
     with pytest.raises(ValueError):
         oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(k), np.array([11], np.int32), 2)
+
+
+# ---- sink + window visibility (Section 3.2: the streaming drafter's cache of 4,096 entries, 4 of them sinks) ----
+
+def _brute_window(q, k, v, ctx, gamma, scale, sink, window):
+    """Loops over an explicitly enumerated key set per row: the sinks, then the window."""
+    q = q.double().numpy(); k = k.double().numpy(); v = v.double().numpy()
+    B, R, Hq, D = q.shape
+    G = Hq // k.shape[1]
+    out = np.zeros((B, R, Hq, D)); lse = np.zeros((B, R, Hq))
+    for b in range(B):
+        L = int(ctx[b])
+        for h in range(Hq):
+            for i in range(R):
+                own = L - R + i
+                keys = sorted(set(range(min(sink, own + 1))) | set(range(max(0, own - window + 1), own + 1)))
+                num = np.zeros(D); den = 0.0
+                for j in keys:
+                    e = np.exp(scale * float(np.dot(q[b, i, h], k[b, h // G, j])))
+                    num += e * v[b, h // G, j]; den += e
+                out[b, i, h] = num / den; lse[b, i, h] = np.log(den)
+    return out, lse
+
+
+@pytest.mark.parametrize("sink,window", [(0, 1), (0, 5), (4, 7), (3, 1), (10, 100), (2, 16)])
+def test_window_brute_force(sink, window):
+    B, Hq, Hkv, D, Lmax, gamma = 2, 4, 2, 8, 48, 3
+    R = gamma + 1
+    q = _rand((B, R, Hq, D), 31); k = _rand((B, Hkv, Lmax, D), 32); v = _rand((B, Hkv, Lmax, D), 33)
+    ctx = np.array([48, 9], dtype=np.int32)
+    out, lse = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx, gamma, sink=sink, window=window)
+    ref, ref_lse = _brute_window(q, k, v, ctx, gamma, 1.0 / np.sqrt(D), sink, window)
+    np.testing.assert_allclose(out, ref, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(lse, ref_lse, rtol=1e-11, atol=1e-12)
+
+
+def test_window_that_covers_everything_is_the_plain_mask():
+    B, Hq, Hkv, D, L, gamma = 1, 4, 2, 8, 37, 2
+    q = _rand((B, gamma + 1, Hq, D), 34); k = _rand((B, Hkv, L, D), 35); v = _rand((B, Hkv, L, D), 36)
+    ctx = np.array([L], dtype=np.int32)
+    full, full_lse = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx, gamma)
+    for sink, window in ((0, L), (0, 10 * L), (5, L), (L, 1)):     # the last: every key is a sink
+        out, lse = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx, gamma, sink=sink, window=window)
+        np.testing.assert_array_equal(out, full)
+        np.testing.assert_array_equal(lse, full_lse)
+
+
+def test_window_of_one_returns_the_rows_own_value_and_hidden_keys_are_never_read():
+    B, Hq, Hkv, D, L, gamma = 1, 2, 1, 8, 30, 3
+    R = gamma + 1
+    q = _rand((B, R, Hq, D), 37); k = _rand((B, Hkv, L, D), 38); v = _rand((B, Hkv, L, D), 39)
+    ctx = np.array([L], dtype=np.int32)
+    out, lse = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx, gamma, sink=0, window=1)
+    for i in range(R):
+        own = L - R + i
+        for h in range(Hq):
+            np.testing.assert_allclose(out[0, i, h], v[0, 0, own].double().numpy(), rtol=1e-15)
+            s = float(q[0, i, h].double() @ k[0, 0, own].double()) / np.sqrt(D)
+            assert abs(lse[0, i, h] - s) < 1e-12
+    # sinks 0..2 and a window of 4: keys 3 .. own-4 are hidden from row i and may hold anything
+    sink, window = 3, 4
+    base, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx, gamma, sink=sink, window=window)
+    k2 = k.clone(); v2 = v.clone()
+    k2[:, :, sink:L - R - window + 1] = float("nan"); v2[:, :, sink:L - R - window + 1] = float("inf")
+    again, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k2), bf16_bits(v2), ctx, gamma, sink=sink, window=window)
+    np.testing.assert_array_equal(base, again)
+    # the key just inside row 0's window is seen by row 0 only (row 1's window starts one key later)
+    k3 = k.clone(); v3 = v.clone()
+    edge = L - R - window + 1
+    k3[:, :, edge] += 1.0; v3[:, :, edge] += 1.0
+    moved, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k3), bf16_bits(v3), ctx, gamma, sink=sink, window=window)
+    assert np.abs(moved[:, 0] - base[:, 0]).max() > 1e-3
+    np.testing.assert_array_equal(moved[:, 1:], base[:, 1:])
+    # a sink key is seen by every row
+    k4 = k.clone(); k4[:, :, 1] += 1.0
+    moved, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k4), bf16_bits(v), ctx, gamma, sink=sink, window=window)
+    assert all(np.abs(moved[:, i] - base[:, i]).max() > 1e-4 for i in range(R))

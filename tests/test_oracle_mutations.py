@@ -35,6 +35,12 @@ MUTATIONS = {
     "sampling_uniform_reused": ("const double u = (double)uniforms[(int64_t)b * R + gamma];",
                                 "const double u = (double)uniforms[(int64_t)b * R + (n < gamma ? n : gamma)];"),
     "keeps_going_after_reject": ("rejected = 1;\n", "rejected = 0; n = 0;\n"),
+    "window_one_key_too_narrow": ("if (!(j < sink || j > own - window)) continue;\n            const double e",
+                                  "if (!(j < sink || j > own - window + 1)) continue;\n            const double e"),
+    "window_anchored_at_last_row": ("const int64_t own = L - R + i; /* the row's own key */",
+                                    "const int64_t own = L - 1; /* the row's own key */"),
+    "sinks_dropped_from_values": ("if (!(j < sink || j > own - window)) continue;\n            const double e",
+                                  "if (!(j > own - window)) continue;\n            const double e"),
 }
 
 
