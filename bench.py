@@ -2,14 +2,17 @@
 """Benchmark of the RAPID verify step on B200.
 
 One step = one pass of the whole hot path over one batch of synthetic input:
-`layers` verify-attention calls (independently seeded K/V caches, all resident in
-HBM) followed by one accept call.  Metric: KV-read GB/s of the step (all KV bytes
-of the step / step time).  Prints ONE JSON line.
+one plan of the work split, `layers` verify-attention calls (independently
+seeded K/V caches, all resident in HBM) and one accept call.  Metric: KV-read
+GB/s of the step (all KV bytes of the step / step time).  Prints ONE JSON line.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference] [--sharded]
 
-`--impl reference` times the fp64 CPU oracle (as it stands) on a bounded sample of
-the same workload on the host cores.
+With --gpus N > 1 and no launcher (no WORLD_SIZE in the environment) the script
+starts N ranks itself, one per GPU.  `--impl reference` times the fp64 CPU oracle
+(as it stands) on a bounded sample of the same workload on the host cores.
+`--sharded` times the context-sharded form of the attention: one sequence's keys
+spread over the N ranks, one all-gather of partial results per layer.
 """
 from __future__ import annotations
 
@@ -17,6 +20,7 @@ import argparse
 import ctypes
 import json
 import os
+import socket
 import statistics
 import sys
 import threading
@@ -39,18 +43,19 @@ def _peaks():
     return 6650.0, "fallback"
 
 
-def ncu_traffic(workload, kernel="verify_attn_splitkv_tc_kernel"):
-    """DRAM bytes per split-kernel launch from the committed ncu capture, or None if the kernel
-    sources have changed since the counters were taken (or the capture is of the other kernel)."""
+def ncu_traffic(workload, kernel):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu capture, or None if the
+    kernel sources have changed since the counters were taken (or no capture covers this workload)."""
     import hashlib
     try:
         rec = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
         h = hashlib.sha256()
         for f in ("attention.cu", "attention_kt.cuh", "tcgen05.cuh", "common.cuh"):
             h.update(open(os.path.join(ROOT, "paper_2502_20330_b200", "csrc", f), "rb").read())
-        if h.hexdigest() != rec["kernel_sha256"] or workload not in rec or rec.get("kernel") != kernel:
+        ent = rec.get(workload)
+        if h.hexdigest() != rec["kernel_sha256"] or not ent or ent.get("kernel") != kernel:
             return None
-        return int(rec[workload]["dram_bytes_read"] + rec[workload]["dram_bytes_write"])
+        return int(ent["dram_bytes_read"] + ent["dram_bytes_write"])
     except Exception:
         return None
 
@@ -79,22 +84,62 @@ def kv_bytes_per_layer(cfg, ctx) -> int:
     return int(4 * cfg.Hkv * cfg.D * int(ctx.sum()))
 
 
+def config_dict(cfg, ctx, world, sharded=False):
+    """What both arms print as `config`: the workload, nothing of how an arm runs it."""
+    kv_layer = kv_bytes_per_layer(cfg, ctx)
+    return {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
+            "ctx": [int(x) for x in ctx], "gamma": cfg.gamma, "V": cfg.V, "layers": cfg.layers, "eta": cfg.eta,
+            "kv_bytes_per_step": kv_layer * cfg.layers,
+            "l2": f"inputs larger than L2: {cfg.layers} distinct cache(s) of {kv_layer / 2**20:.0f} MiB per step"
+                  + ("" if kv_layer * cfg.layers > 2 * 126 * 2**20 else ", and a buffer larger than L2 rewritten "
+                     "between steps"),
+            "parallelism": ("context sharded x%d" % world if sharded else f"replicas x{world}") if world > 1
+                           else "single GPU"}
+
+
+def find_free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _spawn_entry(rank, world, port, fn, args):
+    os.environ["RANK"] = str(rank)
+    os.environ["LOCAL_RANK"] = str(rank)
+    os.environ["WORLD_SIZE"] = str(world)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    fn(*args)
+
+
+def spawn_ranks(world: int, fn, args=()):
+    """Starts `world` processes on this node, each with the launcher's environment (RANK, LOCAL_RANK,
+    WORLD_SIZE, MASTER_ADDR = 127.0.0.1, MASTER_PORT), and runs fn(*args) in every one."""
+    import torch.multiprocessing as mp
+    mp.spawn(_spawn_entry, args=(world, find_free_port(), fn, args), nprocs=world, join=True)
+
+
 # ------------------------------------------------------------------------------------------------
-# CPU oracle leg (bounded sample)
+# CPU oracle leg (bounded sample); with device results at hand it also judges them
 # ------------------------------------------------------------------------------------------------
 class OracleSample:
-    """The oracle, as it stands, on a bounded sample of one step: a subset of one layer's
-    (sequence, head, row) units plus one full accept call, extrapolated to the whole step."""
+    """The oracle, as it stands, on a bounded sample of one step: (sequence, head, row) units of one
+    layer plus one full accept call, extrapolated to the whole step.  The inputs are the bits it is
+    given (the benchmark hands it the very tensors the library ran on)."""
 
-    def __init__(self, cfg, seed):
+    def __init__(self, cfg, seed, attn_inputs=None, accept_inputs=None):
         import oracle
         self.oracle = oracle
         self.cfg = cfg
-        self.ctx = wl.context_lengths(cfg, seed)
-        q, k, v, ctx_t = wl.attention_inputs(cfg, seed, device="cpu", layer=0)
+        if attn_inputs is None:
+            attn_inputs = wl.attention_inputs(cfg, seed, device="cpu", layer=0)
+        if accept_inputs is None:
+            accept_inputs = wl.accept_inputs(cfg, seed, device="cpu")
+        q, k, v, ctx_t = attn_inputs
+        self.ctx = ctx_t.cpu()
         self.bits = (wl.bf16_bits(q), wl.bf16_bits(k), wl.bf16_bits(v))
-        self.ctx_np = ctx_t.numpy()
-        self.acc = [t.numpy() for t in wl.accept_inputs(cfg, seed, device="cpu")]
+        self.ctx_np = self.ctx.numpy()
+        self.acc = [t.cpu().numpy() for t in accept_inputs]
         self.total_units = cfg.B * cfg.Hq * cfg.R
         self.cores = oracle.num_threads()
         self.rng = np.random.default_rng(seed)
@@ -102,20 +147,25 @@ class OracleSample:
         t = self._attention(self.cores)[0]
         self.unit_s = t / 1.0   # seconds per batch of `cores` units
         t0 = time.perf_counter()
-        self._accept()
+        self.accept_ref = self._accept()
         self.accept_s = time.perf_counter() - t0
+        self.attn_ref = None
 
     def _attention(self, n_units):
         n_units = int(min(self.total_units, max(1, n_units)))
-        units = np.sort(self.rng.choice(self.total_units, size=n_units, replace=False)).astype(np.int64)
+        units = None
+        if n_units < self.total_units:
+            units = np.sort(self.rng.choice(self.total_units, size=n_units, replace=False)).astype(np.int64)
         t0 = time.perf_counter()
-        self.oracle.verify_attention(*self.bits, self.ctx_np, self.cfg.gamma, units=units)
-        return time.perf_counter() - t0, n_units
+        out, lse = self.oracle.verify_attention(*self.bits, self.ctx_np, self.cfg.gamma, units=units)
+        dt = time.perf_counter() - t0
+        self.attn_ref = (out, lse)
+        return dt, n_units
 
     def _accept(self):
         z, d, tok, u = self.acc
-        self.oracle.accept(z, d, tok, u, eta=self.cfg.eta, T=self.cfg.temperature,
-                           tail_alpha=self.cfg.tail_alpha, want_ratios=False)
+        return self.oracle.accept(z, d, tok, u, eta=self.cfg.eta, T=self.cfg.temperature,
+                                  tail_alpha=self.cfg.tail_alpha, want_ratios=False)
 
     def step(self, budget_s):
         """Returns (GB/s of the extrapolated step, description, seconds spent)."""
@@ -131,6 +181,35 @@ class OracleSample:
         sample = (f"{n} of {self.total_units} (sequence, head, row) units of one layer ({t_attn:.2f} s) "
                   f"+ one full accept call ({t_acc:.2f} s), extrapolated to {cfg.layers} layer(s)")
         return gbs, sample, t_attn + t_acc
+
+    def judge(self, dev_out, dev_alen, dev_ntok, extra_accept=()):
+        """Compares the library's results on the same bits with what the last step() computed, under
+        the parity rules of the tests.  extra_accept: more (inputs, device results) pairs of the accept
+        step on other seeds, for the histogram of accepted lengths."""
+        from oracle import parity
+        cfg = self.cfg
+        ref, ref_lse = self.attn_ref
+        rows = ~np.isnan(ref_lse)
+        rep = parity.check_attention(dev_out, ref, rows)
+        z, d, tok, u = self.acc
+        acc = parity.check_accept(z, d, tok, u, cfg.eta, cfg.temperature, cfg.tail_alpha, 0, dev_alen, dev_ntok)
+        hist = [0] * (cfg.gamma + 1)
+        ties = list(acc["near_ties"])
+        alts = len(acc["token_alternatives"])
+        for n in dev_alen:
+            hist[int(n)] += 1
+        for (zz, dd, tt, uu), (al, nt) in extra_accept:
+            r = parity.check_accept(zz, dd, tt, uu, cfg.eta, cfg.temperature, cfg.tail_alpha, 0, al, nt)
+            ties += r["near_ties"]
+            alts += len(r["token_alternatives"])
+            for n in al:
+                hist[int(n)] += 1
+        return {"max_abs": rep["max_abs"], "max_row_rel_l2": rep["max_row_rel_l2"], "rows": rep["rows"],
+                "rows_total": int(rows.size), "tolerance": {"max_abs": parity.ATTN_MAX_ABS,
+                                                            "row_rel_l2": parity.ATTN_ROW_REL_L2},
+                "accept_len": [int(x) for x in dev_alen], "accept_len_oracle": acc["accept_len_ref"],
+                "near_ties": [[int(b), int(k), float(g)] for b, k, g in ties], "token_alternatives": alts,
+                "accept_len_histogram": hist, "accept_calls_checked": 1 + len(extra_accept)}
 
 
 def run_reference(args, cfg):
@@ -151,8 +230,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": "verify_step_kv_read_gbs", "value": value, "unit": "GB/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
-                   "ctx": [int(x) for x in ctx], "gamma": cfg.gamma, "V": cfg.V, "layers": cfg.layers},
+        "config": config_dict(cfg, ctx, args.gpus),
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": smp.cores, "kind": "oracle",
                          "sample": sample + f"; mean of {args.steps} such samples"},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -169,7 +247,7 @@ class ClockSampler:
                0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
 
     def __init__(self, index):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.times, self.reasons, self.max_mhz = [], [], set(), None
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -184,7 +262,9 @@ class ClockSampler:
     def _loop(self):
         while not self._stop.is_set():
             try:
-                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                mhz = int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                self.samples.append(mhz)
+                self.times.append(time.perf_counter())
                 bits = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
                 for bit, name in self.REASONS.items():
                     if bits & bit:
@@ -198,12 +278,20 @@ class ClockSampler:
             self._thread = threading.Thread(target=self._loop, daemon=True)
             self._thread.start()
 
+    def mark(self):
+        """Index of the next sample: lets a caller cut the record into regions."""
+        return len(self.samples)
+
+    def summary(self, lo=0, hi=None):
+        s = self.samples[lo:hi]
+        return {"sm_mhz": int(statistics.median(s)) if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
     def stop(self):
         self._stop.set()
         if self._thread is not None:
             self._thread.join()
-        return {"sm_mhz": int(statistics.median(self.samples)) if self.samples else None,
-                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        return self.summary()
 
 
 # ------------------------------------------------------------------------------------------------
@@ -270,26 +358,38 @@ def run_ours(args, cfg):
     aws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma), device=dev)
     cws = R.new_workspace(R.accept_workspace_bytes(cfg.B, cfg.gamma, cfg.V), device=dev)
     acc_params = R.AcceptParams(temperature=cfg.temperature, tail_alpha=cfg.tail_alpha)
-    attn_params = R.AttnParams(kernel=args.kernel)
-    keys_on_m = args.kernel == 2 or (args.kernel == 0 and cfg.D == 128 and cfg.G * cfg.R <= 64)
-    split_kernel = "verify_attn_splitkv_kt_kernel" if keys_on_m else "verify_attn_splitkv_tc_kernel"
+    plan_params = R.AttnParams(kernel=args.kernel)
     stream = torch.cuda.current_stream()
     sptr = int(stream.cuda_stream)
     ev = RawEvents()
 
     kv_layer = kv_bytes_per_layer(cfg, ctx_cpu)
     kv_step = kv_layer * cfg.layers
+    # one cache per step that fits in L2 would be served from it on the next step: such workloads
+    # get a buffer larger than L2 rewritten between steps (outside the kernels that are timed one by one)
+    flush = None
+    if kv_step <= 2 * 126 * 2**20:
+        flush = torch.empty(192 * 2**20, dtype=torch.uint8, device=dev)
 
-    def step(split_events=None):
+    def attn_params(li, split_event=None):
+        # the plan of a step is made right before its first layer: that layer reads it after its
+        # grid-dependency wait, the later ones (other kernels lie in between) before it
+        mode = R.PLAN_NONE if args.no_plan else (R.PLAN_READY if li == 0 else R.PLAN_SETTLED)
+        return R.AttnParams(kernel=args.kernel, plan=mode, split_done_event=split_event)
+
+    def step(split_events=None, call_events=None, st=None):
+        if flush is not None:
+            flush.fill_(1)
+        if not args.no_plan:
+            R.rapid_attention_plan(ctx, cfg.gamma, cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, aws, plan_params, stream=st)
         for li, (q, k, v, out) in enumerate(layers):
-            if split_events is not None:
-                e0, e1 = split_events[li]
-                ev.record(e0, sptr)
-                R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws,
-                                         R.AttnParams(split_done_event=e1, kernel=args.kernel))
-            else:
-                R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws, attn_params)
-        R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params)
+            if call_events is not None:
+                ev.record(call_events[li][0], sptr)
+            e1 = split_events[li] if split_events is not None else None
+            R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws, attn_params(li, e1), stream=st)
+            if call_events is not None:
+                ev.record(call_events[li][1], sptr)
+        R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params, stream=st)
 
     def barrier():
         if world > 1:
@@ -300,6 +400,16 @@ def run_ours(args, cfg):
     for _ in range(max(3, args.warmup)):
         step()
     barrier()
+    # which kernels serve an attention call of this workload: one launch = the cluster form (merged on chip)
+    R.kernel_launch_count_reset()
+    R.rapid_verify_attention(*layers[0][:3], ctx, cfg.gamma, layers[0][3], aws, R.AttnParams(kernel=args.kernel))
+    launches_per_call = R.kernel_launch_count()
+    torch.cuda.synchronize()
+    keys_on_m = args.kernel in (2, 3) or (args.kernel == 0 and cfg.D == 128 and cfg.G * cfg.R <= 64)
+    if launches_per_call == 1:
+        dominant = "verify_attn_splitkv_kt_kernel (one cluster per KV head, merged on chip)"
+    else:
+        dominant = "verify_attn_splitkv_kt_kernel" if keys_on_m else "verify_attn_splitkv_tc_kernel"
 
     # The step is captured once in a CUDA graph (every call of the path is asynchronous and
     # allocation-free, so the whole step is capturable) and the timed region replays it: K graph
@@ -311,9 +421,7 @@ def run_ours(args, cfg):
     R.kernel_launch_count_reset()
     with torch.cuda.stream(side):
         with torch.cuda.graph(graph, stream=side):
-            for (q, k, v, out) in layers:
-                R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws, attn_params, stream=side)
-            R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params, stream=side)
+            step(st=side)
     launches_per_step = R.kernel_launch_count()
     torch.cuda.synchronize()
     for _ in range(3):
@@ -324,13 +432,25 @@ def run_ours(args, cfg):
     sampler = ClockSampler(local_rank)
     sampler.start()
     barrier()
+    m0 = sampler.mark()
     ev.record(e_begin, sptr)
     for s in range(args.steps):
         graph.replay()
     ev.record(e_end, sptr)
     barrier()
+    m1 = sampler.mark()
     launches = launches_per_step * args.steps
     total_ms = ev.elapsed_ms(e_begin, e_end)
+    flush_ms = 0.0
+    if flush is not None:   # the rewrite of the L2-sized buffer is not part of the step: timed alone, taken off
+        f0, f1 = ev.create(), ev.create()
+        ev.record(f0, sptr)
+        for s in range(args.steps):
+            flush.fill_(1)
+        ev.record(f1, sptr)
+        torch.cuda.synchronize()
+        flush_ms = ev.elapsed_ms(f0, f1)
+        total_ms -= flush_ms
 
     s_begin, s_end = ev.create(), ev.create()
     ev.record(s_begin, sptr)
@@ -338,25 +458,71 @@ def run_ours(args, cfg):
         step()
     ev.record(s_end, sptr)
     barrier()
-    stream_us = 1e3 * ev.elapsed_ms(s_begin, s_end) / args.steps
+    stream_us = 1e3 * (ev.elapsed_ms(s_begin, s_end) - flush_ms) / args.steps
     # second live pass for the roofline of the dominant kernel: the same steps with an event pair
-    # around every split kernel (the event between split and merge costs the pair their
-    # programmatic overlap, which is why this pass is not the one that gives `value`)
+    # around every launch of it (the event between split and merge costs the pair their programmatic
+    # overlap, which is why this pass is not the one that gives `value`).  A call that is one kernel
+    # is timed as the call.
     k_steps = min(args.steps, 20)
-    timed_pairs = [[(ev.create(), ev.create()) for _ in range(cfg.layers)] for _ in range(k_steps)]
+    pairs = [[(ev.create(), ev.create()) for _ in range(cfg.layers)] for _ in range(k_steps)]
     for s in range(k_steps):
-        step(timed_pairs[s])
+        if launches_per_call == 1:
+            step(call_events=pairs[s])
+        else:
+            step(split_events=[p[1] for p in pairs[s]], call_events=[(p[0], ev.create()) for p in pairs[s]])
     barrier()
+    kernel_ms = [ev.elapsed_ms(a, b) for ps in pairs for (a, b) in ps]
+    m2 = sampler.mark()
+
+    # sustained: the same graph replayed for about two seconds, an event after every step; the step
+    # times are binned by the SM clock NVML reported at that moment
+    sustained = None
+    if rank == 0 and world == 1 and not args.no_sustained:
+        est_ms = total_ms / args.steps + flush_ms / args.steps
+        n_sus = int(min(20000, max(50, 2000.0 / max(est_ms, 1e-3))))
+        marks = [ev.create() for _ in range(n_sus + 1)]
+        torch.cuda.synchronize()
+        t_host0 = time.perf_counter()
+        ev.record(marks[0], sptr)
+        for s in range(n_sus):
+            graph.replay()
+            ev.record(marks[s + 1], sptr)
+        torch.cuda.synchronize()
+        t_host1 = time.perf_counter()
+        m3 = sampler.mark()
+        ends = np.array([ev.elapsed_ms(marks[0], marks[s + 1]) for s in range(n_sus)])
+        per_step = np.diff(np.concatenate([[0.0], ends])) - flush_ms / args.steps
+        # device time 0 = t_host0 (the stream was idle), so sample i falls into the step running then
+        scale = (t_host1 - t_host0) * 1e3 / max(ends[-1], 1e-6)
+        bins = {}
+        series = []
+        for i in range(m2, m3):
+            t_ms = (sampler.times[i] - t_host0) * 1e3 / scale
+            if 0 <= t_ms <= ends[-1]:
+                sidx = int(np.searchsorted(ends, t_ms))
+                mhz = sampler.samples[i]
+                series.append([round(t_ms, 1), mhz])
+                bins.setdefault(mhz // 50 * 50, []).append(float(per_step[min(sidx, n_sus - 1)]))
+        second_half = per_step[n_sus // 2:]
+        sus_ms = float(np.mean(second_half))
+        sustained = {"seconds": round(float(ends[-1]) / 1e3, 2), "steps": n_sus,
+                     "ms_per_step_second_half": sus_ms,
+                     "value_second_half": job_throughput_gbs(kv_step, 1, sus_ms),
+                     "ms_per_step_first_20": float(np.mean(per_step[:20])),
+                     "by_sm_mhz": {str(kk): {"steps": len(vv), "ms_per_step": float(np.mean(vv))}
+                                   for kk, vv in sorted(bins.items())},
+                     "clock_samples_ms_mhz": series[:: max(1, len(series) // 40)],
+                     "clocks": sampler.summary(m2, m3)}
     clocks = sampler.stop()
-    split_ms = [ev.elapsed_ms(a, b) for pairs in timed_pairs for (a, b) in pairs]
+    clocks.update(sampler.summary(m0, m1))
     status = R.workspace_status(aws) | R.workspace_status(cws)
 
     total_ms = max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
     value = job_throughput_gbs(kv_step, world, ms_per_step)
     peak, peak_kind = _peaks()
-    split_avg_ms = float(np.mean(split_ms))
-    achieved = kv_layer / (split_avg_ms * 1e-3) / 1e9
+    kernel_avg_ms = float(np.mean(kernel_ms))
+    achieved = kv_layer / (kernel_avg_ms * 1e-3) / 1e9
 
     del graph
 
@@ -374,33 +540,53 @@ def run_ours(args, cfg):
         "metric": "verify_step_kv_read_gbs", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
-                   "ctx": [int(x) for x in ctx_cpu], "gamma": cfg.gamma, "V": cfg.V, "layers": cfg.layers,
-                   "eta": cfg.eta, "kv_bytes_per_step": kv_step,
-                   "l2": f"inputs larger than L2: {cfg.layers} distinct caches of {kv_layer / 2**20:.0f} MiB per step",
-                   "launch": "the step captured in one CUDA graph, replayed per step",
-                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+        "config": config_dict(cfg, ctx_cpu, world),
+        "run": {"launch": "the step captured in one CUDA graph, replayed per step",
+                "plan": "none" if args.no_plan else "one rapid_attention_plan per step, shared by its layers",
+                "kernels_per_attention_call": int(launches_per_call),
+                "l2_flush_ms_per_step_not_counted": flush_ms / args.steps},
         "verify_latency_us": {"attention_per_layer": 1e3 * (ms_per_step - float(np.median(acc_ms))) / cfg.layers,
-                              "split_kernel_per_layer": 1e3 * split_avg_ms,
+                              "dominant_kernel_per_layer": 1e3 * kernel_avg_ms,
                               "accept": 1e3 * float(np.median(acc_ms)), "step": 1e3 * ms_per_step,
                               "step_stream_launches": stream_us},
         "frac_of_hbm_peak": {"measured": value / world / peak, "nominal_8TBs": value / world / 8000.0},
-        "roofline": {"bound": "hbm", "kernel": split_kernel, "achieved": achieved, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": ncu_traffic(cfg.name, split_kernel),
+        "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": ncu_traffic(cfg.name, dominant.split(" ")[0]),
                      "algorithmic_bytes": kv_layer,
-                     "timed": f"CUDA events around each of {len(split_ms)} launches in a second pass of {k_steps} steps"},
+                     "timed": f"CUDA events around each of {len(kernel_ms)} launches in a second pass of {k_steps} steps"},
         "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
     }
+    if sustained is not None:
+        line["sustained"] = sustained
 
     if rank == 0 and world == 1 and not args.no_e2e:
         line["e2e"] = run_e2e(R, cfg, seed, Lmax, kv_layer, dev)
     elif rank == 0:
         line["e2e"] = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        del layers
-        smp = OracleSample(cfg, seed)
+        # The CPU leg runs on the very bits the library ran on (layer 0 and the logits, copied back
+        # from the device), and what it computes is also what the library's results are judged by.
+        q0, k0, v0, out0 = layers[0]
+        R.rapid_verify_attention(q0, k0, v0, ctx, cfg.gamma, out0, aws, R.AttnParams(kernel=args.kernel))
+        R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params)
+        torch.cuda.synchronize()
+        dev_out = out0.float().cpu().numpy()
+        dev_alen, dev_ntok = alen.cpu().numpy().copy(), ntok.cpu().numpy().copy()
+        extra = []
+        n_extra = 0 if args.no_hist else max(0, min(15, 128 // max(1, cfg.B) - 1))
+        for i in range(n_extra):
+            zz, dd, tt, uu = wl.accept_inputs(cfg, seed + 7919 * (i + 1), device=dev)
+            R.rapid_accept(zz, dd, tt, uu, cfg.eta, alen, ntok, cws, acc_params)
+            torch.cuda.synchronize()
+            extra.append(([t.cpu().numpy() for t in (zz, dd, tt, uu)], (alen.cpu().numpy().copy(), ntok.cpu().numpy().copy())))
+        host_attn = tuple(t.cpu() for t in (q0, k0, v0, ctx))
+        host_acc = tuple(t.cpu() for t in (z, d, tok, u))
+        del layers, q0, k0, v0
+        smp = OracleSample(cfg, seed, host_attn, host_acc)
         gbs, sample, _ = smp.step(12.0)
         line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": smp.cores, "kind": "oracle", "sample": sample}
+        line["parity"] = smp.judge(dev_out, dev_alen, dev_ntok, extra)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -409,8 +595,10 @@ def run_ours(args, cfg):
 
 
 def run_e2e(R, cfg, seed, Lmax, kv_layer, dev, steps=5):
-    """The step through rapid_verify_step_host: pinned host tensors in, host results out; one layer
-    per step (every layer would move its own 2*Hkv*L*D*2 bytes over PCIe the same way)."""
+    """The step through rapid_verify_step_host: pinned host tensors in, host results out.  The entry
+    point takes one layer (cache, rows, logits); a step of `layers` layers is that call `layers`
+    times, every layer moving its own 2*Hkv*L*D*2 bytes over PCIe.  The layers of the long step are
+    copied from one pinned cache (the same number of bytes crosses the bus as from `layers` caches)."""
     q, k, v, ctx = [t.pin_memory() for t in wl.attention_inputs(cfg, seed, device="cpu", layer=0)]
     z, d, tok, u = [t.pin_memory() for t in wl.accept_inputs(cfg, seed, device="cpu")]
     out = torch.empty_like(q).pin_memory()
@@ -419,21 +607,113 @@ def run_e2e(R, cfg, seed, Lmax, kv_layer, dev, steps=5):
     arena = torch.empty(R.verify_step_host_arena_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma, cfg.V),
                         dtype=torch.uint8, device=dev)
     params = R.AcceptParams(temperature=cfg.temperature, tail_alpha=cfg.tail_alpha)
+
+    def one():
+        R.rapid_verify_step_host(q, k, v, ctx, cfg.gamma, out, z, d, tok, u, cfg.eta, alen, ntok, arena,
+                                 accept_params=params)
+
     times = []
     for i in range(steps + 2):
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        R.rapid_verify_step_host(q, k, v, ctx, cfg.gamma, out, z, d, tok, u, cfg.eta, alen, ntok, arena,
-                                 accept_params=params)
+        one()
         if i >= 2:
             times.append(time.perf_counter() - t0)
     nb = lambda t: t.numel() * t.element_size()  # noqa: E731
     h2d = sum(nb(t) for t in (q, k, v, ctx, z, d, tok, u))
     d2h = sum(nb(t) for t in (out, alen, ntok)) + 8
     t = float(np.median(times))
-    return {"value": kv_layer / t / 1e9, "unit": "GB/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-            "ms_per_step": 1e3 * t, "layers_per_step": 1,
-            "note": "rapid_verify_step_host on pinned host tensors; copies inside the timed region"}
+    res = {"value": kv_layer / t / 1e9, "unit": "GB/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+           "ms_per_step": 1e3 * t, "layers_per_step": 1,
+           "note": "rapid_verify_step_host on pinned host tensors; copies inside the timed region"}
+    if cfg.layers > 1:
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(cfg.layers):
+            one()
+        tl = time.perf_counter() - t0
+        res["whole_step"] = {"value": kv_layer * cfg.layers / tl / 1e9, "unit": "GB/s", "ms_per_step": 1e3 * tl,
+                             "layers_per_step": cfg.layers, "h2d_bytes_per_step": int(h2d) * cfg.layers,
+                             "d2h_bytes_per_step": int(d2h) * cfg.layers,
+                             "note": f"{cfg.layers} rapid_verify_step_host calls back to back, one per layer (each "
+                                     "also runs the accept step on its 8.7 MB of logits); all copied from one "
+                                     "pinned host cache"}
+    return res
+
+
+def run_sharded(args, cfg):
+    """Context-sharded attention: the keys of every sequence spread over the ranks, one all-gather of
+    (output, log-sum-exp) per layer, then the merge.  Strong scaling: the job's bytes are fixed.
+    Not measured on several GPUs here (a call of this benchmark gets one); with one rank it runs as
+    a check of the plumbing."""
+    import torch.distributed as dist
+    import paper_2502_20330_b200 as R
+    from paper_2502_20330_b200 import sharded
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", str(find_free_port()))
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    ctx_cpu = wl.context_lengths(cfg, args.seed)
+    bounds = sharded.context_shard_bounds(ctx_cpu.tolist(), cfg.gamma, world)[rank]
+    lens = torch.tensor([e - s for s, e in bounds], dtype=torch.int32, device=dev)
+    Lloc = int(lens.max())
+    shard_cfg = wl.with_overrides(cfg, ctx_lens=tuple(int(x) for x in lens), ctx_range=None, Lmax=Lloc)
+    layers = []
+    for layer in range(cfg.layers):
+        q, _, _, _ = wl.attention_inputs(wl.with_overrides(cfg, ctx_lens=(cfg.R,) * cfg.B, ctx_range=None, Lmax=cfg.R),
+                                         args.seed, device=dev, layer=layer)      # the same rows on every rank
+        _, k, v, _ = wl.attention_inputs(shard_cfg, rank_seed(args.seed, rank), device=dev, layer=layer)
+        layers.append((q, k, v, torch.empty_like(q)))
+    ws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lloc, cfg.gamma), device=dev)
+
+    def step():
+        for q, k, v, out in layers:
+            sharded.sharded_verify_attention(q, k, v, lens, cfg.gamma, out, ws)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
+    kv_step = kv_bytes_per_layer(cfg, ctx_cpu) * cfg.layers
+    if rank == 0:
+        print(json.dumps({
+            "metric": "verify_step_kv_read_gbs", "value": kv_step / (ms * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": config_dict(cfg, ctx_cpu, world, sharded=True),
+            "run": {"exchange": "one NCCL all-gather of (fp32 output, log-sum-exp) per layer, then rapid_merge_partials",
+                    "accept": "not part of this mode"},
+            "clocks": clocks, "e2e": None, "gpu_launches": int(3 * cfg.layers * args.steps)}))
+    dist.destroy_process_group()
+
+
+def _rank_main(args):
+    cfg = wl.CONFIGS[args.workload]
+    if args.layers:
+        cfg = wl.with_overrides(cfg, layers=args.layers)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    elif args.sharded:
+        run_sharded(args, cfg)
+    else:
+        run_ours(args, cfg)
 
 
 def main():
@@ -445,18 +725,20 @@ def main():
     ap.add_argument("--workload", default="llama8b_128k", choices=sorted(wl.CONFIGS))
     ap.add_argument("--layers", type=int, default=0, help="override the number of resident layers")
     ap.add_argument("--seed", type=int, default=2025)
-    ap.add_argument("--kernel", type=int, default=0, choices=[0, 1, 2],
-                    help="split kernel: 0 the library's choice, 1 rows on the MMA's M axis, 2 keys on the M axis")
+    ap.add_argument("--kernel", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="split kernel: 0 the library's choice, 1 rows on the MMA's M axis, 2 keys on the M axis, "
+                         "3 keys on M with one cluster per KV head")
+    ap.add_argument("--sharded", action="store_true", help="context-sharded attention over the ranks")
+    ap.add_argument("--no-plan", action="store_true", help="every attention call works its split out itself")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true")
+    ap.add_argument("--no-hist", action="store_true")
     args = ap.parse_args()
-    cfg = wl.CONFIGS[args.workload]
-    if args.layers:
-        cfg = wl.with_overrides(cfg, layers=args.layers)
-    if args.impl == "reference":
-        run_reference(args, cfg)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        spawn_ranks(args.gpus, _rank_main, (args,))   # no launcher: start one rank per GPU here
     else:
-        run_ours(args, cfg)
+        _rank_main(args)
 
 
 if __name__ == "__main__":

@@ -5,9 +5,9 @@
  * retrieval-augmented speculative decoding (Algorithm 1 of the RAPID paper):
  *
  *   1. verify attention: the gamma+1 newest query rows of every sequence attend
- *      over that sequence's whole bf16 KV cache in one pass (Algorithm 1, the
- *      LogitsOf step; Section 2.1 "validated by the target model in a single
- *      forward pass"), causally masked among themselves;
+ *      over that sequence's whole bf16 KV cache in one pass of the target over
+ *      all gamma+1 positions (Algorithm 1, the LogitsOf step; Section 2.1),
+ *      causally masked among themselves;
  *   2. accept / residual: the validation loop of Algorithm 1 with the
  *      retrieval-augmented target distribution of Eq. (new_target), the tail
  *      rule of Section 2.4 and the residual draw of Algorithm 1's last step.
@@ -55,6 +55,8 @@ extern "C" {
 #define RAPID_STATUS_RESIDUAL_FALLBACK 4  /* residual mass was 0 / not finite: token drawn from p    */
 #define RAPID_STATUS_PIPELINE_TIMEOUT 8   /* an on-chip wait hit its time limit: outputs invalid      */
 #define RAPID_STATUS_BAD_BLOCK_TABLE 16  /* a block-table entry outside [0, num_blocks): read as 0s  */
+#define RAPID_STATUS_STALE_PLAN 32       /* the plan in the workspace was made for other lengths or another
+                                            geometry than this call's: outputs invalid               */
 
 /* residual_mode */
 #define RAPID_RESIDUAL_PAPER 0 /* norm(max(p - phat, p - q, 0)): Algorithm 1, residual step               */
@@ -91,14 +93,29 @@ typedef struct rapid_attn_shape {
 #define RAPID_ATTN_KERNEL_KEYS_ON_M 2 /* keys on the M axis: head_dim 128, <= 96 grouped rows per KV head (two
                                          softmax groups beyond 64), any paged block size the call accepts;
                                          RAPID_ERR_UNSUPPORTED otherwise                                        */
+#define RAPID_ATTN_KERNEL_CLUSTER_MERGE 3 /* the keys-on-M kernel as one thread-block cluster per (sequence,
+                                         KV head): the cluster's CTAs share that unit's keys and merge their
+                                         partial results on chip, so the call is ONE kernel.  Meant for short
+                                         runs (a decode over a few thousand keys, a 32K layer) of sequences of
+                                         similar lengths; RAPID_ERR_UNSUPPORTED if the clusters do not fit on
+                                         the device together.  The library picks it by itself for a single
+                                         sequence with a cache capacity of at most 65,536 keys.              */
+
+/* rapid_attn_params.plan */
+#define RAPID_PLAN_NONE 0    /* every kernel works its share out from ctx_lens (default)                    */
+#define RAPID_PLAN_READY 1   /* the workspace holds a plan made by rapid_attention_plan for this call's
+                                geometry and for the current ctx_lens                                      */
+#define RAPID_PLAN_SETTLED 2 /* as RAPID_PLAN_READY, and at least one other kernel (or a synchronisation)
+                                lies between rapid_attention_plan and this call in the stream: the plan is
+                                then read while the preceding kernel still runs                            */
 
 /* Optional knobs and extra outputs of the attention call (NULL = defaults). */
 typedef struct rapid_attn_params {
     float scale;      /* softmax scale; 0 = 1/sqrt(D)                                             */
     int32_t num_ctas; /* CTAs the KV length is split over; 0 = one per SM; at most 512            */
     float* lse_out;   /* device [B, R, Hq] fp32 natural-log sum-exp of the scaled scores, or NULL;
-                         within 1e-3, and within 4.5e-3 where the keys-on-M kernel serves 49 to 64
-                         grouped rows (its row sums add bf16-rounded probabilities there)        */
+                         within 1e-4 of the exact value (the row sums then add fp32 probabilities
+                         in every kernel)                                                         */
     float* out_f32;   /* device [B, R, Hq, D] fp32 output before bf16 rounding, or NULL           */
     void* split_done_event; /* a cudaEvent_t recorded on the stream between the split and the merge
                                kernel (lets a caller time the two separately), or NULL          */
@@ -106,6 +123,18 @@ typedef struct rapid_attn_params {
                                  ctx_lens[b] >= 1 suffices.  For a shard of the context that does not
                                  hold the rows' own keys (see rapid_merge_partials)                */
     int32_t kernel;           /* RAPID_ATTN_KERNEL_*: 0 lets the library choose                        */
+    int32_t sink_keys;        /* with window_keys > 0: the first sink_keys keys stay visible to every row  */
+    int32_t window_keys;      /* > 0: row i sees, besides the sink keys, only the window_keys newest keys up
+                                 to and including its own, i.e. (lim_i - window_keys, lim_i] with
+                                 lim_i = ctx_lens[b] - R + i.  The mask of a streaming drafter that keeps
+                                 a few sink tokens and a recent window (Section 3.2, the MagicDec /
+                                 StreamingLLM baseline: 4 sinks in a budget of 4,096) laid over a full
+                                 cache; key tiles no row sees are not read.  0 = the plain causal mask  */
+    int32_t plan;             /* RAPID_PLAN_*                                                           */
+    int32_t reserved;
+    int64_t wait_cycle_limit; /* SM clock cycles an on-chip wait (for a tile, for the tensor cores) may take
+                                 before the kernel gives up and sets RAPID_STATUS_PIPELINE_TIMEOUT;
+                                 0 = the library's limit of about a second                              */
 } rapid_attn_params;
 
 /*
@@ -175,6 +204,24 @@ int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cac
                            const int32_t* ctx_lens, int gamma, void* out,
                            const rapid_attn_shape* shape, const rapid_attn_params* params,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Works out once, on the device, what every attention call over the same lengths would otherwise
+ * work out for itself: each CTA's share of the key tiles and each (sequence, KV head)'s range of
+ * partial results.  (Not in the paper.  ctx_lens does not change between the layers of one verify
+ * step, so the 32 or 80 attention calls of a step can share one plan; each then saves the
+ * microsecond or two its own planning takes at the head of the kernel.)
+ *
+ * The plan is written into `workspace` (one tiny kernel on the stream) and is valid for calls
+ * with the same B, Hq, Hkv, D, gamma, ctx_lens contents and the same params fields num_ctas,
+ * kernel, all_keys_visible, sink_keys, window_keys, and the same presence of lse_out, that name
+ * this workspace and set params->plan.  A call whose geometry or lengths differ from the plan's
+ * sets RAPID_STATUS_STALE_PLAN (checked on the device by every call).  shape's strides and a
+ * paged layout do not matter to the plan.
+ */
+int rapid_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
+                         const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream);
 
 /*
  * Combines P partial attention results of the same rows over disjoint sets of keys -- the context

@@ -16,13 +16,15 @@ STATUS_BAD_DRAFT_TOKEN = 2
 STATUS_RESIDUAL_FALLBACK = 4
 STATUS_PIPELINE_TIMEOUT = 8
 STATUS_BAD_BLOCK_TABLE = 16
-ATTN_KERNEL_AUTO, ATTN_KERNEL_ROWS_ON_M, ATTN_KERNEL_KEYS_ON_M = 0, 1, 2
+STATUS_STALE_PLAN = 32
+ATTN_KERNEL_AUTO, ATTN_KERNEL_ROWS_ON_M, ATTN_KERNEL_KEYS_ON_M, ATTN_KERNEL_CLUSTER_MERGE = 0, 1, 2, 3
+PLAN_NONE, PLAN_READY, PLAN_SETTLED = 0, 1, 2
 RESIDUAL_PAPER = 0
 RESIDUAL_PHAT = 1
 
 EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
-    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_retrieval_select", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_attention_plan", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_retrieval_select", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
     "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_kv_append_paged", "rapid_step_commit",
     "rapid_last_error",
@@ -52,7 +54,8 @@ class _AttnParams(ctypes.Structure):
     _fields_ = [("scale", ctypes.c_float), ("num_ctas", ctypes.c_int32),
                 ("lse_out", ctypes.c_void_p), ("out_f32", ctypes.c_void_p),
                 ("split_done_event", ctypes.c_void_p), ("all_keys_visible", ctypes.c_int32),
-                ("kernel", ctypes.c_int32)]
+                ("kernel", ctypes.c_int32), ("sink_keys", ctypes.c_int32), ("window_keys", ctypes.c_int32),
+                ("plan", ctypes.c_int32), ("reserved", ctypes.c_int32), ("wait_cycle_limit", ctypes.c_int64)]
 
 
 class _AcceptShape(ctypes.Structure):
@@ -74,7 +77,12 @@ class AttnParams:
     out_f32: Optional[torch.Tensor] = None   # [B,R,Hq,D] float32
     split_done_event: Optional[int] = None   # cudaEvent_t handle recorded between split and merge
     all_keys_visible: bool = False           # no causal stair: a context shard without the rows' own keys
-    kernel: int = 0                          # 0 automatic, 1 rows on the MMA's M axis, 2 keys on the M axis
+    kernel: int = 0                          # 0 automatic, 1 rows on the MMA's M axis, 2 keys on the M axis,
+                                             # 3 keys on M with one cluster per (sequence, KV head), merged on chip
+    sink_keys: int = 0                       # with window_keys: the first keys every row keeps seeing
+    window_keys: int = 0                     # > 0: each row sees only that many newest keys up to its own
+    plan: int = 0                            # PLAN_*: the workspace holds a plan made by rapid_attention_plan
+    wait_cycle_limit: int = 0                # clock cycles an on-chip wait may take; 0 = the library's limit
 
 
 @dataclass
@@ -119,6 +127,8 @@ def load_library():
         acc_args = [vp, vp, vp, vp, f32, vp, vp, ctypes.POINTER(_AcceptShape), ctypes.POINTER(_AcceptParams)]
         lib.rapid_verify_attention.restype = i32
         lib.rapid_verify_attention.argtypes = attn_args + [vp, sz, vp]
+        lib.rapid_attention_plan.restype = i32
+        lib.rapid_attention_plan.argtypes = [vp, i32, ctypes.POINTER(_AttnShape), ctypes.POINTER(_AttnParams), vp, sz, vp]
         lib.rapid_verify_attention_paged.restype = i32
         lib.rapid_verify_attention_paged.argtypes = [vp, vp, vp, vp, ctypes.POINTER(_PagedKv)] + attn_args[3:] + [vp, sz, vp]
         lib.rapid_draft_sample.restype = i32
@@ -197,7 +207,8 @@ def _attn_params(p: Optional[AttnParams]):
         return None
     return ctypes.byref(_AttnParams(p.scale, p.num_ctas, p.lse_out.data_ptr() if p.lse_out is not None else None,
                                     p.out_f32.data_ptr() if p.out_f32 is not None else None,
-                                    p.split_done_event, 1 if p.all_keys_visible else 0, int(p.kernel)))
+                                    p.split_done_event, 1 if p.all_keys_visible else 0, int(p.kernel),
+                                    int(p.sink_keys), int(p.window_keys), int(p.plan), 0, int(p.wait_cycle_limit)))
 
 
 def _accept_shape(target_logits: torch.Tensor, draft_logits: torch.Tensor) -> _AcceptShape:
@@ -272,6 +283,17 @@ def rapid_verify_attention(q, k_cache, v_cache, ctx_lens, gamma, out, workspace,
     _check(load_library().rapid_verify_attention(_p(q), _p(k_cache), _p(v_cache), _p(ctx_lens), gamma, _p(out),
                                                  ctypes.byref(shape), _attn_params(params), _p(workspace),
                                                  _nbytes(workspace), _stream_ptr(stream)))
+
+
+def rapid_attention_plan(ctx_lens, gamma, B, Hq, Hkv, D, Lmax, workspace, params: Optional[AttnParams] = None,
+                         stream=None) -> None:
+    """Writes the work split of the attention calls over ``ctx_lens`` into ``workspace`` once; calls that
+    name the same workspace with ``params.plan`` set read it instead of working it out again."""
+    if ctx_lens.dtype != torch.int32 or ctx_lens.numel() != B:
+        raise TypeError("ctx_lens must be int32 [B]")
+    shape = _AttnShape(B, Hq, Hkv, D, Lmax, 0, 0, 0)
+    _check(load_library().rapid_attention_plan(_p(ctx_lens), gamma, ctypes.byref(shape), _attn_params(params),
+                                               _p(workspace), _nbytes(workspace), _stream_ptr(stream)))
 
 
 def rapid_verify_attention_paged(q, k_pool, v_pool, block_table, ctx_lens, gamma, out, workspace,

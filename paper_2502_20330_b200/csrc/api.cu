@@ -236,6 +236,14 @@ int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cac
                                    static_cast<cudaStream_t>(cuda_stream));
 }
 
+int rapid_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
+                         const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream) {
+    clear_error();
+    return launch_attention_plan(ctx_lens, gamma, shape, params, workspace, workspace_bytes,
+                                 static_cast<cudaStream_t>(cuda_stream));
+}
+
 int rapid_verify_attention_paged(const void* q, const void* k_pool, const void* v_pool,
                                  const int32_t* block_table, const rapid_paged_kv* paged,
                                  const int32_t* ctx_lens, int gamma, void* out,

@@ -33,6 +33,8 @@ __host__ __device__ constexpr long long slot_floats(int GR, int D) {
     return ((long long)GR * (D + 2) + 3) / 4 * 4;
 }
 
+struct Walk;
+
 struct AttnArgs {
     const __nv_bfloat16* q;
     const int32_t* ctx_lens;
@@ -58,18 +60,72 @@ struct AttnArgs {
     int pad;
     int kt_half_blocks;  // keys-on-M kernel over a paged cache with 64-key blocks: two boxes per tile
     int tile_keys;  // keys per scheduling tile: what plan, walk and merge count in (64, or 128 for the keys-on-M kernel)
+    // Sink + window visibility (window > 0): row i sees the keys below `sink` and the `window`
+    // newest keys up to its own, (lim_i - window, lim_i].  Tiles no row sees are not streamed.
+    int sink, window;
+    // A plan made by attention_plan_kernel for the same geometry and lengths (plan_mode != 0):
+    // every CTA's walk and every unit's range of partial slots, read instead of computed.
+    int plan_mode;
+    const Walk* plan_walks;
+    const int2* plan_units;  // (first CTA, number of slots) of every unit
+    const int32_t* plan_ctx;  // the lengths the plan was made for
+    const int32_t* plan_sig;  // the geometry the plan was made for (kPlanSigInts words)
+    long long wait_limit;     // clock cycles an on-chip wait may take
+    // One thread-block cluster per unit (cmerge = its size, 0 = off): the cluster's CTAs split the
+    // unit's tiles, exchange their partials through distributed shared memory and write the
+    // output rows themselves; no partial goes to the workspace and no merge kernel follows.
+    int cmerge;
+    __nv_bfloat16* out;
+    float* out_f32;
+    float* lse_out;
 };
 
-struct Walk {
+// Where a CTA stands in its range of the flat tile list.  In sink + window mode a unit streams its
+// tiles [0, ns) and [ns + gap, ...): the real tile behind index t is t + (t >= ns ? gap : 0).
+struct __align__(16) Walk {
     int b, kvh, tile, ntiles, L;
+    int ns, gap;
+    int reserved;
     long long remaining;
     long long total;
 };
+static_assert(sizeof(Walk) == 48, "a walk is three 16-byte words of the plan");
+
+constexpr int kPlanSigInts = 16;
 
 __device__ __forceinline__ int clamp_len(int L, int R, int Lmax) {
     return L < R ? R : (L > Lmax ? Lmax : L);
 }
 __device__ __forceinline__ int tiles_of(int L, int tile_keys) { return (L + tile_keys - 1) / tile_keys; }
+
+// The tiles a unit of L keys streams: all of them, or, with a window, the tiles that hold sink
+// keys and the tiles from the oldest key of row 0's window on (the rows' windows end at their own
+// keys, so row 0's reaches back furthest).
+struct UnitGeom {
+    int nt, ns, gap;
+};
+__device__ __forceinline__ UnitGeom unit_geom(const AttnArgs& a, int L) {
+    UnitGeom g;
+    const int full = tiles_of(L, a.tile_keys);
+    g.nt = full;
+    g.ns = full;
+    g.gap = 0;
+    if (a.window > 0) {
+        const int w0 = L - a.R - a.window + 1;          // the oldest key row 0 sees through its window
+        const int ns = tiles_of(a.sink, a.tile_keys);   // tiles that hold sink keys
+        const int tw0 = w0 > 0 ? w0 / a.tile_keys : 0;  // the tile that key lives in
+        if (tw0 > ns) {
+            g.ns = ns;
+            g.gap = tw0 - ns;
+            g.nt = full - g.gap;
+        }
+    }
+    return g;
+}
+__device__ __forceinline__ int unit_tiles(const AttnArgs& a, int b) {
+    return unit_geom(a, clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax)).nt;
+}
+__device__ __forceinline__ int real_tile(const Walk& w, int t) { return t + (t >= w.ns ? w.gap : 0); }
 
 // The padding applies only when every CTA has a few tiles to stream.
 __device__ __forceinline__ int unit_pad(const AttnArgs& a, long long T) {
@@ -80,7 +136,7 @@ __device__ __forceinline__ int unit_pad(const AttnArgs& a, long long T) {
 __device__ __forceinline__ long long real_tiles_before(const AttnArgs& a, int pad, long long v) {
     long long real = 0;
     for (int b = 0; b < a.B; ++b) {
-        const int nt = tiles_of(clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax), a.tile_keys);
+        const int nt = unit_tiles(a, b);
         const long long ul = nt + pad, span = (long long)a.Hkv * ul;
         if (v >= span) {
             real += (long long)a.Hkv * nt;
@@ -95,11 +151,42 @@ __device__ __forceinline__ long long real_tiles_before(const AttnArgs& a, int pa
     return real;
 }
 
+__device__ __forceinline__ void walk_set_unit(const AttnArgs& a, Walk& w, int b) {
+    w.L = clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax);
+    const UnitGeom g = unit_geom(a, w.L);
+    w.ntiles = g.nt;
+    w.ns = g.ns;
+    w.gap = g.gap;
+}
+
 // Range of CTA c of n in the padded flat list: [c*Tv/n, (c+1)*Tv/n); its real tiles are what it works on.
+// With one cluster per unit (cmerge): CTA c is rank c % cmerge of the cluster of unit c / cmerge and
+// takes an equal share of that unit's tiles.
 __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
+    w.b = 0;
+    w.kvh = 0;
+    w.tile = 0;
+    w.L = 0;
+    w.ntiles = 0;
+    w.ns = 0;
+    w.gap = 0;
+    w.reserved = 0;
+    w.remaining = 0;
+    w.total = 0;
+    if (a.cmerge) {
+        const int unit = cta / a.cmerge, rank = cta % a.cmerge;
+        w.b = unit / a.Hkv;
+        w.kvh = unit % a.Hkv;
+        walk_set_unit(a, w, w.b);
+        const int t0 = (int)((long long)rank * w.ntiles / a.cmerge);
+        const int t1 = (int)((long long)(rank + 1) * w.ntiles / a.cmerge);
+        w.tile = t0;
+        w.remaining = t1 - t0;
+        w.total = w.ntiles;
+        return;
+    }
     long long T = 0;
-    for (int b = 0; b < a.B; ++b)
-        T += (long long)a.Hkv * tiles_of(clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax), a.tile_keys);
+    for (int b = 0; b < a.B; ++b) T += (long long)a.Hkv * unit_tiles(a, b);
     // with fewer tiles than CTAs only the first T CTAs work, one tile each: no CTA inside the
     // range of a unit is ever empty, which the merge relies on
     const long long nc = T < a.num_ctas ? T : a.num_ctas;
@@ -112,23 +199,16 @@ __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     }
     w.total = T;
     w.remaining = t1 - t0;
-    w.b = 0;
-    w.kvh = 0;
-    w.tile = 0;
-    w.L = 0;
-    w.ntiles = 0;
     if (w.remaining <= 0) return;
     long long t = t0;
     for (int b = 0; b < a.B; ++b) {
-        const int L = clamp_len(a.ctx_lens[b], a.Lmin, a.Lmax);
-        const int nt = tiles_of(L, a.tile_keys);
+        const int nt = unit_tiles(a, b);
         const long long span = (long long)a.Hkv * nt;
         if (t < span) {
             w.b = b;
             w.kvh = (int)(t / nt);
             w.tile = (int)(t % nt);
-            w.L = L;
-            w.ntiles = nt;
+            walk_set_unit(a, w, b);
             return;
         }
         t -= span;
@@ -143,11 +223,87 @@ __device__ __forceinline__ void walk_advance(const AttnArgs& a, Walk& w, int seg
         if (++w.kvh == a.Hkv) {
             w.kvh = 0;
             ++w.b;
-            if (w.b < a.B) {
-                w.L = clamp_len(a.ctx_lens[w.b], a.Lmin, a.Lmax);
-                w.ntiles = tiles_of(w.L, a.tile_keys);
-            }
+            if (w.b < a.B && w.remaining > 0) walk_set_unit(a, w, w.b);
         }
+    }
+}
+
+// The partial slots of a unit: first CTA whose range holds one of its tiles, and how many slots
+// (KS per CTA) the merge finds there.
+__device__ __forceinline__ int2 unit_slot_range(const AttnArgs& a, int unit, int KS) {
+    const int b = unit / a.Hkv, kvh = unit % a.Hkv;
+    long long T = 0, t0 = 0;
+    int nt_b = 0;
+    for (int bb = 0; bb < a.B; ++bb) {
+        const int nt = unit_tiles(a, bb);
+        if (bb < b) t0 += (long long)a.Hkv * nt;
+        if (bb == b) nt_b = nt;
+        T += (long long)a.Hkv * nt;
+    }
+    t0 += (long long)kvh * nt_b;
+    const long long units_before = (long long)b * a.Hkv + kvh;
+    const long long nc = T < a.num_ctas ? T : a.num_ctas;
+    // the unit's real tiles in the padded flat list the split kernel cut: [v0, v1)
+    const int pad = unit_pad(a, T);
+    const long long Tv = T + (long long)pad * a.B * a.Hkv;
+    const long long v0 = t0 + (units_before + 1) * pad, v1 = v0 + nt_b;
+    const int c_first = (int)(((v0 + 1) * nc - 1) / Tv);
+    const int c_last = (int)((v1 * nc - 1) / Tv);
+    return make_int2(c_first, (c_last - c_first + 1) * KS);
+}
+
+// A CTA's walk: from the plan (three 16-byte loads) or computed from the lengths.
+__device__ __forceinline__ void load_walk(const AttnArgs& a, int cta, Walk& w) {
+    const uint4* src = reinterpret_cast<const uint4*>(a.plan_walks + cta);
+    uint4* dst = reinterpret_cast<uint4*>(&w);
+    const uint4 x0 = __ldcg(src), x1 = __ldcg(src + 1), x2 = __ldcg(src + 2);
+    dst[0] = x0;
+    dst[1] = x1;
+    dst[2] = x2;
+}
+
+__device__ __forceinline__ void fill_plan_sig(const AttnArgs& a, int KS, int32_t (&sig)[kPlanSigInts]) {
+    const int32_t v[kPlanSigInts] = {a.B, a.Hkv, a.R, a.num_ctas, a.tile_keys, a.pad, a.stair, a.Lmin,
+                                     a.Lmax, a.sink, a.window, a.cmerge, KS, 0x504c414e, 0, 0};
+#pragma unroll
+    for (int i = 0; i < kPlanSigInts; ++i) sig[i] = v[i];
+}
+
+// Checks of CTA 0 that only the device can make: every length inside [Lmin, Lmax], and, when a
+// plan is used, that it was made for this geometry and for these lengths.
+__device__ __forceinline__ void check_call_inputs(const AttnArgs& a, int KS) {
+    bool bad = false, stale = false;
+    for (int b = 0; b < a.B; ++b) {
+        const int L = a.ctx_lens[b];
+        bad |= (L < a.Lmin) || (L > a.Lmax);
+        if (a.plan_mode) stale |= __ldcg(a.plan_ctx + b) != L;
+    }
+    if (a.plan_mode) {
+        int32_t sig[kPlanSigInts];
+        fill_plan_sig(a, KS, sig);
+        for (int i = 0; i < kPlanSigInts; ++i) stale |= __ldcg(a.plan_sig + i) != sig[i];
+    }
+    if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
+    if (stale) atomicOr(a.status, RAPID_STATUS_STALE_PLAN);
+}
+
+// Writes the plan of a call into its workspace: one block; thread c plans CTA c, thread u the
+// slot range of unit u.
+__global__ void __launch_bounds__(512) attention_plan_kernel(const AttnArgs a, int KS, Walk* walks, int2* units,
+                                                             int32_t* ctx_copy, int32_t* sig_out) {
+    const int n_ctas = a.cmerge ? a.B * a.Hkv * a.cmerge : a.num_ctas;
+    for (int c = threadIdx.x; c < n_ctas; c += blockDim.x) {
+        Walk w;
+        plan_cta(a, c, w);
+        walks[c] = w;
+    }
+    if (!a.cmerge)
+        for (int u = threadIdx.x; u < a.B * a.Hkv; u += blockDim.x) units[u] = unit_slot_range(a, u, KS);
+    for (int b = threadIdx.x; b < a.B; b += blockDim.x) ctx_copy[b] = a.ctx_lens[b];
+    if (threadIdx.x == 0) {
+        int32_t sig[kPlanSigInts];
+        fill_plan_sig(a, KS, sig);
+        for (int i = 0; i < kPlanSigInts; ++i) sig_out[i] = sig[i];
     }
 }
 
@@ -194,8 +350,37 @@ __device__ __forceinline__ void walk_advance(const AttnArgs& a, Walk& w, int seg
 //
 // A wait whose outcome is the same for every lane of the warp (needed because the warp goes on
 // to warp-collective TMEM instructions).
-__device__ __forceinline__ bool warp_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    return __all_sync(0xffffffffu, mbar_wait_bounded(bar, parity, abort_flag));
+__device__ __forceinline__ bool warp_wait_bounded(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
+    return __all_sync(0xffffffffu, mbar_wait_bounded(bar, parity, wc));
+}
+
+// Set-up of a split kernel after its input-free prologue: waits for the preceding kernel, lets the
+// dependents launch and hands every thread the CTA's walk.  A settled plan (made at least two
+// kernels earlier in the stream) was read before the wait, and nothing but the wait remains.
+//
+// Order matters here: launch_dependents comes after the wait in every kernel of this library.  A
+// dependent kernel therefore starts only once everything before its predecessor has completed,
+// which is what allows (a) the merge kernel to take the lengths before its own wait although an
+// earlier kernel of the stream may have written them, and (b) a settled plan to be read before
+// the wait.
+__device__ __forceinline__ void split_kernel_walk(const AttnArgs& a, int cta, Walk& w, Walk* s_walk) {
+    const bool settled = a.plan_mode == RAPID_PLAN_SETTLED;
+    if (settled) load_walk(a, cta, w);
+    tc_fence_before_sync();
+    __syncthreads();  // barriers initialised, tensor memory allocated
+    tc_fence_after_sync();
+    griddep_wait();               // inputs are read from here on
+    griddep_launch_dependents();  // the merge blocks may take their seats
+    if (!settled) {
+        if (threadIdx.x == 0) {
+            Walk t;
+            if (a.plan_mode) load_walk(a, cta, t);
+            else plan_cta(a, cta, t);
+            *s_walk = t;
+        }
+        __syncthreads();
+        w = *s_walk;
+    }
 }
 
 constexpr int kTcThreads = 352;
@@ -255,6 +440,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
     __shared__ uint64_t empty_bar[kTcMaxStages];
     __shared__ uint64_t s_full[2], p_full[2][2];
     __shared__ uint64_t q_full, o_free;
+    __shared__ uint64_t drain_bar[2];  // an MMA issuer that leaves early sees its MMAs complete here
     __shared__ uint32_t tmem_slot;
     __shared__ Walk s_walk;
     __shared__ int s_abort;
@@ -285,6 +471,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             mbar_init(&s_full[i], 1);
             mbar_init(&p_full[i][0], lay.n_active);
             mbar_init(&p_full[i][1], lay.n_active);
+            mbar_init(&drain_bar[i], 1);
         }
         mbar_init(&q_full, 1);
         mbar_init(&o_free, 2 * lay.n_active);
@@ -295,29 +482,11 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
         prefetch_tensormap(&tmQ);
     }
     if (warp == 9) tmem_alloc(&tmem_slot, TMEM_COLS);  // warp 9 also frees it at the end
-    // From here on inputs are read (and, much later, the workspace is written): the preceding
-    // kernel must have completed.  Then the merge blocks of this call may take their seats.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;");
-    if (tid == 0) {
-        Walk w;
-        plan_cta(a, cta, w);
-        s_walk = w;
-        if (cta == 0) {
-            bool bad = false;
-            for (int b = 0; b < a.B; ++b) {
-                const int L = a.ctx_lens[b];
-                bad |= (L < a.Lmin) || (L > a.Lmax);
-            }
-            if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
-        }
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
+    Walk w;
+    split_kernel_walk(a, cta, w, &s_walk);
+    if (cta == 0 && warp == 8 && lane == 1) check_call_inputs(a, kStreams);  // an idle lane of the producer warp
     const uint32_t tmem_base = tmem_slot;
-    Walk w = s_walk;
-    volatile int* abort_flag = &s_abort;
+    const WaitCtx wc = {&s_abort, a.wait_limit};
 
     if (warp == 8) {
         // ---------------- TMA producer for K/V tiles ----------------
@@ -333,14 +502,14 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                     // coordinates of the tile: (key, outermost) = (logical position, sequence), or,
                     // paged, (position inside the block, physical block).  The table entry is
                     // fetched before the wait for a free stage, so the two overlap.
-                    int key0 = (w.tile + t) * kTile, outer = w.b;
+                    const int tile = real_tile(w, w.tile + t);
+                    int key0 = tile * kTile, outer = w.b;
                     if (a.block_table) {
-                        const int tile = w.tile + t;
                         outer = __ldg(a.block_table + (size_t)w.b * a.max_blocks + (tile >> a.tile_shift));
                         key0 = (tile & ((1 << a.tile_shift) - 1)) * kTile;
                     }
                     if (n >= nstage)
-                        ok = mbar_wait_bounded_relaxed(&empty_bar[s], ((n / nstage) - 1) & 1, abort_flag);
+                        ok = mbar_wait_bounded_relaxed(&empty_bar[s], ((n / nstage) - 1) & 1, wc);
                     if (!ok) break;
                     if (a.block_table && (unsigned)outer >= (unsigned)a.num_blocks) {
                         // the copy below reads zeros for a block outside the pool (the tensor map
@@ -359,6 +528,13 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 }
                 walk_advance(a, w, seg);
             }
+            // leaving early: the copies already issued must have landed before the CTA gives up its
+            // shared memory
+            if (!ok)
+                for (int s = 0; s < nstage && s < n; ++s) {
+                    const int u = s + (n - 1 - s) / nstage * nstage;  // the stage's latest tile
+                    mbar_wait_drain(&full_bar[s], (u / nstage) & 1);
+                }
         }
     } else if (warp == 9) {
         // ---------------- Q loader and QK^T issuer ----------------
@@ -378,14 +554,15 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 // the previous unit's O rows have been read out, so all its MMAs have completed
                 // and Q may be replaced
-                if (seg_idx > 0) ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, abort_flag);
+                if (seg_idx > 0) ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, wc);
                 if (!ok) break;
                 mbar_arrive_expect_tx(&q_full, (uint32_t)a.GR * D * 2);
 #pragma unroll
                 for (int h = 0; h < NHALF; ++h)
                     tma_load_4d(smem_gen + lay.off_q + h * (128 * 128), &tmQ, &q_full, h * 64,
                                 w.kvh * a.G, 0, w.b);
-                ok = mbar_wait_bounded(&q_full, seg_idx & 1, abort_flag);
+                ok = mbar_wait_bounded(&q_full, seg_idx & 1, wc);
+                if (!ok) mbar_wait_drain(&q_full, seg_idx & 1);  // the Q copy is on its way: let it land
                 const int n_end = n + seg;
                 while (n < n_end && ok) {
                     const int cnt = ((n & 1) || n + 1 >= n_end) ? 1 : 2;  // pairs start at even tiles
@@ -393,10 +570,10 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                     // the S buffer is free once the PVs of the group that used it last have completed
                     for (int i = 0; i < prev_cnt[b] && ok; ++i) {
                         const int pn = prev_first[b] + i;
-                        ok = mbar_wait_bounded(&empty_bar[pn % nstage], (pn / nstage) & 1, abort_flag);
+                        ok = mbar_wait_bounded(&empty_bar[pn % nstage], (pn / nstage) & 1, wc);
                     }
                     for (int i = 0; i < cnt && ok; ++i)
-                        ok = mbar_wait_bounded(&full_bar[(n + i) % nstage], ((n + i) / nstage) & 1, abort_flag);
+                        ok = mbar_wait_bounded(&full_bar[(n + i) % nstage], ((n + i) / nstage) & 1, wc);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint64_t kd = k_desc + (uint64_t)((uint32_t)(n % nstage) * (BLK >> 4));
@@ -416,6 +593,10 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 }
                 walk_advance(a, w, seg);
                 ++seg_idx;
+            }
+            if (!ok) {  // leaving early: every MMA issued here must have completed before tensor memory is freed
+                umma_commit(&drain_bar[0]);
+                mbar_wait_drain(&drain_bar[0], 0);
             }
         }
     } else if (warp == 10) {
@@ -437,7 +618,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                     const int b = ts.group & 1;
                     // P(n) is published only after its stream has read the previous unit's O row
                     const int phase = ts.half ? pairs_seen[b]++ : (ts.group >> 1);
-                    ok = mbar_wait_bounded(&p_full[b][ts.half], phase & 1, abort_flag);
+                    ok = mbar_wait_bounded(&p_full[b][ts.half], phase & 1, wc);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint64_t vd = v_desc + (uint64_t)((uint32_t)(n % nstage) * (BLK >> 4));
@@ -451,6 +632,10 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 }
                 g0 += groups_in_unit(n0, seg);
                 walk_advance(a, w, seg);
+            }
+            if (!ok) {
+                umma_commit(&drain_bar[1]);
+                mbar_wait_drain(&drain_bar[1], 0);
             }
         }
     } else if ((warp & 3) < lay.n_active) {
@@ -474,14 +659,18 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             const int L = w.L;
             const int lim = a.stair ? L - a.R + i_row : L - 1;
             const int all_see = a.stair ? L - a.R : L - 1;  // the last key every row sees
+            // sink + window: keys in [sink, lo] are hidden from this row; lo_max is the newest key
+            // that some row does not see any more
+            const int lo = a.window > 0 ? lim - a.window : -1;
+            const int lo_max = a.window > 0 ? L - 1 - a.window : -1;
             float m_ref = -INFINITY, l_run = 0.f;
             int last_n = -1;  // the stream's latest tile of this unit (CTA-wide index)
 
             for (int n = n0 + ((n0 ^ stream) & 1); n < n0 + seg && ok; n += 2) {
-                const int key0 = (w.tile + (n - n0)) * kTile;
+                const int key0 = real_tile(w, w.tile + (n - n0)) * kTile;
                 const TileSlot ts = tile_slot(n, n0, g0);
                 const uint32_t tS = tmem_base + lane_base + COL_S + 128u * (ts.group & 1) + 64u * ts.half;
-                ok = warp_wait_bounded(&s_full[ts.group & 1], (ts.group >> 1) & 1, abort_flag);
+                ok = warp_wait_bounded(&s_full[ts.group & 1], (ts.group >> 1) & 1, wc);
                 if (!ok) break;
                 tc_fence_after_sync();
                 uint32_t sr[2][32];
@@ -495,6 +684,15 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
                         for (int k = 0; k < 32; ++k)
                             if (key0 + h * 32 + k > lim) sr[h][k] = __float_as_uint(-INFINITY);
+                }
+                if (key0 <= lo_max && key0 + kTile > a.sink) {  // the old edge of the windows
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) {
+                            const int key = key0 + h * 32 + k;
+                            if (key >= a.sink && key <= lo) sr[h][k] = __float_as_uint(-INFINITY);
+                        }
                 }
 
                 uint32_t pk[32];
@@ -535,7 +733,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                     }
                     if (!first) {
                         // O must be at rest (the stream's previous PV complete) while rows are rescaled
-                        ok = warp_wait_bounded(&empty_bar[last_n % nstage], (last_n / nstage) & 1, abort_flag);
+                        ok = warp_wait_bounded(&empty_bar[last_n % nstage], (last_n / nstage) & 1, wc);
                         if (!ok) break;
                         tc_fence_after_sync();
 #pragma unroll
@@ -578,7 +776,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
             const int unit = w.b * a.Hkv + w.kvh;
             float* slot = a.partial + ((size_t)(cta + unit) * 2 + stream) * slot_stride;
             if (last_n >= 0) {
-                ok = warp_wait_bounded(&empty_bar[last_n % nstage], (last_n / nstage) & 1, abort_flag);
+                ok = warp_wait_bounded(&empty_bar[last_n % nstage], (last_n / nstage) & 1, wc);
                 if (!ok) break;
                 tc_fence_after_sync();
 #pragma unroll
@@ -637,24 +835,13 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
 
-    long long T = 0, units_before = 0, t0 = 0;
-    int nt_b = 0;
-    for (int bb = 0; bb < a.B; ++bb) {
-        const int nt = tiles_of(clamp_len(a.ctx_lens[bb], a.Lmin, a.Lmax), a.tile_keys);
-        if (bb < b) t0 += (long long)a.Hkv * nt;
-        if (bb == b) nt_b = nt;
-        T += (long long)a.Hkv * nt;
-    }
-    t0 += (long long)kvh * nt_b;
-    units_before = (long long)b * a.Hkv + kvh;
-    const long long nc = T < a.num_ctas ? T : a.num_ctas;
-    // the unit's real tiles in the padded flat list the split kernel cut: [v0, v1)
-    const int pad = unit_pad(a, T);
-    const long long Tv = T + (long long)pad * a.B * a.Hkv;
-    const long long v0 = t0 + (units_before + 1) * pad, v1 = v0 + nt_b;
-    const int c_first = (int)(((v0 + 1) * nc - 1) / Tv);
-    const int c_last = (int)((v1 * nc - 1) / Tv);
-    const int nslots = (c_last - c_first + 1) * KS;
+    // The unit's slots: from the plan, or from the lengths.  Both are read before the wait although
+    // an earlier kernel of the stream may have written them: this kernel starts only after every
+    // CTA of the split kernel has passed its own wait (it lets its dependents launch after it),
+    // and by then everything before the split kernel has completed.
+    const int2 range = a.plan_mode ? __ldcg(a.plan_units + unit) : unit_slot_range(a, unit, KS);
+    const int c_first = range.x;
+    const int nslots = range.y;
     const size_t slot_stride = (size_t)slot_floats(a.GR, D);
     const float* base = a.partial + (size_t)(c_first + unit) * KS * slot_stride;  // slots are consecutive
 
@@ -825,6 +1012,9 @@ int make_q_map(CUtensorMap* map, const void* q, const rapid_attn_shape& s, int G
 }
 
 constexpr int kMaxSmemOptin = 232448 - 1024;  // 227 KB per CTA on sm_100, less the static barriers
+// Longest cache for which the library itself picks one cluster per KV head: the clusters leave some
+// SMs without work, which a short run wins back by having no merge kernel.
+constexpr int64_t kClusterMaxKeys = 65536;
 
 template <int D, int MR>
 int launch_split_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
@@ -886,34 +1076,115 @@ bool attn_shape_ok(const rapid_attn_shape* s, int gamma) {
 
 }  // namespace
 
-template <int NC, int SG = 1>
-int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ, const AttnArgs& a,
-                    cudaStream_t stream) {
+// Largest cluster (16, 8, 4, 2) of this kernel of which `clusters_needed` fit on the device at once;
+// 0 if none does.  Asked of the runtime once per device, kernel and size.
+// Per-device attributes of a keys-on-M kernel: its dynamic shared memory, and clusters of 16 CTAs.
+template <int NC, int SG>
+cudaError_t kt_configure(int dev) {
     constexpr int smem = kt::smem_bytes(NC);
     static_assert(smem <= kMaxSmemOptin - 4096, "shared memory (dynamic + the kernel's static arrays)");
     static bool configured[64] = {};
+    if (dev >= 0 && dev < 64 && configured[dev]) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC, SG>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC, SG>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+    return cudaSuccess;
+}
+
+template <int NC, int SG>
+int kt_cluster_size_that_fits(int clusters_needed, int dev) {
+    constexpr int smem = kt::smem_bytes(NC);
+    if (kt_configure<NC, SG>(dev) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    static int resident[64][4] = {};  // clusters of 16, 8, 4, 2 CTAs resident together (0 = not asked yet, -1 = none)
+    const int sizes[4] = {16, 8, 4, 2};
+    if (dev < 0 || dev >= 64) return 0;
+    for (int i = 0; i < 4; ++i) {
+        if (!resident[dev][i]) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(sizes[i]);
+            cfg.blockDim = dim3(kt::threads(SG));
+            cfg.dynamicSmemBytes = smem;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = sizes[i];
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kt::verify_attn_splitkv_kt_kernel<NC, SG>, &cfg) != cudaSuccess) {
+                cudaGetLastError();
+                n = 0;
+            }
+            resident[dev][i] = n > 0 ? n : -1;
+        }
+        if (resident[dev][i] >= clusters_needed) return sizes[i];
+    }
+    return 0;
+}
+
+template <int NC, int SG = 1>
+int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ, AttnArgs& a,
+                    cudaStream_t stream, bool want_cluster, bool need_cluster) {
+    constexpr int smem = kt::smem_bytes(NC);
     int dev = 0;
     RAPID_CUDA_CHECK(cudaGetDevice(&dev));
-    if (dev >= 64 || !configured[dev]) {
-        RAPID_CUDA_CHECK(cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC, SG>,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        if (dev < 64) configured[dev] = true;
+    RAPID_CUDA_CHECK((kt_configure<NC, SG>(dev)));
+    const int units = a.B * a.Hkv;
+    a.cmerge = 0;
+    if (want_cluster) {
+        const int cs = kt_cluster_size_that_fits<NC, SG>(units, dev);
+        // on the library's own choice the clusters must also cover most of the machine
+        if (cs && (need_cluster || units * cs * 4 >= sm_count() * 3)) a.cmerge = cs;
+        if (!a.cmerge && need_cluster) {
+            set_error("rapid_verify_attention: %d clusters (one per sequence and KV head) do not fit on the device "
+                      "together", units);
+            return RAPID_ERR_UNSUPPORTED;
+        }
     }
-    RAPID_CUDA_CHECK(launch_dependent(kt::verify_attn_splitkv_kt_kernel<NC, SG>, dim3(a.num_ctas),
-                                      dim3(kt::threads(SG)), (size_t)smem, stream, tmK, tmV, tmQ, a));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.cmerge ? units * a.cmerge : a.num_ctas);
+    cfg.blockDim = dim3(kt::threads(SG));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (a.cmerge) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = a.cmerge;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
+    RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kt::verify_attn_splitkv_kt_kernel<NC, SG>, tmK, tmV, tmQ,
+                                        static_cast<const AttnArgs&>(a)));
     return RAPID_OK;
 }
 
-int dispatch_split_kt(int NC, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
-                      const AttnArgs& a, cudaStream_t stream) {
+// fp32_sums: the caller takes the log-sum-exp, so the row sums must add fp32 probabilities.  With
+// 49 to 64 grouped rows one softmax group has no registers for that (it adds the bf16 values the
+// tensor cores multiply); two groups of 32 columns each do.
+int dispatch_split_kt(int NC, bool fp32_sums, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
+                      AttnArgs& a, cudaStream_t stream, bool want_cluster, bool need_cluster) {
     switch (NC) {
-        case 1: return launch_split_kt<1>(tmK, tmV, tmQ, a, stream);
-        case 2: return launch_split_kt<2>(tmK, tmV, tmQ, a, stream);
-        case 3: return launch_split_kt<3>(tmK, tmV, tmQ, a, stream);
-        case 4: return launch_split_kt<4>(tmK, tmV, tmQ, a, stream);
+        case 1: return launch_split_kt<1>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
+        case 2: return launch_split_kt<2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
+        case 3: return launch_split_kt<3>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
+        case 4:
+            return fp32_sums ? launch_split_kt<4, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster)
+                             : launch_split_kt<4>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
         // more than 64 grouped rows: two softmax groups, each with half of the columns
-        case 5: return launch_split_kt<5, 2>(tmK, tmV, tmQ, a, stream);
-        case 6: return launch_split_kt<6, 2>(tmK, tmV, tmQ, a, stream);
+        case 5: return launch_split_kt<5, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
+        case 6: return launch_split_kt<6, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
     }
     set_error("unsupported number of grouped rows");
     return RAPID_ERR_UNSUPPORTED;
@@ -937,13 +1208,257 @@ int launch_merge_partials(const float* o_parts, const float* lse_parts, int P, i
     return RAPID_OK;
 }
 
+namespace {
+
+// Where things live in an attention workspace (bytes from its start).
+struct WsLayout {
+    size_t sig, walks, units, ctx, partial, total;
+};
+WsLayout ws_layout(int B, int Hkv, int GR, int D) {
+    WsLayout l;
+    size_t off = kWorkspaceHeaderBytes;
+    l.sig = off;
+    off += align_up(kPlanSigInts * sizeof(int32_t), 256);
+    l.walks = off;
+    off += align_up((size_t)kMaxCtas * sizeof(Walk), 256);
+    l.units = off;
+    off += align_up((size_t)B * Hkv * sizeof(int2), 256);
+    l.ctx = off;
+    off += align_up((size_t)B * sizeof(int32_t), 256);
+    l.partial = off;
+    const int64_t slots = ((int64_t)kMaxCtas + (int64_t)B * Hkv) * kStreams;
+    off += (size_t)slots * slot_floats(GR, D) * sizeof(float);
+    l.total = off;
+    return l;
+}
+
+// Everything the attention entry points share: validation, the choice of kernel, the arguments.
+struct AttnCall {
+    AttnArgs a;
+    bool kt_path, kt_half_blocks, fp32_sums, want_cluster, need_cluster;
+    int NC, KS, box_rows;
+    int64_t sl, sh, sb, outer, keys;
+};
+
+int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
+                      const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
+                      const rapid_paged_kv* paged, const int32_t* block_table, AttnCall& c) {
+    if (!ctx_lens || !shape) {
+        set_error("%s: NULL argument", who);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (!attn_shape_ok(shape, gamma)) {
+        set_error("%s: invalid shape (B=%d Hq=%d Hkv=%d Lmax=%lld gamma=%d)", who, shape->B, shape->Hq, shape->Hkv,
+                  (long long)shape->Lmax, gamma);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const rapid_attn_shape& s = *shape;
+    const int R = gamma + 1;
+    const int G = s.Hq / s.Hkv;
+    const int GR = G * R;
+    if (s.D != 64 && s.D != 128) {
+        set_error("%s: head_dim %d is not supported (64 or 128)", who, s.D);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    if (GR > 128) {
+        set_error("%s: %d grouped rows per KV head exceed 128", who, GR);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const bool all_visible = params && params->all_keys_visible;
+    if (s.Lmax < (all_visible ? 1 : R) || s.Lmax > 0x7fffffffLL - kTile) {
+        set_error("%s: Lmax %lld out of range", who, (long long)s.Lmax);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const int sink = params ? params->sink_keys : 0, window = params ? params->window_keys : 0;
+    if (sink < 0 || window < 0 || (sink > 0 && window == 0) || (window > 0 && all_visible)) {
+        set_error("%s: sink_keys and window_keys must not be negative, sink_keys needs a window, and a window "
+                  "cannot be combined with all_keys_visible", who);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    c.outer = s.B;
+    c.keys = s.Lmax;
+    int tile_shift = 0;
+    if (paged) {
+        const int64_t bs = paged->block_size;
+        if (bs < kTile || (bs & (bs - 1)) || paged->num_blocks <= 0 || paged->max_blocks_per_seq <= 0) {
+            set_error("%s: block_size must be a power of two >= %d, num_blocks and max_blocks_per_seq positive", who,
+                      kTile);
+            return RAPID_ERR_UNSUPPORTED;
+        }
+        if (s.Lmax != (int64_t)paged->max_blocks_per_seq * bs) {
+            set_error("%s: shape->Lmax must equal max_blocks_per_seq * block_size", who);
+            return RAPID_ERR_INVALID_ARG;
+        }
+        while ((kTile << tile_shift) < bs) ++tile_shift;
+        c.sl = paged->stride_l ? paged->stride_l : s.D;
+        c.sh = paged->stride_h ? paged->stride_h : bs * c.sl;
+        c.sb = paged->stride_block ? paged->stride_block : s.Hkv * c.sh;
+        c.outer = paged->num_blocks;
+        c.keys = bs;
+    } else {
+        c.sl = s.kv_stride_l ? s.kv_stride_l : s.D;
+        c.sh = s.kv_stride_h ? s.kv_stride_h : s.Lmax * c.sl;
+        c.sb = s.kv_stride_b ? s.kv_stride_b : s.Hkv * c.sh;
+    }
+    if (c.sl < s.D || c.sl % 8 || c.sh % 8 || c.sb % 8 || c.sh <= 0 || c.sb <= 0) {
+        set_error("%s: K/V strides must be positive multiples of 8 elements", who);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const WsLayout lay = ws_layout(s.B, s.Hkv, GR, s.D);
+    if (!workspace || workspace_bytes < lay.total || ((uintptr_t)workspace & 255)) {
+        set_error("%s: workspace of %zu bytes needed (256-byte aligned), got %zu", who, lay.total, workspace_bytes);
+        return RAPID_ERR_WORKSPACE;
+    }
+    int num_ctas = params && params->num_ctas ? params->num_ctas : sm_count();
+    if (num_ctas <= 0 || num_ctas > kMaxCtas) {
+        set_error("%s: num_ctas %d outside [1, %d]", who, num_ctas, kMaxCtas);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const float scale = params && params->scale != 0.f ? params->scale : 1.0f / sqrtf((float)s.D);
+    if (!(scale > 0.f) || !isfinite(scale)) {
+        set_error("%s: scale must be positive and finite", who);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if ((int64_t)s.B * s.Hkv > 65535) {
+        set_error("%s: B*Hkv above 65535 is not supported", who);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const int plan_mode = params ? params->plan : RAPID_PLAN_NONE;
+    if (plan_mode != RAPID_PLAN_NONE && plan_mode != RAPID_PLAN_READY && plan_mode != RAPID_PLAN_SETTLED) {
+        set_error("%s: unknown plan mode %d", who, plan_mode);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    const long long wait_limit = params && params->wait_cycle_limit ? params->wait_cycle_limit : kWaitCycleLimit;
+    if (wait_limit < 0) {
+        set_error("%s: wait_cycle_limit must not be negative", who);
+        return RAPID_ERR_INVALID_ARG;
+    }
+
+    // Which split kernel: keys on the MMA's M axis (a softmax thread per key, probabilities through
+    // shared memory) when the grouped rows fit 64 columns -- faster and cheaper per byte there --,
+    // rows on the M axis otherwise (more rows, head_dim 64).  From 65 to 96 rows the keys-on-M kernel
+    // runs on request only (two softmax groups; measured level with the rows-on-M kernel at 72
+    // rows, not ahead of it).  With one sequence, whose KV heads all have the same length, and a
+    // cache of at most kClusterMaxKeys keys, the keys-on-M kernel runs as one cluster per KV head
+    // and merges on chip; any call can ask for that (RAPID_ATTN_KERNEL_CLUSTER_MERGE).
+    const int want = params ? params->kernel : RAPID_ATTN_KERNEL_AUTO;
+    const bool kt_ok = s.D == 128 && (GR + 15) / 16 <= kt::kMaxNC2;
+    if (want != RAPID_ATTN_KERNEL_AUTO && want != RAPID_ATTN_KERNEL_ROWS_ON_M && want != RAPID_ATTN_KERNEL_KEYS_ON_M &&
+        want != RAPID_ATTN_KERNEL_CLUSTER_MERGE) {
+        set_error("%s: unknown kernel choice %d", who, want);
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if ((want == RAPID_ATTN_KERNEL_KEYS_ON_M || want == RAPID_ATTN_KERNEL_CLUSTER_MERGE) && !kt_ok) {
+        set_error("%s: the keys-on-M kernel needs head_dim 128 and at most %d grouped rows", who, 16 * kt::kMaxNC2);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const bool kt_auto = kt_ok && (GR + 15) / 16 <= kt::kMaxNC;
+    c.kt_path = want == RAPID_ATTN_KERNEL_KEYS_ON_M || want == RAPID_ATTN_KERNEL_CLUSTER_MERGE ||
+                (want == RAPID_ATTN_KERNEL_AUTO && kt_auto);
+    c.need_cluster = want == RAPID_ATTN_KERNEL_CLUSTER_MERGE;
+    c.want_cluster = c.need_cluster ||
+                     (want == RAPID_ATTN_KERNEL_AUTO && c.kt_path && s.B == 1 && s.Lmax <= kClusterMaxKeys &&
+                      !(params && params->split_done_event));
+    if (c.need_cluster && (int64_t)s.B * s.Hkv * 2 > kMaxCtas) {
+        set_error("%s: too many (sequence, KV head) units for one cluster each", who);
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    c.kt_half_blocks = c.kt_path && paged && paged->block_size == kTile;
+    if (c.kt_path && paged && !c.kt_half_blocks) --tile_shift;  // blocks are counted in 128-key tiles
+    c.box_rows = c.kt_path && !c.kt_half_blocks ? kt::kKeys : kTile;
+    c.NC = (GR + 15) / 16;
+    c.KS = c.kt_path ? 1 : kStreams;
+    c.fp32_sums = params && params->lse_out;
+
+    AttnArgs& a = c.a;
+    a = AttnArgs{};
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    a.ctx_lens = ctx_lens;
+    a.partial = reinterpret_cast<float*>(ws + lay.partial);
+    a.status = reinterpret_cast<int32_t*>(ws);
+    a.B = s.B;
+    a.Hq = s.Hq;
+    a.Hkv = s.Hkv;
+    a.G = G;
+    a.R = R;
+    a.GR = GR;
+    a.Lmax = (int)s.Lmax;
+    a.num_ctas = num_ctas;
+    a.scale_log2 = scale * 1.4426950408889634f;
+    a.block_table = paged ? block_table : nullptr;
+    a.max_blocks = paged ? paged->max_blocks_per_seq : 0;
+    a.num_blocks = paged ? paged->num_blocks : 0;
+    a.tile_shift = tile_shift;
+    a.kt_half_blocks = c.kt_half_blocks ? 1 : 0;
+    a.tile_keys = c.kt_path ? kt::kKeys : kTile;
+    a.pad = c.kt_path ? 5 : unit_switch_tiles(s.D);
+    a.stair = all_visible ? 0 : R;
+    a.Lmin = all_visible ? 1 : R;
+    a.sink = window > 0 ? sink : 0;
+    a.window = window;
+    a.plan_mode = plan_mode;
+    a.plan_sig = reinterpret_cast<const int32_t*>(ws + lay.sig);
+    a.plan_walks = reinterpret_cast<const Walk*>(ws + lay.walks);
+    a.plan_units = reinterpret_cast<const int2*>(ws + lay.units);
+    a.plan_ctx = reinterpret_cast<const int32_t*>(ws + lay.ctx);
+    a.wait_limit = wait_limit;
+    a.cmerge = 0;
+    return RAPID_OK;
+}
+
+}  // namespace
+
 size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma) {
     if (!attn_shape_ok(s, gamma)) return 0;
     if (s->D != 64 && s->D != 128) return 0;
     const int64_t GR = (int64_t)(s->Hq / s->Hkv) * (gamma + 1);
     if (GR > 128) return 0;
-    const int64_t slots = ((int64_t)kMaxCtas + (int64_t)s->B * s->Hkv) * kStreams;
-    return kWorkspaceHeaderBytes + (size_t)slots * slot_floats((int)GR, s->D) * sizeof(float);
+    return ws_layout(s->B, s->Hkv, (int)GR, s->D).total;
+}
+
+// The cluster size a keys-on-M call of this geometry would run with (0 = no cluster).
+static int cluster_size_for(const AttnCall& c) {
+    if (!c.kt_path || !c.want_cluster) return 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    const int units = c.a.B * c.a.Hkv;
+    int cs = 0;
+    switch (c.NC) {
+        case 1: cs = kt_cluster_size_that_fits<1, 1>(units, dev); break;
+        case 2: cs = kt_cluster_size_that_fits<2, 1>(units, dev); break;
+        case 3: cs = kt_cluster_size_that_fits<3, 1>(units, dev); break;
+        case 4: cs = c.fp32_sums ? kt_cluster_size_that_fits<4, 2>(units, dev) : kt_cluster_size_that_fits<4, 1>(units, dev); break;
+        case 5: cs = kt_cluster_size_that_fits<5, 2>(units, dev); break;
+        case 6: cs = kt_cluster_size_that_fits<6, 2>(units, dev); break;
+    }
+    if (cs && !c.need_cluster && units * cs * 4 < sm_count() * 3) cs = 0;
+    return cs;
+}
+
+int launch_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
+                          const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
+                          cudaStream_t stream) {
+    AttnCall c;
+    rapid_attn_params p = params ? *params : rapid_attn_params{};
+    p.plan = RAPID_PLAN_NONE;
+    // a paged call plans like a contiguous one: the tiles are the same, only their addresses differ
+    int rc = prepare_attention("rapid_attention_plan", ctx_lens, gamma, shape, &p, workspace, workspace_bytes, nullptr,
+                               nullptr, c);
+    if (rc != RAPID_OK) return rc;
+    c.a.cmerge = cluster_size_for(c);
+    if (c.need_cluster && !c.a.cmerge) {
+        set_error("rapid_attention_plan: the clusters of this call do not fit on the device together");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const WsLayout lay = ws_layout(c.a.B, c.a.Hkv, c.a.GR, shape->D);
+    attention_plan_kernel<<<1, 512, 0, stream>>>(c.a, c.KS, reinterpret_cast<Walk*>(ws + lay.walks),
+                                                 reinterpret_cast<int2*>(ws + lay.units),
+                                                 reinterpret_cast<int32_t*>(ws + lay.ctx),
+                                                 reinterpret_cast<int32_t*>(ws + lay.sig));
+    RAPID_CUDA_CHECK(cudaGetLastError());
+    count_launch(1);
+    return RAPID_OK;
 }
 
 int launch_verify_attention(const void* q, const void* k_cache, const void* v_cache,
@@ -959,170 +1474,55 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
         set_error("rapid_verify_attention_paged: NULL block table");
         return RAPID_ERR_INVALID_ARG;
     }
-    if (!attn_shape_ok(shape, gamma)) {
-        set_error("rapid_verify_attention: invalid shape (B=%d Hq=%d Hkv=%d Lmax=%lld gamma=%d)",
-                  shape->B, shape->Hq, shape->Hkv, (long long)shape->Lmax, gamma);
-        return RAPID_ERR_INVALID_ARG;
-    }
-    const rapid_attn_shape& s = *shape;
-    const int R = gamma + 1;
-    const int G = s.Hq / s.Hkv;
-    const int GR = G * R;
-    if (s.D != 64 && s.D != 128) {
-        set_error("rapid_verify_attention: head_dim %d is not supported (64 or 128)", s.D);
-        return RAPID_ERR_UNSUPPORTED;
-    }
-    if (GR > 128) {
-        set_error("rapid_verify_attention: %d grouped rows per KV head exceed 128", GR);
-        return RAPID_ERR_UNSUPPORTED;
-    }
-    const bool all_visible = params && params->all_keys_visible;
-    if (s.Lmax < (all_visible ? 1 : R) || s.Lmax > 0x7fffffffLL - kTile) {
-        set_error("rapid_verify_attention: Lmax %lld out of range", (long long)s.Lmax);
-        return RAPID_ERR_INVALID_ARG;
-    }
-    int64_t sl, sh, sb, outer = s.B, keys = s.Lmax;
-    int tile_shift = 0;
-    if (paged) {
-        const int64_t bs = paged->block_size;
-        if (bs < kTile || (bs & (bs - 1)) || paged->num_blocks <= 0 || paged->max_blocks_per_seq <= 0) {
-            set_error("rapid_verify_attention_paged: block_size must be a power of two >= %d, num_blocks and "
-                      "max_blocks_per_seq positive", kTile);
-            return RAPID_ERR_UNSUPPORTED;
-        }
-        if (s.Lmax != (int64_t)paged->max_blocks_per_seq * bs) {
-            set_error("rapid_verify_attention_paged: shape->Lmax must equal max_blocks_per_seq * block_size");
-            return RAPID_ERR_INVALID_ARG;
-        }
-        while ((kTile << tile_shift) < bs) ++tile_shift;
-        sl = paged->stride_l ? paged->stride_l : s.D;
-        sh = paged->stride_h ? paged->stride_h : bs * sl;
-        sb = paged->stride_block ? paged->stride_block : s.Hkv * sh;
-        outer = paged->num_blocks;
-        keys = bs;
-    } else {
-        sl = s.kv_stride_l ? s.kv_stride_l : s.D;
-        sh = s.kv_stride_h ? s.kv_stride_h : s.Lmax * sl;
-        sb = s.kv_stride_b ? s.kv_stride_b : s.Hkv * sh;
-    }
-    if (sl < s.D || sl % 8 || sh % 8 || sb % 8 || sh <= 0 || sb <= 0) {
-        set_error("rapid_verify_attention: K/V strides must be positive multiples of 8 elements");
-        return RAPID_ERR_UNSUPPORTED;
-    }
+    AttnCall c;
+    int rc = prepare_attention("rapid_verify_attention", ctx_lens, gamma, shape, params, workspace, workspace_bytes,
+                               paged, block_table, c);
+    if (rc != RAPID_OK) return rc;
     if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q | (uintptr_t)out) & 15) {
         set_error("rapid_verify_attention: q, k_cache, v_cache and out must be 16-byte aligned");
         return RAPID_ERR_UNSUPPORTED;
     }
-    const size_t need = attention_workspace_bytes(shape, gamma);
-    if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) {
-        set_error("rapid_verify_attention: workspace of %zu bytes needed (256-byte aligned), got %zu",
-                  need, workspace_bytes);
-        return RAPID_ERR_WORKSPACE;
-    }
-    int num_ctas = params && params->num_ctas ? params->num_ctas : sm_count();
-    if (num_ctas <= 0 || num_ctas > kMaxCtas) {
-        set_error("rapid_verify_attention: num_ctas %d outside [1, %d]", num_ctas, kMaxCtas);
-        return RAPID_ERR_INVALID_ARG;
-    }
-    const float scale = params && params->scale != 0.f ? params->scale : 1.0f / sqrtf((float)s.D);
-    if (!(scale > 0.f) || !isfinite(scale)) {
-        set_error("rapid_verify_attention: scale must be positive and finite");
-        return RAPID_ERR_INVALID_ARG;
-    }
-    if ((int64_t)s.B * s.Hkv > 65535) {
-        set_error("rapid_verify_attention: B*Hkv above 65535 is not supported");
-        return RAPID_ERR_UNSUPPORTED;
-    }
-
-    CUtensorMap tmK, tmV;
-    // Which split kernel: keys on the MMA's M axis (a softmax thread per key, probabilities through
-    // shared memory) when the grouped rows fit 64 columns -- faster and cheaper per byte there --,
-    // rows on the M axis otherwise (more rows, head_dim 64, paged blocks of 64 keys).  From 65 to 96
-    // rows the keys-on-M kernel runs on request only (two softmax groups; measured level with the
-    // rows-on-M kernel at 72 rows, not ahead of it).
-    const int want = params ? params->kernel : RAPID_ATTN_KERNEL_AUTO;
-    const bool kt_ok = s.D == 128 && (GR + 15) / 16 <= kt::kMaxNC2 && (!paged || paged->block_size >= kTile);
-    if (want != RAPID_ATTN_KERNEL_AUTO && want != RAPID_ATTN_KERNEL_ROWS_ON_M && want != RAPID_ATTN_KERNEL_KEYS_ON_M) {
-        set_error("rapid_verify_attention: unknown kernel choice %d", want);
-        return RAPID_ERR_INVALID_ARG;
-    }
-    if (want == RAPID_ATTN_KERNEL_KEYS_ON_M && !kt_ok) {
-        set_error("rapid_verify_attention: the keys-on-M kernel needs head_dim 128, at most %d grouped rows and, "
-                  "paged, blocks of at least %d keys", 16 * kt::kMaxNC2, kTile);
-        return RAPID_ERR_UNSUPPORTED;
-    }
-    const bool kt_auto = kt_ok && (GR + 15) / 16 <= kt::kMaxNC;
-    const bool kt_path = want == RAPID_ATTN_KERNEL_KEYS_ON_M || (want == RAPID_ATTN_KERNEL_AUTO && kt_auto);
-    const bool kt_half_blocks = kt_path && paged && paged->block_size == kTile;
-    if (kt_path && paged && !kt_half_blocks) --tile_shift;  // blocks are counted in 128-key tiles
-    const int box_rows = kt_path && !kt_half_blocks ? kt::kKeys : kTile;
-    int rc = make_kv_map(&tmK, k_cache, s, outer, keys, sb, sh, sl, box_rows);
-    if (rc != RAPID_OK) return rc;
-    rc = make_kv_map(&tmV, v_cache, s, outer, keys, sb, sh, sl, box_rows);
-    if (rc != RAPID_OK) return rc;
-
-    AttnArgs a;
+    const rapid_attn_shape& s = *shape;
+    AttnArgs& a = c.a;
     a.q = static_cast<const __nv_bfloat16*>(q);
-    a.ctx_lens = ctx_lens;
-    a.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kWorkspaceHeaderBytes);
-    a.status = static_cast<int32_t*>(workspace);
-    a.B = s.B;
-    a.Hq = s.Hq;
-    a.Hkv = s.Hkv;
-    a.G = G;
-    a.R = R;
-    a.GR = GR;
-    a.Lmax = (int)s.Lmax;
-    a.num_ctas = num_ctas;
-    a.scale_log2 = scale * 1.4426950408889634f;
-    a.block_table = paged ? block_table : nullptr;
-    a.max_blocks = paged ? paged->max_blocks_per_seq : 0;
-    a.num_blocks = paged ? paged->num_blocks : 0;
-    a.tile_shift = tile_shift;
-    a.kt_half_blocks = kt_half_blocks ? 1 : 0;
-    a.tile_keys = kt_path ? kt::kKeys : kTile;
-    a.pad = kt_path ? 5 : unit_switch_tiles(s.D);
-    a.stair = all_visible ? 0 : R;
-    a.Lmin = all_visible ? 1 : R;
+    a.out = static_cast<__nv_bfloat16*>(out);
+    a.lse_out = params ? params->lse_out : nullptr;
+    a.out_f32 = params ? params->out_f32 : nullptr;
 
-    CUtensorMap tmQ;
-    rc = make_q_map(&tmQ, q, s, G, R);
+    CUtensorMap tmK, tmV, tmQ;
+    rc = make_kv_map(&tmK, k_cache, s, c.outer, c.keys, c.sb, c.sh, c.sl, c.box_rows);
     if (rc != RAPID_OK) return rc;
-    int n_partials = kStreams;
-    if (kt_path) {
-        n_partials = 1;
-        rc = dispatch_split_kt((GR + 15) / 16, tmK, tmV, tmQ, a, stream);
-    } else if (GR <= 64)
+    rc = make_kv_map(&tmV, v_cache, s, c.outer, c.keys, c.sb, c.sh, c.sl, c.box_rows);
+    if (rc != RAPID_OK) return rc;
+    rc = make_q_map(&tmQ, q, s, a.G, a.R);
+    if (rc != RAPID_OK) return rc;
+
+    if (c.kt_path) {
+        rc = dispatch_split_kt(c.NC, c.fp32_sums, tmK, tmV, tmQ, a, stream, c.want_cluster, c.need_cluster);
+    } else if (a.GR <= 64)
         rc = s.D == 128 ? launch_split_tc<128, 64>(tmK, tmV, tmQ, a, stream)
                         : launch_split_tc<64, 64>(tmK, tmV, tmQ, a, stream);
     else
         rc = s.D == 128 ? launch_split_tc<128, 128>(tmK, tmV, tmQ, a, stream)
                         : launch_split_tc<64, 128>(tmK, tmV, tmQ, a, stream);
     if (rc != RAPID_OK) return rc;
+    if (a.cmerge) {  // merged on chip: one kernel
+        count_launch(1);
+        return RAPID_OK;
+    }
 
     if (params && params->split_done_event)
         RAPID_CUDA_CHECK(cudaEventRecord(static_cast<cudaEvent_t>(params->split_done_event), stream));
 
-    dim3 grid(GR, s.B * s.Hkv);
-    float* lse = params ? params->lse_out : nullptr;
-    float* o32 = params ? params->out_f32 : nullptr;
+    dim3 grid(a.GR, s.B * s.Hkv);
     // programmatic dependent launch: the merge blocks start while the split kernel still runs and
     // hold at their grid-dependency wait until its partials are complete and visible
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(128);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    __nv_bfloat16* out_bf = static_cast<__nv_bfloat16*>(out);
     if (s.D == 128)
-        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<128>, a, n_partials, out_bf, lse, o32));
+        RAPID_CUDA_CHECK(launch_dependent(verify_attn_merge_kernel<128>, grid, dim3(128), 0, stream, a, c.KS, a.out,
+                                          a.lse_out, a.out_f32));
     else
-        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, verify_attn_merge_kernel<64>, a, n_partials, out_bf, lse, o32));
+        RAPID_CUDA_CHECK(launch_dependent(verify_attn_merge_kernel<64>, grid, dim3(128), 0, stream, a, c.KS, a.out,
+                                          a.lse_out, a.out_f32));
     count_launch(2);
     return RAPID_OK;
 }

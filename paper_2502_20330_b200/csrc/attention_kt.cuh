@@ -39,6 +39,21 @@
 // Barriers: every parity wait is on a barrier whose next phase cannot complete before the waiter has
 // passed the current one (per-buffer s_full / p_full, per-stage full / empty; empty doubles as
 // "the PV of this tile has completed").
+//
+// Waits that run out.  Every mbarrier wait is bounded.  The single-thread roles (producer, MMA
+// issuers) leave their loops when a wait fails, after seeing their own asynchronous work land (the
+// producer its bulk copies, the issuers their MMAs).  The softmax warps do NOT leave early: the
+// four warps of a group meet at named barriers, which have no time limit, so a warp that left
+// while another had seen its wait succeed would strand it there.  They run their loops to the end
+// instead; once the abort flag is up every wait returns at once, so that is quick, and what they
+// write is in bounds and flagged invalid by RAPID_STATUS_PIPELINE_TIMEOUT.
+//
+// One cluster per unit (AttnArgs::cmerge).  For calls whose whole run is short (a decode over a
+// few thousand keys) the merge kernel and its two kernel boundaries cost as much as the
+// streaming.  There the CTAs of a thread-block cluster share one unit's tiles, leave their
+// partial (O^T, references, sums) in their own shared memory, and after one cluster barrier CTA r
+// combines the partials of the output rows r, r + cluster size, ... over distributed shared memory
+// and writes them: one kernel per call.
 #pragma once
 
 namespace kt {
@@ -80,6 +95,24 @@ __device__ __forceinline__ bool bar_softmax_or(int grp, bool flag) {
     return res != 0;
 }
 #undef RAPID_KT_BAR_OR
+// Cluster-wide barrier of all threads, release / acquire: what a CTA wrote to its shared memory
+// before it is visible to its peers' distributed-shared-memory loads after it.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// A float of the shared memory of CTA `rank` of the cluster, at the same offset as `addr` here.
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t addr, int rank) {
+    uint32_t raddr;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(raddr) : "memory");
+    return v;
+}
 __device__ __forceinline__ float warp_max32(float v) {
 #pragma unroll
     for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
@@ -118,10 +151,12 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
     __shared__ uint64_t k_full[NK], k_empty[NK], v_full[NV], v_empty[NV];
     __shared__ uint64_t s_full[2], p_full[2];
     __shared__ uint64_t q_full, o_free;
+    __shared__ uint64_t drain_bar[2];  // an MMA issuer that leaves early sees its MMAs complete here
     __shared__ uint32_t tmem_slot;
     __shared__ Walk s_walk;
     __shared__ int s_abort;
     __shared__ __align__(16) float sh_mref[128], sh_fac[128], sh_w[4][128];
+    __shared__ float sh_lfin[128];  // cluster mode: the unit's row sums of this CTA
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -143,6 +178,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
         for (int i = 0; i < 2; ++i) {
             mbar_init(&s_full[i], 1);
             mbar_init(&p_full[i], WS);
+            mbar_init(&drain_bar[i], 1);
         }
         mbar_init(&q_full, 1);
         mbar_init(&o_free, WS);
@@ -153,21 +189,6 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
         prefetch_tensormap(&tmQ);
     }
     if (warp == WS + 1) tmem_alloc(&tmem_slot, TMEM_COLS);  // the same warp frees it at the end
-    griddep_wait();               // inputs are read from here on
-    griddep_launch_dependents();  // the merge blocks may take their seats
-    if (tid == 0) {
-        Walk w;
-        plan_cta(a, cta, w);
-        s_walk = w;
-        if (cta == 0) {
-            bool bad = false;
-            for (int b = 0; b < a.B; ++b) {
-                const int L = a.ctx_lens[b];
-                bad |= (L < a.Lmin) || (L > a.Lmax);
-            }
-            if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
-        }
-    }
     // The Q rows past the grouped rows are never written by the Q loads: zero them once, so that
     // the scores of those columns are 0 whatever the shared memory held.
     {
@@ -178,28 +199,32 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
         }
         fence_proxy_async_smem();
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
+    if (tid < 128) {  // a CTA of a cluster that gets no tile publishes "no partial"
+        sh_mref[tid] = -INFINITY;
+        sh_lfin[tid] = 0.f;
+    }
+    Walk w;
+    split_kernel_walk(a, cta, w, &s_walk);
+    if (cta == 0 && warp == WS && lane == 1) check_call_inputs(a, 1);  // an idle lane of the producer warp
     const uint32_t tmem_base = tmem_slot;
-    Walk w = s_walk;
-    volatile int* abort_flag = &s_abort;
+    const WaitCtx wc = {&s_abort, a.wait_limit};
+    const int unit_b = w.b, unit_kvh = w.kvh;  // cluster mode: the one unit this CTA works on
 
     if (warp == WS) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            int jj = 0;
+            int jj = 0, n_k = 0, n_v = 0;  // tiles met; K and V tiles whose copies were issued
             bool ok = true;
             while (w.remaining > 0 && ok) {
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 for (int t = 0; t < seg && ok; ++t, ++jj) {
                     const int ks = jj % NK, vs = jj % NV;
+                    const int tile = real_tile(w, w.tile + t);
                     // a tile is one box of 128 keys, or, for a paged cache with 64-key blocks, two
                     // boxes of 64 keys from two physical blocks (parts = 2)
                     const int parts = a.kt_half_blocks ? 2 : 1;
-                    int key0[2] = {(w.tile + t) * kKeys, 0}, outer[2] = {w.b, w.b};
+                    int key0[2] = {tile * kKeys, 0}, outer[2] = {w.b, w.b};
                     if (a.block_table) {
-                        const int tile = w.tile + t;
                         for (int p = 0; p < parts; ++p) {
                             const int lb = a.kt_half_blocks ? 2 * tile + p : (tile >> a.tile_shift);
                             key0[p] = a.kt_half_blocks ? 0 : (tile & ((1 << a.tile_shift) - 1)) * kKeys;
@@ -215,7 +240,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         }
                     }
                     const uint32_t part_bytes = kBlk / parts;
-                    if (jj >= NK) ok = mbar_wait_bounded_relaxed(&k_empty[ks], ((jj / NK) - 1) & 1, abort_flag);
+                    if (jj >= NK) ok = mbar_wait_bounded_relaxed(&k_empty[ks], ((jj / NK) - 1) & 1, wc);
                     if (!ok) break;
                     mbar_arrive_expect_tx(&k_full[ks], TILE_TX);
                     for (int p = 0; p < parts; ++p)
@@ -223,7 +248,8 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         for (int h = 0; h < 2; ++h)
                             tma_load_4d(smem_gen + OFF_K + (h * NK + ks) * kBlk + p * part_bytes, &tmK, &k_full[ks],
                                         h * 64, key0[p], w.kvh, outer[p]);
-                    if (jj >= NV) ok = mbar_wait_bounded_relaxed(&v_empty[vs], ((jj / NV) - 1) & 1, abort_flag);
+                    ++n_k;
+                    if (jj >= NV) ok = mbar_wait_bounded_relaxed(&v_empty[vs], ((jj / NV) - 1) & 1, wc);
                     if (!ok) break;
                     mbar_arrive_expect_tx(&v_full[vs], TILE_TX);
                     for (int p = 0; p < parts; ++p)
@@ -231,8 +257,17 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         for (int h = 0; h < 2; ++h)
                             tma_load_4d(smem_gen + OFF_V + (h * NV + vs) * kBlk + p * part_bytes, &tmV, &v_full[vs],
                                         h * 64, key0[p], w.kvh, outer[p]);
+                    ++n_v;
                 }
                 walk_advance(a, w, seg);
+            }
+            // leaving early: the copies already issued must have landed before the CTA gives up its
+            // shared memory
+            if (!ok) {
+                for (int s = 0; s < NK && s < n_k; ++s)
+                    mbar_wait_drain(&k_full[s], ((s + (n_k - 1 - s) / NK * NK) / NK) & 1);
+                for (int s = 0; s < NV && s < n_v; ++s)
+                    mbar_wait_drain(&v_full[s], ((s + (n_v - 1 - s) / NV * NV) / NV) & 1);
             }
         }
     } else if (warp == WS + 1) {
@@ -246,18 +281,19 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
             while (w.remaining > 0 && ok) {
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 // the previous unit has been read out of tensor memory: every MMA of it is complete
-                if (seg_idx > 0) ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, abort_flag);
+                if (seg_idx > 0) ok = mbar_wait_bounded(&o_free, (seg_idx - 1) & 1, wc);
                 if (!ok) break;
                 mbar_arrive_expect_tx(&q_full, (uint32_t)a.GR * D * 2);
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
                     tma_load_4d(smem_gen + OFF_Q + h * (N * 128), &tmQ, &q_full, h * 64, w.kvh * a.G, 0, w.b);
-                ok = mbar_wait_bounded(&q_full, seg_idx & 1, abort_flag);
+                ok = mbar_wait_bounded(&q_full, seg_idx & 1, wc);
+                if (!ok) mbar_wait_drain(&q_full, seg_idx & 1);  // the Q copy is on its way: let it land
                 for (int t = 0; t < seg && ok; ++t, ++jj) {
                     const int s = jj % NK, b = jj & 1;
-                    ok = mbar_wait_bounded(&k_full[s], (jj / NK) & 1, abort_flag);
+                    ok = mbar_wait_bounded(&k_full[s], (jj / NK) & 1, wc);
                     // S^T buffer b is free once the probabilities of tile jj-2 have been published
-                    if (ok && jj >= 2) ok = mbar_wait_bounded(&p_full[b], ((jj - 2) >> 1) & 1, abort_flag);
+                    if (ok && jj >= 2) ok = mbar_wait_bounded(&p_full[b], ((jj - 2) >> 1) & 1, wc);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint32_t d = tmem_base + COL_S + 128u * b;
@@ -272,6 +308,10 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 }
                 walk_advance(a, w, seg);
                 ++seg_idx;
+            }
+            if (!ok) {  // leaving early: every MMA issued here must have completed before tensor memory is freed
+                umma_commit(&drain_bar[0]);
+                mbar_wait_drain(&drain_bar[0], 0);
             }
         }
     } else if (warp == WS + 2) {
@@ -289,8 +329,8 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 for (int t = 0; t < seg && ok; ++t, ++jj) {
                     const int s = jj % NV;
-                    ok = mbar_wait_bounded(&p_full[jj & 1], (jj >> 1) & 1, abort_flag);
-                    if (ok) ok = mbar_wait_bounded(&v_full[s], (jj / NV) & 1, abort_flag);
+                    ok = mbar_wait_bounded(&p_full[jj & 1], (jj >> 1) & 1, wc);
+                    if (ok) ok = mbar_wait_bounded(&v_full[s], (jj / NV) & 1, wc);
                     if (!ok) break;
                     tc_fence_after_sync();
 #pragma unroll
@@ -300,6 +340,10 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                     umma_commit(&v_empty[s]);  // PV complete: the V slot and the P^T buffer are free
                 }
                 walk_advance(a, w, seg);
+            }
+            if (!ok) {
+                umma_commit(&drain_bar[1]);
+                mbar_wait_drain(&drain_bar[1], 0);
             }
         }
     } else if (warp < WS) {
@@ -318,23 +362,32 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
 
         float lsum[NG];  // this key slot's share of the sums of the group's rows
         int jj = 0;
+        // `ok` only records that a wait ran out: these warps run their loops to the end whatever
+        // happens (see "Waits that run out" above)
         bool ok = true;
-        while (w.remaining > 0 && ok) {
+        while (w.remaining > 0) {
             const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
             const int L = w.L;
 #pragma unroll
             for (int i = 0; i < NG; ++i) lsum[i] = 0.f;
 
-            for (int ti = 0; ti < seg && ok; ++ti, ++jj) {
+            for (int ti = 0; ti < seg; ++ti, ++jj) {
                 const int b = jj & 1;
                 const uint32_t tS = tmem_base + lane_base + COL_S + 128u * b + C0;
-                const int key = (w.tile + ti) * kKeys + t;
-                // row i sees keys <= L-R+i; rows are column i*G+g: the masked columns are a prefix
-                // (no stair: every row sees every key below L)
+                const int key0 = real_tile(w, w.tile + ti) * kKeys;  // the tile's first key
+                const int key = key0 + t;
+                // Row i sees keys <= L-R+i and rows are column i*G+g, so the columns the causal stair
+                // hides from this key are a prefix [0, cmin) (no stair: every row sees every key
+                // below L).  With a window the rows too new for this key are a suffix [cmax, N):
+                // row i sees it iff key > L-R+i - window, unless it is a sink key.
                 const int over_ctx = a.stair ? key - (L - a.R) : 0;
                 const int cmin = key >= L ? N : (over_ctx > 0 ? over_ctx * a.G : 0);
-                ok = warp_wait_bounded(&s_full[b], (jj >> 1) & 1, abort_flag);
-                if (!ok) break;
+                int cmax = N;
+                if (a.window > 0 && key >= a.sink) {
+                    const long long rows_in = (long long)key - (L - a.R) + a.window;
+                    cmax = rows_in <= 0 ? 0 : (rows_in * a.G >= N ? N : (int)rows_in * a.G);
+                }
+                ok &= warp_wait_bounded(&s_full[b], (jj >> 1) & 1, wc);
                 tc_fence_after_sync();
 
                 // One pass over the scores: probabilities against the current references, kept in
@@ -365,7 +418,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                                               fmaf(__uint_as_float(sr[e + 3]), c, -m.w)};
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) {
-                                    if (MASKED) x[i] = col + i >= cmin ? x[i] : -INFINITY;
+                                    if (MASKED) x[i] = (col + i >= cmin && col + i < cmax) ? x[i] : -INFINITY;
                                     far |= x[i] > kJump;
                                     x[i] = fast_exp2(x[i]);
                                 }
@@ -380,14 +433,15 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         }
                         return far;
                     };
-                    const bool tile_clear = (w.tile + ti + 1) * kKeys <= L - a.stair;  // the same for every thread
+                    // the same for every thread: no key of the tile is hidden from any row
+                    const bool tile_clear = key0 + kKeys <= L - a.stair &&
+                                            (a.window <= 0 || key0 + kKeys <= a.sink || key0 > L - 1 - a.window);
                     move = tile_clear ? first_pass(std::false_type{}) : first_pass(std::true_type{});
                     move = bar_softmax_or(grp, move);
                 }
                 // PV of the previous tile must be complete: it reads P^T, and O^T may be rescaled now
                 if (jj >= 1) {
-                    ok = warp_wait_bounded(&v_empty[(jj - 1) % NV], ((jj - 1) / NV) & 1, abort_flag);
-                    if (!ok) break;
+                    ok &= warp_wait_bounded(&v_empty[(jj - 1) % NV], ((jj - 1) / NV) & 1, wc);
                     tc_fence_after_sync();
                 }
                 if (move) {
@@ -400,7 +454,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
                         for (int e = 0; e < CH; ++e) {
                             const int col = C0 + CH * ch + e;
-                            const float v = (col >= cmin && col < a.GR) ? __uint_as_float(sr[e]) * c : -INFINITY;
+                            const float v = (col >= cmin && col < cmax && col < a.GR) ? __uint_as_float(sr[e]) * c : -INFINITY;
                             const float wm = warp_max32(v);
                             if (lane == 0) sh_w[wq][col] = wm;
                         }
@@ -442,8 +496,8 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         for (int e = 0; e < CH; e += 2) {
                             const int li = CH * ch + e, col = C0 + li;
                             const float m0 = sh_mref[col], m1 = sh_mref[col + 1];
-                            const float x0 = col >= cmin ? fmaf(__uint_as_float(sr[e]), c, m0 == -INFINITY ? 0.f : -m0) : -INFINITY;
-                            const float x1 = col + 1 >= cmin ? fmaf(__uint_as_float(sr[e + 1]), c, m1 == -INFINITY ? 0.f : -m1) : -INFINITY;
+                            const float x0 = (col >= cmin && col < cmax) ? fmaf(__uint_as_float(sr[e]), c, m0 == -INFINITY ? 0.f : -m0) : -INFINITY;
+                            const float x1 = (col + 1 >= cmin && col + 1 < cmax) ? fmaf(__uint_as_float(sr[e + 1]), c, m1 == -INFINITY ? 0.f : -m1) : -INFINITY;
                             const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                             if (kPacked) {
                                 pq[li >> 1] = pack_bf16x2(p0, p1);
@@ -479,12 +533,11 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                     }
                     *reinterpret_cast<uint4*>(p_gen + (g8 >> 3) * kBlk + (((g8 & 7) ^ p_swz) << 4)) = pk;
                 }
-                if (grp == 0 && key - t + kKeys > L) {
+                if (grp == 0 && key0 + kKeys > L) {
                     // V rows beyond the context may hold any bits: zero them so that 0 * row = 0
                     // (one group does it; PV waits for both groups' arrivals)
-                    ok = warp_wait_bounded(&v_full[jj % NV], (jj / NV) & 1, abort_flag);  // the V tile has landed
-                    if (!ok) break;
-                    const int first_bad = L - (key - t);
+                    ok &= warp_wait_bounded(&v_full[jj % NV], (jj / NV) & 1, wc);  // the V tile has landed
+                    const int first_bad = L - key0;
                     const int chunks = (kKeys - first_bad) * 8;
                     for (int h = 0; h < 2; ++h) {
                         uint8_t* vgen = smem_gen + OFF_V + (h * NV + jj % NV) * kBlk;
@@ -497,14 +550,14 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&p_full[b]);
             }
-            if (!ok) break;
-
             // ---- end of the unit: O^T out of tensor memory, row sums added up, partial written ----
-            ok = warp_wait_bounded(&v_empty[(jj - 1) % NV], ((jj - 1) / NV) & 1, abort_flag);
-            if (!ok) break;
+            ok &= warp_wait_bounded(&v_empty[(jj - 1) % NV], ((jj - 1) / NV) & 1, wc);
             tc_fence_after_sync();
             const int unit = w.b * a.Hkv + w.kvh;
-            float* slot = a.partial + (size_t)(cta + unit) * slot_stride;
+            // the partial goes to the workspace, or, with one cluster per unit, to this CTA's own
+            // shared memory (the K ring: every K tile has been consumed), [column][d] fp32
+            float* slot = a.cmerge ? reinterpret_cast<float*>(smem_gen + OFF_K)
+                                   : a.partial + (size_t)(cta + unit) * slot_stride;
 #pragma unroll
             for (int ch = 0; ch < NG / CH; ++ch) {
                 uint32_t orow[CH];
@@ -524,8 +577,13 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
             bar_softmax(grp);
             if (t < NG && C0 + t < a.GR) {
                 const int col = C0 + t;
-                slot[a.GR * D + col] = sh_mref[col];
-                slot[a.GR * D + a.GR + col] = ((sh_w[0][col] + sh_w[1][col]) + sh_w[2][col]) + sh_w[3][col];
+                const float l_fin = ((sh_w[0][col] + sh_w[1][col]) + sh_w[2][col]) + sh_w[3][col];
+                if (a.cmerge) {
+                    sh_lfin[col] = l_fin;
+                } else {
+                    slot[a.GR * D + col] = sh_mref[col];
+                    slot[a.GR * D + a.GR + col] = l_fin;
+                }
             }
             bar_softmax(grp);  // sh_w / sh_mref are reused by the next unit
             tc_fence_before_sync();
@@ -537,6 +595,35 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
 
     tc_fence_before_sync();
     __syncthreads();
+    if (a.cmerge) {
+        // ---- one cluster per unit: combine the cluster's partials over distributed shared memory ----
+        // CTA r of the cluster takes the output rows (columns) r, r + cmerge, ...; thread d the
+        // output element d.  Fixed order over the ranks: results are bit-identical from run to run.
+        cluster_sync_all();  // every CTA's partial is in its shared memory and visible
+        const uint32_t rank = cluster_cta_rank();
+        const uint32_t xo_addr = smem_base + OFF_K, m_addr = smem_u32(sh_mref), l_addr = smem_u32(sh_lfin);
+        if (tid < D) {
+            for (int col = (int)rank; col < a.GR; col += a.cmerge) {
+                float M = -INFINITY;
+                for (int p = 0; p < a.cmerge; ++p) M = fmaxf(M, ld_dsmem_f32(m_addr + 4u * col, p));
+                float acc = 0.f, l = 0.f;
+                for (int p = 0; p < a.cmerge; ++p) {
+                    const float mp = ld_dsmem_f32(m_addr + 4u * col, p);
+                    if (mp == -INFINITY) continue;  // that CTA saw no key of this row: its partial holds no O
+                    const float wgt = exp2f(mp - M);
+                    l += wgt * ld_dsmem_f32(l_addr + 4u * col, p);
+                    acc += wgt * ld_dsmem_f32(xo_addr + 4u * (col * D + tid), p);
+                }
+                const float val = acc / l;
+                const int i = col / a.G, g = col % a.G;
+                const size_t row = ((size_t)unit_b * a.R + i) * a.Hq + (size_t)unit_kvh * a.G + g;
+                a.out[row * D + tid] = __float2bfloat16_rn(val);
+                if (a.out_f32) a.out_f32[row * D + tid] = val;
+                if (a.lse_out && tid == 0) a.lse_out[row] = (M + log2f(l)) * 0.69314718055994530942f;
+            }
+        }
+        cluster_sync_all();  // no CTA leaves while a peer may still read its shared memory
+    }
     if (warp == WS + 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, TMEM_COLS);

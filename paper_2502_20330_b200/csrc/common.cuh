@@ -57,6 +57,9 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
                             const rapid_attn_shape* shape, const rapid_attn_params* params,
                             void* workspace, size_t workspace_bytes, cudaStream_t stream,
                             const rapid_paged_kv* paged = nullptr, const int32_t* block_table = nullptr);
+int launch_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
+                          const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
+                          cudaStream_t stream);
 int launch_retrieval_select(const float* chunk_emb, const float* query_emb, const int32_t* n_chunks, int B,
                             int Nmax, int Dm, float threshold, int k, float* scores_out, int32_t* sel_idx,
                             int32_t* sel_count, int32_t* status_word, cudaStream_t stream);
@@ -110,41 +113,57 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Every wait on an mbarrier is bounded: after kWaitCycleLimit clock cycles (about a second)
-// the waiter raises *abort_flag (shared memory), which makes every later wait of the CTA
-// return at once, and the caller records RAPID_STATUS_PIPELINE_TIMEOUT.  Returns false on
-// timeout / abort.
+// Every wait on an mbarrier is bounded: after `limit` clock cycles (kWaitCycleLimit, about a
+// second, unless the call names another figure) the waiter raises *abort (shared memory), which
+// makes every later wait of the CTA return at once, and the kernel records
+// RAPID_STATUS_PIPELINE_TIMEOUT.  Returns false on timeout / abort.
 constexpr long long kWaitCycleLimit = 2000000000LL;
+
+struct WaitCtx {
+    volatile int* abort;  // the CTA's abort flag (shared memory)
+    long long limit;      // clock cycles a wait may take
+};
 
 // Same wait for a role that is not on the critical path (the TMA producer runs several stages
 // ahead): it sleeps between polls instead of spinning, which saves power for the clocks.
-__device__ __forceinline__ bool mbar_wait_bounded_relaxed(uint64_t* bar, uint32_t parity,
-                                                          volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_bounded_relaxed(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         __nanosleep(200);
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycleLimit) {
-            *abort_flag = 1;
+        if (*wc.abort) return false;
+        if (clock64() - t0 > wc.limit) {
+            *wc.abort = 1;
             return false;
         }
     }
 }
 
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity,
-                                                  volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycleLimit) {
-            *abort_flag = 1;
+        if (*wc.abort) return false;
+        if (clock64() - t0 > wc.limit) {
+            *wc.abort = 1;
             return false;
         }
     }
+}
+
+// The wait of a role that is leaving after an abort and must see its own asynchronous work land
+// first (a bulk copy it issued, the MMAs it committed): the abort flag does not end it, only the
+// barrier or the library's own limit does.  Such work always completes, so this returns true
+// unless the hardware has stopped.
+__device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitCycleLimit) return false;
+        __nanosleep(100);
+    }
+    return true;
 }
 
 // 4-D tiled TMA load global -> shared, completion counted on an mbarrier (no multicast).
@@ -160,30 +179,6 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* m
 
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
-}
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3,
-                                            uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2,
-                                                  uint32_t& r3, uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-
-// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
-                                               uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
-        "{%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 // Programmatic dependent launch (kernels launched with cudaLaunchAttributeProgrammaticStreamSerialization):

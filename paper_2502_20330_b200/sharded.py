@@ -51,7 +51,8 @@ def exchange_partials(o32: torch.Tensor, lse: torch.Tensor, group=None) -> Tuple
 
 def local_partial(q, k_local, v_local, local_lens, gamma, workspace, holds_newest: bool,
                   params: Optional[_b.AttnParams] = None, stream=None):
-    """This rank's partial: (out_f32 [B,R,Hq,D], lse [B,R,Hq]) over its own keys."""
+    """This rank's partial: (out_f32 [B,R,Hq,D], lse [B,R,Hq]) over its own keys.  The results are
+    allocated on torch's current stream: make ``stream`` that stream (or pass None) when calling this directly."""
     B, R, Hq, D = q.shape
     o32 = torch.empty(B, R, Hq, D, dtype=torch.float32, device=q.device)
     lse = torch.empty(B, R, Hq, dtype=torch.float32, device=q.device)
@@ -68,8 +69,15 @@ def sharded_verify_attention(q, k_local, v_local, local_lens, gamma, out, worksp
 
     ``k_local`` / ``v_local`` [B,Hkv,Lloc,D] hold this rank's run of every sequence's keys and
     ``local_lens`` [B] their counts (see ``context_shard_bounds``); q is the same on every rank.
+
+    Everything runs on ``stream`` (default: the current stream).  The collective and the temporaries
+    follow torch's current stream, so the whole call is made with ``stream`` current: the kernels, the
+    all-gather and the allocator then agree on one order.  The inputs must be ready on that stream.
     """
-    rank, world = dist.get_rank(group), dist.get_world_size(group)
-    o32, lse = local_partial(q, k_local, v_local, local_lens, gamma, workspace, rank == world - 1, params, stream)
-    o_parts, l_parts = exchange_partials(o32, lse, group)
-    _b.rapid_merge_partials(o_parts, l_parts, out=out, stream=stream)
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device)
+    with torch.cuda.stream(stream):
+        rank, world = dist.get_rank(group), dist.get_world_size(group)
+        o32, lse = local_partial(q, k_local, v_local, local_lens, gamma, workspace, rank == world - 1, params, stream)
+        o_parts, l_parts = exchange_partials(o32, lse, group)
+        _b.rapid_merge_partials(o_parts, l_parts, out=out, stream=stream)

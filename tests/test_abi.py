@@ -47,7 +47,7 @@ def test_host_only_calls(lib):
 def test_struct_layouts_match_the_header():
     from paper_2502_20330_b200 import binding
     assert ctypes.sizeof(binding._AttnShape) == 48
-    assert ctypes.sizeof(binding._AttnParams) == 40
+    assert ctypes.sizeof(binding._AttnParams) == 64
     assert ctypes.sizeof(binding._AcceptShape) == 32
     assert ctypes.sizeof(binding._AcceptParams) == 24
     assert ctypes.sizeof(binding._PagedKv) == 40
@@ -62,7 +62,7 @@ def test_struct_layouts_match_what_the_c_compiler_sees(tmp_path):
         '#include <stdio.h>\n#include <stddef.h>\n#include "rapid.h"\n'
         'int main(void) {\n'
         '  printf("%zu %zu\\n", sizeof(rapid_attn_shape), offsetof(rapid_attn_shape, kv_stride_l));\n'
-        '  printf("%zu %zu\\n", sizeof(rapid_attn_params), offsetof(rapid_attn_params, all_keys_visible));\n'
+        '  printf("%zu %zu\\n", sizeof(rapid_attn_params), offsetof(rapid_attn_params, wait_cycle_limit));\n'
         '  printf("%zu %zu\\n", sizeof(rapid_accept_shape), offsetof(rapid_accept_shape, draft_row_stride));\n'
         '  printf("%zu %zu\\n", sizeof(rapid_accept_params), offsetof(rapid_accept_params, ratio_out));\n'
         '  printf("%zu %zu\\n", sizeof(rapid_paged_kv), offsetof(rapid_paged_kv, stride_l));\n'
@@ -72,7 +72,7 @@ def test_struct_layouts_match_what_the_c_compiler_sees(tmp_path):
     got = [tuple(int(x) for x in line.split()) for line in subprocess.run([str(exe)], check=True, capture_output=True,
                                                                           text=True).stdout.splitlines()]
     want = [(ctypes.sizeof(c), getattr(c, f).offset) for c, f in (
-        (binding._AttnShape, "kv_stride_l"), (binding._AttnParams, "all_keys_visible"),
+        (binding._AttnShape, "kv_stride_l"), (binding._AttnParams, "wait_cycle_limit"),
         (binding._AcceptShape, "draft_row_stride"), (binding._AcceptParams, "ratio_out"),
         (binding._PagedKv, "stride_l"))]
     assert got == want

@@ -11,44 +11,52 @@ import workloads as wl
 from workloads import bf16_bits
 
 
-def _run(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, kernel=0):
+# Absolute tolerance of the natural-log sum-exp, one figure for every kernel and shape.  When the
+# caller takes this output, every kernel adds fp32 probabilities into fp32 row sums (the keys-on-M
+# kernel then serves 49 to 64 grouped rows with two softmax groups, which have the registers for
+# it).  What is left: each probability carries the relative error of ex2.approx (2 ulp, 2.4e-7)
+# and of its fp32 argument (scores up to ~30 in log2 units, rounded to 24 bits: 2e-6), and the
+# partial sums of at most 2^17 terms are added in a tree of depth ~17 over threads, CTAs and
+# slots, each step rounding by 6e-8.  All of it is relative to the sum, so ln(sum) moves by at
+# most a few 1e-6; the reference itself (m in base 2, times ln 2) rounds at |lse| * 6e-8 <= 1e-6.
+LSE_TOL = 1e-4
+
+
+def _run(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, kernel=0, sink=0, window=0, plan=0, want_lse=True):
     import paper_2502_20330_b200 as R
     B, Rr, Hq, D = q.shape
     Hkv, Lmax = k.shape[1], k.shape[2]
     ws = R.new_workspace(R.attention_workspace_bytes(B, Hq, Hkv, D, Lmax, gamma))
     out = torch.empty_like(q)
-    lse = torch.empty(B, Rr, Hq, dtype=torch.float32, device=q.device)
+    lse = torch.empty(B, Rr, Hq, dtype=torch.float32, device=q.device) if want_lse else None
     o32 = torch.empty(B, Rr, Hq, D, dtype=torch.float32, device=q.device)
-    R.rapid_verify_attention(q, k, v, ctx, gamma, out, ws,
-                             R.AttnParams(scale=scale, num_ctas=num_ctas, lse_out=lse, out_f32=o32, kernel=kernel))
+    params = R.AttnParams(scale=scale, num_ctas=num_ctas, lse_out=lse, out_f32=o32, kernel=kernel,
+                          sink_keys=sink, window_keys=window, plan=plan)
+    if plan:
+        R.rapid_attention_plan(ctx, gamma, B, Hq, Hkv, D, Lmax, ws, params)
+        if plan == R.PLAN_SETTLED:      # some other kernel between the plan and the call
+            torch.zeros(8, device=q.device).add_(1.0)
+    R.rapid_verify_attention(q, k, v, ctx, gamma, out, ws, params)
     torch.cuda.synchronize()
     return out, lse, o32, R.workspace_status(ws)
 
 
-def _oracle(q, k, v, ctx, gamma, scale=0.0, units=None):
+def _oracle(q, k, v, ctx, gamma, scale=0.0, units=None, sink=0, window=0):
     return oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx.cpu().numpy(), gamma,
-                                   scale=scale, units=units)
+                                   scale=scale, units=units, sink=sink, window=window)
 
 
-def _lse_tolerance(q, k, kernel):
-    """Absolute tolerance of the natural-log sum-exp.  The row sums add fp32 probabilities (1e-3 covers
-    their rounding over 128K keys), except on the keys-on-M kernel from 49 to 64 grouped rows, whose
-    threads have no registers for a tile of fp32 probabilities and add the bf16 values the tensor
-    cores multiply: where one key dominates a row, its rounding (bf16 keeps 8 significant bits, so up
-    to 2^-8 relative) shows in full."""
-    grouped_rows = q.shape[2] // k.shape[1] * q.shape[1]
-    wide_keys_on_m = kernel != 1 and q.shape[3] == 128 and 48 < grouped_rows <= 64
-    return 2.0 ** -8 + 5e-4 if wide_keys_on_m else 1e-3
-
-
-def _compare(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, units=None, kernel=0):
-    out, lse, o32, status = _run(q, k, v, ctx, gamma, num_ctas, scale, kernel)
+def _compare(q, k, v, ctx, gamma, num_ctas=0, scale=0.0, units=None, kernel=0, sink=0, window=0, plan=0,
+             want_lse=True):
+    out, lse, o32, status = _run(q, k, v, ctx, gamma, num_ctas, scale, kernel, sink, window, plan, want_lse)
     assert status == 0
-    ref, ref_lse = _oracle(q, k, v, ctx, gamma, scale, units)
+    ref, ref_lse = _oracle(q, k, v, ctx, gamma, scale, units, sink, window)
     rows = ~np.isnan(ref_lse)
     rep = parity.check_attention(out.float().cpu().numpy(), ref, rows)
     parity.check_attention(o32.cpu().numpy(), ref, rows)
-    assert np.abs(lse.cpu().numpy()[rows] - ref_lse[rows]).max() < _lse_tolerance(q, k, kernel)
+    if want_lse:
+        rep["max_lse_err"] = float(np.abs(lse.cpu().numpy()[rows] - ref_lse[rows]).max())
+        assert rep["max_lse_err"] < LSE_TOL, rep
     return rep, out, o32
 
 
@@ -76,6 +84,8 @@ def test_shapes_against_oracle(Hq, Hkv, D, gamma, L):
     q, k, v, ctx = wl.attention_inputs(cfg, seed=2, device="cuda", poison_padding=True)
     _compare(q, k, v, ctx, gamma)
     _compare(q, k, v, ctx, gamma, kernel=1)
+    # without the log-sum-exp output (49 to 64 rows then run one softmax group with bf16 row sums)
+    _compare(q, k, v, ctx, gamma, want_lse=False)
 
 
 @pytest.mark.parametrize("Hq,Hkv,gamma,L,num_ctas", [
@@ -182,34 +192,50 @@ def test_argument_errors():
     assert R.attention_workspace_bytes(1, 64, 1, 128, 128, 8) == 0        # 576 grouped rows
 
 
-def test_llama8b_32k_sampled_rows():
-    """The 32K workload in the bench's launch configuration; the oracle checks a sample of rows."""
+def _check_every_row(q, k, v, ctx, gamma, variants):
+    """Every row of a full-size workload against the oracle (one oracle pass, several device runs)."""
+    ref, ref_lse = _oracle(q, k, v, ctx, gamma)
+    for kw in variants:
+        out, lse, o32, status = _run(q, k, v, ctx, gamma, **kw)
+        assert status == 0
+        rep = parity.check_attention(out.float().cpu().numpy(), ref)
+        parity.check_attention(o32.cpu().numpy(), ref)
+        assert rep["rows"] == ref_lse.size
+        assert np.abs(lse.cpu().numpy() - ref_lse).max() < LSE_TOL
+
+
+def test_llama8b_32k_every_row():
+    """The 32K workload in the bench's launch configuration (the library's choice there is one cluster
+    per KV head), and the two kernels with a merge launch."""
     cfg = wl.CONFIGS["llama8b_32k"]
     q, k, v, ctx = wl.attention_inputs(cfg, seed=10, device="cuda")
-    units = np.array([0, 8, 37, 100, 143, 200, 287], dtype=np.int64)
-    _compare(q, k, v, ctx, cfg.gamma, units=units)
+    _check_every_row(q, k, v, ctx, cfg.gamma, [dict(), dict(kernel=2), dict(kernel=1), dict(kernel=3),
+                                               dict(plan=2), dict(kernel=2, plan=1)])
 
 
-def test_llama8b_128k_and_70b_sampled_rows():
+def test_llama8b_128k_and_70b_every_row():
     for name in ("llama8b_128k", "llama70b_128k"):
         cfg = wl.CONFIGS[name]
         q, k, v, ctx = wl.attention_inputs(cfg, seed=11, device="cuda")
-        n_units = cfg.B * cfg.Hq * cfg.R
-        units = np.array([0, 8, n_units // 2 + 3, n_units - 1], dtype=np.int64)
-        _compare(q, k, v, ctx, cfg.gamma, units=units)
         if name == "llama8b_128k":
-            _compare(q, k, v, ctx, cfg.gamma, units=units, kernel=1)
+            variants = [dict(), dict(plan=2), dict(kernel=1), dict(kernel=3)]
         else:
-            _compare(q, k, v, ctx, cfg.gamma, units=units, kernel=2)   # two softmax groups at full size
+            variants = [dict(), dict(plan=2), dict(kernel=2)]   # kernel 2: two softmax groups at full size
+        _check_every_row(q, k, v, ctx, cfg.gamma, variants)
         del q, k, v
 
 
-def test_ragged_qwen_batch_sampled_rows():
+def test_ragged_qwen_batch_every_row():
     cfg = wl.CONFIGS["qwen7b_ragged"]
     q, k, v, ctx = wl.attention_inputs(cfg, seed=12, device="cuda", poison_padding=True)
-    n_units = cfg.B * cfg.Hq * cfg.R
-    units = np.arange(3, n_units, n_units // 9, dtype=np.int64)
-    _compare(q, k, v, ctx, cfg.gamma, units=units)
+    _check_every_row(q, k, v, ctx, cfg.gamma, [dict(), dict(plan=2), dict(kernel=1, plan=1)])
+
+
+def test_drafter_8k_every_row():
+    """The drafter-side one-row decode over the retrieved context (gamma = 0)."""
+    cfg = wl.CONFIGS["drafter_8k"]
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=13, device="cuda")
+    _check_every_row(q, k, v, ctx, cfg.gamma, [dict(), dict(kernel=2), dict(kernel=3, plan=2), dict(kernel=1)])
 
 
 def test_random_shapes_and_lengths():
@@ -271,3 +297,159 @@ def test_many_units_per_cta(B, Hq, Hkv, D, gamma, lo, hi, num_ctas):
     rng = np.random.default_rng(B)
     units = rng.choice(B * Hq * (gamma + 1), size=min(96, B * Hq * (gamma + 1)), replace=False).astype(np.int64)
     _compare(q, k, v, ctx, gamma, num_ctas=num_ctas, units=units)
+
+
+# ---- one cluster per (sequence, KV head), merged on chip ----------------------------------------------------
+
+def test_cluster_merge_random_sweep():
+    """Seeded sweep of the cluster variant: every column count up to 96 rows, ragged batches with poisoned
+    padding (units whose cluster has more CTAs than tiles), lengths below one tile, planted large scores.
+    A shape whose clusters do not fit on the device together must be refused, not run."""
+    import paper_2502_20330_b200 as R
+    rng = np.random.default_rng(11)
+    layouts = [(8, 2), (16, 2), (32, 8), (64, 8), (28, 4), (72, 8), (12, 12), (96, 8), (5, 1), (48, 8)]
+    ran = 0
+    for trial in range(70):
+        Hq, Hkv = layouts[int(rng.integers(len(layouts)))]
+        G = Hq // Hkv
+        gamma = int(rng.integers(0, min(11, 96 // G - 1) + 1))
+        B = int(rng.integers(1, 4))
+        Lmax = int(rng.integers(gamma + 1, 6000))
+        lens = tuple(int(rng.integers(gamma + 1, Lmax + 1)) for _ in range(B))
+        cfg = wl.VerifyConfig("cl", B=B, Hq=Hq, Hkv=Hkv, D=128, gamma=gamma, V=4096, ctx_lens=lens, Lmax=Lmax)
+        q, k, v, ctx = wl.attention_inputs(cfg, seed=3000 + trial, device="cuda", poison_padding=True)
+        if rng.random() < 0.3:
+            j = int(rng.integers(0, max(1, min(lens) - 1)))
+            k[:, :, j:j + 3] *= float(rng.choice([4.0, 8.0]))
+        try:
+            _, _, o32 = _compare(q, k, v, ctx, gamma, kernel=3)
+        except R.RapidError as e:
+            assert e.code == 2 and "fit" in str(e)
+            continue
+        ran += 1
+        if trial % 7 == 0:
+            _, _, again, _ = _run(q, k, v, ctx, gamma, kernel=3)
+            assert torch.equal(o32, again)             # bit-identical from run to run
+            _compare(q, k, v, ctx, gamma, kernel=3, plan=1)
+    assert ran >= 40
+
+
+def test_cluster_merge_paged_and_no_lse():
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("clp", B=1, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(5000,), Lmax=5120)
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=71, device="cuda", poison_padding=True)
+    ref, _ = _oracle(q, k, v, ctx, cfg.gamma)
+    for bs in (64, 256):
+        kp, vp, table = wl.paged_layout(k, v, ctx.cpu(), bs, seed=5)
+        ws = R.new_workspace(R.attention_workspace_bytes(1, 32, 8, 128, table.shape[1] * bs, cfg.gamma))
+        out = torch.empty_like(q)
+        R.rapid_verify_attention_paged(q, kp, vp, table, ctx, cfg.gamma, out, ws, R.AttnParams(kernel=3))
+        torch.cuda.synchronize()
+        assert R.workspace_status(ws) == 0
+        parity.check_attention(out.float().cpu().numpy(), ref)
+
+
+# ---- plans -------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kernel", [0, 1, 2])
+@pytest.mark.parametrize("plan", [1, 2])
+def test_planned_calls_match_unplanned_bit_for_bit(kernel, plan):
+    cfg = wl.VerifyConfig("pl", B=3, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(4100, 9, 1111), Lmax=4200)
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=41, device="cuda", poison_padding=True)
+    for num_ctas in (0, 5, 300):
+        a = _run(q, k, v, ctx, cfg.gamma, num_ctas=num_ctas, kernel=kernel)
+        b = _run(q, k, v, ctx, cfg.gamma, num_ctas=num_ctas, kernel=kernel, plan=plan)
+        assert a[3] == 0 and b[3] == 0
+        assert torch.equal(a[2], b[2]) and torch.equal(a[1], b[1])
+
+
+def test_one_plan_serves_many_layers_and_a_stale_plan_is_flagged():
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("pl", B=2, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(9000, 5000))
+    B, Hq, Hkv, D, gamma = cfg.B, cfg.Hq, cfg.Hkv, cfg.D, cfg.gamma
+    layers = [wl.attention_inputs(cfg, seed=50, device="cuda", layer=i) for i in range(3)]
+    ctx = layers[0][3]
+    ws = R.new_workspace(R.attention_workspace_bytes(B, Hq, Hkv, D, 9000, gamma))
+    R.rapid_attention_plan(ctx, gamma, B, Hq, Hkv, D, 9000, ws)
+    outs = []
+    for i, (q, k, v, _) in enumerate(layers):
+        out = torch.empty_like(q)
+        R.rapid_verify_attention(q, k, v, ctx, gamma, out, ws, R.AttnParams(plan=1 if i == 0 else 2))
+        outs.append(out)
+    torch.cuda.synchronize()
+    assert R.workspace_status(ws) == 0
+    for (q, k, v, _), out in zip(layers, outs):
+        ref, _ = _oracle(q, k, v, ctx, gamma)
+        parity.check_attention(out.float().cpu().numpy(), ref)
+    # the lengths move on (a step was committed) but the caller forgets to plan again
+    ctx2 = ctx.clone(); ctx2[1] -= 3
+    q, k, v, _ = layers[0]
+    R.rapid_verify_attention(q, k, v, ctx2, gamma, torch.empty_like(q), ws, R.AttnParams(plan=2))
+    torch.cuda.synchronize()
+    assert R.workspace_status(ws) & R.STATUS_STALE_PLAN
+    # ... and a plan made for another split
+    R.workspace_init(ws)
+    R.rapid_attention_plan(ctx, gamma, B, Hq, Hkv, D, 9000, ws, R.AttnParams(num_ctas=64))
+    R.rapid_verify_attention(q, k, v, ctx, gamma, torch.empty_like(q), ws, R.AttnParams(plan=1))
+    torch.cuda.synchronize()
+    assert R.workspace_status(ws) & R.STATUS_STALE_PLAN
+
+
+# ---- sink + window visibility ------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("Hq,Hkv,D,gamma,lens,sink,window", [
+    (32, 8, 128, 8, (20000, 700), 4, 4092),        # the streaming drafter's budget over a long cache
+    (32, 8, 128, 8, (5000, 4100), 4, 1000),
+    (32, 8, 128, 8, (3000, 300), 0, 257),          # no sinks; the second sequence lies inside the window
+    (64, 8, 128, 8, (6000, 2000), 130, 500),       # 72 rows (rows on M); sinks spill into a second tile
+    (28, 4, 128, 4, (9000, 5), 7, 1),              # a window of one key: each row sees the sinks and itself
+    (8, 2, 64, 4, (4096, 1000), 4, 600),           # head_dim 64
+    (64, 8, 128, 6, (7000, 1500), 64, 128),        # 56 rows; sink and window on tile boundaries
+])
+def test_sink_and_window_mask(Hq, Hkv, D, gamma, lens, sink, window):
+    cfg = wl.VerifyConfig("sw", B=len(lens), Hq=Hq, Hkv=Hkv, D=D, gamma=gamma, V=4096, ctx_lens=lens)
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=60, device="cuda", poison_padding=True)
+    # Keys no row sees: their K may hold anything (a hidden score is never used), and so may the V of
+    # the 128-key tiles that lie wholly in the hidden middle (those tiles are not read at all).  The V
+    # rows of hidden keys that share a tile with visible ones are cache content like any other: finite.
+    for b, L in enumerate(lens):
+        lo, hi = sink, L - (gamma + 1) - window + 1
+        if hi > lo:
+            k[b, :, lo:hi] = float("nan")
+            tlo, thi = (lo + 127) // 128 * 128, hi // 128 * 128
+            if thi > tlo:
+                v[b, :, tlo:thi] = float("nan")
+    kernels = [0, 1] + ([2] if D == 128 and Hq // Hkv * (gamma + 1) <= 96 else [])
+    for kernel in kernels:
+        for num_ctas in (0, 3):
+            _compare(q, k, v, ctx, gamma, num_ctas=num_ctas, kernel=kernel, sink=sink, window=window)
+    _compare(q, k, v, ctx, gamma, sink=sink, window=window, plan=1)
+    if D == 128 and Hq // Hkv * (gamma + 1) <= 96:
+        _compare(q, k, v, ctx, gamma, kernel=3, sink=sink, window=window)
+
+
+def test_window_over_a_128k_cache_reads_only_what_is_visible():
+    """4 sinks + 4,092 recent keys over a 128K cache: parity on every row with the hidden keys poisoned."""
+    cfg = wl.CONFIGS["llama8b_128k"]
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=61, device="cuda")
+    L, R = 131072, cfg.R
+    hi = L - R - 4092 + 1                      # the oldest key of row 0's window
+    k[:, :, 4:hi] = float("nan"); v[:, :, 128:hi // 128 * 128] = float("nan")   # V: the tiles never read
+    ref, ref_lse = _oracle(q, k, v, ctx, cfg.gamma, sink=4, window=4092)
+    for kw in (dict(), dict(kernel=1), dict(kernel=3)):
+        out, lse, o32, status = _run(q, k, v, ctx, cfg.gamma, sink=4, window=4092, **kw)
+        assert status == 0
+        parity.check_attention(out.float().cpu().numpy(), ref)
+        assert np.abs(lse.cpu().numpy() - ref_lse).max() < LSE_TOL
+
+
+def test_window_argument_errors():
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("t", B=1, Hq=8, Hkv=2, D=128, gamma=2, V=4096, ctx_lens=(128,))
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=9, device="cuda")
+    ws = R.new_workspace(R.attention_workspace_bytes(1, 8, 2, 128, 128, 2))
+    for bad in (dict(sink_keys=4), dict(window_keys=-1), dict(sink_keys=-1, window_keys=5),
+                dict(window_keys=5, all_keys_visible=True), dict(plan=7)):
+        with pytest.raises(R.RapidError) as e:
+            R.rapid_verify_attention(q, k, v, ctx, 2, torch.empty_like(q), ws, R.AttnParams(**bad))
+        assert e.value.code == 1

@@ -54,3 +54,36 @@ def test_single_process_is_the_identity():
     import bench
     assert bench.max_over_ranks(1.25) == 1.25
     assert bench.rank_seed(7, 0) == 7
+
+
+def _spawned(results):
+    """What bench.py's own launcher hands every rank: the environment a torchrun rank would see."""
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    assert os.environ["MASTER_ADDR"] == "127.0.0.1" and int(os.environ["LOCAL_RANK"]) == rank
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        results[rank] = bench.max_over_ranks(10.0 * (rank + 1))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_bench_starts_its_own_ranks_without_a_launcher():
+    sys.path.insert(0, ROOT)
+    import bench
+    with mp.Manager() as mgr:
+        results = mgr.dict()
+        bench.spawn_ranks(2, _spawned, (results,))
+        assert dict(results) == {0: 20.0, 1: 20.0}
+
+
+def test_both_arms_print_the_same_config():
+    sys.path.insert(0, ROOT)
+    import bench
+    import workloads as wl
+    cfg = wl.CONFIGS["qwen7b_ragged"]
+    ctx = wl.context_lengths(cfg, 2025)
+    a = bench.config_dict(cfg, ctx, 1)
+    assert a == bench.config_dict(cfg, ctx, 1) and a["workload"] == "qwen7b_ragged" and "model" not in a
+    assert a["kv_bytes_per_step"] == 4 * cfg.Hkv * cfg.D * int(ctx.sum())
