@@ -102,7 +102,7 @@ typedef struct rapid_attn_shape {
                                          sequence with a cache capacity of at most 65,536 keys.              */
 
 /* rapid_attn_params.plan */
-#define RAPID_PLAN_NONE 0    /* every kernel works its share out from ctx_lens (default)                    */
+#define RAPID_PLAN_NONE 0    /* the call plans for itself: one more tiny kernel ahead of its own (default)    */
 #define RAPID_PLAN_READY 1   /* the workspace holds a plan made by rapid_attention_plan for this call's
                                 geometry and for the current ctx_lens                                      */
 #define RAPID_PLAN_SETTLED 2 /* as RAPID_PLAN_READY, and at least one other kernel (or a synchronisation)
@@ -222,6 +222,25 @@ int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cac
 int rapid_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
                          const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
                          void* cuda_stream);
+
+/*
+ * What rapid_verify_attention would launch for this geometry and these params on the current
+ * device (nothing is launched; pointers inside params are only looked at for being NULL or not).
+ */
+typedef struct rapid_attn_launch_info {
+    int32_t kernel;           /* RAPID_ATTN_KERNEL_ROWS_ON_M, _KEYS_ON_M or _CLUSTER_MERGE                 */
+    int32_t kernels_per_call; /* 2 = split + merge, 1 = merged on chip                                   */
+    int32_t ctas;             /* CTAs of the split kernel                                                */
+    int32_t cluster_size;     /* CTAs per thread-block cluster; 0 = launched without clusters            */
+    int32_t softmax_groups;   /* groups of four softmax warps per CTA                                    */
+    int32_t columns;          /* grouped rows as the MMAs see them: padded to a multiple of 16 columns
+                                 (keys on M) or to 64 / 128 rows (rows on M)                             */
+    int32_t max_clusters[4];  /* keys-on-M kernel: clusters of 16, 8, 4, 2 CTAs that fit on the device
+                                 together (0 where that does not apply)                                  */
+} rapid_attn_launch_info;
+
+int rapid_attention_describe(const rapid_attn_shape* shape, int gamma, const rapid_attn_params* params,
+                             rapid_attn_launch_info* info);
 
 /*
  * Combines P partial attention results of the same rows over disjoint sets of keys -- the context

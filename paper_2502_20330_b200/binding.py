@@ -24,7 +24,7 @@ RESIDUAL_PHAT = 1
 
 EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
-    "rapid_workspace_status", "rapid_verify_attention", "rapid_attention_plan", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_retrieval_select", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_attention_plan", "rapid_attention_describe", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_retrieval_select", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
     "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_kv_append_paged", "rapid_step_commit",
     "rapid_last_error",
@@ -56,6 +56,12 @@ class _AttnParams(ctypes.Structure):
                 ("split_done_event", ctypes.c_void_p), ("all_keys_visible", ctypes.c_int32),
                 ("kernel", ctypes.c_int32), ("sink_keys", ctypes.c_int32), ("window_keys", ctypes.c_int32),
                 ("plan", ctypes.c_int32), ("reserved", ctypes.c_int32), ("wait_cycle_limit", ctypes.c_int64)]
+
+
+class _LaunchInfo(ctypes.Structure):
+    _fields_ = [("kernel", ctypes.c_int32), ("kernels_per_call", ctypes.c_int32), ("ctas", ctypes.c_int32),
+                ("cluster_size", ctypes.c_int32), ("softmax_groups", ctypes.c_int32), ("columns", ctypes.c_int32),
+                ("max_clusters", ctypes.c_int32 * 4)]
 
 
 class _AcceptShape(ctypes.Structure):
@@ -129,6 +135,9 @@ def load_library():
         lib.rapid_verify_attention.argtypes = attn_args + [vp, sz, vp]
         lib.rapid_attention_plan.restype = i32
         lib.rapid_attention_plan.argtypes = [vp, i32, ctypes.POINTER(_AttnShape), ctypes.POINTER(_AttnParams), vp, sz, vp]
+        lib.rapid_attention_describe.restype = i32
+        lib.rapid_attention_describe.argtypes = [ctypes.POINTER(_AttnShape), i32, ctypes.POINTER(_AttnParams),
+                                                 ctypes.POINTER(_LaunchInfo)]
         lib.rapid_verify_attention_paged.restype = i32
         lib.rapid_verify_attention_paged.argtypes = [vp, vp, vp, vp, ctypes.POINTER(_PagedKv)] + attn_args[3:] + [vp, sz, vp]
         lib.rapid_draft_sample.restype = i32
@@ -294,6 +303,17 @@ def rapid_attention_plan(ctx_lens, gamma, B, Hq, Hkv, D, Lmax, workspace, params
     shape = _AttnShape(B, Hq, Hkv, D, Lmax, 0, 0, 0)
     _check(load_library().rapid_attention_plan(_p(ctx_lens), gamma, ctypes.byref(shape), _attn_params(params),
                                                _p(workspace), _nbytes(workspace), _stream_ptr(stream)))
+
+
+def rapid_attention_describe(B, Hq, Hkv, D, Lmax, gamma, params: Optional[AttnParams] = None) -> dict:
+    """What an attention call of this geometry would launch on the current device (see include/rapid.h)."""
+    shape = _AttnShape(B, Hq, Hkv, D, Lmax, 0, 0, 0)
+    info = _LaunchInfo()
+    _check(load_library().rapid_attention_describe(ctypes.byref(shape), gamma, _attn_params(params), ctypes.byref(info)))
+    return {"kernel": info.kernel, "kernels_per_call": info.kernels_per_call, "ctas": info.ctas,
+            "cluster_size": info.cluster_size, "softmax_groups": info.softmax_groups, "columns": info.columns,
+            "max_clusters": {16: info.max_clusters[0], 8: info.max_clusters[1], 4: info.max_clusters[2],
+                             2: info.max_clusters[3]}}
 
 
 def rapid_verify_attention_paged(q, k_pool, v_pool, block_table, ctx_lens, gamma, out, workspace,

@@ -244,6 +244,12 @@ int rapid_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_sh
                                  static_cast<cudaStream_t>(cuda_stream));
 }
 
+int rapid_attention_describe(const rapid_attn_shape* shape, int gamma, const rapid_attn_params* params,
+                             rapid_attn_launch_info* info) {
+    clear_error();
+    return describe_attention(shape, gamma, params, info);
+}
+
 int rapid_verify_attention_paged(const void* q, const void* k_pool, const void* v_pool,
                                  const int32_t* block_table, const rapid_paged_kv* paged,
                                  const int32_t* ctx_lens, int gamma, void* out,

@@ -60,12 +60,16 @@ struct AttnArgs {
     int pad;
     int kt_half_blocks;  // keys-on-M kernel over a paged cache with 64-key blocks: two boxes per tile
     int tile_keys;  // keys per scheduling tile: what plan, walk and merge count in (64, or 128 for the keys-on-M kernel)
+    int tile_log2;  // log2(tile_keys)
     // Sink + window visibility (window > 0): row i sees the keys below `sink` and the `window`
     // newest keys up to its own, (lim_i - window, lim_i].  Tiles no row sees are not streamed.
     int sink, window;
-    // A plan made by attention_plan_kernel for the same geometry and lengths (plan_mode != 0):
-    // every CTA's walk and every unit's range of partial slots, read instead of computed.
+    // The plan attention_plan_kernel wrote for this geometry and these lengths: every CTA's walk and
+    // every unit's range of partial slots.  plan_mode says how old it is: RAPID_PLAN_READY = made by
+    // the kernel just before this call's, RAPID_PLAN_SETTLED = at least two kernels ago.  (A call
+    // without a caller's plan launches the plan kernel itself and runs with RAPID_PLAN_READY.)
     int plan_mode;
+    int caller_plan;  // the caller supplied the plan: check it against the call's geometry and lengths
     const Walk* plan_walks;
     const int2* plan_units;  // (first CTA, number of slots) of every unit
     const int32_t* plan_ctx;  // the lengths the plan was made for
@@ -96,7 +100,7 @@ constexpr int kPlanSigInts = 16;
 __device__ __forceinline__ int clamp_len(int L, int R, int Lmax) {
     return L < R ? R : (L > Lmax ? Lmax : L);
 }
-__device__ __forceinline__ int tiles_of(int L, int tile_keys) { return (L + tile_keys - 1) / tile_keys; }
+__device__ __forceinline__ int tiles_of(const AttnArgs& a, int L) { return (L + a.tile_keys - 1) >> a.tile_log2; }
 
 // The tiles a unit of L keys streams: all of them, or, with a window, the tiles that hold sink
 // keys and the tiles from the oldest key of row 0's window on (the rows' windows end at their own
@@ -106,14 +110,14 @@ struct UnitGeom {
 };
 __device__ __forceinline__ UnitGeom unit_geom(const AttnArgs& a, int L) {
     UnitGeom g;
-    const int full = tiles_of(L, a.tile_keys);
+    const int full = tiles_of(a, L);
     g.nt = full;
     g.ns = full;
     g.gap = 0;
     if (a.window > 0) {
         const int w0 = L - a.R - a.window + 1;          // the oldest key row 0 sees through its window
-        const int ns = tiles_of(a.sink, a.tile_keys);   // tiles that hold sink keys
-        const int tw0 = w0 > 0 ? w0 / a.tile_keys : 0;  // the tile that key lives in
+        const int ns = tiles_of(a, a.sink);             // tiles that hold sink keys
+        const int tw0 = w0 > 0 ? w0 >> a.tile_log2 : 0;  // the tile that key lives in
         if (tw0 > ns) {
             g.ns = ns;
             g.gap = tw0 - ns;
@@ -162,6 +166,9 @@ __device__ __forceinline__ void walk_set_unit(const AttnArgs& a, Walk& w, int b)
 // Range of CTA c of n in the padded flat list: [c*Tv/n, (c+1)*Tv/n); its real tiles are what it works on.
 // With one cluster per unit (cmerge): CTA c is rank c % cmerge of the cluster of unit c / cmerge and
 // takes an equal share of that unit's tiles.
+// (Only the plan kernel runs this.  The split kernels read what it wrote: the 64-bit divisions here
+// are tens of kilobytes of code, and a split kernel that carries them no longer shares the SMs'
+// instruction cache with the merge kernel, which costs every launch several microseconds.)
 __device__ __forceinline__ void plan_cta(const AttnArgs& a, int cta, Walk& w) {
     w.b = 0;
     w.kvh = 0;
@@ -271,14 +278,14 @@ __device__ __forceinline__ void fill_plan_sig(const AttnArgs& a, int KS, int32_t
 
 // Checks of CTA 0 that only the device can make: every length inside [Lmin, Lmax], and, when a
 // plan is used, that it was made for this geometry and for these lengths.
-__device__ __forceinline__ void check_call_inputs(const AttnArgs& a, int KS) {
+__device__ __noinline__ void check_call_inputs(const AttnArgs& a, int KS) {
     bool bad = false, stale = false;
     for (int b = 0; b < a.B; ++b) {
         const int L = a.ctx_lens[b];
         bad |= (L < a.Lmin) || (L > a.Lmax);
-        if (a.plan_mode) stale |= __ldcg(a.plan_ctx + b) != L;
+        if (a.caller_plan) stale |= __ldcg(a.plan_ctx + b) != L;
     }
-    if (a.plan_mode) {
+    if (a.caller_plan) {
         int32_t sig[kPlanSigInts];
         fill_plan_sig(a, KS, sig);
         for (int i = 0; i < kPlanSigInts; ++i) stale |= __ldcg(a.plan_sig + i) != sig[i];
@@ -289,8 +296,10 @@ __device__ __forceinline__ void check_call_inputs(const AttnArgs& a, int KS) {
 
 // Writes the plan of a call into its workspace: one block; thread c plans CTA c, thread u the
 // slot range of unit u.
-__global__ void __launch_bounds__(512) attention_plan_kernel(const AttnArgs a, int KS, Walk* walks, int2* units,
+__global__ void __launch_bounds__(512) attention_plan_kernel(const __grid_constant__ AttnArgs a, int KS, Walk* walks, int2* units,
                                                              int32_t* ctx_copy, int32_t* sig_out) {
+    griddep_wait();               // the lengths may come from the kernel just before this one
+    griddep_launch_dependents();  // the split kernel may run its prologue; it reads the plan after its own wait
     const int n_ctas = a.cmerge ? a.B * a.Hkv * a.cmerge : a.num_ctas;
     for (int c = threadIdx.x; c < n_ctas; c += blockDim.x) {
         Walk w;
@@ -374,8 +383,7 @@ __device__ __forceinline__ void split_kernel_walk(const AttnArgs& a, int cta, Wa
     if (!settled) {
         if (threadIdx.x == 0) {
             Walk t;
-            if (a.plan_mode) load_walk(a, cta, t);
-            else plan_cta(a, cta, t);
+            load_walk(a, cta, t);
             *s_walk = t;
         }
         __syncthreads();
@@ -427,7 +435,7 @@ template <int D, int MR>
 __global__ void __launch_bounds__(kTcThreads, 1)
 verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                               const __grid_constant__ CUtensorMap tmV,
-                              const __grid_constant__ CUtensorMap tmQ, const AttnArgs a,
+                              const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ AttnArgs a,
                               const TcLayout lay) {
     constexpr int BLK = kTile * 128;  // bytes of one 64-key x 64-column block
     constexpr int NHALF = D / 64;
@@ -678,20 +686,16 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                 tmem_ld_x32(tS + 32, sr[1]);
                 tmem_wait_ld();
 
-                if (key0 + kTile - 1 > all_see) {  // causal rows and the ragged end of the context
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-#pragma unroll
-                        for (int k = 0; k < 32; ++k)
-                            if (key0 + h * 32 + k > lim) sr[h][k] = __float_as_uint(-INFINITY);
-                }
-                if (key0 <= lo_max && key0 + kTile > a.sink) {  // the old edge of the windows
+                // causal rows and the ragged end of the context, or the old edge of the windows: a key is
+                // hidden from this row if it lies past lim or inside [hid0, lo]
+                if (key0 + kTile - 1 > all_see || (key0 <= lo_max && key0 + kTile > a.sink)) {
+                    const int hid0 = a.window > 0 ? a.sink : 0x7fffffff;
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
 #pragma unroll
                         for (int k = 0; k < 32; ++k) {
                             const int key = key0 + h * 32 + k;
-                            if (key >= a.sink && key <= lo) sr[h][k] = __float_as_uint(-INFINITY);
+                            if (key > lim || (key >= hid0 && key <= lo)) sr[h][k] = __float_as_uint(-INFINITY);
                         }
                 }
 
@@ -822,7 +826,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
 // result does not depend on timing.
 template <int D>
 __global__ void __launch_bounds__(128)
-verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* lse_out,
+verify_attn_merge_kernel(const __grid_constant__ AttnArgs a, int KS, __nv_bfloat16* out, float* lse_out,
                          float* out_f32) {
     constexpr int VEC = D / 32;
     constexpr int UN = 10;
@@ -835,11 +839,11 @@ verify_attn_merge_kernel(const AttnArgs a, int KS, __nv_bfloat16* out, float* ls
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
 
-    // The unit's slots: from the plan, or from the lengths.  Both are read before the wait although
-    // an earlier kernel of the stream may have written them: this kernel starts only after every
-    // CTA of the split kernel has passed its own wait (it lets its dependents launch after it),
-    // and by then everything before the split kernel has completed.
-    const int2 range = a.plan_mode ? __ldcg(a.plan_units + unit) : unit_slot_range(a, unit, KS);
+    // The unit's slots, from the plan.  It is read before the wait although an earlier kernel of the
+    // stream wrote it: this kernel starts only after every CTA of the split kernel has passed its own
+    // wait (it lets its dependents launch after it), and by then everything before the split kernel,
+    // the plan kernel included, has completed.
+    const int2 range = __ldcg(a.plan_units + unit);
     const int c_first = range.x;
     const int nslots = range.y;
     const size_t slot_stride = (size_t)slot_floats(a.GR, D);
@@ -1079,66 +1083,71 @@ bool attn_shape_ok(const rapid_attn_shape* s, int gamma) {
 // Largest cluster (16, 8, 4, 2) of this kernel of which `clusters_needed` fit on the device at once;
 // 0 if none does.  Asked of the runtime once per device, kernel and size.
 // Per-device attributes of a keys-on-M kernel: its dynamic shared memory, and clusters of 16 CTAs.
-template <int NC, int SG>
+template <int NC, int SG, bool WIN>
 cudaError_t kt_configure(int dev) {
     constexpr int smem = kt::smem_bytes(NC);
     static_assert(smem <= kMaxSmemOptin - 4096, "shared memory (dynamic + the kernel's static arrays)");
     static bool configured[64] = {};
     if (dev >= 0 && dev < 64 && configured[dev]) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC, SG>,
+    cudaError_t e = cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC, SG, WIN>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC, SG>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    e = cudaFuncSetAttribute(kt::verify_attn_splitkv_kt_kernel<NC, SG, WIN>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
     return cudaSuccess;
 }
 
-template <int NC, int SG>
-int kt_cluster_size_that_fits(int clusters_needed, int dev) {
+// Clusters of `size` CTAs (16, 8, 4 or 2) of this kernel that can be resident on the device together;
+// 0 if none.  Asked of the runtime once per device, kernel and size.
+template <int NC, int SG, bool WIN = false>
+int kt_resident_clusters(int size, int dev) {
     constexpr int smem = kt::smem_bytes(NC);
-    if (kt_configure<NC, SG>(dev) != cudaSuccess) {
-        cudaGetLastError();
-        return 0;
-    }
-    static int resident[64][4] = {};  // clusters of 16, 8, 4, 2 CTAs resident together (0 = not asked yet, -1 = none)
-    const int sizes[4] = {16, 8, 4, 2};
-    if (dev < 0 || dev >= 64) return 0;
-    for (int i = 0; i < 4; ++i) {
-        if (!resident[dev][i]) {
+    static int resident[64][4] = {};  // by size 16, 8, 4, 2 (0 = not asked yet, -1 = none)
+    const int i = size == 16 ? 0 : size == 8 ? 1 : size == 4 ? 2 : size == 2 ? 3 : -1;
+    if (dev < 0 || dev >= 64 || i < 0) return 0;
+    if (!resident[dev][i]) {
+        int n = 0;
+        if (kt_configure<NC, SG, WIN>(dev) == cudaSuccess) {
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(sizes[i]);
+            cfg.gridDim = dim3(size);
             cfg.blockDim = dim3(kt::threads(SG));
             cfg.dynamicSmemBytes = smem;
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = sizes[i];
+            attr[0].val.clusterDim.x = size;
             attr[0].val.clusterDim.y = 1;
             attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr;
             cfg.numAttrs = 1;
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, kt::verify_attn_splitkv_kt_kernel<NC, SG>, &cfg) != cudaSuccess) {
-                cudaGetLastError();
-                n = 0;
-            }
-            resident[dev][i] = n > 0 ? n : -1;
+            if (cudaOccupancyMaxActiveClusters(&n, kt::verify_attn_splitkv_kt_kernel<NC, SG, WIN>, &cfg) != cudaSuccess) n = 0;
         }
-        if (resident[dev][i] >= clusters_needed) return sizes[i];
+        cudaGetLastError();
+        resident[dev][i] = n > 0 ? n : -1;
     }
+    return resident[dev][i] > 0 ? resident[dev][i] : 0;
+}
+
+// Largest cluster of which `clusters_needed` fit on the device at once; 0 if none does.
+template <int NC, int SG, bool WIN = false>
+int kt_cluster_size_that_fits(int clusters_needed, int dev) {
+    const int sizes[4] = {16, 8, 4, 2};
+    for (int i = 0; i < 4; ++i)
+        if (kt_resident_clusters<NC, SG, WIN>(sizes[i], dev) >= clusters_needed) return sizes[i];
     return 0;
 }
 
-template <int NC, int SG = 1>
-int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ, AttnArgs& a,
-                    cudaStream_t stream, bool want_cluster, bool need_cluster) {
+template <int NC, int SG, bool WIN>
+int launch_split_kt_w(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ, AttnArgs& a,
+                      cudaStream_t stream, bool want_cluster, bool need_cluster) {
     constexpr int smem = kt::smem_bytes(NC);
     int dev = 0;
     RAPID_CUDA_CHECK(cudaGetDevice(&dev));
-    RAPID_CUDA_CHECK((kt_configure<NC, SG>(dev)));
+    RAPID_CUDA_CHECK((kt_configure<NC, SG, WIN>(dev)));
     const int units = a.B * a.Hkv;
     a.cmerge = 0;
     if (want_cluster) {
+        // (the kernel with and without the window mask take the same resources: one answer for both)
         const int cs = kt_cluster_size_that_fits<NC, SG>(units, dev);
         // on the library's own choice the clusters must also cover most of the machine
         if (cs && (need_cluster || units * cs * 4 >= sm_count() * 3)) a.cmerge = cs;
@@ -1165,9 +1174,16 @@ int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
         attr[1].val.clusterDim.z = 1;
         cfg.numAttrs = 2;
     }
-    RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kt::verify_attn_splitkv_kt_kernel<NC, SG>, tmK, tmV, tmQ,
+    RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kt::verify_attn_splitkv_kt_kernel<NC, SG, WIN>, tmK, tmV, tmQ,
                                         static_cast<const AttnArgs&>(a)));
     return RAPID_OK;
+}
+
+template <int NC, int SG = 1>
+int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ, AttnArgs& a,
+                    cudaStream_t stream, bool want_cluster, bool need_cluster) {
+    return a.window > 0 ? launch_split_kt_w<NC, SG, true>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster)
+                        : launch_split_kt_w<NC, SG, false>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
 }
 
 // fp32_sums: the caller takes the log-sum-exp, so the row sums must add fp32 probabilities.  With
@@ -1242,8 +1258,9 @@ struct AttnCall {
 
 int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
                       const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
-                      const rapid_paged_kv* paged, const int32_t* block_table, AttnCall& c) {
-    if (!ctx_lens || !shape) {
+                      const rapid_paged_kv* paged, const int32_t* block_table, AttnCall& c,
+                      bool describe_only = false) {
+    if ((!ctx_lens && !describe_only) || !shape) {
         set_error("%s: NULL argument", who);
         return RAPID_ERR_INVALID_ARG;
     }
@@ -1305,7 +1322,7 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
         return RAPID_ERR_UNSUPPORTED;
     }
     const WsLayout lay = ws_layout(s.B, s.Hkv, GR, s.D);
-    if (!workspace || workspace_bytes < lay.total || ((uintptr_t)workspace & 255)) {
+    if (!describe_only && (!workspace || workspace_bytes < lay.total || ((uintptr_t)workspace & 255))) {
         set_error("%s: workspace of %zu bytes needed (256-byte aligned), got %zu", who, lay.total, workspace_bytes);
         return RAPID_ERR_WORKSPACE;
     }
@@ -1372,7 +1389,7 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
 
     AttnArgs& a = c.a;
     a = AttnArgs{};
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint8_t* ws = static_cast<uint8_t*>(describe_only ? nullptr : workspace);
     a.ctx_lens = ctx_lens;
     a.partial = reinterpret_cast<float*>(ws + lay.partial);
     a.status = reinterpret_cast<int32_t*>(ws);
@@ -1391,12 +1408,14 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
     a.tile_shift = tile_shift;
     a.kt_half_blocks = c.kt_half_blocks ? 1 : 0;
     a.tile_keys = c.kt_path ? kt::kKeys : kTile;
+    a.tile_log2 = c.kt_path ? 7 : 6;
     a.pad = c.kt_path ? 5 : unit_switch_tiles(s.D);
     a.stair = all_visible ? 0 : R;
     a.Lmin = all_visible ? 1 : R;
     a.sink = window > 0 ? sink : 0;
     a.window = window;
     a.plan_mode = plan_mode;
+    a.caller_plan = plan_mode != RAPID_PLAN_NONE;
     a.plan_sig = reinterpret_cast<const int32_t*>(ws + lay.sig);
     a.plan_walks = reinterpret_cast<const Walk*>(ws + lay.walks);
     a.plan_units = reinterpret_cast<const int2*>(ws + lay.units);
@@ -1414,6 +1433,19 @@ size_t attention_workspace_bytes(const rapid_attn_shape* s, int gamma) {
     const int64_t GR = (int64_t)(s->Hq / s->Hkv) * (gamma + 1);
     if (GR > 128) return 0;
     return ws_layout(s->B, s->Hkv, (int)GR, s->D).total;
+}
+
+// Clusters of `size` CTAs of the keys-on-M kernel that serves this call, resident together.
+static int kt_max_clusters(const AttnCall& c, int size, int dev) {
+    switch (c.NC) {
+        case 1: return kt_resident_clusters<1, 1>(size, dev);
+        case 2: return kt_resident_clusters<2, 1>(size, dev);
+        case 3: return kt_resident_clusters<3, 1>(size, dev);
+        case 4: return c.fp32_sums ? kt_resident_clusters<4, 2>(size, dev) : kt_resident_clusters<4, 1>(size, dev);
+        case 5: return kt_resident_clusters<5, 2>(size, dev);
+        case 6: return kt_resident_clusters<6, 2>(size, dev);
+    }
+    return 0;
 }
 
 // The cluster size a keys-on-M call of this geometry would run with (0 = no cluster).
@@ -1435,6 +1467,49 @@ static int cluster_size_for(const AttnCall& c) {
     return cs;
 }
 
+int describe_attention(const rapid_attn_shape* shape, int gamma, const rapid_attn_params* params,
+                       rapid_attn_launch_info* info) {
+    if (!info) {
+        set_error("rapid_attention_describe: NULL info");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    AttnCall c;
+    int rc = prepare_attention("rapid_attention_describe", nullptr, gamma, shape, params, nullptr, 0, nullptr, nullptr,
+                               c, true);
+    if (rc != RAPID_OK) return rc;
+    *info = rapid_attn_launch_info{};
+    const int cs = cluster_size_for(c);
+    const int units = c.a.B * c.a.Hkv;
+    info->kernel = !c.kt_path ? RAPID_ATTN_KERNEL_ROWS_ON_M : (cs ? RAPID_ATTN_KERNEL_CLUSTER_MERGE : RAPID_ATTN_KERNEL_KEYS_ON_M);
+    info->kernels_per_call = cs ? 1 : 2;
+    info->ctas = cs ? units * cs : c.a.num_ctas;
+    info->cluster_size = cs;
+    info->softmax_groups = c.kt_path ? ((c.NC > 4 || (c.NC == 4 && c.fp32_sums)) ? 2 : 1) : 2;
+    info->columns = c.kt_path ? 16 * c.NC : (c.a.GR <= 64 ? 64 : 128);
+    if (c.kt_path) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) {
+            const int sizes[4] = {16, 8, 4, 2};
+            for (int i = 0; i < 4; ++i) info->max_clusters[i] = kt_max_clusters(c, sizes[i], dev);
+        }
+    }
+    if (c.need_cluster && !cs) {
+        set_error("rapid_attention_describe: the clusters of this call do not fit on the device together");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    return RAPID_OK;
+}
+
+static int launch_plan_kernel(const AttnCall& c, void* workspace, int D, cudaStream_t stream) {
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const WsLayout lay = ws_layout(c.a.B, c.a.Hkv, c.a.GR, D);
+    RAPID_CUDA_CHECK(launch_dependent(attention_plan_kernel, dim3(1), dim3(512), 0, stream, c.a, c.KS,
+                                      reinterpret_cast<Walk*>(ws + lay.walks), reinterpret_cast<int2*>(ws + lay.units),
+                                      reinterpret_cast<int32_t*>(ws + lay.ctx), reinterpret_cast<int32_t*>(ws + lay.sig)));
+    count_launch(1);
+    return RAPID_OK;
+}
+
 int launch_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
                           const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
                           cudaStream_t stream) {
@@ -1450,15 +1525,7 @@ int launch_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_s
         set_error("rapid_attention_plan: the clusters of this call do not fit on the device together");
         return RAPID_ERR_UNSUPPORTED;
     }
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
-    const WsLayout lay = ws_layout(c.a.B, c.a.Hkv, c.a.GR, shape->D);
-    attention_plan_kernel<<<1, 512, 0, stream>>>(c.a, c.KS, reinterpret_cast<Walk*>(ws + lay.walks),
-                                                 reinterpret_cast<int2*>(ws + lay.units),
-                                                 reinterpret_cast<int32_t*>(ws + lay.ctx),
-                                                 reinterpret_cast<int32_t*>(ws + lay.sig));
-    RAPID_CUDA_CHECK(cudaGetLastError());
-    count_launch(1);
-    return RAPID_OK;
+    return launch_plan_kernel(c, workspace, shape->D, stream);
 }
 
 int launch_verify_attention(const void* q, const void* k_cache, const void* v_cache,
@@ -1497,6 +1564,14 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     rc = make_q_map(&tmQ, q, s, a.G, a.R);
     if (rc != RAPID_OK) return rc;
 
+    if (!a.caller_plan) {
+        // no plan from the caller: make one now (a tiny kernel ahead of the split kernel, which reads
+        // it after its grid-dependency wait)
+        a.cmerge = cluster_size_for(c);
+        rc = launch_plan_kernel(c, workspace, s.D, stream);
+        if (rc != RAPID_OK) return rc;
+        a.plan_mode = RAPID_PLAN_READY;
+    }
     if (c.kt_path) {
         rc = dispatch_split_kt(c.NC, c.fp32_sums, tmK, tmV, tmQ, a, stream, c.want_cluster, c.need_cluster);
     } else if (a.GR <= 64)

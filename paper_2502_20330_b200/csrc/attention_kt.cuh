@@ -128,11 +128,13 @@ __device__ __forceinline__ float warp_sum32(float v) {
 // group g forms the probabilities of columns [g N/SG, (g+1) N/SG) for all 128 keys of a tile, keeps
 // those rows' references and sums and rescales and reads out those columns of O^T; the groups meet
 // only at the P^T barrier (PV starts when both have published) and at the end of a unit.
-template <int NC, int SG = 1>
+// WIN = the call has a sink + window mask (a kernel of its own, so that calls without one carry none
+// of its code: the kernel's instruction footprint shows in every launch).
+template <int NC, int SG = 1, bool WIN = false>
 __global__ void __launch_bounds__(threads(SG), 1)
 verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                               const __grid_constant__ CUtensorMap tmV,
-                              const __grid_constant__ CUtensorMap tmQ, const AttnArgs a) {
+                              const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ AttnArgs a) {
     constexpr int D = 128;
     constexpr int N = NC * 16;
     constexpr int NG = N / SG;             // columns per softmax group
@@ -219,7 +221,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
                 for (int t = 0; t < seg && ok; ++t, ++jj) {
                     const int ks = jj % NK, vs = jj % NV;
-                    const int tile = real_tile(w, w.tile + t);
+                    const int tile = WIN ? real_tile(w, w.tile + t) : w.tile + t;
                     // a tile is one box of 128 keys, or, for a paged cache with 64-key blocks, two
                     // boxes of 64 keys from two physical blocks (parts = 2)
                     const int parts = a.kt_half_blocks ? 2 : 1;
@@ -374,7 +376,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
             for (int ti = 0; ti < seg; ++ti, ++jj) {
                 const int b = jj & 1;
                 const uint32_t tS = tmem_base + lane_base + COL_S + 128u * b + C0;
-                const int key0 = real_tile(w, w.tile + ti) * kKeys;  // the tile's first key
+                const int key0 = (WIN ? real_tile(w, w.tile + ti) : w.tile + ti) * kKeys;  // the tile's first key
                 const int key = key0 + t;
                 // Row i sees keys <= L-R+i and rows are column i*G+g, so the columns the causal stair
                 // hides from this key are a prefix [0, cmin) (no stair: every row sees every key
@@ -383,9 +385,11 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 const int over_ctx = a.stair ? key - (L - a.R) : 0;
                 const int cmin = key >= L ? N : (over_ctx > 0 ? over_ctx * a.G : 0);
                 int cmax = N;
-                if (a.window > 0 && key >= a.sink) {
-                    const long long rows_in = (long long)key - (L - a.R) + a.window;
-                    cmax = rows_in <= 0 ? 0 : (rows_in * a.G >= N ? N : (int)rows_in * a.G);
+                if constexpr (WIN) {
+                    if (key >= a.sink) {
+                        const long long rows_in = (long long)key - (L - a.R) + a.window;
+                        cmax = rows_in <= 0 ? 0 : (rows_in * a.G >= N ? N : (int)rows_in * a.G);
+                    }
                 }
                 ok &= warp_wait_bounded(&s_full[b], (jj >> 1) & 1, wc);
                 tc_fence_after_sync();
@@ -396,8 +400,34 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                 constexpr bool kPacked = NG > 48;
                 float pv[kPacked ? 2 : NG];
                 uint32_t pq[kPacked ? NG / 2 : 1];
+                // the same for every thread: no key of the tile is hidden from any row
+                const bool tile_clear = key0 + kKeys <= L - a.stair &&
+                                        (!WIN || key0 + kKeys <= a.sink || key0 > L - 1 - a.window);
                 bool move = ti == 0;
-                if (ti > 0) {
+                if (ti == 0 && tile_clear) {
+                    // A unit's first tile, seen whole by every row: the scores of its first key serve as
+                    // the references (any reference will do as long as no visible score sits far above
+                    // it, which the pass below finds out).  That spares this tile the row maxima over its
+                    // 128 keys, the longest stretch of code a CTA would otherwise run before its pipeline
+                    // is full.
+                    if (wq == 0) {
+#pragma unroll
+                        for (int ch = 0; ch < NG / CH; ++ch) {
+                            uint32_t sr[CH];
+                            tmem_ld_cols<CH>(tS + CH * ch, sr);
+                            tmem_wait_ld();
+                            if (lane == 0) {
+#pragma unroll
+                                for (int e = 0; e < CH; ++e) {
+                                    const int col = C0 + CH * ch + e;
+                                    sh_mref[col] = col < a.GR ? __uint_as_float(sr[e]) * c : INFINITY;
+                                }
+                            }
+                        }
+                    }
+                    bar_softmax(grp);
+                }
+                if (ti > 0 || tile_clear) {
                     // MASKED = false for a tile every row sees whole (all of a long context but its end):
                     // no per-column predicate.  Columns past the grouped rows need none either: their
                     // scores are 0 (zero rows of Q) and their reference is +inf, so they come out as 0.
@@ -418,7 +448,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                                               fmaf(__uint_as_float(sr[e + 3]), c, -m.w)};
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) {
-                                    if (MASKED) x[i] = (col + i >= cmin && col + i < cmax) ? x[i] : -INFINITY;
+                                    if (MASKED) x[i] = (col + i >= cmin && (!WIN || col + i < cmax)) ? x[i] : -INFINITY;
                                     far |= x[i] > kJump;
                                     x[i] = fast_exp2(x[i]);
                                 }
@@ -433,9 +463,6 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         }
                         return far;
                     };
-                    // the same for every thread: no key of the tile is hidden from any row
-                    const bool tile_clear = key0 + kKeys <= L - a.stair &&
-                                            (a.window <= 0 || key0 + kKeys <= a.sink || key0 > L - 1 - a.window);
                     move = tile_clear ? first_pass(std::false_type{}) : first_pass(std::true_type{});
                     move = bar_softmax_or(grp, move);
                 }
@@ -454,7 +481,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
                         for (int e = 0; e < CH; ++e) {
                             const int col = C0 + CH * ch + e;
-                            const float v = (col >= cmin && col < cmax && col < a.GR) ? __uint_as_float(sr[e]) * c : -INFINITY;
+                            const float v = (col >= cmin && (!WIN || col < cmax) && col < a.GR) ? __uint_as_float(sr[e]) * c : -INFINITY;
                             const float wm = warp_max32(v);
                             if (lane == 0) sh_w[wq][col] = wm;
                         }
@@ -496,8 +523,8 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         for (int e = 0; e < CH; e += 2) {
                             const int li = CH * ch + e, col = C0 + li;
                             const float m0 = sh_mref[col], m1 = sh_mref[col + 1];
-                            const float x0 = (col >= cmin && col < cmax) ? fmaf(__uint_as_float(sr[e]), c, m0 == -INFINITY ? 0.f : -m0) : -INFINITY;
-                            const float x1 = (col + 1 >= cmin && col + 1 < cmax) ? fmaf(__uint_as_float(sr[e + 1]), c, m1 == -INFINITY ? 0.f : -m1) : -INFINITY;
+                            const float x0 = (col >= cmin && (!WIN || col < cmax)) ? fmaf(__uint_as_float(sr[e]), c, m0 == -INFINITY ? 0.f : -m0) : -INFINITY;
+                            const float x1 = (col + 1 >= cmin && (!WIN || col + 1 < cmax)) ? fmaf(__uint_as_float(sr[e + 1]), c, m1 == -INFINITY ? 0.f : -m1) : -INFINITY;
                             const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                             if (kPacked) {
                                 pq[li >> 1] = pack_bf16x2(p0, p1);

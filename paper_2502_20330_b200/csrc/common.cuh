@@ -60,6 +60,8 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
 int launch_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
                           const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
                           cudaStream_t stream);
+int describe_attention(const rapid_attn_shape* shape, int gamma, const rapid_attn_params* params,
+                       rapid_attn_launch_info* info);
 int launch_retrieval_select(const float* chunk_emb, const float* query_emb, const int32_t* n_chunks, int B,
                             int Nmax, int Dm, float threshold, int k, float* scores_out, int32_t* sel_idx,
                             int32_t* sel_count, int32_t* status_word, cudaStream_t stream);
@@ -157,7 +159,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
 // first (a bulk copy it issued, the MMAs it committed): the abort flag does not end it, only the
 // barrier or the library's own limit does.  Such work always completes, so this returns true
 // unless the hardware has stopped.
-__device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity) {
+static __device__ __noinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity) {
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (clock64() - t0 > kWaitCycleLimit) return false;

@@ -28,7 +28,7 @@ def test_verify_step_chains_both_calls():
     R.kernel_launch_count_reset()
     R.rapid_verify_step(q, k, v, ctx, cfg.gamma, out, aws, z, d, tok, u, cfg.eta, alen, ntok, cws)
     torch.cuda.synchronize()
-    assert R.kernel_launch_count() == 3  # split, merge, accept
+    assert R.kernel_launch_count() == 4  # plan, split, merge, accept
     ref, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx.cpu().numpy(), cfg.gamma)
     parity.check_attention(out.float().cpu().numpy(), ref)
     parity.check_accept(z.cpu().numpy(), d.cpu().numpy(), tok.cpu().numpy(), u.cpu().numpy(), cfg.eta, 1.0, 0.1, 0,
