@@ -160,6 +160,12 @@ typedef struct rapid_accept_params {
     int32_t residual_mode; /* RAPID_RESIDUAL_*                                                  */
     int32_t reserved;
     float* ratio_out;      /* device [B, gamma] fp32: phat(x')/q(x') of every position, or NULL */
+    /* What the drafter already knows about its own rows (Algorithm 1, the drafting loop: x'_j is drawn
+       from q_j, so q_j's normaliser and q_j(x'_j) existed once): rapid_draft_sample returns both, and a
+       caller that kept them spares the accept step the reductions over the draft rows.  Either may be
+       NULL; the values must belong to the same draft_logits and temperature.                          */
+    const float* draft_row_stats; /* device [B, gamma, 2] fp32: (max_v d_v/T, log sum_v exp(d_v/T)), or NULL */
+    const float* draft_logq;      /* device [B, gamma] fp32: natural log of q(x') at the draft token, or NULL */
 } rapid_accept_params;
 
 /* ---- workspaces ---------------------------------------------------------------------------- */
@@ -353,7 +359,7 @@ int rapid_draft_sample(const float* draft_logits, const float* uniforms, float t
  * uniforms and the two output arrays, but has nowhere to put the per-row
  * ratios and candidate tokens the accept kernel leaves for its epilogue.
  *
- * Here that scratch is a fixed array inside the library image (about 5 KB,
+ * Here that scratch is a fixed array inside the library image (7,168 bytes,
  * resident on every GPU that loads the library until the process ends).  The
  * computation, the kernels and the results are those of rapid_accept.
  *

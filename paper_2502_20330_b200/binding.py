@@ -72,7 +72,7 @@ class _AcceptShape(ctypes.Structure):
 class _AcceptParams(ctypes.Structure):
     _fields_ = [("temperature", ctypes.c_float), ("tail_alpha", ctypes.c_float),
                 ("residual_mode", ctypes.c_int32), ("reserved", ctypes.c_int32),
-                ("ratio_out", ctypes.c_void_p)]
+                ("ratio_out", ctypes.c_void_p), ("draft_row_stats", ctypes.c_void_p), ("draft_logq", ctypes.c_void_p)]
 
 
 @dataclass
@@ -97,6 +97,8 @@ class AcceptParams:
     tail_alpha: float = 0.1
     residual_mode: int = RESIDUAL_PAPER
     ratio_out: Optional[torch.Tensor] = None  # [B,gamma] float32
+    draft_row_stats: Optional[torch.Tensor] = None  # [B,gamma,2] float32: rapid_draft_sample's out_row_stats
+    draft_logq: Optional[torch.Tensor] = None       # [B,gamma] float32: rapid_draft_sample's out_logq
 
 
 _lib = None
@@ -234,8 +236,13 @@ def _accept_shape(target_logits: torch.Tensor, draft_logits: torch.Tensor) -> _A
 def _accept_params(p: Optional[AcceptParams]):
     if p is None:
         return None
+    for t in (p.draft_row_stats, p.draft_logq):
+        if t is not None and (t.dtype != torch.float32 or not t.is_contiguous()):
+            raise TypeError("draft_row_stats and draft_logq must be dense float32")
     return ctypes.byref(_AcceptParams(p.temperature, p.tail_alpha, p.residual_mode, 0,
-                                      p.ratio_out.data_ptr() if p.ratio_out is not None else None))
+                                      p.ratio_out.data_ptr() if p.ratio_out is not None else None,
+                                      p.draft_row_stats.data_ptr() if p.draft_row_stats is not None else None,
+                                      p.draft_logq.data_ptr() if p.draft_logq is not None else None))
 
 
 def attention_workspace_bytes(B, Hq, Hkv, D, Lmax, gamma) -> int:

@@ -1,8 +1,8 @@
 // Accept / residual step (Algorithm 1, validation loop and residual draw; Eq. (new_target);
 // tail rule of Section 2.4), vocabulary-parallel, in ONE launch.
 //
-// A thread-block cluster of kCluster CTAs owns one logit row (one draft position of one sequence,
-// or the bonus row).  Each CTA reads its 1/kCluster slice of the target and the draft row from
+// A thread-block cluster of 16 (or 8) CTAs owns one logit row (one draft position of one sequence,
+// or the bonus row).  Each CTA reads its slice of the target and the draft row from
 // global memory exactly once, keeps it in shared memory, and the cluster then walks the steps of
 // Algorithm 1 over those resident slices, exchanging a few floats through distributed shared
 // memory between the steps:
@@ -20,6 +20,8 @@
 #include <cooperative_groups.h>
 #include <math.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace cg = cooperative_groups;
@@ -28,11 +30,12 @@ namespace rapid {
 
 namespace {
 
-constexpr int kThreads = 512;
-constexpr int kWarps = kThreads / 32;
-constexpr int kCluster = 8;
-constexpr int kMaxSlice = 24576;  // floats of one array a CTA keeps: 2 * 96 KiB of shared memory
-constexpr int kBatch = 4;         // float4 loads per thread and array in flight together
+// A portable cluster of 8 CTAs of 1024 threads per row.  (The kernel is written for any cluster size
+// and thread count; a cluster of 16 CTAs of 512 threads, which puts the nine rows of gamma = 8 on 144
+// SMs instead of 72, measured the same 20 us: the kernel's time is the chain of its barriers and
+// exchanges, not the work between them.)
+constexpr int kClusterPortable = 8, kThreadsPortable = 1024;
+constexpr int kMaxSlice = 24576;  // floats of one array a CTA keeps: 2 * 96 KiB
 
 struct AcceptArgs {
     const float* z;  // target logits [B, R, V]
@@ -48,6 +51,8 @@ struct AcceptArgs {
     int32_t* cand;     // [B*R] candidate token of every row; bit 31 = drawn from p as a fallback
     float* logq_out;   // optional [B]: natural log of the drawn token's probability (gamma = 0 calls)
     float* stats_out;  // optional [B, 2]: max and log-sum-exp of the row's logits / T (gamma = 0 calls)
+    const float* d_stats;  // optional [B, gamma, 2]: (max, log-sum-exp) of every draft row / T, natural log
+    const float* d_logq;   // optional [B, gamma]: natural log of q at the draft token
     int B, gamma, R, V;
     int slice;  // entries per CTA (multiple of 4)
     int per;    // consecutive entries per thread in the search (odd: conflict-free shared reads)
@@ -70,25 +75,32 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-// Block-wide maximum / sum of two values at once, in a fixed order; sh holds 2 * kWarps floats.
+// Block-wide maximum / sum of two values at once, in a fixed order: every warp reduces by shuffles,
+// warp 0 reduces the NW <= 32 warp results the same way, everybody reads the two totals.  sh holds
+// 2 * NW + 2 floats.
+template <int NW>
 __device__ __forceinline__ void block_max2(float& x, float& y, float* sh) {
     x = warp_max(x);
     y = warp_max(y);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    __syncthreads();
+    __syncthreads();  // the previous use of sh has been read
     if (lane == 0) {
         sh[warp] = x;
-        sh[kWarps + warp] = y;
+        sh[NW + warp] = y;
     }
     __syncthreads();
-    x = sh[0];
-    y = sh[kWarps];
-#pragma unroll
-    for (int i = 1; i < kWarps; ++i) {
-        x = fmaxf(x, sh[i]);
-        y = fmaxf(y, sh[kWarps + i]);
+    if (warp == 0) {
+        const float a = warp_max(lane < NW ? sh[lane] : -INFINITY), b = warp_max(lane < NW ? sh[NW + lane] : -INFINITY);
+        if (lane == 0) {
+            sh[2 * NW] = a;
+            sh[2 * NW + 1] = b;
+        }
     }
+    __syncthreads();
+    x = sh[2 * NW];
+    y = sh[2 * NW + 1];
 }
+template <int NW>
 __device__ __forceinline__ void block_sum2(float& x, float& y, float* sh) {
     x = warp_sum(x);
     y = warp_sum(y);
@@ -96,16 +108,19 @@ __device__ __forceinline__ void block_sum2(float& x, float& y, float* sh) {
     __syncthreads();
     if (lane == 0) {
         sh[warp] = x;
-        sh[kWarps + warp] = y;
+        sh[NW + warp] = y;
     }
     __syncthreads();
-    x = 0.f;
-    y = 0.f;
-#pragma unroll
-    for (int i = 0; i < kWarps; ++i) {
-        x += sh[i];
-        y += sh[kWarps + i];
+    if (warp == 0) {
+        const float a = warp_sum(lane < NW ? sh[lane] : 0.f), b = warp_sum(lane < NW ? sh[NW + lane] : 0.f);
+        if (lane == 0) {
+            sh[2 * NW] = a;
+            sh[2 * NW + 1] = b;
+        }
     }
+    __syncthreads();
+    x = sh[2 * NW];
+    y = sh[2 * NW + 1];
 }
 
 __device__ __forceinline__ float max4(const float4& v) { return fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)); }
@@ -120,37 +135,42 @@ __device__ __forceinline__ float warp_incl_scan(float v) {
     return v;
 }
 
-// Every CTA of the cluster publishes one float4 and gets all kCluster of them, in rank order.
-// Each step of the kernel uses its own slot, so a slot is never rewritten while a peer reads it.
-__device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, float4* slot,
-                                                 float4* gathered, float4 mine) {
-    if (threadIdx.x == 0) *slot = mine;
+// Every CTA of the cluster hands one float4 to all of them: thread r < CL of CTA c stores it
+// into slot[c] of CTA r's shared memory (a distributed-shared-memory store), and the cluster barrier
+// that follows makes all CL stores visible everywhere.  Each step of the kernel uses a slot
+// array of its own, so none is rewritten while a peer may still read it.
+template <int CL>
+__device__ __forceinline__ void cluster_publish(cg::cluster_group& cluster, float4* slots, int my_rank, float4 mine) {
+    if (threadIdx.x < CL) cluster.map_shared_rank(slots, threadIdx.x)[my_rank] = mine;
     cluster.sync();
-    if (threadIdx.x < kCluster) gathered[threadIdx.x] = *cluster.map_shared_rank(slot, threadIdx.x);
-    __syncthreads();
 }
 
 // Combine the per-CTA (max, sum relative to that max) pairs of a row, in rank order.
+template <int CL>
 __device__ __forceinline__ void combine_ms(const float4* g, bool second, float& M, float& S) {
     M = -INFINITY;
 #pragma unroll
-    for (int r = 0; r < kCluster; ++r) M = fmaxf(M, second ? g[r].z : g[r].x);
+    for (int r = 0; r < CL; ++r) M = fmaxf(M, second ? g[r].z : g[r].x);
     S = 0.f;
 #pragma unroll
-    for (int r = 0; r < kCluster; ++r) {
+    for (int r = 0; r < CL; ++r) {
         const float m = second ? g[r].z : g[r].x, s = second ? g[r].w : g[r].y;
         S += (m == -INFINITY) ? 0.f : s * exp2f(m - M);
     }
 }
 
-// NV4 = float4 groups a thread owns in each array (group i belongs to thread i % kThreads).
-template <int NV4>
-__global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptArgs a) {
+// CL = CTAs per cluster (= per row), NT = threads per CTA, NV4 = float4 groups a thread owns in each
+// array (group i belongs to thread i % NT).
+template <int CL, int NT, int NV4>
+__global__ void __launch_bounds__(NT, 2048 / NT / 2) accept_fused_kernel(const AcceptArgs a) {
+    constexpr int NW = NT / 32;
     extern __shared__ __align__(16) float slice_mem[];
-    __shared__ float4 xch[3];
-    __shared__ float4 gath[3][kCluster];
-    __shared__ float sh_red[2 * kWarps];
+    __shared__ float4 gath[3][CL];
+    __shared__ float sh_red[2 * NW + 2];
+    __shared__ float sh_ms[4];
     __shared__ int sh_tok, sh_last, sh_final;
+    __shared__ int sh_tl;       // the draft token's place in this CTA's slice, or -1
+    __shared__ float sh_pq[2];  // p and q at the draft token, kept by the thread that forms them
 
     cg::cluster_group cluster = cg::this_cluster();
     const int c = (int)cluster.block_rank();
@@ -166,25 +186,51 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
     const float4* z = reinterpret_cast<const float4*>(a.z + (size_t)row * a.zs + v0);
     const float4* d = draft ? reinterpret_cast<const float4*>(a.d + (size_t)drow * a.ds + v0) : nullptr;
     const float c2 = a.inv_T_log2;
+    // the drafter's own statistics of this row, if the caller kept them: the row's maximum and sum
+    // need not be found again
+    const bool have_dstats = draft && a.d_stats != nullptr;
 
+    // Distributed shared memory may be written only once every CTA of the cluster is running: each
+    // CTA says so here and waits for the others just before its first store into a peer.
+    cluster.barrier_arrive();
     griddep_wait();  // the logits may come from the kernel just before this one
     griddep_launch_dependents();
 
+    // The draft token and the two logits at it are needed late (step 2), by one thread, on the CTA's
+    // critical path: thread 0 asks for them now, so that they arrive while step 0 runs.
+    int tok = 0;
+    float z_tok = 0.f, d_tok = 0.f, lq_given = 0.f;
+    bool tok_here = false;
+    if (draft && tid == 0) {
+        tok = a.tokens[drow];
+        if (tok < 0 || tok >= a.V) {
+            if (c == 0) atomicOr(a.status, RAPID_STATUS_BAD_DRAFT_TOKEN);
+            tok = tok < 0 ? 0 : a.V - 1;
+        }
+        tok_here = tok >= v0 && tok < v1;
+        if (tok_here) {
+            z_tok = __ldg(a.z + (size_t)row * a.zs + tok);
+            if (a.d_logq) lq_given = __ldg(a.d_logq + drow);
+            else d_tok = __ldg(a.d + (size_t)drow * a.ds + tok);
+        }
+    }
+    if (tid == 0) sh_tl = tok_here ? tok - v0 : -1;  // read after the block reductions of step 0
+
     // ---- step 0: the only pass over global memory; p = softmax(z/T), q = softmax(d/T) ----
-    float mz = -INFINITY, md = -INFINITY;
+    // every load of the thread is in flight before the first is used
+    float sz = 0.f, sd = 0.f, mz = -INFINITY, md = -INFINITY;
+    {
+        float4 xz[NV4], xd[NV4];
 #pragma unroll
-    for (int k0 = 0; k0 < NV4; k0 += kBatch) {
-        float4 xz[kBatch], xd[kBatch];
-#pragma unroll
-        for (int e = 0; e < kBatch; ++e) {
-            const int i = (k0 + e) * kThreads + tid;
+        for (int e = 0; e < NV4; ++e) {
+            const int i = e * NT + tid;
             const bool ok = i < n4;
             xz[e] = ok ? __ldg(z + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
             xd[e] = (ok && draft) ? __ldg(d + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
         }
 #pragma unroll
-        for (int e = 0; e < kBatch; ++e) {
-            const int i = (k0 + e) * kThreads + tid;
+        for (int e = 0; e < NV4; ++e) {
+            const int i = e * NT + tid;
             if (i < n4) {
                 zc[i] = xz[e];
                 if (draft) dc[i] = xd[e];
@@ -192,39 +238,51 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
             mz = fmaxf(mz, max4(xz[e]));
             md = fmaxf(md, max4(xd[e]));
         }
-    }
-    block_max2(mz, md, sh_red);
-    // slice maxima in base-2 units (scaling by log2(e)/T > 0 keeps the order); an empty or all -inf
-    // slice contributes (-inf, 0)
-    const float Mzb = mz * c2, Mdb = md * c2;
-    const float refz = (mz == -INFINITY) ? 0.f : Mzb, refd = (md == -INFINITY) ? 0.f : Mdb;
-    float sz = 0.f, sd = 0.f;
+        block_max2<NW>(mz, md, sh_red);
+        // slice maxima in base-2 units (scaling by log2(e)/T > 0 keeps the order); an empty or all -inf
+        // slice contributes (-inf, 0)
+        const float refz = (mz == -INFINITY) ? 0.f : mz * c2, refd = (md == -INFINITY) ? 0.f : md * c2;
 #pragma unroll
-    for (int kk = 0; kk < NV4; ++kk) {
-        const int i = kk * kThreads + tid;
-        if (i < n4) {
-            const float4 x = zc[i];
-            sz += fast_exp2(fmaf(x.x, c2, -refz)) + fast_exp2(fmaf(x.y, c2, -refz)) +
-                  fast_exp2(fmaf(x.z, c2, -refz)) + fast_exp2(fmaf(x.w, c2, -refz));
-            if (draft) {
-                const float4 y = dc[i];
-                sd += fast_exp2(fmaf(y.x, c2, -refd)) + fast_exp2(fmaf(y.y, c2, -refd)) +
-                      fast_exp2(fmaf(y.z, c2, -refd)) + fast_exp2(fmaf(y.w, c2, -refd));
-            }
+        for (int e = 0; e < NV4; ++e) {
+            sz += fast_exp2(fmaf(xz[e].x, c2, -refz)) + fast_exp2(fmaf(xz[e].y, c2, -refz)) +
+                  fast_exp2(fmaf(xz[e].z, c2, -refz)) + fast_exp2(fmaf(xz[e].w, c2, -refz));
+            if (draft && !have_dstats)
+                sd += fast_exp2(fmaf(xd[e].x, c2, -refd)) + fast_exp2(fmaf(xd[e].y, c2, -refd)) +
+                      fast_exp2(fmaf(xd[e].z, c2, -refd)) + fast_exp2(fmaf(xd[e].w, c2, -refd));
         }
     }
-    block_sum2(sz, sd, sh_red);
-    cluster_exchange(cluster, &xch[0], gath[0], make_float4(mz == -INFINITY ? -INFINITY : Mzb, sz,
-                                                            md == -INFINITY ? -INFINITY : Mdb, sd));
+    block_sum2<NW>(sz, sd, sh_red);
+    const float Mzb = mz * c2, Mdb = md * c2;
+    cluster.barrier_wait();  // every CTA of the cluster has started
+    cluster_publish<CL>(cluster, gath[0], c, make_float4(mz == -INFINITY ? -INFINITY : Mzb, sz,
+                                                     md == -INFINITY ? -INFINITY : Mdb, sd));
     // p = 2^(z * c2 - Mz) / Sz, q = 2^(d * c2 - Md) / Sd.  The row maximum is taken off inside the
     // fused multiply-add, before anything is rounded, and the normaliser is applied as a factor:
     // at a low temperature the scaled logits are in the hundreds, and a constant folded from
     // Mz + log2 Sz would be rounded at that magnitude, scaling every p of the row by the same
     // 1 + 1e-5 -- more than the whole residual mass when p and phat nearly coincide.  This way the
     // top entry is exactly 1/Sz, and phat's top entry exactly 1/Sy.
-    float Mz, Sz, Md = 0.f, Sd = 1.f;
-    combine_ms(gath[0], false, Mz, Sz);
-    if (draft) combine_ms(gath[0], true, Md, Sd);
+    if (warp == 0) {  // one warp combines the eight (max, sum) pairs; everybody reads the result
+        float Mz_, Sz_, Md_ = 0.f, Sd_ = 1.f;
+        combine_ms<CL>(gath[0], false, Mz_, Sz_);
+        if (draft) {
+            if (have_dstats) {
+                const float mx = __ldg(a.d_stats + 2 * drow), lse = __ldg(a.d_stats + 2 * drow + 1);
+                Md_ = mx * 1.4426950408889634f;
+                Sd_ = exp2f((lse - mx) * 1.4426950408889634f);
+            } else {
+                combine_ms<CL>(gath[0], true, Md_, Sd_);
+            }
+        }
+        if (lane == 0) {
+            sh_ms[0] = Mz_;
+            sh_ms[1] = Sz_;
+            sh_ms[2] = Md_;
+            sh_ms[3] = Sd_;
+        }
+    }
+    __syncthreads();
+    const float Mz = sh_ms[0], Sz = sh_ms[1], Md = sh_ms[2], Sd = sh_ms[3];
     const float iSz = 1.f / Sz, iSd = 1.f / Sd;
 
     float sw = 0.f, sp = 0.f;
@@ -234,9 +292,10 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
         // p and q replace the logits in shared memory; y stays in registers
         float ev[NV4 * 4];
         float my = -INFINITY, unused = -INFINITY;
+        const int tl = sh_tl;
 #pragma unroll
         for (int kk = 0; kk < NV4; ++kk) {
-            const int i = kk * kThreads + tid;
+            const int i = kk * NT + tid;
             if (i < n4) {
                 const float4 x = zc[i], y = dc[i];
                 const float lp[4] = {fmaf(x.x, c2, -Mz), fmaf(x.y, c2, -Mz), fmaf(x.z, c2, -Mz), fmaf(x.w, c2, -Mz)};
@@ -253,12 +312,17 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
                 }
                 zc[i] = make_float4(p[0], p[1], p[2], p[3]);
                 dc[i] = make_float4(q[0], q[1], q[2], q[3]);
+                if (i == (tl >> 2)) {  // the draft token's entry: step 2 overwrites the slices, keep a copy
+                    const int e = tl & 3;
+                    sh_pq[0] = e == 0 ? p[0] : e == 1 ? p[1] : e == 2 ? p[2] : p[3];
+                    sh_pq[1] = e == 0 ? q[0] : e == 1 ? q[1] : e == 2 ? q[2] : q[3];
+                }
             } else {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) ev[4 * kk + e] = -INFINITY;
             }
         }
-        block_max2(my, unused, sh_red);
+        block_max2<NW>(my, unused, sh_red);
         const float refy = (my == -INFINITY) ? 0.f : my;
         float sy = 0.f, zero = 0.f;
 #pragma unroll
@@ -266,25 +330,30 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
             ev[e] = fast_exp2(ev[e] - refy);  // phat up to the factor 2^(my - My) / Sy
             sy += ev[e];
         }
-        block_sum2(sy, zero, sh_red);
-        cluster_exchange(cluster, &xch[1], gath[1], make_float4(my, sy, 0.f, 0.f));
-        combine_ms(gath[1], false, My, Sy);
+        block_sum2<NW>(sy, zero, sh_red);
+        cluster_publish<CL>(cluster, gath[1], c, make_float4(my, sy, 0.f, 0.f));
+        if (warp == 0) {
+            float My_, Sy_;
+            combine_ms<CL>(gath[1], false, My_, Sy_);
+            if (lane == 0) {
+                sh_ms[0] = My_;
+                sh_ms[1] = Sy_;
+            }
+        }
+        __syncthreads();
+        My = sh_ms[0];
+        Sy = sh_ms[1];
         const float rel = (my == -INFINITY) ? 0.f : exp2f(my - My);  // phat / max(phat) = ev * rel
         const float to_phat = rel / Sy;
 
         // ---- step 2: the ratio at the draft token, then the residual weights ----
-        int tok = a.tokens[drow];
-        if (tok < 0 || tok >= a.V) {
-            if (c == 0 && tid == 0) atomicOr(a.status, RAPID_STATUS_BAD_DRAFT_TOKEN);
-            tok = tok < 0 ? 0 : a.V - 1;
-        }
-        const int tl = tok - v0;
-        if (tl >= 0 && tl < v1 - v0 && ((tl >> 2) % kThreads) == tid) {
+        if (tok_here) {  // thread 0 of the CTA whose slice holds the draft token
             // formed from log-probabilities: a draft token deep in the tail has p, phat and q far
-            // below the fp32 normal range while their ratio is O(1)
-            const float p = slice_mem[tl], q = slice_mem[a.slice + tl];
-            const float az = fmaf(__ldg(a.z + (size_t)row * a.zs + tok), c2, -Mz);
-            const float lq = fmaf(__ldg(a.d + (size_t)drow * a.ds + tok), c2, -Md) - log2f(Sd);
+            // below the fp32 normal range while their ratio is O(1).  (p and q of the token were set
+            // aside in step 1; the block reductions since then have made them visible.)
+            const float p = sh_pq[0], q = sh_pq[1];
+            const float az = fmaf(z_tok, c2, -Mz);
+            const float lq = a.d_logq ? lq_given * 1.4426950408889634f : fmaf(d_tok, c2, -Md) - log2f(Sd);
             const float y2 = fmaf(a.eta_log2, q - p, az);
             const float lph = (y2 - My < a.log2_alpha) ? az - log2f(Sz) : (y2 - My) - log2f(Sy);
             const float ratio = (lq == -INFINITY) ? INFINITY : exp2f(lph - lq);
@@ -294,7 +363,7 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
         // the weights replace p in shared memory, p moves to where q was (the fallback draws from it)
 #pragma unroll
         for (int kk = 0; kk < NV4; ++kk) {
-            const int i = kk * kThreads + tid;
+            const int i = kk * NT + tid;
             if (i < n4) {
                 const float4 p4 = zc[i], q4 = dc[i];
                 const float p[4] = {p4.x, p4.y, p4.z, p4.w};
@@ -317,7 +386,7 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
         // bonus row: the weights are p itself
 #pragma unroll
         for (int kk = 0; kk < NV4; ++kk) {
-            const int i = kk * kThreads + tid;
+            const int i = kk * NT + tid;
             if (i < n4) {
                 const float4 x = zc[i];
                 const float4 p = make_float4(fast_exp2(fmaf(x.x, c2, -Mz)) * iSz, fast_exp2(fmaf(x.y, c2, -Mz)) * iSz,
@@ -328,22 +397,22 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
         }
         sw = sp;
     }
-    block_sum2(sw, sp, sh_red);
-    cluster_exchange(cluster, &xch[2], gath[2], make_float4(sw, sp, 0.f, 0.f));  // also a CTA barrier
+    block_sum2<NW>(sw, sp, sh_red);
+    cluster_publish<CL>(cluster, gath[2], c, make_float4(sw, sp, 0.f, 0.f));  // also a CTA barrier
 
     // ---- step 3: the row's candidate token by inverse CDF (every CTA finds the same slice) ----
     const float u = a.uniforms[b * a.R + a.gamma];
     bool use_p = !draft;
     float W = 0.f;
 #pragma unroll
-    for (int rr = 0; rr < kCluster; ++rr) W += use_p ? gath[2][rr].y : gath[2][rr].x;
+    for (int rr = 0; rr < CL; ++rr) W += use_p ? gath[2][rr].y : gath[2][rr].x;
     int fell_back = 0;  // reported only if this row turns out to be the one Algorithm 1 reaches
     if (!(W > 0.f) || !isfinite(W)) {  // empty residual: defined fallback, draw from p
         if (!use_p) fell_back = (int)0x80000000;
         use_p = true;
         W = 0.f;
 #pragma unroll
-        for (int rr = 0; rr < kCluster; ++rr) W += gath[2][rr].y;
+        for (int rr = 0; rr < CL; ++rr) W += gath[2][rr].y;
     }
     const float target = u * W;
     int owner = -1, last_mass = -1;
@@ -351,7 +420,7 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
     {
         float run = 0.f;
 #pragma unroll
-        for (int rr = 0; rr < kCluster; ++rr) {
+        for (int rr = 0; rr < CL; ++rr) {
             const float own = use_p ? gath[2][rr].y : gath[2][rr].x;
             if (own > 0.f) {
                 if (owner < 0 && run + own > target) {
@@ -385,9 +454,13 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
         }
         if (lane == 31) sh_red[warp] = incl_w;
         __syncthreads();
-        float cum = before;
-        for (int wdx = 0; wdx < warp; ++wdx) cum += sh_red[wdx];
-        cum += incl_w - mine;
+        if (warp == 0) {  // exclusive prefix of the warp totals
+            const float tot = lane < NW ? sh_red[lane] : 0.f;
+            const float excl = warp_incl_scan(tot) - tot;
+            if (lane < NW) sh_red[NW + lane] = excl;
+        }
+        __syncthreads();
+        float cum = before + sh_red[NW + warp] + (incl_w - mine);
         int found = 0x7fffffff, last = -1;
         for (int i = t0; i < t1; ++i) {
             const float w = wsrc[i];
@@ -413,10 +486,13 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
     }
 
     // ---- the last cluster to finish settles every sequence ----
-    __threadfence();  // ratio and candidate of this row, before the cluster is counted as done
-    cluster.sync();   // also: no CTA leaves while a peer may still read its exchange slots
+    // This row's ratio and candidate were stored by threads of this cluster before the barrier below;
+    // the barrier (release / acquire over the cluster) orders them before thread 0's fence, which is
+    // cumulative, so they are visible device-wide before the count that announces them.
+    cluster.sync();  // also: no CTA leaves while a peer may still write into its exchange slots
     if (c != 0) return;
     if (tid == 0) {
+        __threadfence();
         const int total = (int)gridDim.y;
         const int old = atomicAdd(a.done, 1);
         sh_final = (old == total - 1);
@@ -424,29 +500,79 @@ __global__ void __launch_bounds__(kThreads, 1) accept_fused_kernel(const AcceptA
     }
     __syncthreads();
     if (!sh_final) return;
-    for (int s = tid; s < a.B; s += kThreads) {
-        int n = 0;
-        for (; n < a.gamma; ++n) {
-            const float ratio = __ldcg(a.ratio + s * a.gamma + n);
-            const float us = a.uniforms[s * a.R + n];
-            if (!(us <= fminf(1.f, ratio))) break;
+    // A warp per sequence: lane n takes position n's ratio, uniform and candidate in one round of
+    // loads and a ballot finds the first rejection (drafts longer than 31 positions: one lane walks them).
+    for (int s = warp; s < a.B; s += NW) {
+        int n, cand;
+        if (a.R <= 32) {
+            const bool is_draft = lane < a.gamma;
+            const float ratio = is_draft ? __ldcg(a.ratio + s * a.gamma + lane) : 0.f;
+            const float us = is_draft ? a.uniforms[s * a.R + lane] : 0.f;
+            const int cnd = lane < a.R ? __ldcg(a.cand + s * a.R + lane) : 0;
+            const unsigned rej = __ballot_sync(0xffffffffu, is_draft && !(us <= fminf(1.f, ratio)));
+            n = rej ? __ffs(rej) - 1 : a.gamma;
+            cand = __shfl_sync(0xffffffffu, cnd, n);
+        } else {
+            n = 0;
+            cand = 0;
+            if (lane == 0) {
+                for (; n < a.gamma; ++n) {
+                    const float ratio = __ldcg(a.ratio + s * a.gamma + n);
+                    if (!(a.uniforms[s * a.R + n] <= fminf(1.f, ratio))) break;
+                }
+                cand = __ldcg(a.cand + s * a.R + n);
+            }
         }
-        const int cand = __ldcg(a.cand + s * a.R + n);  // bit 31: the row fell back to p
-        if (cand < 0) atomicOr(a.status, RAPID_STATUS_RESIDUAL_FALLBACK);
-        a.accept_len[s] = n;
-        a.next_token[s] = cand & 0x7fffffff;
+        if (lane == 0) {
+            if (cand < 0) atomicOr(a.status, RAPID_STATUS_RESIDUAL_FALLBACK);  // bit 31: the row fell back to p
+            a.accept_len[s] = n;
+            a.next_token[s] = cand & 0x7fffffff;
+        }
     }
+    __syncthreads();
     if (tid == 0) *a.done = 0;  // ready for the next call on this workspace
 }
 
 bool accept_shape_ok(const rapid_accept_shape* s) {
     // a CTA keeps its slice of both rows in shared memory; grid.y carries the rows
-    return s && s->B > 0 && s->gamma >= 0 && s->V > 0 && s->V <= (int64_t)kCluster * kMaxSlice &&
+    return s && s->B > 0 && s->gamma >= 0 && s->V > 0 && s->V <= (int64_t)kClusterPortable * kMaxSlice &&
            (int64_t)s->B * (s->gamma + 1) <= 65535;
 }
 
 constexpr int kMaxDevices = 64;
-bool g_smem_opted[kMaxDevices] = {};  // the kernel's dynamic shared memory limit, raised per device
+std::atomic<int> g_accept_config[kMaxDevices];  // per device: the kernels' shared-memory limits have been raised
+
+template <int CL, int NT, int NV4>
+cudaError_t configure_accept_kernel(int max_slice_floats) {
+    return cudaFuncSetAttribute(accept_fused_kernel<CL, NT, NV4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                2 * max_slice_floats * (int)sizeof(float));
+}
+
+template <int CL, int NT>
+int launch_accept_shape(AcceptArgs& a, size_t rows, cudaStream_t stream) {
+    a.slice = (int)(((a.V / 4 + CL - 1) / CL) * 4);
+    a.per = ((a.slice + NT - 1) / NT) | 1;
+    // one cluster per logit row; a programmatic dependent of whatever precedes it in the stream
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(CL, (unsigned)rows);
+    cfg.blockDim = dim3(NT);
+    cfg.dynamicSmemBytes = 2 * (size_t)a.slice * sizeof(float);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CL;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    if (a.slice <= 4 * 4 * NT)
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, accept_fused_kernel<CL, NT, 4>, static_cast<const AcceptArgs&>(a)));
+    else
+        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, accept_fused_kernel<CL, NT, 6>, static_cast<const AcceptArgs&>(a)));
+    return RAPID_OK;
+}
 
 }  // namespace
 
@@ -518,14 +644,14 @@ int launch_accept(const float* target_logits, const float* draft_logits,
                                                                align_up((size_t)s.B * sizeof(int32_t), 256));
     a.logq_out = logq_out;
     a.stats_out = stats_out;
+    a.d_stats = params ? params->draft_row_stats : nullptr;
+    a.d_logq = params ? params->draft_logq : nullptr;
     a.next_token = out_next_token;
     a.ratio_out = params ? params->ratio_out : nullptr;
     a.B = s.B;
     a.gamma = s.gamma;
     a.R = R;
     a.V = (int)s.V;
-    a.slice = (int)(((s.V / 4 + kCluster - 1) / kCluster) * 4);
-    a.per = ((a.slice + kThreads - 1) / kThreads) | 1;
     a.zs = zs;
     a.ds = ds;
     a.inv_T_log2 = 1.4426950408889634f / T;
@@ -536,32 +662,14 @@ int launch_accept(const float* target_logits, const float* draft_logits,
 
     int dev = 0;
     RAPID_CUDA_CHECK(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= kMaxDevices || !g_smem_opted[dev]) {
-        RAPID_CUDA_CHECK(cudaFuncSetAttribute(accept_fused_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              2 * 8 * 4 * kThreads * (int)sizeof(float)));
-        RAPID_CUDA_CHECK(cudaFuncSetAttribute(accept_fused_kernel<12>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              2 * kMaxSlice * (int)sizeof(float)));
-        if (dev >= 0 && dev < kMaxDevices) g_smem_opted[dev] = true;
+    constexpr int P = kClusterPortable, PT = kThreadsPortable;
+    if (dev < 0 || dev >= kMaxDevices || !g_accept_config[dev].load(std::memory_order_acquire)) {
+        RAPID_CUDA_CHECK((configure_accept_kernel<P, PT, 4>(4 * 4 * PT)));
+        RAPID_CUDA_CHECK((configure_accept_kernel<P, PT, 6>(kMaxSlice)));
+        if (dev >= 0 && dev < kMaxDevices) g_accept_config[dev].store(1, std::memory_order_release);
     }
-    // one cluster per logit row; a programmatic dependent of whatever precedes it in the stream
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kCluster, (unsigned)rows);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = 2 * (size_t)a.slice * sizeof(float);
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kCluster;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    if (a.slice <= 8 * 4 * kThreads)
-        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, accept_fused_kernel<8>, a));
-    else
-        RAPID_CUDA_CHECK(cudaLaunchKernelEx(&cfg, accept_fused_kernel<12>, a));
+    const int rc = launch_accept_shape<P, PT>(a, rows, stream);
+    if (rc != RAPID_OK) return rc;
     count_launch(1);
     return RAPID_OK;
 }
@@ -582,7 +690,9 @@ constexpr size_t kStaticScratchBytes =
 
 static __device__ __align__(256) unsigned char g_accept_scratch[kStaticScratchBytes];
 
-void* g_scratch_addr[kMaxDevices] = {};  // device address of g_accept_scratch, per device
+// device address of g_accept_scratch, per device; atomic because first calls on a device may come
+// from several host threads at once (they would all look up, and store, the same address)
+std::atomic<void*> g_scratch_addr[kMaxDevices];
 
 }  // namespace
 }  // namespace rapid
@@ -614,12 +724,13 @@ extern "C" int rapid_accept_static(const float* target_logits, const float* draf
     }
     // In host code the array's name is only a handle for the runtime, not a device address: the
     // address the kernels can use has to be asked for, once per device, with that device current.
-    if (!g_scratch_addr[dev]) {
+    void* scratch = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
         void* ptr = nullptr;
         RAPID_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_accept_scratch));
-        g_scratch_addr[dev] = ptr;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
+        scratch = ptr;
     }
-    void* scratch = g_scratch_addr[dev];
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     // the array keeps whatever the previous call left: the status word must start at zero
     RAPID_CUDA_CHECK(cudaMemsetAsync(scratch, 0, kWorkspaceHeaderBytes, st));

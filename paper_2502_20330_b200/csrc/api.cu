@@ -274,7 +274,7 @@ int rapid_draft_sample(const float* draft_logits, const float* uniforms, float t
         return RAPID_ERR_INVALID_ARG;
     }
     rapid_accept_shape shape = {B, 0, V, row_stride, 0};
-    rapid_accept_params params = {temperature, 0.f, RAPID_RESIDUAL_PAPER, 0, nullptr};
+    rapid_accept_params params = {temperature, 0.f, RAPID_RESIDUAL_PAPER, 0, nullptr, nullptr, nullptr};
     return launch_accept(draft_logits, nullptr, nullptr, uniforms, 0.f, nullptr, out_token, &shape, &params,
                          workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream), out_logq,
                          out_row_stats);

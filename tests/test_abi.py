@@ -49,7 +49,7 @@ def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(binding._AttnShape) == 48
     assert ctypes.sizeof(binding._AttnParams) == 64
     assert ctypes.sizeof(binding._AcceptShape) == 32
-    assert ctypes.sizeof(binding._AcceptParams) == 24
+    assert ctypes.sizeof(binding._AcceptParams) == 40
     assert ctypes.sizeof(binding._PagedKv) == 40
 
 
@@ -64,7 +64,7 @@ def test_struct_layouts_match_what_the_c_compiler_sees(tmp_path):
         '  printf("%zu %zu\\n", sizeof(rapid_attn_shape), offsetof(rapid_attn_shape, kv_stride_l));\n'
         '  printf("%zu %zu\\n", sizeof(rapid_attn_params), offsetof(rapid_attn_params, wait_cycle_limit));\n'
         '  printf("%zu %zu\\n", sizeof(rapid_accept_shape), offsetof(rapid_accept_shape, draft_row_stride));\n'
-        '  printf("%zu %zu\\n", sizeof(rapid_accept_params), offsetof(rapid_accept_params, ratio_out));\n'
+        '  printf("%zu %zu\\n", sizeof(rapid_accept_params), offsetof(rapid_accept_params, draft_logq));\n'
         '  printf("%zu %zu\\n", sizeof(rapid_paged_kv), offsetof(rapid_paged_kv, stride_l));\n'
         '  return 0;\n}\n')
     exe = tmp_path / "layout"
@@ -73,7 +73,7 @@ def test_struct_layouts_match_what_the_c_compiler_sees(tmp_path):
                                                                           text=True).stdout.splitlines()]
     want = [(ctypes.sizeof(c), getattr(c, f).offset) for c, f in (
         (binding._AttnShape, "kv_stride_l"), (binding._AttnParams, "wait_cycle_limit"),
-        (binding._AcceptShape, "draft_row_stride"), (binding._AcceptParams, "ratio_out"),
+        (binding._AcceptShape, "draft_row_stride"), (binding._AcceptParams, "draft_logq"),
         (binding._PagedKv, "stride_l"))]
     assert got == want
 

@@ -158,3 +158,40 @@ def test_full_vocabulary_workloads(name):
     z, d, tok, u = wl.accept_inputs(cfg, seed=13, device="cuda")
     _check(z, d, tok, u, cfg.eta)
     _check(z, d, tok, u, 20.0, T=0.1)
+
+
+@pytest.mark.parametrize("T", [1.0, 0.5])
+def test_drafter_statistics_handed_to_the_accept_step(T):
+    """Algorithm 1's drafting loop draws x'_j from q_j; rapid_draft_sample returns log q_j(x'_j) and the
+    row's (max, log-sum-exp) from that pass.  Handed to the accept step they replace its own reductions
+    over the draft rows: same accepted lengths, same tokens, ratios equal to rounding."""
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("t", B=6, Hq=8, Hkv=2, D=64, gamma=5, V=32000, ctx_lens=(64,) * 6, target_sigma=1.0,
+                          temperature=T)
+    z, d, _, u = wl.accept_inputs(cfg, seed=14, device="cuda")
+    B, gamma, V = cfg.B, cfg.gamma, cfg.V
+    rows = d.reshape(B * gamma, V)
+    g = torch.Generator(device="cuda").manual_seed(15)
+    du = torch.rand(B * gamma, generator=g, device="cuda")
+    tok = torch.zeros(B * gamma, dtype=torch.int32, device="cuda")
+    logq = torch.zeros(B * gamma, device="cuda")
+    stats = torch.zeros(B * gamma, 2, device="cuda")
+    ws0 = R.new_workspace(R.accept_workspace_bytes(B * gamma, 0, V))
+    R.rapid_draft_sample(rows, du, T, tok, logq, ws0, out_row_stats=stats)
+    tok = tok.reshape(B, gamma)
+    outs = []
+    for params in (R.AcceptParams(temperature=T), R.AcceptParams(temperature=T, draft_row_stats=stats, draft_logq=logq),
+                   R.AcceptParams(temperature=T, draft_row_stats=stats), R.AcceptParams(temperature=T, draft_logq=logq)):
+        ws = R.new_workspace(R.accept_workspace_bytes(B, gamma, V))
+        alen = torch.zeros(B, dtype=torch.int32, device="cuda"); ntok = torch.zeros_like(alen)
+        params.ratio_out = torch.zeros(B, gamma, device="cuda")
+        R.rapid_accept(z, d, tok, u, 5.0, alen, ntok, ws, params)
+        torch.cuda.synchronize()
+        assert R.workspace_status(ws) == 0
+        outs.append((alen.cpu().numpy(), ntok.cpu().numpy(), params.ratio_out.cpu().numpy()))
+        parity.check_accept(z.cpu().numpy(), d.cpu().numpy(), tok.cpu().numpy(), u.cpu().numpy(), 5.0, T, 0.1, 0,
+                            outs[-1][0], outs[-1][1], outs[-1][2])
+    for o in outs[1:]:
+        np.testing.assert_array_equal(o[0], outs[0][0])
+        np.testing.assert_array_equal(o[1], outs[0][1])
+        np.testing.assert_allclose(o[2], outs[0][2], rtol=2e-5)
