@@ -64,6 +64,13 @@ def _load():
             vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, c_i64,
             ctypes.c_int, c_i64, c_i64, c_i64, c_dbl, c_i64, c_i64, vp, c_i64, vp, vp,
         ]
+        lib.oracle_e4m3_to_double.restype = c_dbl
+        lib.oracle_e4m3_to_double.argtypes = [ctypes.c_uint8]
+        lib.oracle_verify_attention_fp8.restype = ctypes.c_int
+        lib.oracle_verify_attention_fp8.argtypes = [
+            vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, c_i64,
+            ctypes.c_int, c_i64, c_i64, c_i64, c_dbl, vp, c_i64, vp, vp,
+        ]
         lib.oracle_rapid_distributions.restype = None
         lib.oracle_rapid_distributions.argtypes = [vp, vp, c_i64, c_dbl, c_dbl, c_dbl, vp, vp, vp, vp]
         lib.oracle_residual_weights.restype = None
@@ -139,6 +146,41 @@ def verify_attention(q_bits, k_bits, v_bits, ctx_lens, gamma, scale=0.0, units=N
             sb, sh, sl, float(scale), _ptr(units), n_units, _ptr(out), _ptr(lse))
     if rc != 0:
         raise ValueError(f"oracle_verify_attention failed with {rc}")
+    return out, lse
+
+
+def e4m3_to_double(code: int) -> float:
+    """Value of one FP8 E4M3 code (OCP 8-bit floating point: bias 7, no infinities, S.1111.111 = NaN)."""
+    return float(_load().oracle_e4m3_to_double(int(code) & 0xFF))
+
+
+def verify_attention_fp8(q_bits, k_codes, v_codes, k_scale, v_scale, ctx_lens, gamma, scale=0.0, units=None):
+    """Verify attention over an FP8 E4M3 cache with one fp32 scale per (sequence, KV head) for K and for V:
+    the attention definition applied to K = k_scale * decode(k_codes), V = v_scale * decode(v_codes), in fp64.
+    q_bits [B,R,Hq,D] uint16 (bf16 bits); k_codes, v_codes [B,Hkv,Lmax,D] uint8; k_scale, v_scale [B,Hkv] float32.
+    Returns (out [B,R,Hq,D] float64, lse [B,R,Hq] float64); ``units`` as in verify_attention."""
+    lib = _load()
+    q_bits = _c(q_bits, np.uint16)
+    B, R, Hq, D = q_bits.shape
+    assert R == gamma + 1
+    k_codes = _c(k_codes, np.uint8)
+    v_codes = _c(v_codes, np.uint8)
+    _, Hkv, Lmax, Dk = k_codes.shape
+    assert Dk == D and v_codes.shape == k_codes.shape and k_codes.shape[0] == B
+    k_scale = _c(k_scale, np.float32).reshape(B, Hkv)
+    v_scale = _c(v_scale, np.float32).reshape(B, Hkv)
+    ctx_lens = _c(ctx_lens, np.int32)
+    out = np.full((B, R, Hq, D), np.nan, dtype=np.float64)
+    lse = np.full((B, R, Hq), np.nan, dtype=np.float64)
+    n_units = 0
+    if units is not None:
+        units = _c(units, np.int64)
+        n_units = units.size
+    rc = lib.oracle_verify_attention_fp8(
+        _ptr(q_bits), _ptr(k_codes), _ptr(v_codes), _ptr(k_scale), _ptr(v_scale), _ptr(ctx_lens), B, Hq, Hkv, D,
+        Lmax, gamma, Hkv * Lmax * D, Lmax * D, D, float(scale), _ptr(units), n_units, _ptr(out), _ptr(lse))
+    if rc != 0:
+        raise ValueError(f"oracle_verify_attention_fp8 failed with {rc}")
     return out, lse
 
 

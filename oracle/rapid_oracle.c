@@ -214,6 +214,97 @@ int oracle_verify_attention_window(const uint16_t* q, const uint16_t* k, const u
 }
 
 /* ------------------------------------------------------------------------ */
+/* Verify attention over an 8-bit KV cache.                                  */
+/*                                                                           */
+/* The paper's case for this path is that reading the long context's KV      */
+/* cache is memory-bound (Introduction; Section 2.1), and it fixes no        */
+/* storage precision.  Reading taken here: a cache stored as FP8 E4M3 codes  */
+/* (1 sign, 4 exponent, 3 mantissa bits, bias 7, no infinities, S.1111.111   */
+/* = NaN, exponent 0 = subnormals: the OCP 8-bit floating point format) with */
+/* one fp32 scale per (sequence, KV head) for K and one for V:               */
+/*     K[b,h,j,:] = k_scale[b,h] * decode(k_codes[b,h,j,:]),  V likewise.    */
+/* The attention is the definition above applied to those K and V, in fp64;  */
+/* q stays bf16.  Same masks, layouts (strides in elements = bytes),         */
+/* unit_list and return codes as oracle_verify_attention.                    */
+/* ------------------------------------------------------------------------ */
+double oracle_e4m3_to_double(uint8_t code) {
+    const int sign = code >> 7, e = (code >> 3) & 15, m = code & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m, -9);          /* subnormal: m/8 * 2^-6 */
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);  /* normal: 1.m * 2^(e-7) */
+    return sign ? -v : v;
+}
+
+int oracle_verify_attention_fp8(const uint16_t* q, const uint8_t* k, const uint8_t* v,
+                                const float* k_scale, const float* v_scale,
+                                const int32_t* ctx_lens, int B, int Hq, int Hkv, int D, int64_t Lmax,
+                                int gamma, int64_t kv_stride_b, int64_t kv_stride_h,
+                                int64_t kv_stride_l, double scale, const int64_t* unit_list,
+                                int64_t n_units, double* out, double* lse) {
+    const int R = gamma + 1;
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || gamma < 0 || Hq % Hkv != 0) return -1;
+    const int G = Hq / Hkv;
+    for (int b = 0; b < B; ++b)
+        if (ctx_lens[b] < R || (int64_t)ctx_lens[b] > Lmax) return -1;
+    if (scale == 0.0) scale = 1.0 / sqrt((double)D);
+    const int64_t all_units = (int64_t)B * Hq * R;
+    if (!unit_list) n_units = all_units;
+    for (int64_t t = 0; unit_list && t < n_units; ++t)
+        if (unit_list[t] < 0 || unit_list[t] >= all_units) return -1;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t t = 0; t < n_units; ++t) {
+        const int64_t unit = unit_list ? unit_list[t] : t;
+        const int b = (int)(unit / ((int64_t)Hq * R));
+        const int h = (int)((unit / R) % Hq);
+        const int i = (int)(unit % R);
+        const int head8 = h / G;
+        const int64_t L = ctx_lens[b];
+        const int64_t last = L - R + i; /* last visible key */
+        const double ks = (double)k_scale[(int64_t)b * Hkv + head8];
+        const double vs = (double)v_scale[(int64_t)b * Hkv + head8];
+        const uint16_t* qrow = q + (((int64_t)b * R + i) * Hq + h) * D;
+        const uint8_t* kbase = k + b * kv_stride_b + head8 * kv_stride_h;
+        const uint8_t* vbase = v + b * kv_stride_b + head8 * kv_stride_h;
+        double* sc = (double*)malloc((size_t)(last + 1) * sizeof(double));
+        double* acc = (double*)calloc((size_t)D, sizeof(double));
+        double* qd = (double*)malloc((size_t)D * sizeof(double));
+        if (!sc || !acc || !qd) {
+#pragma omp atomic write
+            failed = 1;
+            free(sc);
+            free(acc);
+            free(qd);
+            continue;
+        }
+        for (int d = 0; d < D; ++d) qd[d] = bf16_bits_to_double(qrow[d]);
+        double m = -INFINITY;
+        for (int64_t j = 0; j <= last; ++j) {
+            const uint8_t* kcodes = kbase + j * kv_stride_l;
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += qd[d] * (ks * oracle_e4m3_to_double(kcodes[d]));
+            sc[j] = scale * dot;
+            if (sc[j] > m) m = sc[j];
+        }
+        double denom = 0.0;
+        for (int64_t j = 0; j <= last; ++j) {
+            const double e = exp(sc[j] - m);
+            denom += e;
+            const uint8_t* vcodes = vbase + j * kv_stride_l;
+            for (int d = 0; d < D; ++d) acc[d] += e * (vs * oracle_e4m3_to_double(vcodes[d]));
+        }
+        double* orow = out + (((int64_t)b * R + i) * Hq + h) * D;
+        for (int d = 0; d < D; ++d) orow[d] = acc[d] / denom;
+        if (lse) lse[((int64_t)b * R + i) * Hq + h] = m + log(denom);
+        free(sc);
+        free(acc);
+        free(qd);
+    }
+    return failed ? -2 : 0;
+}
+
+/* ------------------------------------------------------------------------ */
 /* Accept / residual (Algorithm 1, validation loop and residual step).       */
 /* ------------------------------------------------------------------------ */
 

@@ -255,3 +255,77 @@ def test_window_of_one_returns_the_rows_own_value_and_hidden_keys_are_never_read
     k4 = k.clone(); k4[:, :, 1] += 1.0
     moved, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k4), bf16_bits(v), ctx, gamma, sink=sink, window=window)
     assert all(np.abs(moved[:, i] - base[:, i]).max() > 1e-4 for i in range(R))
+
+
+# ---- FP8 E4M3 cache with per-(sequence, KV head) scales ----------------------------------------------------
+
+def _codes(shape, seed):
+    """Random E4M3 codes without the two NaN patterns."""
+    g = torch.Generator().manual_seed(seed)
+    c = torch.randint(0, 256, shape, generator=g, dtype=torch.int32)
+    c[(c & 0x7F) == 0x7F] = 0x3A
+    return c.to(torch.uint8)
+
+
+def test_e4m3_decoding_of_every_code():
+    """All 256 codes: against the library's own E4M3 type, and a few values known by heart from the format
+    (bias 7, 3 mantissa bits, subnormals at exponent 0, no infinities, S.1111.111 = NaN, largest 448)."""
+    lib = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).double().numpy()
+    for code in range(256):
+        v = oracle.e4m3_to_double(code)
+        if np.isnan(lib[code]):
+            assert np.isnan(v) and code in (0x7F, 0xFF)
+        else:
+            assert v == lib[code], hex(code)
+    known = {0x00: 0.0, 0x01: 2.0 ** -9, 0x07: 7 * 2.0 ** -9, 0x08: 2.0 ** -6, 0x38: 1.0, 0x39: 1.125, 0x40: 2.0,
+             0x7E: 448.0, 0x78: 256.0, 0xB8: -1.0, 0xFE: -448.0, 0x80: 0.0}
+    for code, val in known.items():
+        assert oracle.e4m3_to_double(code) == val
+    assert np.copysign(1.0, oracle.e4m3_to_double(0x80)) == -1.0
+
+
+def test_fp8_cache_equals_the_bf16_definition_on_values_both_can_hold():
+    """Every E4M3 value times a power-of-two scale is a bf16 number: the bf16 oracle on those numbers must
+    give the same bits."""
+    B, Hq, Hkv, D, Lmax, gamma = 2, 4, 2, 16, 40, 3
+    q = _rand((B, gamma + 1, Hq, D), 41)
+    kc, vc = _codes((B, Hkv, Lmax, D), 42), _codes((B, Hkv, Lmax, D), 43)
+    ks = torch.tensor([[0.5, 2.0], [0.125, 1.0]]); vs = torch.tensor([[4.0, 0.25], [1.0, 0.0625]])
+    ctx = np.array([40, 9], dtype=np.int32)
+    out8, lse8 = oracle.verify_attention_fp8(bf16_bits(q), kc.numpy(), vc.numpy(), ks.numpy(), vs.numpy(), ctx, gamma)
+    k = (kc.view(torch.float8_e4m3fn).float() * ks[:, :, None, None]).to(torch.bfloat16)
+    v = (vc.view(torch.float8_e4m3fn).float() * vs[:, :, None, None]).to(torch.bfloat16)
+    assert torch.equal(k.float(), kc.view(torch.float8_e4m3fn).float() * ks[:, :, None, None])   # nothing was rounded
+    out16, lse16 = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx, gamma)
+    np.testing.assert_array_equal(out8, out16)
+    np.testing.assert_array_equal(lse8, lse16)
+
+
+def test_fp8_scales_act_as_the_definition_says():
+    B, Hq, Hkv, D, Lmax, gamma = 1, 4, 2, 8, 30, 2
+    q = _rand((B, gamma + 1, Hq, D), 44)
+    kc, vc = _codes((B, Hkv, Lmax, D), 45), _codes((B, Hkv, Lmax, D), 46)
+    ks = np.array([[0.37, 1.9]], np.float32); vs = np.array([[0.8, 3.1]], np.float32)
+    ctx = np.array([30], dtype=np.int32)
+    base, lse = oracle.verify_attention_fp8(bf16_bits(q), kc.numpy(), vc.numpy(), ks, vs, ctx, gamma)
+    # the value scale multiplies the output of its own KV head's query heads, and nothing else
+    vs2 = vs.copy(); vs2[0, 1] *= 4.0
+    out, lse2 = oracle.verify_attention_fp8(bf16_bits(q), kc.numpy(), vc.numpy(), ks, vs2, ctx, gamma)
+    np.testing.assert_allclose(out[:, :, 2:], 4.0 * base[:, :, 2:], rtol=1e-12)
+    np.testing.assert_array_equal(out[:, :, :2], base[:, :, :2])
+    np.testing.assert_array_equal(lse2, lse)
+    # a key scale of 2 with the query halved (exact in bf16) leaves every score as it was
+    ks2 = ks * 2.0
+    out, lse3 = oracle.verify_attention_fp8(bf16_bits((q.float() * 0.5).to(torch.bfloat16)), kc.numpy(), vc.numpy(),
+                                            ks2, vs, ctx, gamma)
+    np.testing.assert_allclose(out, base, rtol=1e-12)
+    np.testing.assert_allclose(lse3, lse, rtol=1e-12)
+    # and it is the brute-force softmax of the decoded cache
+    kd = kc.view(torch.float8_e4m3fn).double() * torch.tensor(ks, dtype=torch.float64)[:, :, None, None]
+    vd = vc.view(torch.float8_e4m3fn).double() * torch.tensor(vs, dtype=torch.float64)[:, :, None, None]
+    for i in range(gamma + 1):
+        n = 30 - (gamma + 1) + i + 1
+        for h in range(Hq):
+            s = (kd[0, h // 2, :n] @ q[0, i, h].double()) / np.sqrt(D)
+            ref = torch.softmax(s, 0) @ vd[0, h // 2, :n]
+            np.testing.assert_allclose(base[0, i, h], ref.numpy(), rtol=1e-10, atol=1e-13)

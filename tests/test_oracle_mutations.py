@@ -35,6 +35,12 @@ MUTATIONS = {
     "sampling_uniform_reused": ("const double u = (double)uniforms[(int64_t)b * R + gamma];",
                                 "const double u = (double)uniforms[(int64_t)b * R + (n < gamma ? n : gamma)];"),
     "keeps_going_after_reject": ("rejected = 1;\n", "rejected = 0; n = 0;\n"),
+    "e4m3_bias_off_by_one": ("else v = ldexp(1.0 + (double)m / 8.0, e - 7);", "else v = ldexp(1.0 + (double)m / 8.0, e - 8);"),
+    "e4m3_subnormal_as_normal": ("if (e == 0) v = ldexp((double)m, -9);", "if (e == 0) v = ldexp(1.0 + (double)m / 8.0, -7);"),
+    "fp8_value_scale_taken_from_keys": ("const double vs = (double)v_scale[(int64_t)b * Hkv + head8];",
+                                        "const double vs = (double)k_scale[(int64_t)b * Hkv + head8];"),
+    "fp8_scale_of_the_wrong_head": ("const double ks = (double)k_scale[(int64_t)b * Hkv + head8];",
+                                    "const double ks = (double)k_scale[(int64_t)b * Hkv];"),
     "window_one_key_too_narrow": ("if (!(j < sink || j > own - window)) continue;\n            const double e",
                                   "if (!(j < sink || j > own - window + 1)) continue;\n            const double e"),
     "window_anchored_at_last_row": ("const int64_t own = L - R + i; /* the row's own key */",
