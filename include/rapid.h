@@ -131,7 +131,9 @@ typedef struct rapid_attn_params {
                                  StreamingLLM baseline: 4 sinks in a budget of 4,096) laid over a full
                                  cache; key tiles no row sees are not read.  0 = the plain causal mask  */
     int32_t plan;             /* RAPID_PLAN_*                                                           */
-    int32_t reserved;
+    int32_t kv_fp8;           /* non-zero in a call of rapid_attention_plan or rapid_attention_describe:
+                                 the plan is for rapid_verify_attention_fp8 (which always runs the
+                                 keys-on-M kernel); ignored elsewhere                                   */
     int64_t wait_cycle_limit; /* SM clock cycles an on-chip wait (for a tile, for the tensor cores) may take
                                  before the kernel gives up and sets RAPID_STATUS_PIPELINE_TIMEOUT;
                                  0 = the library's limit of about a second                              */
@@ -210,6 +212,29 @@ int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cac
                            const int32_t* ctx_lens, int gamma, void* out,
                            const rapid_attn_shape* shape, const rapid_attn_params* params,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * rapid_verify_attention over an 8-bit KV cache.  (The paper fixes no storage precision; its case for
+ * this path is that reading the long context's KV cache is memory-bound -- Introduction, Section 2.1 --
+ * and a cache of half the bytes is read in half the time.)
+ *
+ *   k_cache, v_cache : device [B, Hkv, Lmax, D] FP8 E4M3 codes (one byte each: 1 sign, 4 exponent,
+ *                      3 mantissa bits, bias 7, no infinities), geometry and strides (in elements,
+ *                      multiples of 16) of `shape`;  K = k_scale[b, kvh] * decode(code), V likewise
+ *   k_scale, v_scale : device fp32 [B, Hkv], positive and finite
+ *   q, out           : bf16 as in rapid_verify_attention
+ * The result is the attention of rapid_verify_attention over those K and V.  Inside, q and the softmax
+ * probabilities enter the 8-bit tensor-core products as the sum of two E4M3 numbers each (8 significant
+ * bits, what bf16 carries), so the output meets the bf16 call's tolerances against the exact result
+ * over the same codes; lse_out is within 5e-3.  head_dim 128, at most 96 grouped rows per KV head, a
+ * contiguous cache, the plain causal mask; params->kernel 0 or RAPID_ATTN_KERNEL_KEYS_ON_M;
+ * RAPID_ERR_UNSUPPORTED otherwise.  Workspace, plan, errors and status bits as in
+ * rapid_verify_attention (a plan made by rapid_attention_plan for the same geometry serves both).
+ */
+int rapid_verify_attention_fp8(const void* q, const void* k_cache, const void* v_cache, const float* k_scale,
+                               const float* v_scale, const int32_t* ctx_lens, int gamma, void* out,
+                               const rapid_attn_shape* shape, const rapid_attn_params* params, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream);
 
 /*
  * Works out once, on the device, what every attention call over the same lengths would otherwise

@@ -24,7 +24,7 @@ RESIDUAL_PHAT = 1
 
 EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
-    "rapid_workspace_status", "rapid_verify_attention", "rapid_attention_plan", "rapid_attention_describe", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_retrieval_select", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_fp8", "rapid_attention_plan", "rapid_attention_describe", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_retrieval_select", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
     "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_kv_append_paged", "rapid_step_commit",
     "rapid_last_error",
@@ -55,7 +55,7 @@ class _AttnParams(ctypes.Structure):
                 ("lse_out", ctypes.c_void_p), ("out_f32", ctypes.c_void_p),
                 ("split_done_event", ctypes.c_void_p), ("all_keys_visible", ctypes.c_int32),
                 ("kernel", ctypes.c_int32), ("sink_keys", ctypes.c_int32), ("window_keys", ctypes.c_int32),
-                ("plan", ctypes.c_int32), ("reserved", ctypes.c_int32), ("wait_cycle_limit", ctypes.c_int64)]
+                ("plan", ctypes.c_int32), ("kv_fp8", ctypes.c_int32), ("wait_cycle_limit", ctypes.c_int64)]
 
 
 class _LaunchInfo(ctypes.Structure):
@@ -89,6 +89,7 @@ class AttnParams:
     window_keys: int = 0                     # > 0: each row sees only that many newest keys up to its own
     plan: int = 0                            # PLAN_*: the workspace holds a plan made by rapid_attention_plan
     wait_cycle_limit: int = 0                # clock cycles an on-chip wait may take; 0 = the library's limit
+    kv_fp8: bool = False                     # rapid_attention_plan / describe: the plan is for the FP8-cache call
 
 
 @dataclass
@@ -135,6 +136,8 @@ def load_library():
         acc_args = [vp, vp, vp, vp, f32, vp, vp, ctypes.POINTER(_AcceptShape), ctypes.POINTER(_AcceptParams)]
         lib.rapid_verify_attention.restype = i32
         lib.rapid_verify_attention.argtypes = attn_args + [vp, sz, vp]
+        lib.rapid_verify_attention_fp8.restype = i32
+        lib.rapid_verify_attention_fp8.argtypes = [vp, vp, vp, vp, vp] + attn_args[3:] + [vp, sz, vp]
         lib.rapid_attention_plan.restype = i32
         lib.rapid_attention_plan.argtypes = [vp, i32, ctypes.POINTER(_AttnShape), ctypes.POINTER(_AttnParams), vp, sz, vp]
         lib.rapid_attention_describe.restype = i32
@@ -219,7 +222,8 @@ def _attn_params(p: Optional[AttnParams]):
     return ctypes.byref(_AttnParams(p.scale, p.num_ctas, p.lse_out.data_ptr() if p.lse_out is not None else None,
                                     p.out_f32.data_ptr() if p.out_f32 is not None else None,
                                     p.split_done_event, 1 if p.all_keys_visible else 0, int(p.kernel),
-                                    int(p.sink_keys), int(p.window_keys), int(p.plan), 0, int(p.wait_cycle_limit)))
+                                    int(p.sink_keys), int(p.window_keys), int(p.plan), 1 if p.kv_fp8 else 0,
+                                    int(p.wait_cycle_limit)))
 
 
 def _accept_shape(target_logits: torch.Tensor, draft_logits: torch.Tensor) -> _AcceptShape:
@@ -299,6 +303,29 @@ def rapid_verify_attention(q, k_cache, v_cache, ctx_lens, gamma, out, workspace,
     _check(load_library().rapid_verify_attention(_p(q), _p(k_cache), _p(v_cache), _p(ctx_lens), gamma, _p(out),
                                                  ctypes.byref(shape), _attn_params(params), _p(workspace),
                                                  _nbytes(workspace), _stream_ptr(stream)))
+
+
+def rapid_verify_attention_fp8(q, k_cache, v_cache, k_scale, v_scale, ctx_lens, gamma, out, workspace,
+                               params: Optional[AttnParams] = None, stream=None) -> None:
+    """Verify attention over an FP8 E4M3 cache: k_cache / v_cache [B,Hkv,Lmax,D] uint8 (or torch.float8_e4m3fn)
+    codes, k_scale / v_scale [B,Hkv] float32; q and out bfloat16."""
+    if q.dtype != torch.bfloat16 or out.dtype != torch.bfloat16 or ctx_lens.dtype != torch.int32:
+        raise TypeError("q/out must be bfloat16 and ctx_lens int32")
+    if k_cache.element_size() != 1 or v_cache.element_size() != 1:
+        raise TypeError("k_cache / v_cache must hold one-byte E4M3 codes")
+    if k_scale.dtype != torch.float32 or v_scale.dtype != torch.float32 or not (k_scale.is_contiguous() and v_scale.is_contiguous()):
+        raise TypeError("k_scale / v_scale must be dense float32 [B, Hkv]")
+    if not (q.is_contiguous() and out.is_contiguous()) or q.shape[1] != gamma + 1 or out.shape != q.shape:
+        raise ValueError("q and out must be dense [B, gamma+1, Hq, D]")
+    if k_cache.stride() != v_cache.stride() or k_cache.shape != v_cache.shape:
+        raise ValueError("k_cache and v_cache must share shape and strides")
+    if k_scale.shape != (q.shape[0], k_cache.shape[1]) or v_scale.shape != k_scale.shape:
+        raise ValueError("k_scale / v_scale must be [B, Hkv]")
+    shape = _attn_shape(q, k_cache)
+    _check(load_library().rapid_verify_attention_fp8(_p(q), _p(k_cache), _p(v_cache), _p(k_scale), _p(v_scale),
+                                                     _p(ctx_lens), gamma, _p(out), ctypes.byref(shape),
+                                                     _attn_params(params), _p(workspace), _nbytes(workspace),
+                                                     _stream_ptr(stream)))
 
 
 def rapid_attention_plan(ctx_lens, gamma, B, Hq, Hkv, D, Lmax, workspace, params: Optional[AttnParams] = None,

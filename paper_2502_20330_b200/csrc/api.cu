@@ -236,6 +236,15 @@ int rapid_verify_attention(const void* q, const void* k_cache, const void* v_cac
                                    static_cast<cudaStream_t>(cuda_stream));
 }
 
+int rapid_verify_attention_fp8(const void* q, const void* k_cache, const void* v_cache, const float* k_scale,
+                               const float* v_scale, const int32_t* ctx_lens, int gamma, void* out,
+                               const rapid_attn_shape* shape, const rapid_attn_params* params, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream) {
+    clear_error();
+    return launch_verify_attention_fp8(q, k_cache, v_cache, k_scale, v_scale, ctx_lens, gamma, out, shape, params,
+                                       workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int rapid_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
                          const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
                          void* cuda_stream) {

@@ -79,6 +79,9 @@ struct AttnArgs {
     // unit's tiles, exchange their partials through distributed shared memory and write the
     // output rows themselves; no partial goes to the workspace and no merge kernel follows.
     int cmerge;
+    // FP8 cache: one fp32 scale per (sequence, KV head) for the K codes and one for the V codes
+    const float* k_scale;
+    const float* v_scale;
     __nv_bfloat16* out;
     float* out_f32;
     float* lse_out;
@@ -259,14 +262,39 @@ __device__ __forceinline__ int2 unit_slot_range(const AttnArgs& a, int unit, int
     return make_int2(c_first, (c_last - c_first + 1) * KS);
 }
 
-// A CTA's walk: from the plan (three 16-byte loads) or computed from the lengths.
-__device__ __forceinline__ void load_walk(const AttnArgs& a, int cta, Walk& w) {
+__device__ __forceinline__ void fill_plan_sig(const AttnArgs& a, int KS, int32_t (&sig)[kPlanSigInts]);
+
+// True if the plan in the workspace was made for this call's geometry, kernel and split (the lengths
+// it was made for are checked by CTA 0 alone: lengths that have moved on cannot send a kernel outside
+// its buffers, a walk made for another geometry could).
+__device__ __forceinline__ bool plan_matches(const AttnArgs& a, int KS) {
+    int32_t want[kPlanSigInts];
+    fill_plan_sig(a, KS, want);
+    const uint4* src = reinterpret_cast<const uint4*>(a.plan_sig);
+    bool same = true;
+#pragma unroll
+    for (int i = 0; i < kPlanSigInts / 4; ++i) {
+        const uint4 x = __ldcg(src + i);
+        same &= x.x == (uint32_t)want[4 * i] && x.y == (uint32_t)want[4 * i + 1] && x.z == (uint32_t)want[4 * i + 2] &&
+                x.w == (uint32_t)want[4 * i + 3];
+    }
+    return same;
+}
+
+// A CTA's walk from the plan (three 16-byte loads); no work at all if the plan is not this call's.
+__device__ __forceinline__ void load_walk(const AttnArgs& a, int cta, int KS, Walk& w) {
     const uint4* src = reinterpret_cast<const uint4*>(a.plan_walks + cta);
     uint4* dst = reinterpret_cast<uint4*>(&w);
     const uint4 x0 = __ldcg(src), x1 = __ldcg(src + 1), x2 = __ldcg(src + 2);
+    const bool ok = plan_matches(a, KS);
     dst[0] = x0;
     dst[1] = x1;
     dst[2] = x2;
+    if (!ok) {
+        w.remaining = 0;
+        w.b = 0;
+        w.kvh = 0;
+    }
 }
 
 __device__ __forceinline__ void fill_plan_sig(const AttnArgs& a, int KS, int32_t (&sig)[kPlanSigInts]) {
@@ -285,11 +313,7 @@ __device__ __noinline__ void check_call_inputs(const AttnArgs& a, int KS) {
         bad |= (L < a.Lmin) || (L > a.Lmax);
         if (a.caller_plan) stale |= __ldcg(a.plan_ctx + b) != L;
     }
-    if (a.caller_plan) {
-        int32_t sig[kPlanSigInts];
-        fill_plan_sig(a, KS, sig);
-        for (int i = 0; i < kPlanSigInts; ++i) stale |= __ldcg(a.plan_sig + i) != sig[i];
-    }
+    stale |= !plan_matches(a, KS);
     if (bad) atomicOr(a.status, RAPID_STATUS_BAD_CTX_LEN);
     if (stale) atomicOr(a.status, RAPID_STATUS_STALE_PLAN);
 }
@@ -372,9 +396,9 @@ __device__ __forceinline__ bool warp_wait_bounded(uint64_t* bar, uint32_t parity
 // which is what allows (a) the merge kernel to take the lengths before its own wait although an
 // earlier kernel of the stream may have written them, and (b) a settled plan to be read before
 // the wait.
-__device__ __forceinline__ void split_kernel_walk(const AttnArgs& a, int cta, Walk& w, Walk* s_walk) {
+__device__ __forceinline__ void split_kernel_walk(const AttnArgs& a, int cta, int KS, Walk& w, Walk* s_walk) {
     const bool settled = a.plan_mode == RAPID_PLAN_SETTLED;
-    if (settled) load_walk(a, cta, w);
+    if (settled) load_walk(a, cta, KS, w);
     tc_fence_before_sync();
     __syncthreads();  // barriers initialised, tensor memory allocated
     tc_fence_after_sync();
@@ -383,7 +407,7 @@ __device__ __forceinline__ void split_kernel_walk(const AttnArgs& a, int cta, Wa
     if (!settled) {
         if (threadIdx.x == 0) {
             Walk t;
-            load_walk(a, cta, t);
+            load_walk(a, cta, KS, t);
             *s_walk = t;
         }
         __syncthreads();
@@ -491,7 +515,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
     }
     if (warp == 9) tmem_alloc(&tmem_slot, TMEM_COLS);  // warp 9 also frees it at the end
     Walk w;
-    split_kernel_walk(a, cta, w, &s_walk);
+    split_kernel_walk(a, cta, kStreams, w, &s_walk);
     if (cta == 0 && warp == 8 && lane == 1) check_call_inputs(a, kStreams);  // an idle lane of the producer warp
     const uint32_t tmem_base = tmem_slot;
     const WaitCtx wc = {&s_abort, a.wait_limit};
@@ -819,6 +843,7 @@ verify_attn_splitkv_tc_kernel(const __grid_constant__ CUtensorMap tmK,
 }
 
 #include "attention_kt.cuh"
+#include "attention_kt8.cuh"
 
 // Merge: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the partials of a unit.
 // One block of 4 warps per (grouped row, unit): warp w takes the slots j = w, w+4, ... (four
@@ -843,7 +868,7 @@ verify_attn_merge_kernel(const __grid_constant__ AttnArgs a, int KS, __nv_bfloat
     // stream wrote it: this kernel starts only after every CTA of the split kernel has passed its own
     // wait (it lets its dependents launch after it), and by then everything before the split kernel,
     // the plan kernel included, has completed.
-    const int2 range = __ldcg(a.plan_units + unit);
+    const int2 range = plan_matches(a, KS) ? __ldcg(a.plan_units + unit) : make_int2(0, 0);  // not this call's plan: nothing to merge
     const int c_first = range.x;
     const int nslots = range.y;
     const size_t slot_stride = (size_t)slot_floats(a.GR, D);
@@ -852,6 +877,17 @@ verify_attn_merge_kernel(const __grid_constant__ AttnArgs a, int KS, __nv_bfloat
     // everything above depends on the call's inputs only; the partials need the split kernel
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");  // a following dependent launch may begin its prologue
+    if (nslots <= 0) {  // the plan is not this call's (status says so): defined output, nothing read
+        if (warp == 0) {
+            const size_t row = ((size_t)b * a.R + m / a.G) * a.Hq + (size_t)kvh * a.G + m % a.G;
+            for (int d = lane; d < D; d += 32) {
+                out[row * D + d] = __float2bfloat16_rn(0.f);
+                if (out_f32) out_f32[row * D + d] = 0.f;
+            }
+            if (lse_out && lane == 0) lse_out[row] = -INFINITY;
+        }
+        return;
+    }
 
     // Warp w takes the slots j = w, w + 4, ...  The O rows of its first UN slots are requested at
     // once, together with every slot's running maximum: neither depends on the other, so the common
@@ -972,17 +1008,19 @@ EncodeTiledFn get_encode_fn() {
 // Tensor map of a cache [outer][Hkv][keys][D] with element strides sb / sh / sl: outer = sequences
 // and keys = Lmax for a contiguous cache, outer = physical blocks and keys = block size for a paged one.
 int make_kv_map(CUtensorMap* map, const void* base, const rapid_attn_shape& s, int64_t outer,
-                int64_t keys, int64_t sb, int64_t sh, int64_t sl, int box_rows) {
+                int64_t keys, int64_t sb, int64_t sh, int64_t sl, int box_rows, bool fp8 = false) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) {
         set_error("cuTensorMapEncodeTiled is not available from the CUDA driver");
         return RAPID_ERR_CUDA;
     }
     cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)keys, (cuuint64_t)s.Hkv, (cuuint64_t)outer};
-    cuuint64_t strides[3] = {(cuuint64_t)sl * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+    // bf16: boxes of 64 columns (128 bytes); E4M3 codes: the whole 128-byte row of a key
+    const cuuint64_t esz = fp8 ? 1 : 2;
+    cuuint64_t strides[3] = {(cuuint64_t)sl * esz, (cuuint64_t)sh * esz, (cuuint64_t)sb * esz};
+    cuuint32_t box[4] = {fp8 ? 128u : 64u, (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+    CUresult r = enc(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
                      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -1259,7 +1297,7 @@ struct AttnCall {
 int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
                       const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
                       const rapid_paged_kv* paged, const int32_t* block_table, AttnCall& c,
-                      bool describe_only = false) {
+                      bool describe_only = false, bool fp8 = false) {
     if ((!ctx_lens && !describe_only) || !shape) {
         set_error("%s: NULL argument", who);
         return RAPID_ERR_INVALID_ARG;
@@ -1269,6 +1307,7 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
                   (long long)shape->Lmax, gamma);
         return RAPID_ERR_INVALID_ARG;
     }
+    if (params && params->kv_fp8) fp8 = true;  // planning for, or describing, a call over an 8-bit cache
     const rapid_attn_shape& s = *shape;
     const int R = gamma + 1;
     const int G = s.Hq / s.Hkv;
@@ -1317,9 +1356,19 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
         c.sh = s.kv_stride_h ? s.kv_stride_h : s.Lmax * c.sl;
         c.sb = s.kv_stride_b ? s.kv_stride_b : s.Hkv * c.sh;
     }
-    if (c.sl < s.D || c.sl % 8 || c.sh % 8 || c.sb % 8 || c.sh <= 0 || c.sb <= 0) {
-        set_error("%s: K/V strides must be positive multiples of 8 elements", who);
+    const int stride_unit = fp8 ? 16 : 8;  // 16 bytes either way
+    if (c.sl < s.D || c.sl % stride_unit || c.sh % stride_unit || c.sb % stride_unit || c.sh <= 0 || c.sb <= 0) {
+        set_error("%s: K/V strides must be positive multiples of %d elements", who, stride_unit);
         return RAPID_ERR_UNSUPPORTED;
+    }
+    if (fp8) {
+        const int want8 = params ? params->kernel : RAPID_ATTN_KERNEL_AUTO;
+        if (s.D != 128 || GR > 96 || sink || window || paged ||
+            (want8 != RAPID_ATTN_KERNEL_AUTO && want8 != RAPID_ATTN_KERNEL_KEYS_ON_M)) {
+            set_error("%s: the 8-bit cache needs head_dim 128, at most 96 grouped rows, a contiguous cache, no window "
+                      "and the keys-on-M kernel", who);
+            return RAPID_ERR_UNSUPPORTED;
+        }
     }
     const WsLayout lay = ws_layout(s.B, s.Hkv, GR, s.D);
     if (!describe_only && (!workspace || workspace_bytes < lay.total || ((uintptr_t)workspace & 255))) {
@@ -1372,10 +1421,11 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
     const bool kt_auto = kt_ok && (GR + 15) / 16 <= kt::kMaxNC;
     c.kt_path = want == RAPID_ATTN_KERNEL_KEYS_ON_M || want == RAPID_ATTN_KERNEL_CLUSTER_MERGE ||
                 (want == RAPID_ATTN_KERNEL_AUTO && kt_auto);
-    c.need_cluster = want == RAPID_ATTN_KERNEL_CLUSTER_MERGE;
-    c.want_cluster = c.need_cluster ||
+    if (fp8) c.kt_path = true;
+    c.need_cluster = !fp8 && want == RAPID_ATTN_KERNEL_CLUSTER_MERGE;
+    c.want_cluster = !fp8 && (c.need_cluster ||
                      (want == RAPID_ATTN_KERNEL_AUTO && c.kt_path && s.B == 1 && s.Lmax <= kClusterMaxKeys &&
-                      !(params && params->split_done_event));
+                      !(params && params->split_done_event)));
     if (c.need_cluster && (int64_t)s.B * s.Hkv * 2 > kMaxCtas) {
         set_error("%s: too many (sequence, KV head) units for one cluster each", who);
         return RAPID_ERR_UNSUPPORTED;
@@ -1526,6 +1576,74 @@ int launch_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_s
         return RAPID_ERR_UNSUPPORTED;
     }
     return launch_plan_kernel(c, workspace, shape->D, stream);
+}
+
+template <int NC, int SG>
+int launch_split_kt8(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t stream) {
+    constexpr int smem = kt8::smem_bytes(NC);
+    static_assert(smem <= kMaxSmemOptin - 4096, "shared memory (dynamic + the kernel's static arrays)");
+    static bool configured[64] = {};
+    int dev = 0;
+    RAPID_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        RAPID_CUDA_CHECK(cudaFuncSetAttribute(kt8::verify_attn_splitkv_kt8_kernel<NC, SG>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    RAPID_CUDA_CHECK(launch_dependent(kt8::verify_attn_splitkv_kt8_kernel<NC, SG>, dim3(a.num_ctas),
+                                      dim3(kt8::threads(SG)), (size_t)smem, stream, tmK, tmV, a));
+    return RAPID_OK;
+}
+
+int launch_verify_attention_fp8(const void* q, const void* k_cache, const void* v_cache, const float* k_scale,
+                                const float* v_scale, const int32_t* ctx_lens, int gamma, void* out,
+                                const rapid_attn_shape* shape, const rapid_attn_params* params, void* workspace,
+                                size_t workspace_bytes, cudaStream_t stream) {
+    if (!q || !k_cache || !v_cache || !k_scale || !v_scale || !ctx_lens || !out || !shape) {
+        set_error("rapid_verify_attention_fp8: NULL argument");
+        return RAPID_ERR_INVALID_ARG;
+    }
+    AttnCall c;
+    int rc = prepare_attention("rapid_verify_attention_fp8", ctx_lens, gamma, shape, params, workspace, workspace_bytes,
+                               nullptr, nullptr, c, false, true);
+    if (rc != RAPID_OK) return rc;
+    if (((uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)q | (uintptr_t)out) & 15) {
+        set_error("rapid_verify_attention_fp8: q, k_cache, v_cache and out must be 16-byte aligned");
+        return RAPID_ERR_UNSUPPORTED;
+    }
+    const rapid_attn_shape& s = *shape;
+    AttnArgs& a = c.a;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.out = static_cast<__nv_bfloat16*>(out);
+    a.lse_out = params ? params->lse_out : nullptr;
+    a.out_f32 = params ? params->out_f32 : nullptr;
+    a.k_scale = k_scale;
+    a.v_scale = v_scale;
+    CUtensorMap tmK, tmV;
+    rc = make_kv_map(&tmK, k_cache, s, c.outer, c.keys, c.sb, c.sh, c.sl, kt8::kKeys, true);
+    if (rc != RAPID_OK) return rc;
+    rc = make_kv_map(&tmV, v_cache, s, c.outer, c.keys, c.sb, c.sh, c.sl, kt8::kKeys, true);
+    if (rc != RAPID_OK) return rc;
+    if (!a.caller_plan) {
+        rc = launch_plan_kernel(c, workspace, s.D, stream);
+        if (rc != RAPID_OK) return rc;
+        a.plan_mode = RAPID_PLAN_READY;
+    }
+    switch (c.NC) {
+        case 1: rc = launch_split_kt8<1, 1>(tmK, tmV, a, stream); break;
+        case 2: rc = launch_split_kt8<2, 1>(tmK, tmV, a, stream); break;
+        case 3: rc = launch_split_kt8<3, 1>(tmK, tmV, a, stream); break;
+        case 4: rc = launch_split_kt8<4, 2>(tmK, tmV, a, stream); break;
+        default: rc = launch_split_kt8<6, 2>(tmK, tmV, a, stream); break;  // 65 to 96 rows: 96 columns, two groups
+    }
+    if (rc != RAPID_OK) return rc;
+    if (params && params->split_done_event)
+        RAPID_CUDA_CHECK(cudaEventRecord(static_cast<cudaEvent_t>(params->split_done_event), stream));
+    dim3 grid(a.GR, s.B * s.Hkv);
+    RAPID_CUDA_CHECK(launch_dependent(verify_attn_merge_kernel<128>, grid, dim3(128), 0, stream, a, c.KS, a.out,
+                                      a.lse_out, a.out_f32));
+    count_launch(2);
+    return RAPID_OK;
 }
 
 int launch_verify_attention(const void* q, const void* k_cache, const void* v_cache,

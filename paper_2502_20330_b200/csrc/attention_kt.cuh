@@ -206,7 +206,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
         sh_lfin[tid] = 0.f;
     }
     Walk w;
-    split_kernel_walk(a, cta, w, &s_walk);
+    split_kernel_walk(a, cta, 1, w, &s_walk);
     if (cta == 0 && warp == WS && lane == 1) check_call_inputs(a, 1);  // an idle lane of the producer warp
     const uint32_t tmem_base = tmem_slot;
     const WaitCtx wc = {&s_abort, a.wait_limit};
@@ -564,7 +564,7 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                     // V rows beyond the context may hold any bits: zero them so that 0 * row = 0
                     // (one group does it; PV waits for both groups' arrivals)
                     ok &= warp_wait_bounded(&v_full[jj % NV], (jj / NV) & 1, wc);  // the V tile has landed
-                    const int first_bad = L - key0;
+                    const int first_bad = max(L - key0, 0);
                     const int chunks = (kKeys - first_bad) * 8;
                     for (int h = 0; h < 2; ++h) {
                         uint8_t* vgen = smem_gen + OFF_V + (h * NV + jj % NV) * kBlk;

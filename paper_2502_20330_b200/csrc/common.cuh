@@ -57,6 +57,10 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
                             const rapid_attn_shape* shape, const rapid_attn_params* params,
                             void* workspace, size_t workspace_bytes, cudaStream_t stream,
                             const rapid_paged_kv* paged = nullptr, const int32_t* block_table = nullptr);
+int launch_verify_attention_fp8(const void* q, const void* k_cache, const void* v_cache, const float* k_scale,
+                                const float* v_scale, const int32_t* ctx_lens, int gamma, void* out,
+                                const rapid_attn_shape* shape, const rapid_attn_params* params, void* workspace,
+                                size_t workspace_bytes, cudaStream_t stream);
 int launch_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_shape* shape,
                           const rapid_attn_params* params, void* workspace, size_t workspace_bytes,
                           cudaStream_t stream);

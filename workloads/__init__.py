@@ -186,3 +186,34 @@ def accept_inputs(cfg: VerifyConfig, seed: int, device="cpu"):
 def bf16_bits(t: torch.Tensor):
     """Raw bits of a bf16 tensor as a numpy uint16 array on the host."""
     return t.detach().contiguous().cpu().view(torch.int16).numpy().view("uint16")
+
+
+def attention_inputs_fp8(cfg: VerifyConfig, seed: int, device="cpu", layer: int = 0, poison_padding: bool = False):
+    """The same draws as ``attention_inputs`` with the cache stored as FP8 E4M3 codes: every (sequence,
+    KV head) slab of K and of V ~ N(0,1) is divided by its own scale (largest magnitude / 448, the
+    format's largest value) and rounded to E4M3 by the library's conversion.
+    Returns q [B,R,Hq,D] bf16, k_codes, v_codes [B,Hkv,Lmax,D] uint8, k_scale, v_scale [B,Hkv] float32,
+    ctx_lens [B] int32.  ``poison_padding`` fills positions >= ctx_lens[b] with the NaN code."""
+    ctx = context_lengths(cfg, seed)
+    Lmax = cache_capacity(cfg, ctx)
+    g = _gen(seed * 1000003 + 17 * layer + 1, device)
+    q = (torch.randn(cfg.B, cfg.R, cfg.Hq, cfg.D, generator=g, device=device,
+                     dtype=torch.float32) * cfg.q_scale).to(torch.bfloat16)
+    kc = torch.empty(cfg.B, cfg.Hkv, Lmax, cfg.D, device=device, dtype=torch.uint8)
+    vc = torch.empty_like(kc)
+    ks = torch.empty(cfg.B, cfg.Hkv, device=device, dtype=torch.float32)
+    vs = torch.empty_like(ks)
+    for b in range(cfg.B):
+        for h in range(cfg.Hkv):
+            for codes, scales in ((kc, ks), (vc, vs)):
+                x = torch.randn(Lmax, cfg.D, generator=g, device=device, dtype=torch.float32)
+                s = x.abs().max() / 448.0
+                scales[b, h] = s
+                codes[b, h] = (x / s).to(torch.float8_e4m3fn).view(torch.uint8)
+    if poison_padding:
+        for b in range(cfg.B):
+            L = int(ctx[b])
+            if L < Lmax:
+                kc[b, :, L:] = 0x7F
+                vc[b, :, L:] = 0xFF
+    return q, kc, vc, ks, vs, ctx.to(device)
