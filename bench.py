@@ -80,8 +80,11 @@ def job_throughput_gbs(bytes_per_rank_step: int, world: int, ms_per_step: float)
     return bytes_per_rank_step * world / (ms_per_step * 1e-3) / 1e9
 
 
+KV_ELEMENT_BYTES = 2   # set to 1 by --kv fp8: the algorithmic bytes are those of the cache as it is stored
+
+
 def kv_bytes_per_layer(cfg, ctx) -> int:
-    return int(4 * cfg.Hkv * cfg.D * int(ctx.sum()))
+    return int(2 * KV_ELEMENT_BYTES * cfg.Hkv * cfg.D * int(ctx.sum()))
 
 
 L2_BYTES = 126 * 2**20
@@ -101,7 +104,8 @@ def with_layer_chain(cfg, ctx):
 def config_dict(cfg, ctx, world, sharded=False):
     """What both arms print as `config`: the workload, nothing of how an arm runs it."""
     kv_layer = kv_bytes_per_layer(cfg, ctx)
-    return {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
+    return {"workload": cfg.name, "kv_cache": "fp8 e4m3 + fp32 scale per (sequence, KV head)" if KV_ELEMENT_BYTES == 1 else "bf16",
+            "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
             "ctx": [int(x) for x in ctx], "gamma": cfg.gamma, "V": cfg.V, "layers": cfg.layers, "eta": cfg.eta,
             "kv_bytes_per_step": kv_layer * cfg.layers,
             "l2": f"inputs larger than L2: {cfg.layers} distinct cache(s) of {kv_layer / 2**20:.0f} MiB per step"
@@ -149,9 +153,16 @@ class OracleSample:
             attn_inputs = wl.attention_inputs(cfg, seed, device="cpu", layer=0)
         if accept_inputs is None:
             accept_inputs = wl.accept_inputs(cfg, seed, device="cpu")
-        q, k, v, ctx_t = attn_inputs
+        self.fp8 = KV_ELEMENT_BYTES == 1
+        if self.fp8:
+            if len(attn_inputs) == 4:      # the reference arm generates its own inputs
+                attn_inputs = wl.attention_inputs_fp8(cfg, seed, device="cpu", layer=0)
+            q, k, v, ks, vs, ctx_t = attn_inputs
+            self.bits = (wl.bf16_bits(q), k.cpu().numpy(), v.cpu().numpy(), ks.cpu().numpy(), vs.cpu().numpy())
+        else:
+            q, k, v, ctx_t = attn_inputs
+            self.bits = (wl.bf16_bits(q), wl.bf16_bits(k), wl.bf16_bits(v))
         self.ctx = ctx_t.cpu()
-        self.bits = (wl.bf16_bits(q), wl.bf16_bits(k), wl.bf16_bits(v))
         self.ctx_np = self.ctx.numpy()
         self.acc = [t.cpu().numpy() for t in accept_inputs]
         self.total_units = cfg.B * cfg.Hq * cfg.R
@@ -171,7 +182,8 @@ class OracleSample:
         if n_units < self.total_units:
             units = np.sort(self.rng.choice(self.total_units, size=n_units, replace=False)).astype(np.int64)
         t0 = time.perf_counter()
-        out, lse = self.oracle.verify_attention(*self.bits, self.ctx_np, self.cfg.gamma, units=units)
+        fn = self.oracle.verify_attention_fp8 if self.fp8 else self.oracle.verify_attention
+        out, lse = fn(*self.bits, self.ctx_np, self.cfg.gamma, units=units)
         dt = time.perf_counter() - t0
         self.attn_ref = (out, lse)
         return dt, n_units
@@ -365,17 +377,30 @@ def run_ours(args, cfg):
     if not args.layers:
         cfg = with_layer_chain(cfg, ctx_cpu)
     Lmax = wl.cache_capacity(cfg, ctx_cpu)
+    fp8 = KV_ELEMENT_BYTES == 1
     layers = []
     for layer in range(cfg.layers):
-        q, k, v, ctx = wl.attention_inputs(cfg, seed, device=dev, layer=layer)
-        layers.append((q, k, v, torch.empty_like(q)))
+        if fp8:
+            q, k, v, ks, vs, ctx = wl.attention_inputs_fp8(cfg, seed, device=dev, layer=layer)
+            layers.append((q, k, v, torch.empty_like(q), ks, vs))
+        else:
+            q, k, v, ctx = wl.attention_inputs(cfg, seed, device=dev, layer=layer)
+            layers.append((q, k, v, torch.empty_like(q)))
+
+    def attention(layer, params, st=None):
+        if fp8:
+            q_, k_, v_, out_, ks_, vs_ = layer
+            R.rapid_verify_attention_fp8(q_, k_, v_, ks_, vs_, ctx, cfg.gamma, out_, aws, params, stream=st)
+        else:
+            q_, k_, v_, out_ = layer
+            R.rapid_verify_attention(q_, k_, v_, ctx, cfg.gamma, out_, aws, params, stream=st)
     z, d, tok, u = wl.accept_inputs(cfg, seed, device=dev)
     alen = torch.zeros(cfg.B, dtype=torch.int32, device=dev)
     ntok = torch.zeros_like(alen)
     aws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma), device=dev)
     cws = R.new_workspace(R.accept_workspace_bytes(cfg.B, cfg.gamma, cfg.V), device=dev)
     acc_params = R.AcceptParams(temperature=cfg.temperature, tail_alpha=cfg.tail_alpha)
-    plan_params = R.AttnParams(kernel=args.kernel)
+    plan_params = R.AttnParams(kernel=args.kernel, kv_fp8=fp8)
     stream = torch.cuda.current_stream()
     sptr = int(stream.cuda_stream)
     ev = RawEvents()
@@ -399,11 +424,11 @@ def run_ours(args, cfg):
             flush.fill_(1)
         if not args.no_plan:
             R.rapid_attention_plan(ctx, cfg.gamma, cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, aws, plan_params, stream=st)
-        for li, (q, k, v, out) in enumerate(layers):
+        for li, layer in enumerate(layers):
             if call_events is not None:
                 ev.record(call_events[li][0], sptr)
             e1 = split_events[li] if split_events is not None else None
-            R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, aws, attn_params(li, e1), stream=st)
+            attention(layer, attn_params(li, e1), st)
             if call_events is not None:
                 ev.record(call_events[li][1], sptr)
         R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params, stream=st)
@@ -418,9 +443,11 @@ def run_ours(args, cfg):
         step()
     barrier()
     # which kernels serve an attention call of this workload
-    info = R.rapid_attention_describe(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma, R.AttnParams(kernel=args.kernel))
+    info = R.rapid_attention_describe(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma, plan_params)
     launches_per_call = info["kernels_per_call"]
-    if info["kernel"] == R.ATTN_KERNEL_CLUSTER_MERGE:
+    if fp8:
+        dominant = "verify_attn_splitkv_kt8_kernel"
+    elif info["kernel"] == R.ATTN_KERNEL_CLUSTER_MERGE:
         dominant = f"verify_attn_splitkv_kt_kernel (clusters of {info['cluster_size']} CTAs, merged on chip)"
     else:
         dominant = "verify_attn_splitkv_kt_kernel" if info["kernel"] == R.ATTN_KERNEL_KEYS_ON_M \
@@ -563,7 +590,7 @@ def run_ours(args, cfg):
     line = {
         "metric": "verify_step_kv_read_gbs", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "vs_baseline": None, "dtype": "fp8 e4m3 cache, bf16 q/out, fp32 accumulate" if fp8 else "bf16", "data": "synthetic",
         "config": config_dict(cfg, ctx_cpu, world),
         "run": {"launch": "the step captured in one CUDA graph, replayed per step",
                 "plan": "none" if args.no_plan else "one rapid_attention_plan per step, shared by its layers",
@@ -584,15 +611,15 @@ def run_ours(args, cfg):
     if sustained is not None:
         line["sustained"] = sustained
 
-    if rank == 0 and world == 1 and not args.no_e2e:
+    if rank == 0 and world == 1 and not args.no_e2e and not fp8:
         line["e2e"] = run_e2e(R, cfg, seed, Lmax, kv_layer, dev)
     elif rank == 0:
         line["e2e"] = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         # The CPU leg runs on the very bits the library ran on (layer 0 and the logits, copied back
         # from the device), and what it computes is also what the library's results are judged by.
-        q0, k0, v0, out0 = layers[0]
-        R.rapid_verify_attention(q0, k0, v0, ctx, cfg.gamma, out0, aws, R.AttnParams(kernel=args.kernel))
+        out0 = layers[0][3]
+        attention(layers[0], R.AttnParams(kernel=args.kernel))
         R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params)
         torch.cuda.synchronize()
         dev_out = out0.float().cpu().numpy()
@@ -604,9 +631,10 @@ def run_ours(args, cfg):
             R.rapid_accept(zz, dd, tt, uu, cfg.eta, alen, ntok, cws, acc_params)
             torch.cuda.synchronize()
             extra.append(([t.cpu().numpy() for t in (zz, dd, tt, uu)], (alen.cpu().numpy().copy(), ntok.cpu().numpy().copy())))
-        host_attn = tuple(t.cpu() for t in (q0, k0, v0, ctx))
+        l0 = layers[0]
+        host_attn = tuple(t.cpu() for t in ((l0[0], l0[1], l0[2], l0[4], l0[5], ctx) if fp8 else (l0[0], l0[1], l0[2], ctx)))
         host_acc = tuple(t.cpu() for t in (z, d, tok, u))
-        del layers, q0, k0, v0
+        del layers, l0
         smp = OracleSample(cfg, seed, host_attn, host_acc)
         gbs, sample, _ = smp.step(12.0)
         line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": smp.cores, "kind": "oracle", "sample": sample}
@@ -729,6 +757,8 @@ def run_sharded(args, cfg):
 
 
 def _rank_main(args):
+    global KV_ELEMENT_BYTES
+    KV_ELEMENT_BYTES = 1 if args.kv == "fp8" else 2
     cfg = wl.CONFIGS[args.workload]
     if args.layers:
         cfg = wl.with_overrides(cfg, layers=args.layers)
@@ -752,6 +782,8 @@ def main():
     ap.add_argument("--kernel", type=int, default=0, choices=[0, 1, 2, 3],
                     help="split kernel: 0 the library's choice, 1 rows on the MMA's M axis, 2 keys on the M axis, "
                          "3 keys on M with one cluster per KV head")
+    ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"],
+                    help="storage of the KV cache: bf16, or FP8 E4M3 codes with a scale per (sequence, KV head)")
     ap.add_argument("--sharded", action="store_true", help="context-sharded attention over the ranks")
     ap.add_argument("--no-plan", action="store_true", help="every attention call works its split out itself")
     ap.add_argument("--no-e2e", action="store_true")

@@ -1578,7 +1578,7 @@ int launch_attention_plan(const int32_t* ctx_lens, int gamma, const rapid_attn_s
     return launch_plan_kernel(c, workspace, shape->D, stream);
 }
 
-template <int NC, int SG>
+template <int NC>
 int launch_split_kt8(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t stream) {
     constexpr int smem = kt8::smem_bytes(NC);
     static_assert(smem <= kMaxSmemOptin - 4096, "shared memory (dynamic + the kernel's static arrays)");
@@ -1586,12 +1586,12 @@ int launch_split_kt8(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnA
     int dev = 0;
     RAPID_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        RAPID_CUDA_CHECK(cudaFuncSetAttribute(kt8::verify_attn_splitkv_kt8_kernel<NC, SG>,
+        RAPID_CUDA_CHECK(cudaFuncSetAttribute(kt8::verify_attn_splitkv_kt8_kernel<NC>,
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    RAPID_CUDA_CHECK(launch_dependent(kt8::verify_attn_splitkv_kt8_kernel<NC, SG>, dim3(a.num_ctas),
-                                      dim3(kt8::threads(SG)), (size_t)smem, stream, tmK, tmV, a));
+    RAPID_CUDA_CHECK(launch_dependent(kt8::verify_attn_splitkv_kt8_kernel<NC>, dim3(a.num_ctas),
+                                      dim3(kt8::threads(NC)), (size_t)smem, stream, tmK, tmV, a));
     return RAPID_OK;
 }
 
@@ -1630,11 +1630,12 @@ int launch_verify_attention_fp8(const void* q, const void* k_cache, const void* 
         a.plan_mode = RAPID_PLAN_READY;
     }
     switch (c.NC) {
-        case 1: rc = launch_split_kt8<1, 1>(tmK, tmV, a, stream); break;
-        case 2: rc = launch_split_kt8<2, 1>(tmK, tmV, a, stream); break;
-        case 3: rc = launch_split_kt8<3, 1>(tmK, tmV, a, stream); break;
-        case 4: rc = launch_split_kt8<4, 2>(tmK, tmV, a, stream); break;
-        default: rc = launch_split_kt8<6, 2>(tmK, tmV, a, stream); break;  // 65 to 96 rows: 96 columns, two groups
+        case 1: rc = launch_split_kt8<1>(tmK, tmV, a, stream); break;
+        case 2: rc = launch_split_kt8<2>(tmK, tmV, a, stream); break;
+        case 3: rc = launch_split_kt8<3>(tmK, tmV, a, stream); break;
+        case 4: rc = launch_split_kt8<4>(tmK, tmV, a, stream); break;
+        case 5: rc = launch_split_kt8<5>(tmK, tmV, a, stream); break;
+        default: rc = launch_split_kt8<6>(tmK, tmV, a, stream); break;
     }
     if (rc != RAPID_OK) return rc;
     if (params && params->split_done_event)

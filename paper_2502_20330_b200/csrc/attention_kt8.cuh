@@ -30,16 +30,25 @@
 
 namespace kt8 {
 
-using kt::bar_softmax;
-using kt::bar_softmax_or;
 using kt::warp_max32;
 using kt::warp_sum32;
 
-// Barrier of all softmax threads (one group: its own barrier; two groups: a third one over both).
+// Named barriers: one per softmax group of 128 threads (ids 1 .. SG), one over all groups (id 15).
+__device__ __forceinline__ void bar_softmax(int grp) {
+    asm volatile("bar.sync %0, 128;" ::"r"(grp + 1) : "memory");
+}
+__device__ __forceinline__ bool bar_softmax_or(int grp, bool flag) {
+    uint32_t res;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %2, 0;\n\tbar.red.or.pred p, %1, 128, q;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(res)
+                 : "r"(grp + 1), "r"((uint32_t)flag)
+                 : "memory");
+    return res != 0;
+}
 template <int SG>
 __device__ __forceinline__ void bar_softmax_all() {
-    if (SG == 1) asm volatile("bar.sync 1, 128;" ::: "memory");
-    else asm volatile("bar.sync 3, 256;" ::: "memory");
+    asm volatile("bar.sync 15, %0;" ::"n"(128 * SG) : "memory");
 }
 
 constexpr int kKeys = 128;           // keys per tile
@@ -47,7 +56,11 @@ constexpr int kBlk = kKeys * 128;    // bytes of one tile: 128 keys x 128 E4M3 c
 constexpr int kNK = 4, kNV = 6;      // K and V slots
 constexpr float kShift = 4.f;        // a new reference sits this far (log2) below the maximum it was taken from
 constexpr float kJump = 8.f;         // a score this far above the reference (p' > 256) moves it
-__host__ __device__ constexpr int threads(int SG) { return 128 * SG + 96; }
+// Columns per softmax group.  (The kernel also runs with 8: six groups at 48 columns measured 75 us per
+// 8B-128K layer against 68 us for three groups of 16 -- every group pays its own waits and barriers per
+// tile, and the schedulers' issue slots, 47 % busy with three groups, are what runs out.)
+__host__ __device__ constexpr int group_cols(int NC) { return 16; }
+__host__ __device__ constexpr int threads(int NC) { return 128 * (NC * 16 / group_cols(NC)) + 96; }  // + three role warps
 __host__ __device__ constexpr int smem_bytes(int NC) {
     // K ring + V ring + Q hi, lo (N rows of 128 bytes each) + P^T hi, lo (128 keys x 128 bytes each)
     return (kNK + kNV) * kBlk + 2 * (NC * 16) * 128 + 2 * kBlk + 1024;
@@ -69,36 +82,38 @@ __host__ __device__ constexpr uint32_t umma_idesc_e4m3(int M, int N, int a_mn_ma
     return (1u << 4) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
            ((uint32_t)(M >> 4) << 24);
 }
-// Two fp32 -> two E4M3 codes (round to nearest even, saturating), `hi` in bits 8..15, `lo` in bits 0..7.
-__device__ __forceinline__ uint32_t cvt_e4m3x2(float hi, float lo) {
-    uint16_t r;
-    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-// Two E4M3 codes (bits 0..15) -> their values.
-__device__ __forceinline__ float2 e4m3x2_to_float2(uint32_t codes) {
-    uint32_t h2;
-    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)codes));
-    return __half22float2(*reinterpret_cast<__half2*>(&h2));
-}
-// A non-negative value below 448 as hi + rest: hi keeps 3 mantissa bits (an E4M3 normal, or 0 below
-// 2^-6); returns hi's E4M3 code and leaves the remainder in `rest`.
-__device__ __forceinline__ uint32_t split_hi(float v, float& rest) {
-    uint32_t h = (__float_as_uint(v) + 0x00080000u) & 0xFFF00000u;
-    h = v >= 0.015625f ? h : 0u;
-    rest = v - __uint_as_float(h);
-    return h ? ((h >> 20) - 960u) & 0x7Fu : 0u;
+// Two values as hi + lo E4M3 pairs: hi = E4M3(v) by the hardware conversion, the remainders formed in
+// packed half precision (v < 448 and its remainder need far fewer than half's 11 bits) and converted
+// the same way.  Returns hi's two codes in bits 0..15 (v0 low), lo's two in `lo`.
+__device__ __forceinline__ uint32_t split_e4m3x2(float v0, float v1, uint32_t& lo) {
+    uint16_t h;
+    uint32_t hf2, vf2, rf2;
+    uint16_t l;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(h) : "f"(v1), "f"(v0));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(hf2) : "h"(h));
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(vf2) : "f"(v1), "f"(v0));
+    asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(rf2) : "r"(vf2), "r"(hf2));
+    asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(l) : "r"(rf2));
+    lo = l;
+    return h;
 }
 
-template <int NC, int SG = 1>
-__global__ void __launch_bounds__(threads(SG), 1)
+// NC = N / 16 column chunks.  There are SG = N / NG softmax groups of 128 threads each (thread t of
+// every group is key t of the tile): a group forms the probabilities of its own NG = 8 or 16 columns --
+// half or all of a 16-byte chunk of the key's P^T hi row, and of its lo row -- and keeps those rows'
+// references and sums.  What a tile costs is the time ONE warp takes over its 32 keys x NG columns
+// (some 8 cycles per instruction: a latency chain, not an issue limit), and this cache delivers
+// twice the keys per byte: narrow groups, several warps per scheduler, keep that chain short.
+template <int NC>
+__global__ void __launch_bounds__(threads(NC), 1)
 verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                                const __grid_constant__ AttnArgs a) {
     constexpr int D = 128;
     constexpr int N = NC * 16;
-    constexpr int NG = N / SG;  // columns per softmax group
-    constexpr int WS = 4 * SG;  // softmax warps; the role warps follow
-    static_assert(NG % 16 == 0 && NG <= 48, "a group's columns are whole 16-byte chunks of a P^T row, held as fp32");
+    constexpr int NG = group_cols(NC);  // columns per softmax group
+    constexpr int SG = N / NG;          // softmax groups
+    constexpr int WS = 4 * SG;          // softmax warps; the role warps follow
+    static_assert(SG <= 6, "named barriers 1..6 and 1024 threads at most");
     constexpr int NK = kNK, NV = kNV;
     constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t COL_S = 0;    // S^T buffer b at COL_S + 128 b
@@ -138,7 +153,7 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
             mbar_init(&p_full[i], WS);
             mbar_init(&drain_bar[i], 1);
         }
-        mbar_init(&q_full, 4);  // the four warps of the first softmax group
+        mbar_init(&q_full, WS);  // every softmax warp
         fence_mbar_init();
         s_abort = 0;
         prefetch_tensormap(&tmK);
@@ -148,7 +163,7 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
     // The rows of both Q operands past the grouped rows are never written: zero them once (scores 0).
     {
         const int pad_chunks = (N - a.GR) * 8;  // 16-byte chunks per operand
-        for (int i = tid; i < 2 * pad_chunks; i += threads(SG)) {
+        for (int i = tid; i < 2 * pad_chunks; i += threads(NC)) {
             const int h = i >= pad_chunks, k16 = h ? i - pad_chunks : i;
             *reinterpret_cast<uint4*>(smem_gen + (h ? OFF_QL : OFF_QH) + a.GR * 128 + k16 * 16) = make_uint4(0, 0, 0, 0);
         }
@@ -280,56 +295,50 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
         while (w.remaining > 0) {
             const int seg = (int)min((long long)(w.ntiles - w.tile), w.remaining);
             const int L = w.L;
-            // ---- the unit's Q: row t of the first group, quantised to hi + lo codes on the row's own scale ----
-            if (grp == 0) {
-                if (t < a.GR) {
-                    const int i = t / a.G, g = t % a.G;
+            // ---- the unit's Q, quantised to hi + lo codes on every row's own scale ----
+            // softmax thread st takes 16 consecutive elements (one 16-byte chunk of codes) of grouped row
+            // st / 8: the eight threads of a row find its largest magnitude with three shuffles
+            {
+                const int st = grp * 128 + t;
+                const int row = st >> 3, j2 = st & 7;
+                const bool has = row < a.GR;
+                uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
+                if (has) {
+                    const int i = row / a.G, g = row % a.G;
                     const uint4* src = reinterpret_cast<const uint4*>(
-                        a.q + (((size_t)w.b * a.R + i) * a.Hq + (size_t)w.kvh * a.G + g) * D);
-                    uint4 raw[16];
+                        a.q + (((size_t)w.b * a.R + i) * a.Hq + (size_t)w.kvh * a.G + g) * D) + 2 * j2;
+                    r0 = __ldg(src);
+                    r1 = __ldg(src + 1);
+                }
+                const uint32_t u[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+                float amax = 0.f;
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) raw[j] = __ldg(src + j);
-                    float amax = 0.f;
+                for (int e = 0; e < 8; ++e) {
+                    amax = fmaxf(amax, fabsf(__uint_as_float(u[e] << 16)));
+                    amax = fmaxf(amax, fabsf(__uint_as_float(u[e] & 0xffff0000u)));
+                }
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const uint32_t u[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+                for (int o = 1; o < 8; o <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                // 2^s with 128 <= amax * 2^s < 256 (s clamped to what fp32 holds; a zero row: 2^0)
+                int s2 = amax > 0.f ? 7 - ((int)((__float_as_uint(amax) >> 23) & 0xff) - 127) : 0;
+                s2 = s2 > 126 ? 126 : (s2 < -126 ? -126 : s2);
+                const float up = __uint_as_float((uint32_t)(s2 + 127) << 23), down = __uint_as_float((uint32_t)(127 - s2) << 23);
+                if (has) {
+                    if (j2 == 0) sh_c[row] = a.scale_log2 * __ldg(a.k_scale + (size_t)w.b * a.Hkv + w.kvh) * down;
+                    uint32_t hw[4], lw[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            amax = fmaxf(amax, fabsf(__uint_as_float(u[e] << 16)));
-                            amax = fmaxf(amax, fabsf(__uint_as_float(u[e] & 0xffff0000u)));
-                        }
+                    for (int e = 0; e < 8; e += 2) {
+                        uint32_t l01, l23;
+                        const uint32_t h01 = split_e4m3x2(__uint_as_float(u[e] << 16) * up, __uint_as_float(u[e] & 0xffff0000u) * up, l01);
+                        const uint32_t h23 = split_e4m3x2(__uint_as_float(u[e + 1] << 16) * up, __uint_as_float(u[e + 1] & 0xffff0000u) * up, l23);
+                        hw[e >> 1] = h01 | (h23 << 16);
+                        lw[e >> 1] = l01 | (l23 << 16);
                     }
-                    // 2^s with 128 <= amax * 2^s < 256 (s clamped to what fp32 holds; a zero row: 2^0)
-                    int s2 = amax > 0.f ? 7 - ((int)((__float_as_uint(amax) >> 23) & 0xff) - 127) : 0;
-                    s2 = s2 > 126 ? 126 : (s2 < -126 ? -126 : s2);
-                    const float up = __uint_as_float((uint32_t)(s2 + 127) << 23), down = __uint_as_float((uint32_t)(127 - s2) << 23);
-                    sh_c[t] = a.scale_log2 * __ldg(a.k_scale + (size_t)w.b * a.Hkv + w.kvh) * down;
-                    uint8_t* qh = smem_gen + OFF_QH + t * 128;
-                    uint8_t* ql = smem_gen + OFF_QL + t * 128;
-#pragma unroll
-                    for (int j2 = 0; j2 < 8; ++j2) {  // 16 codes = one 16-byte chunk = two loads of 8 bf16
-                        uint32_t hw[4], lw[4];
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            const uint4 r = raw[2 * j2 + half];
-                            const uint32_t u[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-                            for (int e = 0; e < 4; e += 2) {
-                                const float x0 = __uint_as_float(u[e] << 16) * up, x1 = __uint_as_float(u[e] & 0xffff0000u) * up;
-                                const float x2 = __uint_as_float(u[e + 1] << 16) * up, x3 = __uint_as_float(u[e + 1] & 0xffff0000u) * up;
-                                const uint32_t h01 = cvt_e4m3x2(x1, x0), h23 = cvt_e4m3x2(x3, x2);
-                                const float2 d01 = e4m3x2_to_float2(h01), d23 = e4m3x2_to_float2(h23);
-                                const uint32_t l01 = cvt_e4m3x2(x1 - d01.y, x0 - d01.x), l23 = cvt_e4m3x2(x3 - d23.y, x2 - d23.x);
-                                hw[2 * half + (e >> 1)] = h01 | (h23 << 16);
-                                lw[2 * half + (e >> 1)] = l01 | (l23 << 16);
-                            }
-                        }
-                        const int off = ((j2 ^ (t & 7)) << 4);
-                        *reinterpret_cast<uint4*>(qh + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-                        *reinterpret_cast<uint4*>(ql + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-                    }
-                } else if (t < N) {
-                    sh_c[t] = 0.f;
+                    const int off = row * 128 + ((j2 ^ (row & 7)) << 4);
+                    *reinterpret_cast<uint4*>(smem_gen + OFF_QH + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                    *reinterpret_cast<uint4*>(smem_gen + OFF_QL + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                } else if (j2 == 0 && row < N) {
+                    sh_c[row] = 0.f;
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
@@ -353,28 +362,27 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
                 float pv[NG];
                 bool move = ti == 0;
                 if (ti > 0) {
-                    bool far = false;
+                    float xmax = -INFINITY;
+                    uint32_t sr[NG];
+                    tmem_ld_cols<NG>(tS, sr);
+                    tmem_wait_ld();
+                    // a tile every row sees whole (all of a long context but its end) needs no mask
+                    const bool tile_clear = key0 + kKeys <= L - a.stair;
 #pragma unroll
-                    for (int ch = 0; ch < NG / 16; ++ch) {
-                        uint32_t sr[16];
-                        tmem_ld_x16(tS + 16 * ch, sr);
-                        tmem_wait_ld();
+                    for (int e = 0; e < NG; e += 4) {
+                        const int col = C0 + e;
+                        const float4 m = *reinterpret_cast<const float4*>(&sh_mref[col]);
+                        const float4 cc = *reinterpret_cast<const float4*>(&sh_c[col]);
+                        float x[4] = {fmaf(__uint_as_float(sr[e]), cc.x, -m.x), fmaf(__uint_as_float(sr[e + 1]), cc.y, -m.y),
+                                      fmaf(__uint_as_float(sr[e + 2]), cc.z, -m.z), fmaf(__uint_as_float(sr[e + 3]), cc.w, -m.w)};
 #pragma unroll
-                        for (int e = 0; e < 16; e += 4) {
-                            const int li = 16 * ch + e, col = C0 + li;
-                            const float4 m = *reinterpret_cast<const float4*>(&sh_mref[col]);
-                            const float4 cc = *reinterpret_cast<const float4*>(&sh_c[col]);
-                            float x[4] = {fmaf(__uint_as_float(sr[e]), cc.x, -m.x), fmaf(__uint_as_float(sr[e + 1]), cc.y, -m.y),
-                                          fmaf(__uint_as_float(sr[e + 2]), cc.z, -m.z), fmaf(__uint_as_float(sr[e + 3]), cc.w, -m.w)};
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                x[i] = col + i >= cmin ? x[i] : -INFINITY;
-                                far |= x[i] > kJump;
-                                pv[li + i] = fast_exp2(x[i]);
-                            }
+                        for (int i = 0; i < 4; ++i) {
+                            if (!tile_clear) x[i] = col + i >= cmin ? x[i] : -INFINITY;
+                            xmax = fmaxf(xmax, x[i]);
+                            pv[e + i] = fast_exp2(x[i]);
                         }
                     }
-                    move = bar_softmax_or(grp, far);
+                    move = bar_softmax_or(grp, xmax > kJump);
                 }
                 if (jj >= 1) {  // PV of the previous tile is complete: P^T is free, O^T at rest
                     ok &= warp_wait_bounded(&v_empty[(jj - 1) % NV], ((jj - 1) / NV) & 1, wc);
@@ -382,14 +390,13 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
                 }
                 if (move) {
                     // new reference = max(old, this tile's row maxima over the 128 keys - kShift)
-#pragma unroll
-                    for (int ch = 0; ch < NG / 16; ++ch) {
-                        uint32_t sr[16];
-                        tmem_ld_x16(tS + 16 * ch, sr);
+                    {
+                        uint32_t sr[NG];
+                        tmem_ld_cols<NG>(tS, sr);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            const int col = C0 + 16 * ch + e;
+                        for (int e = 0; e < NG; ++e) {
+                            const int col = C0 + e;
                             const float v = (col >= cmin && col < a.GR) ? __uint_as_float(sr[e]) * sh_c[col] : -INFINITY;
                             const float wm = warp_max32(v);
                             if (lane == 0) sh_w[wq][col] = wm;
@@ -409,55 +416,57 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
                     if (ti > 0) {
 #pragma unroll
                         for (int i = 0; i < NG; ++i) lsum[i] *= sh_fac[C0 + i];
-#pragma unroll
-                        for (int ch = 0; ch < NG / 16; ++ch) {
-                            uint32_t orow[16];
-                            tmem_ld_x16(tO + 16 * ch, orow);
+                        {
+                            uint32_t orow[NG];
+                            tmem_ld_cols<NG>(tO, orow);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 16; ++e)
-                                orow[e] = __float_as_uint(__uint_as_float(orow[e]) * sh_fac[C0 + 16 * ch + e]);
-                            tmem_st_x16(tO + 16 * ch, orow);
+                            for (int e = 0; e < NG; ++e)
+                                orow[e] = __float_as_uint(__uint_as_float(orow[e]) * sh_fac[C0 + e]);
+                            tmem_st_cols<NG>(tO, orow);
                         }
                         tmem_wait_st();
                     }
-#pragma unroll
-                    for (int ch = 0; ch < NG / 16; ++ch) {
-                        uint32_t sr[16];
-                        tmem_ld_x16(tS + 16 * ch, sr);
+                    {
+                        uint32_t sr[NG];
+                        tmem_ld_cols<NG>(tS, sr);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            const int li = 16 * ch + e, col = C0 + li;
+                        for (int e = 0; e < NG; ++e) {
+                            const int col = C0 + e;
                             const float m0 = sh_mref[col];
                             const float x0 = col >= cmin
                                                  ? fmaf(__uint_as_float(sr[e]), sh_c[col], m0 == -INFINITY ? 0.f : -m0)
                                                  : -INFINITY;
-                            pv[li] = fast_exp2(x0);
+                            pv[e] = fast_exp2(x0);
                         }
                     }
                 }
-                // this key's rows of P^T: every probability as hi + lo codes, 16 columns per 16-byte chunk
+                // this key's rows of P^T: every probability as hi + lo codes; the group's NG columns are
+                // all or half of one 16-byte chunk of either row
+                {
+                    uint32_t hw[NG / 4], lw[NG / 4];
 #pragma unroll
-                for (int c16 = 0; c16 < NG / 16; ++c16) {
-                    uint32_t hw[4], lw[4];
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        float r0, r1, r2, r3;
-                        const int o = 16 * c16 + 4 * q4;
-                        const uint32_t h0 = split_hi(pv[o], r0), h1 = split_hi(pv[o + 1], r1), h2 = split_hi(pv[o + 2], r2),
-                                       h3 = split_hi(pv[o + 3], r3);
-                        hw[q4] = h0 | (h1 << 8) | (h2 << 16) | (h3 << 24);
-                        lw[q4] = cvt_e4m3x2(r1, r0) | (cvt_e4m3x2(r3, r2) << 16);
+                    for (int q4 = 0; q4 < NG / 4; ++q4) {
+                        const int o = 4 * q4;
+                        uint32_t l01, l23;
+                        const uint32_t h01 = split_e4m3x2(pv[o], pv[o + 1], l01), h23 = split_e4m3x2(pv[o + 2], pv[o + 3], l23);
+                        hw[q4] = h01 | (h23 << 16);
+                        lw[q4] = l01 | (l23 << 16);
                         lsum[o] += pv[o];
                         lsum[o + 1] += pv[o + 1];
                         lsum[o + 2] += pv[o + 2];
                         lsum[o + 3] += pv[o + 3];
                     }
-                    const int g16 = C0 / 16 + c16;  // the chunk's place in the row
-                    const int off = ((g16 ^ p_swz) << 4);
-                    *reinterpret_cast<uint4*>(ph_gen + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-                    *reinterpret_cast<uint4*>(pl_gen + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                    if constexpr (NG == 16) {
+                        const int off = ((grp ^ p_swz) << 4);
+                        *reinterpret_cast<uint4*>(ph_gen + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                        *reinterpret_cast<uint4*>(pl_gen + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                    } else {
+                        const int off = (((grp >> 1) ^ p_swz) << 4) + ((grp & 1) << 3);
+                        *reinterpret_cast<uint2*>(ph_gen + off) = make_uint2(hw[0], hw[1]);
+                        *reinterpret_cast<uint2*>(pl_gen + off) = make_uint2(lw[0], lw[1]);
+                    }
                 }
                 if (grp == 0 && key0 + kKeys > L) {
                     // V rows beyond the context may hold any codes (NaN among them): zero them so that 0 * row = 0
@@ -480,14 +489,13 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
             const int unit = w.b * a.Hkv + w.kvh;
             const float vs = __ldg(a.v_scale + unit);
             float* slot = a.partial + (size_t)(cta + unit) * slot_stride;
-#pragma unroll
-            for (int ch = 0; ch < NG / 16; ++ch) {
-                uint32_t orow[16];
-                tmem_ld_x16(tO + 16 * ch, orow);
+            {
+                uint32_t orow[NG];
+                tmem_ld_cols<NG>(tO, orow);
                 tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const int col = C0 + 16 * ch + e;
+                for (int e = 0; e < NG; ++e) {
+                    const int col = C0 + e;
                     if (col < a.GR && sh_mref[col] != -INFINITY) slot[(size_t)col * D + t] = __uint_as_float(orow[e]) * vs;
                 }
             }

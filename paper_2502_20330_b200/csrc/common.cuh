@@ -119,6 +119,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// The same test, but the hardware may park the thread until the phase completes or `ns` nanoseconds
+// have passed: a waiting warp then costs its scheduler no issue slots.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
 // Every wait on an mbarrier is bounded: after `limit` clock cycles (kWaitCycleLimit, about a
 // second, unless the call names another figure) the waiter raises *abort (shared memory), which
 // makes every later wait of the CTA return at once, and the kernel records
@@ -150,7 +164,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_parked(bar, parity, 2000)) return true;
         if (*wc.abort) return false;
         if (clock64() - t0 > wc.limit) {
             *wc.abort = 1;
