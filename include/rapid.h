@@ -474,6 +474,16 @@ int rapid_retrieval_select(const float* chunk_emb, const float* query_emb, const
                            int32_t Nmax, int32_t Dm, float threshold, int32_t k, float* scores_out,
                            int32_t* sel_idx, int32_t* sel_count, int32_t* status_word, void* cuda_stream);
 
+/*
+ * Size of the drafter's retrieved context (Section 3.1, "RAG Setup": the retrieved text is bounded
+ * by the larger of a fixed floor, 4,096 tokens, and 1/24 of the full context, in chunks of 512
+ * tokens).  Host arithmetic only: returns floor(max(floor_tokens, context_tokens / divisor) /
+ * chunk_tokens), the k to hand to rapid_retrieval_select, or -1 (with rapid_last_error set) when
+ * context_tokens < 0 or one of the other three is not positive.
+ */
+int64_t rapid_retrieval_budget_chunks(int64_t context_tokens, int32_t chunk_tokens, int32_t floor_tokens,
+                                      int32_t divisor);
+
 /* ---- bookkeeping around the step --------------------------------------------------------------- */
 
 /*

@@ -24,7 +24,7 @@ RESIDUAL_PHAT = 1
 
 EXPORTS = [
     "rapid_attention_workspace_bytes", "rapid_accept_workspace_bytes", "rapid_workspace_init",
-    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_fp8", "rapid_attention_plan", "rapid_attention_describe", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_retrieval_select", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
+    "rapid_workspace_status", "rapid_verify_attention", "rapid_verify_attention_fp8", "rapid_attention_plan", "rapid_attention_describe", "rapid_verify_attention_paged", "rapid_merge_partials", "rapid_retrieval_select", "rapid_retrieval_budget_chunks", "rapid_draft_sample", "rapid_accept", "rapid_accept_static",
     "rapid_verify_step",
     "rapid_verify_step_host", "rapid_verify_step_host_arena_bytes", "rapid_kv_append", "rapid_kv_append_paged", "rapid_step_commit",
     "rapid_last_error",
@@ -149,6 +149,8 @@ def load_library():
         lib.rapid_draft_sample.argtypes = [vp, vp, f32, vp, vp, vp, i32, i64, i64, vp, sz, vp]
         lib.rapid_retrieval_select.restype = i32
         lib.rapid_retrieval_select.argtypes = [vp, vp, vp, i32, i32, i32, f32, i32, vp, vp, vp, vp, vp]
+        lib.rapid_retrieval_budget_chunks.restype = i64
+        lib.rapid_retrieval_budget_chunks.argtypes = [i64, i32, i32, i32]
         lib.rapid_merge_partials.restype = i32
         lib.rapid_merge_partials.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp]
         lib.rapid_accept.restype = i32
@@ -395,10 +397,14 @@ def rapid_draft_sample(draft_logits, uniforms, temperature, out_token, out_logq,
                                              _p(workspace), _nbytes(workspace), _stream_ptr(stream)))
 
 
-def retrieval_budget_chunks(context_tokens: int, chunk_tokens: int = 512, floor_tokens: int = 4096,
-                            fraction: int = 24) -> int:
-    """Chunks the retrieved context may hold: its length is bounded by max(floor_tokens, context / fraction)."""
-    return max(floor_tokens, context_tokens // fraction) // chunk_tokens
+def rapid_retrieval_budget_chunks(context_tokens: int, chunk_tokens: int = 512, floor_tokens: int = 4096,
+                                  divisor: int = 24) -> int:
+    """Chunks the retrieved context may hold (the library's rapid_retrieval_budget_chunks)."""
+    k = load_library().rapid_retrieval_budget_chunks(int(context_tokens), int(chunk_tokens), int(floor_tokens),
+                                                     int(divisor))
+    if k < 0:
+        raise ValueError(load_library().rapid_last_error().decode())
+    return int(k)
 
 
 def rapid_retrieval_select(chunk_emb, query_emb, k, status_word, threshold=0.3, n_chunks=None, stream=None):

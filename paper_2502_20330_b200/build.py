@@ -42,7 +42,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    subprocess.run(["nvcc", "-shared", "-o", LIB] + objs + ["-lcudart"], check=True)
+    subprocess.run(["nvcc", "-shared", "-Wno-deprecated-gpu-targets", "-o", LIB] + objs + ["-lcudart"], check=True)
     return LIB
 
 

@@ -297,6 +297,17 @@ int rapid_retrieval_select(const float* chunk_emb, const float* query_emb, const
                                    sel_count, status_word, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int64_t rapid_retrieval_budget_chunks(int64_t context_tokens, int32_t chunk_tokens, int32_t floor_tokens,
+                                      int32_t divisor) {
+    clear_error();
+    if (context_tokens < 0 || chunk_tokens <= 0 || floor_tokens <= 0 || divisor <= 0) {
+        set_error("rapid_retrieval_budget_chunks: context_tokens >= 0 and positive chunk, floor and divisor wanted");
+        return -1;
+    }
+    const int64_t share = context_tokens / divisor;
+    return (share > floor_tokens ? share : (int64_t)floor_tokens) / chunk_tokens;
+}
+
 int rapid_merge_partials(const float* o_parts, const float* lse_parts, int P, int64_t rows, int D, void* out,
                          float* out_f32, float* lse_out, void* cuda_stream) {
     clear_error();

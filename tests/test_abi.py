@@ -44,6 +44,19 @@ def test_host_only_calls(lib):
     assert a > 2 * 2 * 4096 * 64 * 2
 
 
+def test_retrieval_budget_rule():
+    """Section 3.1, RAG set-up: max(4,096 tokens, context / 24) in chunks of 512 (host arithmetic of the library)."""
+    import paper_2502_20330_b200 as R
+    assert R.rapid_retrieval_budget_chunks(131072) == 10      # 131072/24 = 5461 tokens -> 10 chunks of 512
+    assert R.rapid_retrieval_budget_chunks(32768) == 8        # the 4096-token floor
+    assert R.rapid_retrieval_budget_chunks(1_000_000) == 81
+    assert R.rapid_retrieval_budget_chunks(0) == 8
+    with pytest.raises(ValueError):
+        R.rapid_retrieval_budget_chunks(-1)
+    with pytest.raises(ValueError):
+        R.rapid_retrieval_budget_chunks(1000, chunk_tokens=0)
+
+
 def test_struct_layouts_match_the_header():
     from paper_2502_20330_b200 import binding
     assert ctypes.sizeof(binding._AttnShape) == 48

@@ -57,13 +57,6 @@ def test_ragged_requests_ties_and_degenerate_vectors():
     _check(E, q, 200, -1.0, n_chunks=[128, 50, 0])      # k above the count, a request without chunks
 
 
-def test_budget_rule():
-    import paper_2502_20330_b200 as R
-    assert R.retrieval_budget_chunks(131072) == 10      # 131072/24 = 5461 tokens -> 10 chunks of 512
-    assert R.retrieval_budget_chunks(32768) == 8        # the 4096-token floor
-    assert R.retrieval_budget_chunks(1_000_000) == 81
-
-
 def test_argument_errors():
     import paper_2502_20330_b200 as R
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
