@@ -43,17 +43,26 @@ def _peaks():
     return 6650.0, "fallback"
 
 
+TRAFFIC_SOURCES = ("attention.cu", "attention_kt.cuh", "attention_kt8.cuh", "tcgen05.cuh", "common.cuh")
+
+
+def kernel_sources_sha256() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for f in TRAFFIC_SOURCES:
+        h.update(open(os.path.join(ROOT, "paper_2502_20330_b200", "csrc", f), "rb").read())
+    return h.hexdigest()
+
+
 def ncu_traffic(workload, kernel):
     """DRAM bytes per launch of the dominant kernel from the committed ncu capture, or None if the
-    kernel sources have changed since the counters were taken (or no capture covers this workload)."""
-    import hashlib
+    kernel sources have changed since the counters were taken (or no capture covers this kernel on this
+    workload, cache type and mask)."""
     try:
         rec = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
-        h = hashlib.sha256()
-        for f in ("attention.cu", "attention_kt.cuh", "tcgen05.cuh", "common.cuh"):
-            h.update(open(os.path.join(ROOT, "paper_2502_20330_b200", "csrc", f), "rb").read())
-        ent = rec.get(workload)
-        if h.hexdigest() != rec["kernel_sha256"] or not ent or ent.get("kernel") != kernel:
+        key = f"{kernel}:{workload}" + (":fp8" if KV_ELEMENT_BYTES == 1 else "") + (":window" if MASK[1] > 0 else "")
+        ent = rec["captures"].get(key)
+        if kernel_sources_sha256() != rec["sources_sha256"] or not ent:
             return None
         return int(ent["dram_bytes_read"] + ent["dram_bytes_write"])
     except Exception:
@@ -83,8 +92,25 @@ def job_throughput_gbs(bytes_per_rank_step: int, world: int, ms_per_step: float)
 KV_ELEMENT_BYTES = 2   # set to 1 by --kv fp8: the algorithmic bytes are those of the cache as it is stored
 
 
+MASK = (0, 0)          # set by --sink / --window: (sink_keys, window_keys); (0, 0) is the full causal mask
+
+
+def visible_keys(cfg, ctx) -> int:
+    """Keys some row of a sequence can see, summed over the sequences: all of them under the full mask,
+    the sinks and the union of the rows' windows otherwise.  These are the keys the method has to read."""
+    sink, window = MASK
+    total = 0
+    for L in (int(x) for x in ctx):
+        if window <= 0:
+            total += L
+        else:
+            lo = max(0, L - cfg.R - window + 1)      # first key of the oldest row's window
+            total += (L - lo) + min(sink, lo)
+    return total
+
+
 def kv_bytes_per_layer(cfg, ctx) -> int:
-    return int(2 * KV_ELEMENT_BYTES * cfg.Hkv * cfg.D * int(ctx.sum()))
+    return int(2 * KV_ELEMENT_BYTES * cfg.Hkv * cfg.D * visible_keys(cfg, ctx))
 
 
 L2_BYTES = 126 * 2**20
@@ -105,6 +131,7 @@ def config_dict(cfg, ctx, world, sharded=False):
     """What both arms print as `config`: the workload, nothing of how an arm runs it."""
     kv_layer = kv_bytes_per_layer(cfg, ctx)
     return {"workload": cfg.name, "kv_cache": "fp8 e4m3 + fp32 scale per (sequence, KV head)" if KV_ELEMENT_BYTES == 1 else "bf16",
+            "mask": "causal" if MASK[1] <= 0 else f"{MASK[0]} sink keys + a window of {MASK[1]} keys per row",
             "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
             "ctx": [int(x) for x in ctx], "gamma": cfg.gamma, "V": cfg.V, "layers": cfg.layers, "eta": cfg.eta,
             "kv_bytes_per_step": kv_layer * cfg.layers,
@@ -183,7 +210,8 @@ class OracleSample:
             units = np.sort(self.rng.choice(self.total_units, size=n_units, replace=False)).astype(np.int64)
         t0 = time.perf_counter()
         fn = self.oracle.verify_attention_fp8 if self.fp8 else self.oracle.verify_attention
-        out, lse = fn(*self.bits, self.ctx_np, self.cfg.gamma, units=units)
+        kw = {} if self.fp8 else {"sink": MASK[0], "window": MASK[1]}
+        out, lse = fn(*self.bits, self.ctx_np, self.cfg.gamma, units=units, **kw)
         dt = time.perf_counter() - t0
         self.attn_ref = (out, lse)
         return dt, n_units
@@ -400,7 +428,7 @@ def run_ours(args, cfg):
     aws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma), device=dev)
     cws = R.new_workspace(R.accept_workspace_bytes(cfg.B, cfg.gamma, cfg.V), device=dev)
     acc_params = R.AcceptParams(temperature=cfg.temperature, tail_alpha=cfg.tail_alpha)
-    plan_params = R.AttnParams(kernel=args.kernel, kv_fp8=fp8)
+    plan_params = R.AttnParams(kernel=args.kernel, kv_fp8=fp8, sink_keys=MASK[0], window_keys=MASK[1])
     stream = torch.cuda.current_stream()
     sptr = int(stream.cuda_stream)
     ev = RawEvents()
@@ -417,7 +445,8 @@ def run_ours(args, cfg):
         # the plan of a step is made right before its first layer: that layer reads it after its
         # grid-dependency wait, the later ones (other kernels lie in between) before it
         mode = R.PLAN_NONE if args.no_plan else (R.PLAN_READY if li == 0 else R.PLAN_SETTLED)
-        return R.AttnParams(kernel=args.kernel, plan=mode, split_done_event=split_event)
+        return R.AttnParams(kernel=args.kernel, plan=mode, split_done_event=split_event, sink_keys=MASK[0],
+                            window_keys=MASK[1])
 
     def step(split_events=None, call_events=None, st=None):
         if flush is not None:
@@ -611,7 +640,7 @@ def run_ours(args, cfg):
     if sustained is not None:
         line["sustained"] = sustained
 
-    if rank == 0 and world == 1 and not args.no_e2e and not fp8:
+    if rank == 0 and world == 1 and not args.no_e2e and not fp8 and MASK[1] <= 0:
         line["e2e"] = run_e2e(R, cfg, seed, Lmax, kv_layer, dev)
     elif rank == 0:
         line["e2e"] = None
@@ -619,7 +648,7 @@ def run_ours(args, cfg):
         # The CPU leg runs on the very bits the library ran on (layer 0 and the logits, copied back
         # from the device), and what it computes is also what the library's results are judged by.
         out0 = layers[0][3]
-        attention(layers[0], R.AttnParams(kernel=args.kernel))
+        attention(layers[0], R.AttnParams(kernel=args.kernel, sink_keys=MASK[0], window_keys=MASK[1]))
         R.rapid_accept(z, d, tok, u, cfg.eta, alen, ntok, cws, acc_params)
         torch.cuda.synchronize()
         dev_out = out0.float().cpu().numpy()
@@ -757,8 +786,12 @@ def run_sharded(args, cfg):
 
 
 def _rank_main(args):
-    global KV_ELEMENT_BYTES
+    global KV_ELEMENT_BYTES, MASK
     KV_ELEMENT_BYTES = 1 if args.kv == "fp8" else 2
+    if args.window > 0:
+        if args.kv == "fp8" or args.sharded:
+            raise SystemExit("--window is for the bf16 cache on one rank's own context")
+        MASK = (max(0, args.sink), args.window)
     cfg = wl.CONFIGS[args.workload]
     if args.layers:
         cfg = wl.with_overrides(cfg, layers=args.layers)
@@ -784,6 +817,9 @@ def main():
                          "3 keys on M with one cluster per KV head")
     ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"],
                     help="storage of the KV cache: bf16, or FP8 E4M3 codes with a scale per (sequence, KV head)")
+    ap.add_argument("--sink", type=int, default=0, help="with --window: the first keys every row sees")
+    ap.add_argument("--window", type=int, default=0,
+                    help="every row sees the sinks and its own newest WINDOW keys only (0: the full causal mask)")
     ap.add_argument("--sharded", action="store_true", help="context-sharded attention over the ranks")
     ap.add_argument("--no-plan", action="store_true", help="every attention call works its split out itself")
     ap.add_argument("--no-e2e", action="store_true")

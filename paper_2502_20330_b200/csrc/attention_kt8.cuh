@@ -84,7 +84,7 @@ __host__ __device__ constexpr uint32_t umma_idesc_e4m3(int M, int N, int a_mn_ma
 }
 // Two values as hi + lo E4M3 pairs: hi = E4M3(v) by the hardware conversion, the remainders formed in
 // packed half precision (v < 448 and its remainder need far fewer than half's 11 bits) and converted
-// the same way.  Returns hi's two codes in bits 0..15 (v0 low), lo's two in `lo`.
+// the same way.  v0's codes go to the low bytes of hi and lo.
 __device__ __forceinline__ uint32_t split_e4m3x2(float v0, float v1, uint32_t& lo) {
     uint16_t h;
     uint32_t hf2, vf2, rf2;
@@ -98,6 +98,12 @@ __device__ __forceinline__ uint32_t split_e4m3x2(float v0, float v1, uint32_t& l
     return h;
 }
 
+__device__ __forceinline__ void split_e4m3x4(float v0, float v1, float v2, float v3, uint32_t& hi, uint32_t& lo) {
+    uint32_t l01, l23;
+    const uint32_t h01 = split_e4m3x2(v0, v1, l01), h23 = split_e4m3x2(v2, v3, l23);
+    hi = h01 | (h23 << 16);
+    lo = l01 | (l23 << 16);
+}
 // NC = N / 16 column chunks.  There are SG = N / NG softmax groups of 128 threads each (thread t of
 // every group is key t of the tile): a group forms the probabilities of its own NG = 8 or 16 columns --
 // half or all of a 16-byte chunk of the key's P^T hi row, and of its lo row -- and keeps those rows'
@@ -327,13 +333,10 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
                     if (j2 == 0) sh_c[row] = a.scale_log2 * __ldg(a.k_scale + (size_t)w.b * a.Hkv + w.kvh) * down;
                     uint32_t hw[4], lw[4];
 #pragma unroll
-                    for (int e = 0; e < 8; e += 2) {
-                        uint32_t l01, l23;
-                        const uint32_t h01 = split_e4m3x2(__uint_as_float(u[e] << 16) * up, __uint_as_float(u[e] & 0xffff0000u) * up, l01);
-                        const uint32_t h23 = split_e4m3x2(__uint_as_float(u[e + 1] << 16) * up, __uint_as_float(u[e + 1] & 0xffff0000u) * up, l23);
-                        hw[e >> 1] = h01 | (h23 << 16);
-                        lw[e >> 1] = l01 | (l23 << 16);
-                    }
+                    for (int e = 0; e < 8; e += 2)
+                        split_e4m3x4(__uint_as_float(u[e] << 16) * up, __uint_as_float(u[e] & 0xffff0000u) * up,
+                                     __uint_as_float(u[e + 1] << 16) * up, __uint_as_float(u[e + 1] & 0xffff0000u) * up,
+                                     hw[e >> 1], lw[e >> 1]);
                     const int off = row * 128 + ((j2 ^ (row & 7)) << 4);
                     *reinterpret_cast<uint4*>(smem_gen + OFF_QH + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
                     *reinterpret_cast<uint4*>(smem_gen + OFF_QL + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
@@ -366,20 +369,36 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
                     uint32_t sr[NG];
                     tmem_ld_cols<NG>(tS, sr);
                     tmem_wait_ld();
-                    // a tile every row sees whole (all of a long context but its end) needs no mask
-                    const bool tile_clear = key0 + kKeys <= L - a.stair;
+                    // a tile every row sees whole (all of a long context but its end) takes the loop
+                    // without any mask; the two loops are separate code so that the common one carries
+                    // no predicate at all
+                    if (key0 + kKeys <= L - a.stair) {
 #pragma unroll
-                    for (int e = 0; e < NG; e += 4) {
-                        const int col = C0 + e;
-                        const float4 m = *reinterpret_cast<const float4*>(&sh_mref[col]);
-                        const float4 cc = *reinterpret_cast<const float4*>(&sh_c[col]);
-                        float x[4] = {fmaf(__uint_as_float(sr[e]), cc.x, -m.x), fmaf(__uint_as_float(sr[e + 1]), cc.y, -m.y),
-                                      fmaf(__uint_as_float(sr[e + 2]), cc.z, -m.z), fmaf(__uint_as_float(sr[e + 3]), cc.w, -m.w)};
+                        for (int e = 0; e < NG; e += 4) {
+                            const float4 m = *reinterpret_cast<const float4*>(&sh_mref[C0 + e]);
+                            const float4 cc = *reinterpret_cast<const float4*>(&sh_c[C0 + e]);
+                            const float x0 = fmaf(__uint_as_float(sr[e]), cc.x, -m.x), x1 = fmaf(__uint_as_float(sr[e + 1]), cc.y, -m.y);
+                            const float x2 = fmaf(__uint_as_float(sr[e + 2]), cc.z, -m.z), x3 = fmaf(__uint_as_float(sr[e + 3]), cc.w, -m.w);
+                            xmax = fmaxf(fmaxf(xmax, x0), fmaxf(fmaxf(x1, x2), x3));
+                            pv[e] = fast_exp2(x0);
+                            pv[e + 1] = fast_exp2(x1);
+                            pv[e + 2] = fast_exp2(x2);
+                            pv[e + 3] = fast_exp2(x3);
+                        }
+                    } else {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            if (!tile_clear) x[i] = col + i >= cmin ? x[i] : -INFINITY;
-                            xmax = fmaxf(xmax, x[i]);
-                            pv[e + i] = fast_exp2(x[i]);
+                        for (int e = 0; e < NG; e += 4) {
+                            const int col = C0 + e;
+                            const float4 m = *reinterpret_cast<const float4*>(&sh_mref[col]);
+                            const float4 cc = *reinterpret_cast<const float4*>(&sh_c[col]);
+                            float x[4] = {fmaf(__uint_as_float(sr[e]), cc.x, -m.x), fmaf(__uint_as_float(sr[e + 1]), cc.y, -m.y),
+                                          fmaf(__uint_as_float(sr[e + 2]), cc.z, -m.z), fmaf(__uint_as_float(sr[e + 3]), cc.w, -m.w)};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                x[i] = col + i >= cmin ? x[i] : -INFINITY;
+                                xmax = fmaxf(xmax, x[i]);
+                                pv[e + i] = fast_exp2(x[i]);
+                            }
                         }
                     }
                     move = bar_softmax_or(grp, xmax > kJump);
@@ -449,10 +468,7 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
 #pragma unroll
                     for (int q4 = 0; q4 < NG / 4; ++q4) {
                         const int o = 4 * q4;
-                        uint32_t l01, l23;
-                        const uint32_t h01 = split_e4m3x2(pv[o], pv[o + 1], l01), h23 = split_e4m3x2(pv[o + 2], pv[o + 3], l23);
-                        hw[q4] = h01 | (h23 << 16);
-                        lw[q4] = l01 | (l23 << 16);
+                        split_e4m3x4(pv[o], pv[o + 1], pv[o + 2], pv[o + 3], hw[q4], lw[q4]);
                         lsum[o] += pv[o];
                         lsum[o + 1] += pv[o + 1];
                         lsum[o + 2] += pv[o + 2];
