@@ -445,8 +445,10 @@ def run_ours(args, cfg):
         # the plan of a step is made right before its first layer: that layer reads it after its
         # grid-dependency wait, the later ones (other kernels lie in between) before it
         mode = R.PLAN_NONE if args.no_plan else (R.PLAN_READY if li == 0 else R.PLAN_SETTLED)
+        # every cache of the step was written long before the step: all but a layer's newest rows may be
+        # copied while the preceding kernel still runs (what a decode loop can state as well)
         return R.AttnParams(kernel=args.kernel, plan=mode, split_done_event=split_event, sink_keys=MASK[0],
-                            window_keys=MASK[1])
+                            window_keys=MASK[1], kv_settled=not args.no_early_kv)
 
     def step(split_events=None, call_events=None, st=None):
         if flush is not None:
@@ -623,6 +625,8 @@ def run_ours(args, cfg):
         "config": config_dict(cfg, ctx_cpu, world),
         "run": {"launch": "the step captured in one CUDA graph, replayed per step",
                 "plan": "none" if args.no_plan else "one rapid_attention_plan per step, shared by its layers",
+                "early_kv": "off" if (args.no_early_kv or args.no_plan) else
+                            "kv_settled: a layer's first tiles below its newest rows are copied before its stream-order wait",
                 "kernels_per_attention_call": int(launches_per_call), "attention_launch": info,
                 "l2_flush_ms_per_step_not_counted": flush_ms / args.steps},
         "verify_latency_us": {"attention_per_layer": 1e3 * (ms_per_step - float(np.median(acc_ms))) / cfg.layers,
@@ -822,6 +826,8 @@ def main():
                     help="every row sees the sinks and its own newest WINDOW keys only (0: the full causal mask)")
     ap.add_argument("--sharded", action="store_true", help="context-sharded attention over the ranks")
     ap.add_argument("--no-plan", action="store_true", help="every attention call works its split out itself")
+    ap.add_argument("--no-early-kv", action="store_true",
+                    help="do not let a layer copy its first (old) K/V tiles while the preceding kernel runs")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sustained", action="store_true")

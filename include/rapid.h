@@ -137,6 +137,15 @@ typedef struct rapid_attn_params {
     int64_t wait_cycle_limit; /* SM clock cycles an on-chip wait (for a tile, for the tensor cores) may take
                                  before the kernel gives up and sets RAPID_STATUS_PIPELINE_TIMEOUT;
                                  0 = the library's limit of about a second                              */
+    int32_t kv_settled;       /* non-zero, together with plan = RAPID_PLAN_SETTLED and a contiguous cache: the
+                                 caller states that every K/V entry OLDER than the R newest keys of each
+                                 sequence (positions below ctx_lens[b] - R) was final before the work that
+                                 precedes this call on the stream was issued.  The split kernel then starts
+                                 copying its first such tiles while that preceding work still runs (before
+                                 its own stream-order wait); the newest R rows, q and everything else are
+                                 read after the wait as always.  True of a decode loop, where only the newest
+                                 rows of a layer's cache are written inside a step.  0 = nothing is read
+                                 early (default)                                                        */
 } rapid_attn_params;
 
 /*

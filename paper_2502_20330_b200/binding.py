@@ -55,7 +55,8 @@ class _AttnParams(ctypes.Structure):
                 ("lse_out", ctypes.c_void_p), ("out_f32", ctypes.c_void_p),
                 ("split_done_event", ctypes.c_void_p), ("all_keys_visible", ctypes.c_int32),
                 ("kernel", ctypes.c_int32), ("sink_keys", ctypes.c_int32), ("window_keys", ctypes.c_int32),
-                ("plan", ctypes.c_int32), ("kv_fp8", ctypes.c_int32), ("wait_cycle_limit", ctypes.c_int64)]
+                ("plan", ctypes.c_int32), ("kv_fp8", ctypes.c_int32), ("wait_cycle_limit", ctypes.c_int64),
+                ("kv_settled", ctypes.c_int32)]
 
 
 class _LaunchInfo(ctypes.Structure):
@@ -90,6 +91,8 @@ class AttnParams:
     plan: int = 0                            # PLAN_*: the workspace holds a plan made by rapid_attention_plan
     wait_cycle_limit: int = 0                # clock cycles an on-chip wait may take; 0 = the library's limit
     kv_fp8: bool = False                     # rapid_attention_plan / describe: the plan is for the FP8-cache call
+    kv_settled: bool = False                 # with plan = PLAN_SETTLED: all but the newest R keys were final before
+                                             # the preceding work was issued; their tiles may be copied early
 
 
 @dataclass
@@ -225,7 +228,7 @@ def _attn_params(p: Optional[AttnParams]):
                                     p.out_f32.data_ptr() if p.out_f32 is not None else None,
                                     p.split_done_event, 1 if p.all_keys_visible else 0, int(p.kernel),
                                     int(p.sink_keys), int(p.window_keys), int(p.plan), 1 if p.kv_fp8 else 0,
-                                    int(p.wait_cycle_limit)))
+                                    int(p.wait_cycle_limit), 1 if p.kv_settled else 0))
 
 
 def _accept_shape(target_logits: torch.Tensor, draft_logits: torch.Tensor) -> _AcceptShape:

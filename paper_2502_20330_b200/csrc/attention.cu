@@ -69,6 +69,9 @@ struct AttnArgs {
     // the kernel just before this call's, RAPID_PLAN_SETTLED = at least two kernels ago.  (A call
     // without a caller's plan launches the plan kernel itself and runs with RAPID_PLAN_READY.)
     int plan_mode;
+    // kv_settled: tiles wholly below the newest R keys may be copied before the grid-dependency wait
+    // (the caller vouches for them; needs a settled plan and a contiguous cache)
+    int kv_settled;
     int caller_plan;  // the caller supplied the plan: check it against the call's geometry and lengths
     const Walk* plan_walks;
     const int2* plan_units;  // (first CTA, number of slots) of every unit
@@ -391,11 +394,13 @@ __device__ __forceinline__ bool warp_wait_bounded(uint64_t* bar, uint32_t parity
 // dependents launch and hands every thread the CTA's walk.  A settled plan (made at least two
 // kernels earlier in the stream) was read before the wait, and nothing but the wait remains.
 //
-// Order matters here: launch_dependents comes after the wait in every kernel of this library.  A
-// dependent kernel therefore starts only once everything before its predecessor has completed,
-// which is what allows (a) the merge kernel to take the lengths before its own wait although an
-// earlier kernel of the stream may have written them, and (b) a settled plan to be read before
-// the wait.
+// Order matters here: in the plan kernel and in every split kernel launch_dependents comes after the
+// wait.  A merge kernel therefore starts only once everything before its split kernel has completed,
+// which is what allows it (a) to take the unit's slots from the plan before its own wait.  The merge
+// kernels let their dependents go before their wait, so the next call's split kernel may start
+// while this call's split kernel still runs; by then everything before THIS call's split kernel
+// has completed, the plan kernel of the step included, which is what allows (b) a settled plan to be
+// read before the wait, and (c) old K/V tiles to be copied there when the caller vouches for them.
 __device__ __forceinline__ void split_kernel_walk(const AttnArgs& a, int cta, int KS, Walk& w, Walk* s_walk) {
     const bool settled = a.plan_mode == RAPID_PLAN_SETTLED;
     if (settled) load_walk(a, cta, KS, w);
@@ -875,8 +880,10 @@ verify_attn_merge_kernel(const __grid_constant__ AttnArgs a, int KS, __nv_bfloat
     const float* base = a.partial + (size_t)(c_first + unit) * KS * slot_stride;  // slots are consecutive
 
     // everything above depends on the call's inputs only; the partials need the split kernel
+    // Dependents may launch BEFORE this kernel's own wait: see verify_attn_merge_rows_kernel for why that
+    // is safe for what the library's kernels do ahead of their waits.
+    asm volatile("griddepcontrol.launch_dependents;");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;");  // a following dependent launch may begin its prologue
     if (nslots <= 0) {  // the plan is not this call's (status says so): defined output, nothing read
         if (warp == 0) {
             const size_t row = ((size_t)b * a.R + m / a.G) * a.Hq + (size_t)kvh * a.G + m % a.G;
@@ -949,6 +956,116 @@ verify_attn_merge_kernel(const __grid_constant__ AttnArgs a, int KS, __nv_bfloat
         }
         if (lse_out && lane == 0) lse_out[row] = (M + log2f(l)) * 0.69314718055994530942f;
     }
+}
+
+// The same merge as one WARP per (grouped row, unit), four rows to a block, for the keys-on-M kernel with
+// one softmax group (one partial per CTA and unit: some twenty slots per unit when the SMs share eight
+// units).  It uses no shared memory and few enough registers for a block to sit on an SM BESIDE a CTA of
+// that split kernel: the merge blocks of a layer are resident while its split kernel runs and start
+// the moment it completes, with every slot of a row requested at once.
+//
+// It lets its dependents launch BEFORE its own wait.  The kernel that follows it on the stream may
+// therefore start while this layer's split kernel still runs (its CTAs take the SMs as this layer's
+// CTAs leave them).  That is safe for what the library's kernels do ahead of their own waits: they
+// read a settled plan (complete before this layer's split kernel passed its wait, or this kernel
+// could not have been launched) and, where the caller vouches for it, old entries of a K/V cache
+// (rapid_attn_params.kv_settled); everything else they read after their wait, which ends only when
+// this kernel has completed.
+template <int D>
+__global__ void __launch_bounds__(128)
+verify_attn_merge_rows_kernel(const __grid_constant__ AttnArgs a, __nv_bfloat16* out, float* lse_out,
+                              float* out_f32) {
+    constexpr int VEC = D / 32;
+    constexpr int UN = 20;
+    const int lane = threadIdx.x & 31;
+    const int m = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int unit = blockIdx.y;
+    const int b = unit / a.Hkv;
+    const int kvh = unit % a.Hkv;
+    // the unit's slots, from the plan (read before the wait: see verify_attn_merge_kernel)
+    const int2 range = plan_matches(a, 1) ? __ldcg(a.plan_units + unit) : make_int2(0, 0);
+    const int c_first = range.x;
+    const int nslots = range.y;
+    const size_t slot_stride = (size_t)slot_floats(a.GR, D);
+    const float* base = a.partial + (size_t)(c_first + unit) * slot_stride;  // slots are consecutive
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (m >= a.GR) return;
+    const size_t row = ((size_t)b * a.R + m / a.G) * a.Hq + (size_t)kvh * a.G + m % a.G;
+    if (nslots <= 0) {  // the plan is not this call's (status says so): defined output, nothing read
+        for (int d = lane; d < D; d += 32) {
+            out[row * D + d] = __float2bfloat16_rn(0.f);
+            if (out_f32) out_f32[row * D + d] = 0.f;
+        }
+        if (lse_out && lane == 0) lse_out[row] = -INFINITY;
+        return;
+    }
+    // Slots are taken UN at a time (usually all at once): their O rows are requested first, lane u then
+    // fetches the reference and the sum of slot u, and the weights go round by shuffle.
+    float ov[UN][VEC];
+    auto fetch = [&](int j0) {
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const int j = min(j0 + u, nslots - 1);  // past the end: any valid slot, never used
+            const float* slot = base + (size_t)j * slot_stride + (size_t)m * D + lane * VEC;
+            if (VEC == 4) {
+                const float4 t = *reinterpret_cast<const float4*>(slot);
+                ov[u][0] = t.x; ov[u][1] = t.y; ov[u][2] = t.z; ov[u][VEC - 1] = t.w;
+            } else {
+                const float2 t = *reinterpret_cast<const float2*>(slot);
+                ov[u][0] = t.x; ov[u][1] = t.y;
+            }
+        }
+    };
+    fetch(0);
+    // lane u's slot of the first round: its reference and its sum, requested together with the O rows
+    // (the sum of an untouched slot is garbage and is never used: selected away, not multiplied)
+    float mj = -INFINITY, lj = 0.f;
+    if (lane < UN && lane < nslots) {
+        mj = base[(size_t)lane * slot_stride + a.GR * D + m];
+        lj = base[(size_t)lane * slot_stride + a.GR * D + a.GR + m];
+    }
+    float M = mj;
+    for (int j = UN + lane; j < nslots; j += 32) M = fmaxf(M, base[j * slot_stride + a.GR * D + m]);  // rarely any
+#pragma unroll
+    for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float acc[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+    float lpart = 0.f;  // lane u: the sums of the slots u, u + UN, ...
+    for (int j0 = 0; j0 < nslots; j0 += UN) {  // slots in their order: the result does not depend on timing
+        if (j0) {
+            fetch(j0);
+            mj = -INFINITY;
+            if (lane < UN && j0 + lane < nslots) {
+                mj = base[(size_t)(j0 + lane) * slot_stride + a.GR * D + m];
+                lj = base[(size_t)(j0 + lane) * slot_stride + a.GR * D + a.GR + m];
+            }
+        }
+        float w = 0.f;
+        if (mj != -INFINITY) {  // an untouched slot holds neither a sum nor an O row
+            w = exp2f(mj - M);
+            lpart += w * lj;
+        }
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const float wu = __shfl_sync(0xffffffffu, w, u);
+            if (wu == 0.f) continue;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] += wu * ov[u][e];
+        }
+    }
+    float lsum = lpart;  // a fixed tree over the lanes
+#pragma unroll
+    for (int o = 16; o; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+        const int d = lane * VEC + e;
+        const float val = acc[e] / lsum;
+        out[row * D + d] = __float2bfloat16_rn(val);
+        if (out_f32) out_f32[row * D + d] = val;
+    }
+    if (lse_out && lane == 0) lse_out[row] = (M + log2f(lsum)) * 0.69314718055994530942f;
 }
 
 // Combines P partial attention results of the same rows over disjoint key sets (each normalised
@@ -1471,6 +1588,7 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
     a.plan_units = reinterpret_cast<const int2*>(ws + lay.units);
     a.plan_ctx = reinterpret_cast<const int32_t*>(ws + lay.ctx);
     a.wait_limit = wait_limit;
+    a.kv_settled = params && params->kv_settled && plan_mode == RAPID_PLAN_SETTLED && !paged;
     a.cmerge = 0;
     return RAPID_OK;
 }
@@ -1711,7 +1829,17 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     dim3 grid(a.GR, s.B * s.Hkv);
     // programmatic dependent launch: the merge blocks start while the split kernel still runs and
     // hold at their grid-dependency wait until its partials are complete and visible
-    if (s.D == 128)
+    // Which merge: a warp per row (blocks that sit on an SM beside a CTA of the one-group keys-on-M kernel,
+    // a quarter of the blocks) where a row has few slots or the call few rows; four warps per row
+    // otherwise.  Measured per layer (split + merge, chains of layers): ragged batch of 8 132.5 against
+    // 136.4 us, one-row decode at 8K 13.05 against 13.5, but 8 units of 36 rows 33.1 against 32.1 at
+    // 32K and 86.9 against 86.3 at 128K.
+    const bool one_group = c.kt_path && (c.NC <= 3 || (c.NC == 4 && !c.fp32_sums));
+    const bool warp_per_row = one_group && (a.GR <= 8 || a.num_ctas <= 8 * s.B * s.Hkv);
+    if (warp_per_row)
+        RAPID_CUDA_CHECK(launch_dependent(verify_attn_merge_rows_kernel<128>, dim3((a.GR + 3) / 4, s.B * s.Hkv),
+                                          dim3(128), 0, stream, a, a.out, a.lse_out, a.out_f32));
+    else if (s.D == 128)
         RAPID_CUDA_CHECK(launch_dependent(verify_attn_merge_kernel<128>, grid, dim3(128), 0, stream, a, c.KS, a.out,
                                           a.lse_out, a.out_f32));
     else

@@ -205,8 +205,48 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
         sh_mref[tid] = -INFINITY;
         sh_lfin[tid] = 0.f;
     }
+    // The walk, the stream-order wait, and between the two, where the caller vouches for the older part
+    // of the cache (kv_settled, which implies a settled plan), the first tiles' copies: they overlap
+    // the work that precedes this kernel on the stream.  Only tiles wholly below the newest R keys
+    // are taken early; everything else is read after the wait.
     Walk w;
-    split_kernel_walk(a, cta, 1, w, &s_walk);
+    const bool settled = a.plan_mode == RAPID_PLAN_SETTLED;
+    if (settled) load_walk(a, cta, 1, w);
+    tc_fence_before_sync();
+    __syncthreads();  // barriers initialised, tensor memory allocated
+    tc_fence_after_sync();
+    int pre_k = 0, pre_v = 0;  // tiles whose K / V copies were issued before the wait (producer lane only)
+    if (a.kv_settled && warp == WS && lane == 0 && w.remaining > 0) {
+        const int seg0 = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+        const int old_tiles = (w.L - a.R) >> 7;  // tiles 0 .. old_tiles-1 hold none of the newest R keys
+        for (int t = 0; t < seg0 && t < NV; ++t) {
+            const int tile = WIN ? real_tile(w, w.tile + t) : w.tile + t;
+            if (tile >= old_tiles) break;
+            if (t < NK) {
+                mbar_arrive_expect_tx(&k_full[t], TILE_TX);
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                    tma_load_4d(smem_gen + OFF_K + (h * NK + t) * kBlk, &tmK, &k_full[t], h * 64, tile * kKeys, w.kvh, w.b);
+                ++pre_k;
+            }
+            mbar_arrive_expect_tx(&v_full[t], TILE_TX);
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+                tma_load_4d(smem_gen + OFF_V + (h * NV + t) * kBlk, &tmV, &v_full[t], h * 64, tile * kKeys, w.kvh, w.b);
+            ++pre_v;
+        }
+    }
+    griddep_wait();               // inputs are read from here on
+    griddep_launch_dependents();  // the merge blocks may take their seats (after the wait: see split_kernel_walk)
+    if (!settled) {
+        if (threadIdx.x == 0) {
+            Walk t;
+            load_walk(a, cta, 1, t);
+            s_walk = t;
+        }
+        __syncthreads();
+        w = s_walk;
+    }
     if (cta == 0 && warp == WS && lane == 1) check_call_inputs(a, 1);  // an idle lane of the producer warp
     const uint32_t tmem_base = tmem_slot;
     const WaitCtx wc = {&s_abort, a.wait_limit};
@@ -242,23 +282,27 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
                         }
                     }
                     const uint32_t part_bytes = kBlk / parts;
-                    if (jj >= NK) ok = mbar_wait_bounded_relaxed(&k_empty[ks], ((jj / NK) - 1) & 1, wc);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(&k_full[ks], TILE_TX);
-                    for (int p = 0; p < parts; ++p)
+                    if (jj >= pre_k) {  // (the first pre_k tiles' K copies went out before the wait)
+                        if (jj >= NK) ok = mbar_wait_bounded_relaxed(&k_empty[ks], ((jj / NK) - 1) & 1, wc);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&k_full[ks], TILE_TX);
+                        for (int p = 0; p < parts; ++p)
 #pragma unroll
-                        for (int h = 0; h < 2; ++h)
-                            tma_load_4d(smem_gen + OFF_K + (h * NK + ks) * kBlk + p * part_bytes, &tmK, &k_full[ks],
-                                        h * 64, key0[p], w.kvh, outer[p]);
+                            for (int h = 0; h < 2; ++h)
+                                tma_load_4d(smem_gen + OFF_K + (h * NK + ks) * kBlk + p * part_bytes, &tmK, &k_full[ks],
+                                            h * 64, key0[p], w.kvh, outer[p]);
+                    }
                     ++n_k;
-                    if (jj >= NV) ok = mbar_wait_bounded_relaxed(&v_empty[vs], ((jj / NV) - 1) & 1, wc);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(&v_full[vs], TILE_TX);
-                    for (int p = 0; p < parts; ++p)
+                    if (jj >= pre_v) {
+                        if (jj >= NV) ok = mbar_wait_bounded_relaxed(&v_empty[vs], ((jj / NV) - 1) & 1, wc);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&v_full[vs], TILE_TX);
+                        for (int p = 0; p < parts; ++p)
 #pragma unroll
-                        for (int h = 0; h < 2; ++h)
-                            tma_load_4d(smem_gen + OFF_V + (h * NV + vs) * kBlk + p * part_bytes, &tmV, &v_full[vs],
-                                        h * 64, key0[p], w.kvh, outer[p]);
+                            for (int h = 0; h < 2; ++h)
+                                tma_load_4d(smem_gen + OFF_V + (h * NV + vs) * kBlk + p * part_bytes, &tmV, &v_full[vs],
+                                            h * 64, key0[p], w.kvh, outer[p]);
+                    }
                     ++n_v;
                 }
                 walk_advance(a, w, seg);
@@ -266,6 +310,8 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
             // leaving early: the copies already issued must have landed before the CTA gives up its
             // shared memory
             if (!ok) {
+                n_k = max(n_k, pre_k);  // copies that went out before the wait count too
+                n_v = max(n_v, pre_v);
                 for (int s = 0; s < NK && s < n_k; ++s)
                     mbar_wait_drain(&k_full[s], ((s + (n_k - 1 - s) / NK * NK) / NK) & 1);
                 for (int s = 0; s < NV && s < n_v; ++s)

@@ -176,7 +176,40 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
         fence_proxy_async_smem();
     }
     Walk w;
-    split_kernel_walk(a, cta, 1, w, &s_walk);
+    // The walk, the stream-order wait and, between the two, the first tiles' copies where the caller
+    // vouches for the older part of the cache (see the bf16 keys-on-M kernel).
+    const bool settled = a.plan_mode == RAPID_PLAN_SETTLED;
+    if (settled) load_walk(a, cta, 1, w);
+    tc_fence_before_sync();
+    __syncthreads();  // barriers initialised, tensor memory allocated
+    tc_fence_after_sync();
+    int pre_k = 0, pre_v = 0;  // tiles whose K / V copies were issued before the wait (producer lane only)
+    if (a.kv_settled && warp == WS && lane == 0 && w.remaining > 0) {
+        const int seg0 = (int)min((long long)(w.ntiles - w.tile), w.remaining);
+        const int old_tiles = (w.L - a.R) >> 7;  // tiles 0 .. old_tiles-1 hold none of the newest R keys
+        for (int t = 0; t < seg0 && t < NV && w.tile + t < old_tiles; ++t) {
+            const int key0 = (w.tile + t) * kKeys;
+            if (t < NK) {
+                mbar_arrive_expect_tx(&k_full[t], kBlk);
+                tma_load_4d(smem_gen + OFF_K + t * kBlk, &tmK, &k_full[t], 0, key0, w.kvh, w.b);
+                ++pre_k;
+            }
+            mbar_arrive_expect_tx(&v_full[t], kBlk);
+            tma_load_4d(smem_gen + OFF_V + t * kBlk, &tmV, &v_full[t], 0, key0, w.kvh, w.b);
+            ++pre_v;
+        }
+    }
+    griddep_wait();               // inputs are read from here on
+    griddep_launch_dependents();  // the merge blocks may take their seats (after the wait: see split_kernel_walk)
+    if (!settled) {
+        if (threadIdx.x == 0) {
+            Walk t;
+            load_walk(a, cta, 1, t);
+            s_walk = t;
+        }
+        __syncthreads();
+        w = s_walk;
+    }
     if (cta == 0 && warp == WS && lane == 1) check_call_inputs(a, 1);
     const uint32_t tmem_base = tmem_slot;
     const WaitCtx wc = {&s_abort, a.wait_limit};
@@ -191,20 +224,26 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
                 for (int t = 0; t < seg && ok; ++t, ++jj) {
                     const int ks = jj % NK, vs = jj % NV;
                     const int key0 = (w.tile + t) * kKeys;
-                    if (jj >= NK) ok = mbar_wait_bounded_relaxed(&k_empty[ks], ((jj / NK) - 1) & 1, wc);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(&k_full[ks], kBlk);
-                    tma_load_4d(smem_gen + OFF_K + ks * kBlk, &tmK, &k_full[ks], 0, key0, w.kvh, w.b);
+                    if (jj >= pre_k) {  // (the first pre_k tiles' K copies went out before the wait)
+                        if (jj >= NK) ok = mbar_wait_bounded_relaxed(&k_empty[ks], ((jj / NK) - 1) & 1, wc);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&k_full[ks], kBlk);
+                        tma_load_4d(smem_gen + OFF_K + ks * kBlk, &tmK, &k_full[ks], 0, key0, w.kvh, w.b);
+                    }
                     ++n_k;
-                    if (jj >= NV) ok = mbar_wait_bounded_relaxed(&v_empty[vs], ((jj / NV) - 1) & 1, wc);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(&v_full[vs], kBlk);
-                    tma_load_4d(smem_gen + OFF_V + vs * kBlk, &tmV, &v_full[vs], 0, key0, w.kvh, w.b);
+                    if (jj >= pre_v) {
+                        if (jj >= NV) ok = mbar_wait_bounded_relaxed(&v_empty[vs], ((jj / NV) - 1) & 1, wc);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&v_full[vs], kBlk);
+                        tma_load_4d(smem_gen + OFF_V + vs * kBlk, &tmV, &v_full[vs], 0, key0, w.kvh, w.b);
+                    }
                     ++n_v;
                 }
                 walk_advance(a, w, seg);
             }
             if (!ok) {  // leaving early: the copies already issued must land first
+                n_k = max(n_k, pre_k);
+                n_v = max(n_v, pre_v);
                 for (int s = 0; s < NK && s < n_k; ++s)
                     mbar_wait_drain(&k_full[s], ((s + (n_k - 1 - s) / NK * NK) / NK) & 1);
                 for (int s = 0; s < NV && s < n_v; ++s)

@@ -60,7 +60,7 @@ def test_retrieval_budget_rule():
 def test_struct_layouts_match_the_header():
     from paper_2502_20330_b200 import binding
     assert ctypes.sizeof(binding._AttnShape) == 48
-    assert ctypes.sizeof(binding._AttnParams) == 64
+    assert ctypes.sizeof(binding._AttnParams) == 72
     assert ctypes.sizeof(binding._AcceptShape) == 32
     assert ctypes.sizeof(binding._AcceptParams) == 40
     assert ctypes.sizeof(binding._PagedKv) == 40
@@ -75,7 +75,7 @@ def test_struct_layouts_match_what_the_c_compiler_sees(tmp_path):
         '#include <stdio.h>\n#include <stddef.h>\n#include "rapid.h"\n'
         'int main(void) {\n'
         '  printf("%zu %zu\\n", sizeof(rapid_attn_shape), offsetof(rapid_attn_shape, kv_stride_l));\n'
-        '  printf("%zu %zu\\n", sizeof(rapid_attn_params), offsetof(rapid_attn_params, wait_cycle_limit));\n'
+        '  printf("%zu %zu\\n", sizeof(rapid_attn_params), offsetof(rapid_attn_params, kv_settled));\n'
         '  printf("%zu %zu\\n", sizeof(rapid_accept_shape), offsetof(rapid_accept_shape, draft_row_stride));\n'
         '  printf("%zu %zu\\n", sizeof(rapid_accept_params), offsetof(rapid_accept_params, draft_logq));\n'
         '  printf("%zu %zu\\n", sizeof(rapid_paged_kv), offsetof(rapid_paged_kv, stride_l));\n'
@@ -85,7 +85,7 @@ def test_struct_layouts_match_what_the_c_compiler_sees(tmp_path):
     got = [tuple(int(x) for x in line.split()) for line in subprocess.run([str(exe)], check=True, capture_output=True,
                                                                           text=True).stdout.splitlines()]
     want = [(ctypes.sizeof(c), getattr(c, f).offset) for c, f in (
-        (binding._AttnShape, "kv_stride_l"), (binding._AttnParams, "wait_cycle_limit"),
+        (binding._AttnShape, "kv_stride_l"), (binding._AttnParams, "kv_settled"),
         (binding._AcceptShape, "draft_row_stride"), (binding._AcceptParams, "draft_logq"),
         (binding._PagedKv, "stride_l"))]
     assert got == want

@@ -453,3 +453,62 @@ def test_window_argument_errors():
         with pytest.raises(R.RapidError) as e:
             R.rapid_verify_attention(q, k, v, ctx, 2, torch.empty_like(q), ws, R.AttnParams(**bad))
         assert e.value.code == 1
+
+
+@pytest.mark.parametrize("Hq,Hkv,gamma,lens,kernel,sink,window", [
+    (32, 8, 8, (9000, 517), 0, 0, 0),       # keys on M; the short sequence has old tiles for few CTAs only
+    (32, 8, 0, (8192,), 0, 0, 0),           # the drafter's one-row decode
+    (32, 8, 8, (40000,), 3, 0, 0),          # one cluster per KV head
+    (32, 8, 8, (30000, 4100), 0, 4, 1020),  # window variant: the early tiles are the sink tile and the window's
+    (64, 8, 8, (5000, 300), 0, 0, 0),       # rows on M: the flag changes nothing there
+])
+def test_early_copies_of_the_settled_cache_change_nothing(Hq, Hkv, gamma, lens, kernel, sink, window):
+    """kv_settled: two layers back to back on one stream, each layer's newest rows written by the kernels just
+    ahead of its call (the older keys long before).  The second layer's first tiles are then copied while the
+    first layer's merge still runs; results must equal the oracle and, bit for bit, the calls without the flag."""
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("e", B=len(lens), Hq=Hq, Hkv=Hkv, D=128, gamma=gamma, V=4096, ctx_lens=lens)
+    Rr = cfg.R
+    layers = [wl.attention_inputs(cfg, seed=60 + i, device="cuda") for i in range(2)]
+    ctx = layers[0][3]
+    Lmax = layers[0][1].shape[2]
+    news, caches = [], []
+    for q, k, v, _ in layers:                       # take the newest rows out of the caches, poison their place
+        kn = torch.stack([k[b, :, L - Rr:L].clone() for b, L in enumerate(lens)])
+        vn = torch.stack([v[b, :, L - Rr:L].clone() for b, L in enumerate(lens)])
+        kc, vc = k.clone(), v.clone()
+        for b, L in enumerate(lens):
+            kc[b, :, L - Rr:L] = float("nan")
+            vc[b, :, L - Rr:L] = float("nan")
+        news.append((kn, vn))
+        caches.append((kc, vc))
+    ws = R.new_workspace(R.attention_workspace_bytes(cfg.B, Hq, Hkv, 128, Lmax, gamma))
+    outs = [torch.zeros_like(layers[0][0]) for _ in range(2)]
+    o32s = [torch.zeros(cfg.B, Rr, Hq, 128, device="cuda") for _ in range(2)]
+    torch.cuda.synchronize()
+
+    def run(flag):
+        base = R.AttnParams(kernel=kernel, sink_keys=sink, window_keys=window)
+        R.rapid_attention_plan(ctx, gamma, cfg.B, Hq, Hkv, 128, Lmax, ws, base)
+        for i, ((q, _, _, _), (kc, vc), (kn, vn)) in enumerate(zip(layers, caches, news)):
+            for b, L in enumerate(lens):            # the layer's newest rows arrive right before its call
+                kc[b, :, L - Rr:L] = kn[b]
+                vc[b, :, L - Rr:L] = vn[b]
+            R.rapid_verify_attention(q, kc, vc, ctx, gamma, outs[i], ws,
+                                     R.AttnParams(kernel=kernel, sink_keys=sink, window_keys=window,
+                                                  plan=R.PLAN_SETTLED, kv_settled=flag, out_f32=o32s[i]))
+        torch.cuda.synchronize()
+        assert R.workspace_status(ws) == 0
+        return [o.clone() for o in o32s]
+
+    plain = run(False)
+    for (kc, vc) in caches:                         # poison the newest rows again for the second pass
+        for b, L in enumerate(lens):
+            kc[b, :, L - Rr:L] = float("nan")
+            vc[b, :, L - Rr:L] = float("nan")
+    torch.cuda.synchronize()
+    early = run(True)
+    for i, (q, k, v, _) in enumerate(layers):
+        ref, ref_lse = _oracle(q, k, v, ctx, gamma, sink=sink, window=window)
+        parity.check_attention(early[i].cpu().numpy(), ref, ~np.isnan(ref_lse))
+        assert torch.equal(early[i], plain[i])

@@ -147,3 +147,42 @@ def test_a_plan_made_for_another_kernel_is_refused_not_followed():
     R.rapid_verify_attention(q2, k2, v2, ctx2, 8, out, ws2, R.AttnParams(plan=R.PLAN_SETTLED))
     torch.cuda.synchronize()
     assert R.workspace_status(ws2) & R.STATUS_STALE_PLAN
+
+
+def test_early_copies_of_the_settled_cache_change_nothing():
+    """kv_settled over the 8-bit cache: two layers back to back, the second one's first tiles copied while
+    the first one's merge still runs; the newest rows of each layer arrive right before its call."""
+    import paper_2502_20330_b200 as R
+    lens, gamma = (9000, 700), 8
+    cfg = wl.VerifyConfig("f8", B=2, Hq=32, Hkv=8, D=128, gamma=gamma, V=4096, ctx_lens=lens)
+    layers = [wl.attention_inputs_fp8(cfg, seed=70 + i, device="cuda") for i in range(2)]
+    ctx, Lmax, Rr = layers[0][5], layers[0][1].shape[2], gamma + 1
+    ws = R.new_workspace(R.attention_workspace_bytes(2, 32, 8, 128, Lmax, gamma))
+    news = [[(kc[b, :, L - Rr:L].clone(), vc[b, :, L - Rr:L].clone()) for b, L in enumerate(lens)]
+            for _, kc, vc, _, _, _ in layers]
+    o32s = [torch.zeros(2, Rr, 32, 128, device="cuda") for _ in range(2)]
+    outs = [torch.zeros_like(layers[0][0]) for _ in range(2)]
+
+    def run(flag):
+        for _, kc, vc, _, _, _ in layers:           # the newest rows are not there yet (NaN codes)
+            for b, L in enumerate(lens):
+                kc[b, :, L - Rr:L] = 0x7F
+                vc[b, :, L - Rr:L] = 0x7F
+        torch.cuda.synchronize()
+        R.rapid_attention_plan(ctx, gamma, 2, 32, 8, 128, Lmax, ws, R.AttnParams(kv_fp8=True))
+        for i, (q, kc, vc, ks, vs, _) in enumerate(layers):
+            for b, L in enumerate(lens):
+                kc[b, :, L - Rr:L] = news[i][b][0]
+                vc[b, :, L - Rr:L] = news[i][b][1]
+            R.rapid_verify_attention_fp8(q, kc, vc, ks, vs, ctx, gamma, outs[i], ws,
+                                         R.AttnParams(plan=R.PLAN_SETTLED, kv_settled=flag, out_f32=o32s[i], kv_fp8=True))
+        torch.cuda.synchronize()
+        assert R.workspace_status(ws) == 0
+        return [o.clone() for o in o32s]
+
+    plain, early = run(False), run(True)
+    for i, (q, kc, vc, ks, vs, _) in enumerate(layers):
+        ref, ref_lse = oracle.verify_attention_fp8(bf16_bits(q), kc.cpu().numpy(), vc.cpu().numpy(), ks.cpu().numpy(),
+                                                   vs.cpu().numpy(), ctx.cpu().numpy(), gamma)
+        parity.check_attention(early[i].cpu().numpy(), ref, ~np.isnan(ref_lse))
+        assert torch.equal(early[i], plain[i])
