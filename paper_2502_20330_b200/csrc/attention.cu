@@ -1344,12 +1344,14 @@ int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
 // fp32_sums: the caller takes the log-sum-exp, so the row sums must add fp32 probabilities.  With
 // 49 to 64 grouped rows one softmax group has no registers for that (it adds the bf16 values the
 // tensor cores multiply); two groups of 32 columns each do.
-int dispatch_split_kt(int NC, bool fp32_sums, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
-                      AttnArgs& a, cudaStream_t stream, bool want_cluster, bool need_cluster) {
+int dispatch_split_kt(int NC, bool fp32_sums, bool two_groups, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                      const CUtensorMap& tmQ, AttnArgs& a, cudaStream_t stream, bool want_cluster, bool need_cluster) {
     switch (NC) {
         case 1: return launch_split_kt<1>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
         case 2: return launch_split_kt<2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
-        case 3: return launch_split_kt<3>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
+        case 3:
+            return two_groups ? launch_split_kt<3, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster)
+                              : launch_split_kt<3>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
         case 4:
             return fp32_sums ? launch_split_kt<4, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster)
                              : launch_split_kt<4>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
@@ -1406,7 +1408,7 @@ WsLayout ws_layout(int B, int Hkv, int GR, int D) {
 // Everything the attention entry points share: validation, the choice of kernel, the arguments.
 struct AttnCall {
     AttnArgs a;
-    bool kt_path, kt_half_blocks, fp32_sums, want_cluster, need_cluster;
+    bool kt_path, kt_half_blocks, fp32_sums, want_cluster, need_cluster, few_slots, two_groups;
     int NC, KS, box_rows;
     int64_t sl, sh, sb, outer, keys;
 };
@@ -1553,6 +1555,14 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
     c.NC = (GR + 15) / 16;
     c.KS = c.kt_path ? 1 : kStreams;
     c.fp32_sums = params && params->lse_out;
+    // Few partial slots per unit, or few rows: the warp-per-row merge whose blocks sit beside the split
+    // kernel's CTAs pays (it needs the one-group kernel's registers).  Otherwise 33 to 48 grouped rows
+    // run with two softmax groups of 24 columns: measured 30.2 against 32.0 us per 32K layer and 83.8
+    // against 84.5 per 128K layer of the 8-unit shape (the ragged batch of 32 units, with the other
+    // merge: 134.2 against 131.6, which is why it keeps one group).
+    c.few_slots = GR <= 8 || num_ctas <= 8 * s.B * s.Hkv;
+    c.two_groups = c.kt_path && !fp8 && c.NC == 3 && !c.few_slots && !c.need_cluster;
+    if (c.two_groups) c.want_cluster = false;
 
     AttnArgs& a = c.a;
     a = AttnArgs{};
@@ -1652,7 +1662,7 @@ int describe_attention(const rapid_attn_shape* shape, int gamma, const rapid_att
     info->kernels_per_call = cs ? 1 : 2;
     info->ctas = cs ? units * cs : c.a.num_ctas;
     info->cluster_size = cs;
-    info->softmax_groups = c.kt_path ? ((c.NC > 4 || (c.NC == 4 && c.fp32_sums)) ? 2 : 1) : 2;
+    info->softmax_groups = c.kt_path ? ((c.NC > 4 || (c.NC == 4 && c.fp32_sums) || c.two_groups) ? 2 : 1) : 2;
     info->columns = c.kt_path ? 16 * c.NC : (c.a.GR <= 64 ? 64 : 128);
     if (c.kt_path) {
         int dev = 0;
@@ -1810,7 +1820,7 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
         a.plan_mode = RAPID_PLAN_READY;
     }
     if (c.kt_path) {
-        rc = dispatch_split_kt(c.NC, c.fp32_sums, tmK, tmV, tmQ, a, stream, c.want_cluster, c.need_cluster);
+        rc = dispatch_split_kt(c.NC, c.fp32_sums, c.two_groups, tmK, tmV, tmQ, a, stream, c.want_cluster, c.need_cluster);
     } else if (a.GR <= 64)
         rc = s.D == 128 ? launch_split_tc<128, 64>(tmK, tmV, tmQ, a, stream)
                         : launch_split_tc<64, 64>(tmK, tmV, tmQ, a, stream);
@@ -1834,8 +1844,8 @@ int launch_verify_attention(const void* q, const void* k_cache, const void* v_ca
     // otherwise.  Measured per layer (split + merge, chains of layers): ragged batch of 8 132.5 against
     // 136.4 us, one-row decode at 8K 13.05 against 13.5, but 8 units of 36 rows 33.1 against 32.1 at
     // 32K and 86.9 against 86.3 at 128K.
-    const bool one_group = c.kt_path && (c.NC <= 3 || (c.NC == 4 && !c.fp32_sums));
-    const bool warp_per_row = one_group && (a.GR <= 8 || a.num_ctas <= 8 * s.B * s.Hkv);
+    const bool one_group = c.kt_path && !c.two_groups && (c.NC <= 3 || (c.NC == 4 && !c.fp32_sums));
+    const bool warp_per_row = one_group && c.few_slots;
     if (warp_per_row)
         RAPID_CUDA_CHECK(launch_dependent(verify_attn_merge_rows_kernel<128>, dim3((a.GR + 3) / 4, s.B * s.Hkv),
                                           dim3(128), 0, stream, a, a.out, a.lse_out, a.out_f32));
