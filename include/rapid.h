@@ -88,7 +88,7 @@ typedef struct rapid_attn_shape {
 } rapid_attn_shape;
 
 /* Which split kernel rapid_verify_attention uses (rapid_attn_params.kernel). */
-#define RAPID_ATTN_KERNEL_AUTO 0      /* keys on M for head_dim 128 and <= 64 grouped rows, rows on M otherwise */
+#define RAPID_ATTN_KERNEL_AUTO 0      /* keys on M for head_dim 128 and <= 80 grouped rows, rows on M otherwise */
 #define RAPID_ATTN_KERNEL_ROWS_ON_M 1 /* grouped rows on the MMA's M axis: any supported shape           */
 #define RAPID_ATTN_KERNEL_KEYS_ON_M 2 /* keys on the M axis: head_dim 128, <= 96 grouped rows per KV head (two
                                          softmax groups beyond 64), any paged block size the call accepts;
@@ -98,8 +98,8 @@ typedef struct rapid_attn_shape {
                                          partial results on chip, so the call is ONE kernel.  Meant for short
                                          runs (a decode over a few thousand keys, a 32K layer) of sequences of
                                          similar lengths; RAPID_ERR_UNSUPPORTED if the clusters do not fit on
-                                         the device together.  The library picks it by itself for a single
-                                         sequence with a cache capacity of at most 65,536 keys.              */
+                                         the device together.  The library picks it by itself only where the
+                                         clusters would fill three quarters of the SMs.                      */
 
 /* rapid_attn_params.plan */
 #define RAPID_PLAN_NONE 0    /* the call plans for itself: one more tiny kernel ahead of its own (default)    */

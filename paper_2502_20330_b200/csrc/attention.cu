@@ -72,6 +72,10 @@ struct AttnArgs {
     // kv_settled: tiles wholly below the newest R keys may be copied before the grid-dependency wait
     // (the caller vouches for them; needs a settled plan and a contiguous cache)
     int kv_settled;
+    // merge_early: the 4-warp merge lets its dependents launch before its own wait (after a keys-on-M
+    // split kernel; after the rows-on-M kernel it measured 2.5 us slower per layer of the smallest
+    // workload and no faster on the largest, so there the order stays wait, then launch)
+    int merge_early;
     int caller_plan;  // the caller supplied the plan: check it against the call's geometry and lengths
     const Walk* plan_walks;
     const int2* plan_units;  // (first CTA, number of slots) of every unit
@@ -880,10 +884,12 @@ verify_attn_merge_kernel(const __grid_constant__ AttnArgs a, int KS, __nv_bfloat
     const float* base = a.partial + (size_t)(c_first + unit) * KS * slot_stride;  // slots are consecutive
 
     // everything above depends on the call's inputs only; the partials need the split kernel
-    // Dependents may launch BEFORE this kernel's own wait: see verify_attn_merge_rows_kernel for why that
-    // is safe for what the library's kernels do ahead of their waits.
-    asm volatile("griddepcontrol.launch_dependents;");
+    // After a keys-on-M split kernel dependents may launch BEFORE this kernel's own wait: see
+    // verify_attn_merge_rows_kernel for why that is safe for what the library's kernels do ahead of
+    // their waits.
+    if (a.merge_early) asm volatile("griddepcontrol.launch_dependents;");
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!a.merge_early) asm volatile("griddepcontrol.launch_dependents;");
     if (nslots <= 0) {  // the plan is not this call's (status says so): defined output, nothing read
         if (warp == 0) {
             const size_t row = ((size_t)b * a.R + m / a.G) * a.Hq + (size_t)kvh * a.G + m % a.G;
@@ -1521,9 +1527,10 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
 
     // Which split kernel: keys on the MMA's M axis (a softmax thread per key, probabilities through
     // shared memory) when the grouped rows fit 64 columns -- faster and cheaper per byte there --,
-    // rows on the M axis otherwise (more rows, head_dim 64).  From 65 to 96 rows the keys-on-M kernel
-    // runs on request only (two softmax groups; measured level with the rows-on-M kernel at 72
-    // rows, not ahead of it).  With one sequence, whose KV heads all have the same length, and a
+    // rows on the M axis otherwise (more rows, head_dim 64).  From 65 to 80 rows the keys-on-M kernel
+    // with two softmax groups is the choice as well (chains of eight 128K layers: 93.7 against 97.2 us
+    // per layer at 72 rows, 94.1 against 97.9 at 80); at 88 and 96 rows it runs on request only (104.7
+    // against 98.8, 109.4 against 101.5).  With one sequence, whose KV heads all have the same length, and a
     // cache of at most kClusterMaxKeys keys, the keys-on-M kernel runs as one cluster per KV head
     // and merges on chip; any call can ask for that (RAPID_ATTN_KERNEL_CLUSTER_MERGE).
     const int want = params ? params->kernel : RAPID_ATTN_KERNEL_AUTO;
@@ -1537,7 +1544,7 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
         set_error("%s: the keys-on-M kernel needs head_dim 128 and at most %d grouped rows", who, 16 * kt::kMaxNC2);
         return RAPID_ERR_UNSUPPORTED;
     }
-    const bool kt_auto = kt_ok && (GR + 15) / 16 <= kt::kMaxNC;
+    const bool kt_auto = kt_ok && (GR + 15) / 16 <= kt::kMaxNC + 1;
     c.kt_path = want == RAPID_ATTN_KERNEL_KEYS_ON_M || want == RAPID_ATTN_KERNEL_CLUSTER_MERGE ||
                 (want == RAPID_ATTN_KERNEL_AUTO && kt_auto);
     if (fp8) c.kt_path = true;
@@ -1599,6 +1606,7 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
     a.plan_ctx = reinterpret_cast<const int32_t*>(ws + lay.ctx);
     a.wait_limit = wait_limit;
     a.kv_settled = params && params->kv_settled && plan_mode == RAPID_PLAN_SETTLED && !paged;
+    a.merge_early = c.kt_path;
     a.cmerge = 0;
     return RAPID_OK;
 }

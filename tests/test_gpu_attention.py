@@ -512,3 +512,22 @@ def test_early_copies_of_the_settled_cache_change_nothing(Hq, Hkv, gamma, lens, 
         ref, ref_lse = _oracle(q, k, v, ctx, gamma, sink=sink, window=window)
         parity.check_attention(early[i].cpu().numpy(), ref, ~np.isnan(ref_lse))
         assert torch.equal(early[i], plain[i])
+
+
+def test_describe_names_the_kernels_the_workloads_get():
+    """rapid_attention_describe against the library's documented choices for the named workloads."""
+    import paper_2502_20330_b200 as R
+    want = {"llama8b_128k": (2, 2, 48), "llama8b_32k": (2, 2, 48), "llama70b_128k": (2, 2, 80),
+            "qwen7b_ragged": (2, 1, 48), "drafter_8k": (2, 1, 16), "tiny": (1, 2, 64)}
+    for name, (kernel, groups, cols) in want.items():
+        cfg = wl.CONFIGS[name]
+        Lmax = cfg.Lmax or max(cfg.ctx_lens)
+        d = R.rapid_attention_describe(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma)
+        assert (d["kernel"], d["softmax_groups"], d["columns"]) == (kernel, groups, cols), (name, d)
+        assert d["kernels_per_call"] == 2 and d["ctas"] > 0
+    d = R.rapid_attention_describe(1, 64, 8, 128, 131072, 10)          # 88 grouped rows: rows on M
+    assert d["kernel"] == 1
+    d = R.rapid_attention_describe(1, 32, 8, 128, 8192, 0, R.AttnParams(kernel=R.ATTN_KERNEL_CLUSTER_MERGE))
+    assert d["kernel"] == 3 and d["kernels_per_call"] == 1 and d["cluster_size"] >= 2
+    d = R.rapid_attention_describe(1, 32, 8, 128, 131072, 8, R.AttnParams(kv_fp8=True))
+    assert d["kernel"] == 2

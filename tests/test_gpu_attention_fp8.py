@@ -125,14 +125,13 @@ def test_argument_errors():
 
 
 def test_a_plan_made_for_another_kernel_is_refused_not_followed():
-    """72 grouped rows: a plan made without kv_fp8 is the rows-on-M kernel's (64-key tiles, two partials per
-    CTA).  The 8-bit call must not walk it: every CTA compares the plan's signature with its own call, does
+    """72 grouped rows: a plan made for the rows-on-M kernel (64-key tiles, two partials per CTA).  The 8-bit call must not walk it: every CTA compares the plan's signature with its own call, does
     nothing on a mismatch, and the status word says why the output is empty."""
     import paper_2502_20330_b200 as R
     cfg = wl.VerifyConfig("f8", B=2, Hq=64, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(1500, 500))
     q, kc, vc, ks, vs, ctx = wl.attention_inputs_fp8(cfg, seed=2, device="cuda")
     ws = R.new_workspace(R.attention_workspace_bytes(2, 64, 8, 128, 1500, 8))
-    R.rapid_attention_plan(ctx, 8, 2, 64, 8, 128, 1500, ws)               # no kv_fp8: rows on M
+    R.rapid_attention_plan(ctx, 8, 2, 64, 8, 128, 1500, ws, R.AttnParams(kernel=R.ATTN_KERNEL_ROWS_ON_M))
     out = torch.full_like(q, 7.0)
     R.rapid_verify_attention_fp8(q, kc, vc, ks, vs, ctx, 8, out, ws, R.AttnParams(plan=R.PLAN_SETTLED))
     torch.cuda.synchronize()
@@ -144,7 +143,7 @@ def test_a_plan_made_for_another_kernel_is_refused_not_followed():
     R.rapid_verify_attention_fp8(q, kc, vc, ks, vs, ctx, 8, out, ws2, R.AttnParams(plan=R.PLAN_READY))
     q2, k2, v2, ctx2 = wl.attention_inputs(cfg, seed=2, device="cuda")
     R.rapid_verify_attention(q2, k2, v2, ctx2, 8, out, ws2, R.AttnParams(plan=R.PLAN_SETTLED, kernel=2))
-    R.rapid_verify_attention(q2, k2, v2, ctx2, 8, out, ws2, R.AttnParams(plan=R.PLAN_SETTLED))
+    R.rapid_verify_attention(q2, k2, v2, ctx2, 8, out, ws2, R.AttnParams(plan=R.PLAN_SETTLED, kernel=R.ATTN_KERNEL_ROWS_ON_M))
     torch.cuda.synchronize()
     assert R.workspace_status(ws2) & R.STATUS_STALE_PLAN
 
