@@ -618,6 +618,7 @@ def run_ours(args, cfg):
         acc_ms.append(ev.elapsed_ms(a0, a1) / 20)
     del agraph
 
+    attn_layer_us = 1e3 * (ms_per_step - float(np.median(acc_ms))) / cfg.layers
     line = {
         "metric": "verify_step_kv_read_gbs", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -629,7 +630,7 @@ def run_ours(args, cfg):
                             "kv_settled: a layer's first tiles below its newest rows are copied before its stream-order wait",
                 "kernels_per_attention_call": int(launches_per_call), "attention_launch": info,
                 "l2_flush_ms_per_step_not_counted": flush_ms / args.steps},
-        "verify_latency_us": {"attention_per_layer": 1e3 * (ms_per_step - float(np.median(acc_ms))) / cfg.layers,
+        "verify_latency_us": {"attention_per_layer": attn_layer_us,
                               "dominant_kernel_per_layer": 1e3 * kernel_avg_ms,
                               "accept": 1e3 * float(np.median(acc_ms)), "step": 1e3 * ms_per_step,
                               "step_stream_launches": stream_us},
@@ -638,7 +639,14 @@ def run_ours(args, cfg):
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": ncu_traffic(cfg.name, dominant.split(" ")[0]),
                      "algorithmic_bytes": kv_layer,
-                     "timed": f"CUDA events around each of {len(kernel_ms)} launches in a second pass of {k_steps} steps"},
+                     "timed": f"CUDA events around each of {len(kernel_ms)} launches in a second pass of {k_steps} steps "
+                              "(an event between two launches costs them their overlap as programmatic dependents: "
+                              "the launch is timed alone, launch latency and prologue included)",
+                     # the same bytes over a layer's share of the timed steps themselves, where the layers overlap
+                     # as they do in use; that time holds the merge kernel as well
+                     "in_the_timed_steps": {"us_per_layer_split_and_merge": attn_layer_us,
+                                            "achieved": kv_layer / (attn_layer_us * 1e-6) / 1e9,
+                                            "frac": kv_layer / (attn_layer_us * 1e-6) / 1e9 / peak}},
         "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
     }
     if sustained is not None:
@@ -799,6 +807,8 @@ def _rank_main(args):
     cfg = wl.CONFIGS[args.workload]
     if args.layers:
         cfg = wl.with_overrides(cfg, layers=args.layers)
+    if args.gamma >= 0:
+        cfg = wl.with_overrides(cfg, gamma=args.gamma)
     if args.impl == "reference":
         run_reference(args, cfg)
     elif args.sharded:
@@ -815,6 +825,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_128k", choices=sorted(wl.CONFIGS))
     ap.add_argument("--layers", type=int, default=0, help="override the number of resident layers")
+    ap.add_argument("--gamma", type=int, default=-1, help="override the workload's number of draft tokens")
     ap.add_argument("--seed", type=int, default=2025)
     ap.add_argument("--kernel", type=int, default=0, choices=[0, 1, 2, 3],
                     help="split kernel: 0 the library's choice, 1 rows on the MMA's M axis, 2 keys on the M axis, "
