@@ -219,7 +219,10 @@ verify_attn_splitkv_kt_kernel(const __grid_constant__ CUtensorMap tmK,
     if (a.kv_settled && warp == WS && lane == 0 && w.remaining > 0) {
         const int seg0 = (int)min((long long)(w.ntiles - w.tile), w.remaining);
         const int old_tiles = (w.L - a.R) >> 7;  // tiles 0 .. old_tiles-1 hold none of the newest R keys
-        for (int t = 0; t < seg0 && t < NV; ++t) {
+        // a short walk takes only as many tiles early as there are K slots: more V tiles ahead would hold
+        // up the K tiles it needs next (one-row decode at 8K: 12.7 against 13.3 us per layer)
+        const int n_early = seg0 > 2 * NV ? NV : NK;
+        for (int t = 0; t < seg0 && t < n_early; ++t) {
             const int tile = WIN ? real_tile(w, w.tile + t) : w.tile + t;
             if (tile >= old_tiles) break;
             if (t < NK) {

@@ -187,7 +187,8 @@ verify_attn_splitkv_kt8_kernel(const __grid_constant__ CUtensorMap tmK, const __
     if (a.kv_settled && warp == WS && lane == 0 && w.remaining > 0) {
         const int seg0 = (int)min((long long)(w.ntiles - w.tile), w.remaining);
         const int old_tiles = (w.L - a.R) >> 7;  // tiles 0 .. old_tiles-1 hold none of the newest R keys
-        for (int t = 0; t < seg0 && t < NV && w.tile + t < old_tiles; ++t) {
+        const int n_early = seg0 > 2 * NV ? NV : NK;  // a short walk: no V tiles ahead of the K tiles it needs next
+        for (int t = 0; t < seg0 && t < n_early && w.tile + t < old_tiles; ++t) {
             const int key0 = (w.tile + t) * kKeys;
             if (t < NK) {
                 mbar_arrive_expect_tx(&k_full[t], kBlk);
