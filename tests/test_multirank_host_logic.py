@@ -87,3 +87,28 @@ def test_both_arms_print_the_same_config():
     a = bench.config_dict(cfg, ctx, 1)
     assert a == bench.config_dict(cfg, ctx, 1) and a["workload"] == "qwen7b_ragged" and "model" not in a
     assert a["kv_bytes_per_step"] == 4 * cfg.Hkv * cfg.D * int(ctx.sum())
+
+
+def test_visible_keys_under_a_window_by_brute_force():
+    """bench.py's algorithmic bytes under --sink/--window: the keys SOME row can see, counted one by one."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import workloads as wl
+    saved = bench.MASK
+    try:
+        for gamma in (0, 3, 8):
+            cfg = wl.VerifyConfig("w", B=3, Hq=8, Hkv=2, D=64, gamma=gamma, V=4096, ctx_lens=(300, 40, gamma + 1))
+            for sink, window in ((0, 0), (4, 16), (0, 1), (50, 7), (4, 4092), (400, 3)):
+                bench.MASK = (sink, window)
+                want = 0
+                for L in cfg.ctx_lens:
+                    seen = set()
+                    for i in range(cfg.R):
+                        own = L - cfg.R + i
+                        for j in range(own + 1):
+                            if window <= 0 or j < sink or j > own - window:
+                                seen.add(j)
+                    want += len(seen)
+                assert bench.visible_keys(cfg, cfg.ctx_lens) == want, (gamma, sink, window)
+    finally:
+        bench.MASK = saved
