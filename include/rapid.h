@@ -107,7 +107,10 @@ typedef struct rapid_attn_shape {
                                 geometry and for the current ctx_lens                                      */
 #define RAPID_PLAN_SETTLED 2 /* as RAPID_PLAN_READY, and at least one other kernel (or a synchronisation)
                                 lies between rapid_attention_plan and this call in the stream: the plan is
-                                then read while the preceding kernel still runs                            */
+                                then read while the preceding kernel still runs.  That kernel must be one
+                                of this library's or an ordinary launch: a foreign kernel launched with
+                                programmatic stream serialisation that lets its dependents go before the
+                                plan kernel has completed does not settle anything                         */
 
 /* Optional knobs and extra outputs of the attention call (NULL = defaults). */
 typedef struct rapid_attn_params {
