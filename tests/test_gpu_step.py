@@ -86,3 +86,45 @@ def test_verify_step_replays_from_a_cuda_graph():
     parity.check_accept(z.cpu().numpy(), d.cpu().numpy(), tok.cpu().numpy(), u.cpu().numpy(), 5.0, 1.0, 0.1, 0,
                         alen.cpu().numpy(), ntok.cpu().numpy())
     assert R.workspace_status(aws) == 0 and R.workspace_status(cws) == 0
+
+
+@pytest.mark.parametrize("name,nlayers", [("llama8b_32k", 4), ("drafter_8k", 6)])
+def test_overlapping_layers_replay_bit_identically(name, nlayers):
+    """A step's layers in one CUDA graph, every layer but the first with a settled plan and early copies of its
+    old keys: the next layer's split kernel starts while this layer's still runs.  Forty replays must reproduce
+    the first run bit for bit, and layer 0 must match the oracle."""
+    import numpy as np
+    import oracle
+    from oracle import parity
+    from workloads import bf16_bits
+    import paper_2502_20330_b200 as R
+    cfg = wl.CONFIGS[name]
+    layers = [wl.attention_inputs(cfg, seed=9 + i, device="cuda", layer=i) for i in range(nlayers)]
+    ctx, Lmax = layers[0][3], layers[0][1].shape[2]
+    ws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma))
+    outs = [torch.zeros_like(l[0]) for l in layers]
+
+    def step():
+        R.rapid_attention_plan(ctx, cfg.gamma, cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, ws, R.AttnParams())
+        for i, (q, k, v, _) in enumerate(layers):
+            R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, outs[i], ws,
+                                     R.AttnParams(plan=R.PLAN_READY if i == 0 else R.PLAN_SETTLED, kv_settled=True))
+
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        step()
+        torch.cuda.synchronize()
+        first = [o.clone() for o in outs]
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            step()
+        for _ in range(40):
+            for o in outs:
+                o.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            assert all(torch.equal(o, r) for o, r in zip(outs, first))
+    assert R.workspace_status(ws) == 0
+    q, k, v, _ = layers[0]
+    ref, ref_lse = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx.cpu().numpy(), cfg.gamma)
+    parity.check_attention(first[0].float().cpu().numpy(), ref, ~np.isnan(ref_lse))
