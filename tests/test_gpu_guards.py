@@ -146,6 +146,38 @@ def test_sharded_merge_guard_bands():
     np.testing.assert_allclose(o32.t.cpu().numpy(), ref, rtol=0, atol=2e-5)
 
 
+@pytest.mark.parametrize("Hq,gamma,lens,num_ctas,plan", [
+    (32, 8, (3000, 777), 0, 0), (64, 8, (1500, 500), 0, 2), (32, 0, (2048,), 512, 1),
+])
+def test_fp8_attention_guard_bands(Hq, gamma, lens, num_ctas, plan):
+    """The 8-bit-cache call inside sentinel bands, planned and unplanned, early copies included."""
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("g8", B=len(lens), Hq=Hq, Hkv=8, D=128, gamma=gamma, V=4096, ctx_lens=lens)
+    q, kc, vc, ks, vs, ctx = wl.attention_inputs_fp8(cfg, seed=91, device="cuda", poison_padding=True)
+    Lmax = kc.shape[2]
+    nbytes = R.attention_workspace_bytes(cfg.B, Hq, 8, 128, Lmax, gamma)
+    out, o32 = Banded(q.shape, torch.bfloat16), Banded(q.shape, torch.float32)
+    lse, ws = Banded(q.shape[:3], torch.float32), Banded((nbytes,), torch.uint8)
+    lens_b = Banded(ctx.shape, torch.int32, fill=ctx)
+    ksb, vsb = Banded(ks.shape, torch.float32, fill=ks), Banded(vs.shape, torch.float32, fill=vs)
+    R.workspace_init(ws.t)
+    params = R.AttnParams(num_ctas=num_ctas, lse_out=lse.t, out_f32=o32.t, plan=plan, kv_fp8=True,
+                          kv_settled=plan == R.PLAN_SETTLED)
+    if plan:
+        R.rapid_attention_plan(lens_b.t, gamma, cfg.B, Hq, 8, 128, Lmax, ws.t, params)
+        if plan == R.PLAN_SETTLED:
+            torch.zeros(8, device="cuda").add_(1.0)
+    R.rapid_verify_attention_fp8(q, kc, vc, ksb.t, vsb.t, lens_b.t, gamma, out.t, ws.t, params)
+    torch.cuda.synchronize()
+    assert R.workspace_status(ws.t) == 0
+    for name, b in (("out", out), ("out_f32", o32), ("lse", lse), ("workspace", ws), ("ctx_lens", lens_b),
+                    ("k_scale", ksb), ("v_scale", vsb)):
+        assert b.intact(), f"bytes around {name} were written"
+    ref, ref_lse = oracle.verify_attention_fp8(bf16_bits(q), kc.cpu().numpy(), vc.cpu().numpy(), ks.cpu().numpy(),
+                                               vs.cpu().numpy(), ctx.cpu().numpy(), gamma)
+    parity.check_attention(out.t.float().cpu().numpy(), ref, ~np.isnan(ref_lse))
+
+
 # ---- RAPID_STATUS_RESIDUAL_FALLBACK ----------------------------------------------------------------------
 
 def _accept(z, d, tok, u, eta, mode=0):
@@ -208,6 +240,59 @@ def test_empty_residual_of_a_row_the_loop_never_reaches_raises_nothing():
 
 
 # ---- RAPID_STATUS_PIPELINE_TIMEOUT -----------------------------------------------------------------------
+
+@pytest.mark.parametrize("limit", [1, 3000, 40000])
+def test_a_wait_that_runs_out_after_early_copies_went_out(limit):
+    """The same with a settled plan and kv_settled: the producer has copies in flight from before its
+    stream-order wait when its first bounded wait gives up, and must see them land before the CTA ends."""
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("to", B=2, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(40000, 30000))
+    q, k, v, ctx = wl.attention_inputs(cfg, seed=89, device="cuda")
+    Lmax = k.shape[2]
+    ws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, cfg.gamma))
+    out = torch.empty_like(q)
+    ref, _ = oracle.verify_attention(bf16_bits(q), bf16_bits(k), bf16_bits(v), ctx.cpu().numpy(), cfg.gamma)
+
+    def call(lim):
+        R.rapid_attention_plan(ctx, cfg.gamma, cfg.B, cfg.Hq, cfg.Hkv, cfg.D, Lmax, ws, R.AttnParams())
+        torch.zeros(8, device="cuda").add_(1.0)
+        R.rapid_verify_attention(q, k, v, ctx, cfg.gamma, out, ws,
+                                 R.AttnParams(plan=R.PLAN_SETTLED, kv_settled=True, wait_cycle_limit=lim))
+        torch.cuda.synchronize()
+        return R.workspace_status(ws)
+
+    status = call(limit)
+    if limit == 1:
+        assert status == R.STATUS_PIPELINE_TIMEOUT
+    else:
+        assert status in (0, R.STATUS_PIPELINE_TIMEOUT)
+    R.workspace_init(ws)
+    assert call(0) == 0
+    parity.check_attention(out.float().cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("limit", [1, 3000, 40000])
+def test_a_wait_that_runs_out_over_the_fp8_cache(limit):
+    import paper_2502_20330_b200 as R
+    cfg = wl.VerifyConfig("to8", B=2, Hq=32, Hkv=8, D=128, gamma=8, V=4096, ctx_lens=(40000, 30000))
+    q, kc, vc, ks, vs, ctx = wl.attention_inputs_fp8(cfg, seed=90, device="cuda")
+    ws = R.new_workspace(R.attention_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, kc.shape[2], cfg.gamma))
+    out = torch.empty_like(q)
+    R.rapid_verify_attention_fp8(q, kc, vc, ks, vs, ctx, cfg.gamma, out, ws, R.AttnParams(wait_cycle_limit=limit))
+    torch.cuda.synchronize()
+    status = R.workspace_status(ws)
+    if limit == 1:
+        assert status == R.STATUS_PIPELINE_TIMEOUT
+    else:
+        assert status in (0, R.STATUS_PIPELINE_TIMEOUT)
+    R.workspace_init(ws)
+    R.rapid_verify_attention_fp8(q, kc, vc, ks, vs, ctx, cfg.gamma, out, ws)
+    torch.cuda.synchronize()
+    assert R.workspace_status(ws) == 0
+    ref, ref_lse = oracle.verify_attention_fp8(bf16_bits(q), kc.cpu().numpy(), vc.cpu().numpy(), ks.cpu().numpy(),
+                                               vs.cpu().numpy(), ctx.cpu().numpy(), cfg.gamma)
+    parity.check_attention(out.float().cpu().numpy(), ref, ~np.isnan(ref_lse))
+
 
 @pytest.mark.parametrize("kernel", [1, 2, 3])
 @pytest.mark.parametrize("limit", [1, 3000, 40000])
