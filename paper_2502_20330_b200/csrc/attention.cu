@@ -1353,13 +1353,17 @@ int launch_split_kt(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtens
 int dispatch_split_kt(int NC, bool fp32_sums, bool two_groups, const CUtensorMap& tmK, const CUtensorMap& tmV,
                       const CUtensorMap& tmQ, AttnArgs& a, cudaStream_t stream, bool want_cluster, bool need_cluster) {
     switch (NC) {
-        case 1: return launch_split_kt<1>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
-        case 2: return launch_split_kt<2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
+        case 1:
+            return two_groups ? launch_split_kt<1, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster)
+                              : launch_split_kt<1>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
+        case 2:
+            return two_groups ? launch_split_kt<2, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster)
+                              : launch_split_kt<2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
         case 3:
             return two_groups ? launch_split_kt<3, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster)
                               : launch_split_kt<3>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
         case 4:
-            return fp32_sums ? launch_split_kt<4, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster)
+            return (fp32_sums || two_groups) ? launch_split_kt<4, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster)
                              : launch_split_kt<4>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
         // more than 64 grouped rows: two softmax groups, each with half of the columns
         case 5: return launch_split_kt<5, 2>(tmK, tmV, tmQ, a, stream, want_cluster, need_cluster);
@@ -1563,12 +1567,13 @@ int prepare_attention(const char* who, const int32_t* ctx_lens, int gamma, const
     c.KS = c.kt_path ? 1 : kStreams;
     c.fp32_sums = params && params->lse_out;
     // Few partial slots per unit, or few rows: the warp-per-row merge whose blocks sit beside the split
-    // kernel's CTAs pays (it needs the one-group kernel's registers).  Otherwise 33 to 48 grouped rows
-    // run with two softmax groups of 24 columns: measured 30.2 against 32.0 us per 32K layer and 83.8
-    // against 84.5 per 128K layer of the 8-unit shape (the ragged batch of 32 units, with the other
-    // merge: 134.2 against 131.6, which is why it keeps one group).
+    // kernel's CTAs pays (it needs the one-group kernel's registers).  Otherwise up to 64 grouped rows
+    // run with two softmax groups of 8 to 32 columns: measured 30.2 against 32.0 us per 32K layer and
+    // 83.8 against 84.5 per 128K layer of the 8-unit shape at 36 rows, 33.4 against 36.3 and 89.5 against
+    // 91.1 at 63 rows, 14.5 against 16.1 per 8K layer at 20 rows, 12.6 against 13.0 at 12 rows (the
+    // ragged batch of 32 units, with the other merge: 134.2 against 131.6, which is why it keeps one group).
     c.few_slots = GR <= 8 || num_ctas <= 8 * s.B * s.Hkv;
-    c.two_groups = c.kt_path && !fp8 && c.NC == 3 && !c.few_slots && !c.need_cluster;
+    c.two_groups = c.kt_path && !fp8 && c.NC <= 4 && !c.few_slots && !c.need_cluster;
     if (c.two_groups) c.want_cluster = false;
 
     AttnArgs& a = c.a;
