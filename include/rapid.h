@@ -21,7 +21,14 @@
  *     and must not be shared by calls that can overlap on the GPU.
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as
  *     void*; NULL is the default stream).  There is no host synchronisation
- *     unless an entry point says so.
+ *     unless an entry point says so.  Work issued to the stream after a call
+ *     sees its results, as after any kernel launch.  Among themselves the
+ *     library's kernels are programmatic dependent launches (a kernel's
+ *     prologue, and where the caller allows it the first copies of old cache
+ *     tiles, overlap the kernel before it); a caller's own kernel launched
+ *     with programmatic stream serialisation right after a call may likewise
+ *     start while the call's kernels run and must pass its grid-dependency
+ *     wait before it touches anything the call reads or writes.
  *   - Return value: RAPID_OK or one of the RAPID_ERR_* codes.  No exception
  *     crosses the boundary.  rapid_last_error() describes the last failure on
  *     the calling thread.
