@@ -43,6 +43,10 @@ def _oracle_paged(q, kp, vp, table, ctx, gamma):
     (28, 4, 128, 4, 128, (1500, 2300), True),        # [block, token, head, D] storage
     (8, 2, 64, 4, 512, (1000, 70), False),           # head_dim 64, a sequence inside one block
     (32, 8, 128, 0, 128, (777,), True),              # one-row decode
+    (32, 8, 128, 2, 64, (5000, 900), False),         # 12 grouped rows: two softmax groups of 8 columns, 64-key blocks
+    (32, 8, 128, 4, 256, (7000,), True),             # 20 rows: two groups of 16 columns
+    (56, 8, 128, 8, 128, (4000, 2100), False),       # 63 rows: two groups of 32 columns
+    (64, 8, 128, 8, 64, (3000, 1000), False),        # 72 rows: two groups of 40 columns, two boxes per tile
 ])
 def test_paged_against_oracle(Hq, Hkv, D, gamma, bs, lens, token_major):
     cfg = wl.VerifyConfig("p", B=len(lens), Hq=Hq, Hkv=Hkv, D=D, gamma=gamma, V=4096, ctx_lens=lens)
